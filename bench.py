@@ -1,0 +1,451 @@
+#!/usr/bin/env python
+"""Benchmark of libfsoftmax: last-dimension softmax, achieved HBM GB/s against the roofline.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference] [--all]
+
+A step is one fs_softmax call (dispatcher -> one kernel) over one batch of the headline workload:
+the bf16 attention-score tensor, 16384 rows x 2048 columns (cfg2). Inputs are seeded synthetic data
+already resident in HBM; successive steps rotate over enough independent (x, y) buffer pairs that
+the working set is several times the L2 size, so every step reads and writes DRAM. Timing is on the
+device with CUDA events recorded on the launching stream, max over ranks.
+
+One JSON line goes to stdout (rank 0). Beyond the base keys it carries
+  roofline      algorithmic bytes (read x once + write y once) per launch / average launch time,
+                against the measured copy bandwidth of this GPU pool (MEASURED_PEAKS.json)
+  e2e           the same metric through fs_softmax_host: pinned host buffers, H2D and D2H copies
+                inside the timed region
+  cpu_baseline  the fp64 oracle, as it stands, on the host cores over a bounded sample
+  workloads     the other four workloads, each timed the same way (--all, default on at N=1)
+With N > 1 (launched by torch.distributed.run) every rank runs the same per-GPU workload on its
+own GPU: rows are independent, so there is no collective on the data path ("weak" scaling).
+
+--impl reference times the CPU oracle instead (rank 0 only), on a bounded sample per step.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2607_24762_b200 import workloads as W  # noqa: E402
+
+METRIC = "softmax achieved HBM GB/s (min read+write bytes/time)"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
+# summarised under profiles/; None where no capture has been taken.
+NCU_TRAFFIC_BYTES = {
+}
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks
+# ---------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index          # nvidia-smi -i accepts an index or a GPU UUID
+        self.proc = None
+        self.file = None
+
+    def start(self):
+        try:
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
+                 "-i", str(self.index)], stdout=self.file, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def n_samples(self) -> int:
+        if not self.file:
+            return 0
+        try:
+            with open(self.file.name) as f:
+                return sum(1 for _ in f)
+        except Exception:
+            return 0
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if not self.proc:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        rows = []
+        try:
+            with open(self.file.name) as f:
+                for line in f:
+                    parts = [p.strip() for p in line.split(",")]
+                    if len(parts) >= 8:
+                        rows.append(parts)
+            os.unlink(self.file.name)
+        except Exception:
+            pass
+        sm = []
+        reasons = set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for p in rows:
+            try:
+                sm.append(float(p[0]))
+                out["sm_max_mhz"] = float(p[1])
+            except ValueError:
+                continue
+            for name, v in zip(names, p[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if sm:
+            out["sm_mhz"] = statistics.median(sm)
+        out["reasons"] = sorted(reasons)
+        out["samples"] = len(sm)
+        return out
+
+
+# ---------------------------------------------------------------------------------------------
+# GPU arm
+# ---------------------------------------------------------------------------------------------
+
+def device_buffers(w: W.Workload, n_pairs: int, threads: int):
+    """n_pairs independent (x, y) device buffer pairs holding the workload's seeded input."""
+    import torch
+    tdtype = torch.float32 if w.dtype == W.FP32 else torch.int16
+    slab = max(1, (64 << 20) // (w.cols * w.elem_size))
+    x0 = torch.empty((w.rows, w.cols), dtype=tdtype, device="cuda")
+    for r0 in range(0, w.rows, slab):
+        r1 = min(w.rows, r0 + slab)
+        h = W.generate_rows(w, r0, r1, threads=threads)
+        x0[r0:r1].copy_(torch.from_numpy(h.view(np.int16) if w.dtype != W.FP32 else h))
+    xs = [x0] + [x0.clone() for _ in range(n_pairs - 1)]
+    ys = [torch.empty_like(x0) for _ in range(n_pairs)]
+    return xs, ys
+
+
+def time_device(w: W.Workload, steps: int, warmup: int, l2_bytes: int, sampler: ClockSampler | None = None,
+                barrier=None, min_clock_samples: int = 0):
+    """Times `steps` fs_softmax launches with CUDA events on the launching stream."""
+    import torch
+
+    import paper_2607_24762_b200 as fs
+    free, _ = torch.cuda.mem_get_info()
+    pair_bytes = w.min_bytes
+    want = max(1, math.ceil(4 * l2_bytes / pair_bytes))
+    n_pairs = int(max(1, min(want, 256, (free * 0.6) // pair_bytes)))
+    xs, ys = device_buffers(w, n_pairs, threads=min(8, os.cpu_count() or 1))
+    stream = torch.cuda.current_stream()
+    sh = stream.cuda_stream
+    lib = fs.binding.lib()
+    ptrs = [(x.data_ptr(), y.data_ptr()) for x, y in zip(xs, ys)]
+    scale = w.scale_f32
+
+    def launch(i):
+        xp, yp = ptrs[i % n_pairs]
+        st = lib.fs_softmax(xp, yp, w.rows, w.cols, w.dtype, scale, sh)
+        if st != 0:
+            raise RuntimeError(f"fs_softmax failed: {fs.fs_strerror(st)}")
+
+    for i in range(max(3, warmup)):
+        launch(i)
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+    if sampler:
+        sampler.start()
+        time.sleep(0.12)
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    start.record(stream)
+    for i in range(steps):
+        launch(i)
+    stop.record(stream)
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+    ms = start.elapsed_time(stop)
+    extension_s = 0.0
+    if sampler and min_clock_samples:
+        # the timed region can be shorter than nvidia-smi's sampling period: keep the same loop
+        # running (untimed) until enough clock samples were taken under load
+        t0 = time.time()
+        i = 0
+        while sampler.n_samples() < min_clock_samples + 3 and time.time() - t0 < 3.0:
+            for _ in range(64):
+                launch(i)
+                i += 1
+            torch.cuda.synchronize()
+        extension_s = time.time() - t0
+    clocks = sampler.stop() if sampler else None
+    if clocks is not None:
+        clocks["sampled_over"] = "timed region" + (f" + {extension_s:.1f} s of the same launches" if extension_s else "")
+    status = fs.fs_device_status()
+    if status != 0:
+        raise RuntimeError(f"device status: {fs.fs_strerror(status)}")
+    kernel = fs.fs_kernel_name(fs.fs_select_kernel(w.rows, w.cols, w.dtype))
+    del xs, ys
+    torch.cuda.empty_cache()
+    return {"ms_per_step": ms / steps, "n_pairs": n_pairs, "kernel": kernel, "clocks": clocks}
+
+
+def time_e2e(w: W.Workload, steps: int, warmup: int):
+    """The same metric through fs_softmax_host: pinned host buffers in, pinned host buffers out."""
+    import torch
+
+    import paper_2607_24762_b200 as fs
+    rows = w.rows
+    tdtype = torch.float32 if w.dtype == W.FP32 else torch.int16
+    h = W.generate_rows(w, 0, rows, threads=min(8, os.cpu_count() or 1))
+    xh = torch.from_numpy(h.view(np.int16) if w.dtype != W.FP32 else h).pin_memory()
+    yh = torch.empty((rows, w.cols), dtype=tdtype).pin_memory()
+    for _ in range(max(1, warmup)):
+        fs.fs_softmax_host(xh, yh, rows, w.cols, w.dtype, w.scale_f32)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        fs.fs_softmax_host(xh, yh, rows, w.cols, w.dtype, w.scale_f32)     # blocks until y_host is complete
+    dt = (time.perf_counter() - t0) / steps
+    nbytes = rows * w.cols * w.elem_size
+    fs.fs_release()
+    return {"value": round(2 * nbytes / dt / 1e9, 2), "unit": UNIT, "ms_per_step": round(dt * 1e3, 4),
+            "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": nbytes,
+            "api": "fs_softmax_host (pinned host buffers, 16 MiB chunks pipelined over 3 streams)"}
+
+
+# ---------------------------------------------------------------------------------------------
+# CPU oracle arm (reported baseline; also --impl reference)
+# ---------------------------------------------------------------------------------------------
+
+def oracle_sample(w: W.Workload, target_cpu_seconds: float):
+    """A bounded sample of the workload: evenly spaced row blocks, sized for ~target_cpu_seconds."""
+    ns_per_elem = 30.0 if w.index == 5 else 11.0
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+    rows = int(target_cpu_seconds * 1e9 / ns_per_elem / w.cols)
+    rows = max(cores, min(w.rows, rows))
+    rows -= rows % cores if rows >= 2 * cores else 0
+    stride = max(1, w.rows // rows)
+    idx = [min(w.rows - 1, i * stride) for i in range(rows)]
+    x = np.concatenate([W.generate_rows(w, i, i + 1) for i in idx]) if stride > 1 else W.generate_rows(w, 0, rows)
+    return x, cores, f"{rows} of {w.rows} rows (every {stride}th), all {w.cols} columns"
+
+
+def run_oracle(w: W.Workload, x: np.ndarray, cores: int) -> float:
+    """Seconds for the single-threaded oracle run on `cores` threads over a row partition of x."""
+    from oracle import fso
+    parts = [p for p in np.array_split(np.arange(x.shape[0]), cores) if len(p)]
+    outs = [None] * len(parts)
+
+    def work(k):
+        outs[k] = fso.softmax_f64(x[parts[k][0]:parts[k][-1] + 1], w.dtype, w.scale_f32)
+
+    ths = [threading.Thread(target=work, args=(k,)) for k in range(len(parts))]
+    t0 = time.perf_counter()
+    for t in ths:
+        t.start()
+    for t in ths:
+        t.join()
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(w: W.Workload, target_cpu_seconds: float = 16.0):
+    from oracle import fso
+    fso.build()
+    x, cores, what = oracle_sample(w, target_cpu_seconds)
+    run_oracle(w, x[:cores], cores)                        # load the library, touch the code
+    # a workload smaller than the target is passed over several times (about 10 s of CPU work)
+    est = x.size * 11e-9
+    passes = int(max(1, min(200, round(10.0 / max(est, 1e-3)))))
+    dt = sum(run_oracle(w, x, cores) for _ in range(passes)) / passes
+    nbytes = 2 * x.size * w.elem_size
+    if passes > 1:
+        what += f", mean of {passes} passes"
+    return {"value": round(nbytes / dt / 1e9, 4), "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": what, "seconds": round(dt, 4), "rows_per_s": round(x.shape[0] / dt, 1)}
+
+
+def reference_arm(args, w: W.Workload):
+    """--impl reference: the oracle, as it stands, on the host cores; a step is one bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import fso
+    fso.build()
+    x, cores, what = oracle_sample(w, 4.0)
+    for _ in range(max(1, min(args.warmup, 2))):
+        run_oracle(w, x, cores)
+    steps = max(1, min(args.steps, 20))
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        run_oracle(w, x, cores)
+    dt = (time.perf_counter() - t0) / steps
+    value = round(2 * x.size * w.elem_size / dt / 1e9, 4)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": args.warmup, "ms_per_step": round(dt * 1e3, 3), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "shape": [w.rows, w.cols], "storage_dtype": W.DTYPE_NAME[w.dtype],
+                       "step": "the fp64 oracle over a bounded sample of the workload: " + what},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------
+# main
+# ---------------------------------------------------------------------------------------------
+
+def smi_id(props, local_rank: int) -> str:
+    """The GPU's UUID (CUDA_VISIBLE_DEVICES may renumber indices), else its index."""
+    try:
+        u = str(props.uuid)
+        return u if u.startswith("GPU-") else "GPU-" + u
+    except Exception:
+        return str(local_rank)
+
+
+def roofline_obj(w: W.Workload, ms_per_step: float, kernel: str):
+    peak, which = measured_peak()
+    achieved = w.min_bytes / (ms_per_step * 1e-3) / 1e9
+    traffic = NCU_TRAFFIC_BYTES.get(w.name)
+    return {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+            "frac": round(achieved / peak, 4), "peak_source": f"of {which} (copy bandwidth)",
+            "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
+            "traffic": traffic, "algorithmic_bytes_per_launch": w.min_bytes, "kernel": kernel}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--workload", default="cfg2", choices=sorted(W.WORKLOADS))
+    ap.add_argument("--impl", default="fsoftmax", choices=["fsoftmax", "reference"])
+    ap.add_argument("--rows", type=int, default=0,
+                    help="use only the first ROWS rows of the workload (small cases for profiler captures)")
+    ap.add_argument("--all", dest="all_workloads", action="store_true", default=None,
+                    help="also time the other workloads (default: on at --gpus 1)")
+    ap.add_argument("--no-all", dest="all_workloads", action="store_false")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the cpu_baseline leg")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the end-to-end leg")
+    ap.add_argument("--no-clocks", action="store_true", help="do not sample nvidia-smi clocks (profiler captures)")
+    args = ap.parse_args()
+    w = W.WORKLOADS[args.workload]
+    if args.rows:
+        import dataclasses
+        w = dataclasses.replace(w, rows=min(w.rows, args.rows), note=w.note + f" (first {args.rows} rows)")
+
+    if args.impl == "reference":
+        reference_arm(args, w)
+        return
+
+    import torch
+
+    import __graft_entry__ as entry
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: libfsoftmax has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        entry.build()
+    if dist:
+        dist.barrier()
+    import paper_2607_24762_b200 as fs
+    fs.binding.lib()
+
+    def barrier():
+        if dist:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    props = torch.cuda.get_device_properties(local_rank)
+    l2 = int(getattr(props, "L2_cache_size", 126 << 20))
+    sampler = ClockSampler(smi_id(props, local_rank)) if rank == 0 and not args.no_clocks else None
+    res = time_device(w, args.steps, args.warmup, l2, sampler=sampler, barrier=barrier, min_clock_samples=8)
+    ms = res["ms_per_step"]
+    if dist:
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    value = world * w.min_bytes / (ms * 1e-3) / 1e9
+
+    line = {"metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": round(ms, 6), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "what": w.note, "shape": [w.rows, w.cols],
+                       "storage_dtype": W.DTYPE_NAME[w.dtype], "scale": w.scale_f32, "kernel": res["kernel"],
+                       "parallelism": f"rows independent: {world} replica(s) of the per-GPU workload, no collective",
+                       "l2": f"rotating over {res['n_pairs']} independent (x,y) buffer pairs = "
+                             f"{res['n_pairs'] * w.min_bytes / 2**20:.0f} MiB, L2 is {l2 / 2**20:.0f} MiB",
+                       "rows_per_s": round(world * w.rows / (ms * 1e-3), 1)},
+            "roofline": roofline_obj(w, ms, res["kernel"]),
+            "gpu_launches": args.steps,
+            "clocks": res["clocks"]}
+
+    if rank == 0 and world == 1:
+        if not args.no_e2e:
+            line["e2e"] = time_e2e(w, steps=max(3, min(args.steps, 20)), warmup=2)
+        if args.all_workloads is None or args.all_workloads:
+            others = {}
+            for name, ow in W.WORKLOADS.items():
+                if name == w.name:
+                    continue
+                free, _ = torch.cuda.mem_get_info()
+                if free < ow.min_bytes * 1.3:
+                    others[name] = {"skipped": "not enough free device memory"}
+                    continue
+                k = max(20, min(2000, int(0.08 / max(ow.min_bytes / 6.0e12, 4e-6))))
+                r = time_device(ow, k, 10, l2)
+                gbs = ow.min_bytes / (r["ms_per_step"] * 1e-3) / 1e9
+                peak, which = measured_peak()
+                others[name] = {"what": ow.note, "kernel": r["kernel"], "steps": k, "ms_per_step": round(r["ms_per_step"], 6),
+                                "GB/s": round(gbs, 1), "rows_per_s": round(ow.rows / (r["ms_per_step"] * 1e-3), 1),
+                                "frac_of_measured_copy": round(gbs / peak, 4),
+                                "frac_of_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 4), "n_pairs": r["n_pairs"]}
+            line["workloads"] = others
+        if not args.no_cpu:
+            line["cpu_baseline"] = cpu_baseline(w)
+    elif rank == 0:
+        line["e2e"] = None
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if dist:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

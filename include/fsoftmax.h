@@ -1,0 +1,126 @@
+/*
+ * libfsoftmax -- last-dimension softmax for NVIDIA B200 (sm_100a), C ABI.
+ *
+ * The operation is the `softmax` operator the paper reports its largest gains on (abstract and
+ * Sec. IV-C: Gemma 4 E2B and Qwen 3.5 35B-A3B eager-attention softmax); its semantics are the
+ * eager framework's on the same inputs (Sec. III-C, "Kernel Validator"):
+ *
+ *     y[i][j] = exp(z[i][j] - max_k z[i][k]) / sum_k exp(z[i][k] - max_k z[i][k]),   z = scale * x
+ *
+ * over the last dimension of a contiguous row-major [rows, cols] tensor. Arithmetic is fp32 inside
+ * (fp32 accumulation of the row sum), the result is rounded once, to nearest even, to the tensor's
+ * dtype. IEEE special values follow the formula literally: a -inf entry beside finite ones gives
+ * exactly +0; a NaN or +inf entry (after scaling), or a row holding only -inf, makes that whole row
+ * NaN. `scale` may be zero or negative.
+ *
+ * General conventions
+ *   - Pointers named `x`/`y` are DEVICE pointers unless the entry point says "host".
+ *   - The caller owns every buffer and the stream. Device entry points only enqueue work on
+ *     `stream` (a cudaStream_t passed as void*, NULL = default stream): they never synchronise
+ *     and keep no reference to the buffers after the enqueued work has run.
+ *   - All entry points return an fs_status as int and enqueue nothing when they return an error.
+ *   - The library works on the calling thread's current CUDA device. One GPU; no host fallback:
+ *     without a usable CUDA device every compute entry point returns FS_ERR_CUDA.
+ *   - Thread-safe. Per-device attributes are cached on first use.
+ */
+#ifndef FSOFTMAX_H_
+#define FSOFTMAX_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { FS_DTYPE_FP32 = 0, FS_DTYPE_BF16 = 1, FS_DTYPE_FP16 = 2 } fs_dtype;
+
+typedef enum {
+    FS_OK = 0,
+    FS_ERR_INVALID_ARG = 1,    /* null pointer, negative size, unknown dtype/kernel, non-finite scale, partial overlap */
+    FS_ERR_UNSUPPORTED = 2,    /* a forced kernel cannot handle this shape/alignment/launch geometry */
+    FS_ERR_CUDA = 3,           /* a CUDA call failed; see fs_last_cuda_error() */
+    FS_ERR_DEVICE_TIMEOUT = 4  /* a bounded device-side wait expired (reported by fs_device_status) */
+} fs_status;
+
+/* The kernels behind the size-based dispatcher (the "variants" of the operator in the sense of
+ * the paper's Sec. III-A: same operator, different shape/dtype/layout -> different kernel). */
+typedef enum {
+    FS_KERNEL_AUTO = 0,
+    FS_KERNEL_WARP = 1,       /* (sub-)warp per row, row held in registers */
+    FS_KERNEL_BLOCK = 2,      /* block per row, 128-bit global loads, row held in registers */
+    FS_KERNEL_BLOCK_TMA = 3,  /* block per row, rows prefetched into a shared-memory ring by bulk async copies */
+    FS_KERNEL_CLUSTER = 4,    /* thread-block cluster per row, (max,sum) pairs exchanged through distributed shared memory */
+    FS_KERNEL_GENERIC = 5     /* any cols, any alignment; reads the row twice */
+} fs_kernel;
+
+/*
+ * fs_softmax -- y = softmax(scale * x) over the last dimension; the dispatcher picks the kernel.
+ *   x, y   device pointers to rows*cols elements of `dtype`, row-major, row pitch = cols elements.
+ *          x == y (exact aliasing) is allowed; any other overlap returns FS_ERR_INVALID_ARG.
+ *          Any alignment is accepted; the fast kernels need 16-byte aligned x and y and a row size
+ *          that is a multiple of 16 bytes, other cases run the generic kernel.
+ *   rows, cols  >= 0. rows == 0 or cols == 0 returns FS_OK without a launch.
+ *   dtype  an fs_dtype; x and y share it.
+ *   scale  finite float, multiplies x before the max is taken (scale <= 0 is legal).
+ *   stream cudaStream_t as void*.
+ */
+int fs_softmax(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale, void* stream);
+
+/*
+ * fs_softmax_ex -- as fs_softmax, with the kernel and its launch geometry forced (tests, tuning).
+ *   kernel   an fs_kernel; FS_KERNEL_AUTO behaves like fs_softmax.
+ *   threads  threads per block, 0 = the kernel's own choice. Must be a multiple of 32.
+ *   cluster  blocks per cluster for FS_KERNEL_CLUSTER (1, 2, 4, 8 or 16), 0 = the kernel's choice;
+ *            ignored by the other kernels.
+ * Returns FS_ERR_UNSUPPORTED when the forced kernel cannot run this shape, alignment or geometry.
+ */
+int fs_softmax_ex(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale,
+                  void* stream, int kernel, int threads, int cluster);
+
+/*
+ * fs_select_kernel -- the dispatcher's decision, without a launch (no CUDA call is made when the
+ * device attributes are already cached or `x_align`/`y_align` rule the fast paths out).
+ *   x_align, y_align  the largest power of two (<= 16 is enough) dividing each base address.
+ * Returns an fs_kernel (>= 1), or a negative fs_status on invalid arguments.
+ */
+int fs_select_kernel(int64_t rows, int64_t cols, int dtype, int x_align, int y_align);
+
+/*
+ * fs_softmax_host -- the same operation on HOST buffers, end to end.
+ *   x_host, y_host  host pointers (pinned memory gives full copy bandwidth; pageable works).
+ * Splits the rows into chunks and pipelines host->device copy, kernel and device->host copy on
+ * internal streams through device staging buffers the library allocates on first use and keeps
+ * (grown on demand, released by fs_release). Blocks until y_host is complete.
+ */
+int fs_softmax_host(const void* x_host, void* y_host, int64_t rows, int64_t cols, int dtype, float scale);
+
+/*
+ * fs_copy -- speed-of-light calibration: copies `bytes` bytes from x to y (device pointers, both
+ * 16-byte aligned, bytes a multiple of 16) with the same 128-bit streaming accesses and grid
+ * sizing as the softmax kernels. Same traffic as a softmax over the same buffers, no arithmetic.
+ */
+int fs_copy(const void* x, void* y, int64_t bytes, void* stream);
+
+/*
+ * fs_device_status -- reads and clears the device-side status word of the current device
+ * (synchronises the device). FS_OK, or FS_ERR_DEVICE_TIMEOUT if a bounded wait on an async copy
+ * expired inside a kernel since the last call (the outputs of that launch are then undefined).
+ */
+int fs_device_status(void);
+
+/* fs_release -- frees the staging buffers and streams fs_softmax_host created on the current device. */
+int fs_release(void);
+
+/* The cudaError_t behind the last FS_ERR_CUDA returned on this thread (0 if none). */
+int fs_last_cuda_error(void);
+
+/* Static strings. */
+const char* fs_strerror(int status);
+const char* fs_kernel_name(int kernel);
+const char* fs_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FSOFTMAX_H_ */

@@ -1,0 +1,147 @@
+"""Thin ctypes binding of libfsoftmax's C ABI (see include/fsoftmax.h).
+
+Argument marshalling only: every step of the softmax runs in the CUDA library. Functions carry
+the C entry points' names. Device buffers may be given as torch CUDA tensors (their ``data_ptr``
+is passed) or as raw integer addresses; host buffers as numpy arrays or torch CPU tensors.
+There is no fallback: if the shared library is missing, or no CUDA device is usable, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import threading
+
+FS_DTYPE_FP32, FS_DTYPE_BF16, FS_DTYPE_FP16 = 0, 1, 2
+FS_OK, FS_ERR_INVALID_ARG, FS_ERR_UNSUPPORTED, FS_ERR_CUDA, FS_ERR_DEVICE_TIMEOUT = 0, 1, 2, 3, 4
+FS_KERNEL_AUTO, FS_KERNEL_WARP, FS_KERNEL_BLOCK, FS_KERNEL_BLOCK_TMA, FS_KERNEL_CLUSTER, FS_KERNEL_GENERIC = range(6)
+KERNELS = {"auto": 0, "warp": 1, "block": 2, "block_tma": 3, "cluster": 4, "generic": 5}
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libfsoftmax.so")
+_lock = threading.Lock()
+_lib = None
+
+
+class FsError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().fs_strerror(status).decode()
+        if status == FS_ERR_CUDA:
+            msg += f" [cudaError {lib().fs_last_cuda_error()}]"
+        super().__init__(f"{where}: {msg} (status {status})")
+
+
+def lib() -> ctypes.CDLL:
+    """Load libfsoftmax.so (built in-tree by ``_build.build_library``). Raises if it is missing."""
+    global _lib
+    with _lock:
+        if _lib is None:
+            if not os.path.exists(LIB_PATH):
+                raise RuntimeError(
+                    f"{LIB_PATH} is missing: build it with "
+                    "`python -c 'import __graft_entry__ as g; g.build()'` (needs nvcc). "
+                    "There is no CPU or PyTorch fallback.")
+            L = ctypes.CDLL(LIB_PATH)
+            vp, i64, ci, f32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_float
+            L.fs_softmax.argtypes = [vp, vp, i64, i64, ci, f32, vp]
+            L.fs_softmax.restype = ci
+            L.fs_softmax_ex.argtypes = [vp, vp, i64, i64, ci, f32, vp, ci, ci, ci]
+            L.fs_softmax_ex.restype = ci
+            L.fs_select_kernel.argtypes = [i64, i64, ci, ci, ci]
+            L.fs_select_kernel.restype = ci
+            L.fs_softmax_host.argtypes = [vp, vp, i64, i64, ci, f32]
+            L.fs_softmax_host.restype = ci
+            L.fs_copy.argtypes = [vp, vp, i64, vp]
+            L.fs_copy.restype = ci
+            L.fs_device_status.argtypes = []
+            L.fs_device_status.restype = ci
+            L.fs_release.argtypes = []
+            L.fs_release.restype = ci
+            L.fs_last_cuda_error.argtypes = []
+            L.fs_last_cuda_error.restype = ci
+            L.fs_strerror.argtypes = [ci]
+            L.fs_strerror.restype = ctypes.c_char_p
+            L.fs_kernel_name.argtypes = [ci]
+            L.fs_kernel_name.restype = ctypes.c_char_p
+            L.fs_version.argtypes = []
+            L.fs_version.restype = ctypes.c_char_p
+            _lib = L
+    return _lib
+
+
+def _ptr(buf) -> int:
+    if buf is None:
+        return 0
+    if isinstance(buf, int):
+        return buf
+    if hasattr(buf, "data_ptr"):
+        return int(buf.data_ptr())
+    if hasattr(buf, "ctypes"):
+        return int(buf.ctypes.data)
+    raise TypeError(f"cannot take the address of {type(buf)!r}")
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return 0
+    if isinstance(stream, int):
+        return stream
+    return int(stream.cuda_stream)          # torch.cuda.Stream
+
+
+def _check(status: int, where: str) -> None:
+    if status != FS_OK:
+        raise FsError(status, where)
+
+
+def fs_softmax(x, y, rows: int, cols: int, dtype: int, scale: float = 1.0, stream=None) -> None:
+    """y = softmax(scale * x) over the last dimension of a [rows, cols] device tensor."""
+    _check(lib().fs_softmax(_ptr(x), _ptr(y), rows, cols, dtype, scale, _stream(stream)), "fs_softmax")
+
+
+def fs_softmax_ex(x, y, rows: int, cols: int, dtype: int, scale: float = 1.0, stream=None,
+                  kernel: int = FS_KERNEL_AUTO, threads: int = 0, cluster: int = 0) -> None:
+    _check(lib().fs_softmax_ex(_ptr(x), _ptr(y), rows, cols, dtype, scale, _stream(stream), kernel, threads, cluster),
+           "fs_softmax_ex")
+
+
+def fs_softmax_status(x, y, rows, cols, dtype, scale=1.0, stream=None, kernel=FS_KERNEL_AUTO, threads=0,
+                      cluster=0) -> int:
+    """fs_softmax_ex returning the raw status instead of raising (for error-path tests)."""
+    return lib().fs_softmax_ex(_ptr(x), _ptr(y), rows, cols, dtype, scale, _stream(stream), kernel, threads, cluster)
+
+
+def fs_select_kernel(rows: int, cols: int, dtype: int, x_align: int = 16, y_align: int = 16) -> int:
+    return lib().fs_select_kernel(rows, cols, dtype, x_align, y_align)
+
+
+def fs_softmax_host(x_host, y_host, rows: int, cols: int, dtype: int, scale: float = 1.0) -> None:
+    _check(lib().fs_softmax_host(_ptr(x_host), _ptr(y_host), rows, cols, dtype, scale), "fs_softmax_host")
+
+
+def fs_copy(x, y, nbytes: int, stream=None) -> None:
+    _check(lib().fs_copy(_ptr(x), _ptr(y), nbytes, _stream(stream)), "fs_copy")
+
+
+def fs_device_status() -> int:
+    return lib().fs_device_status()
+
+
+def fs_release() -> None:
+    _check(lib().fs_release(), "fs_release")
+
+
+def fs_last_cuda_error() -> int:
+    return lib().fs_last_cuda_error()
+
+
+def fs_strerror(status: int) -> str:
+    return lib().fs_strerror(status).decode()
+
+
+def fs_kernel_name(kernel: int) -> str:
+    return lib().fs_kernel_name(kernel).decode()
+
+
+def fs_version() -> str:
+    return lib().fs_version().decode()

@@ -1,0 +1,312 @@
+// Block-per-row and cluster-per-row softmax kernels. One pass over the data: every thread keeps
+// its share of the row in registers as 2^((x - r_t) c) against its OWN reference r_t (the max of
+// its elements), so each element costs one ex2; the (r, s) partial pairs are then merged with the
+// online-softmax rule (Milakov-Gimelshein)
+//     (r, s) (+) (r', s') = (R = max(r, r'),  s 2^((r-R)c) + s' 2^((r'-R)c))
+// across the warp (shuffles), the block (shared memory, one __syncthreads per row) and, for the
+// split-row kernel, the thread-block cluster (distributed shared memory, one cluster barrier per
+// row). The output is e * 2^((r_t - R)c) / S.
+//
+// Three front ends share that arithmetic:
+//   block_row_kernel      128-bit global loads straight into registers
+//   block_row_tma_kernel  rows prefetched into a shared-memory ring by cp.async.bulk (no multicast),
+//                         completion tracked per stage by an mbarrier
+//   cluster_row_kernel    a row split over the blocks of a cluster, each block prefetching its
+//                         own slice like block_row_tma_kernel
+#pragma once
+#include "common.cuh"
+
+namespace fsm {
+
+// Threads per block the register budget allows for a payload of VPT*VE floats per thread.
+template <int DT, int VPT> struct BlockCfg {
+    static constexpr int PAYLOAD = VPT * Traits<DT>::VE;
+    static constexpr int MAX_THREADS = PAYLOAD <= 16 ? 1024 : 512;
+};
+
+// Per-thread part: e[k][i] = 2^((x - r_use) c), r = own reference, s = sum of e.
+// valid(k) says whether this thread's k-th vector exists.
+template <int DT, int VPT, typename Valid>
+__device__ __forceinline__ void thread_partial(const uint4 (&raw)[VPT], float (&e)[VPT][Traits<DT>::VE],
+                                               float& r, float& s, const Params& p, float ident, Valid valid) {
+    constexpr int VE = Traits<DT>::VE;
+    r = ident;
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+        unpack<DT>(raw[k], e[k]);
+        if (valid(k)) {
+#pragma unroll
+            for (int i = 0; i < VE; ++i) r = ref_pick(r, e[k][i], p.neg);
+        }
+    }
+    // A thread whose elements are all masked (or that has none) subtracts 0 instead of the identity.
+    const float r_use = (r == ident) ? 0.0f : r;
+    s = 0.0f;
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+        if (valid(k)) {
+#pragma unroll
+            for (int i = 0; i < VE; ++i) {
+                e[k][i] = ex2<DT>((e[k][i] - r_use) * p.c);
+                s += e[k][i];
+            }
+        }
+    }
+}
+
+// Block-wide merge of (r, s). `wp` points at 32 float2 slots; the caller alternates between two
+// such arrays from row to row so that one __syncthreads per row is enough.
+__device__ __forceinline__ void block_merge_pairs(float& r, float& s, float2* wp, float c, int neg, float ident) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    warp_merge_pairs(r, s, c, neg, ident);
+    if (nwarps == 1) return;
+    if (lane == 0) wp[warp] = make_float2(r, s);
+    __syncthreads();
+    const float2 v = (lane < nwarps) ? wp[lane] : make_float2(ident, 0.0f);
+    r = v.x; s = v.y;
+    warp_merge_pairs(r, s, c, neg, ident);
+}
+
+template <int DT, int VPT, typename Valid, typename VecIndex>
+__device__ __forceinline__ void scale_and_store(float (&e)[VPT][Traits<DT>::VE], float r_t, float R, float S,
+                                                const Params& p, float ident, uint4* yrow, Valid valid, VecIndex vec) {
+    constexpr int VE = Traits<DT>::VE;
+    const float f = ref_factor(r_t, R, p.c, ident) * (1.0f / S);
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+        if (valid(k)) {
+#pragma unroll
+            for (int i = 0; i < VE; ++i) e[k][i] *= f;
+            st_stream(yrow + vec(k), pack<DT>(e[k]));
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// block per row, direct global loads
+// ---------------------------------------------------------------------------------------------
+template <int DT, int VPT>
+__global__ void __launch_bounds__(BlockCfg<DT, VPT>::MAX_THREADS, 1)
+block_row_kernel(const Params p) {
+    constexpr int VE = Traits<DT>::VE;
+    __shared__ float2 wp[2][32];
+    const int T = blockDim.x, tid = threadIdx.x;
+    const int nvec = static_cast<int>(p.nvec);
+    const float ident = ref_identity(p.neg);
+    const uint4* __restrict__ xv = static_cast<const uint4*>(p.x);
+    uint4* __restrict__ yv = static_cast<uint4*>(p.y);
+    auto valid = [&](int k) { return tid + k * T < nvec; };
+    auto vec = [&](int k) { return tid + k * T; };
+    int par = 0;
+    for (int64_t row = blockIdx.x; row < p.rows; row += gridDim.x, par ^= 1) {
+        uint4 raw[VPT];
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            raw[k] = make_uint4(0u, 0u, 0u, 0u);
+            if (valid(k)) raw[k] = ld_stream(xv + row * p.nvec + vec(k));
+        }
+        float e[VPT][VE], r_t, s;
+        thread_partial<DT, VPT>(raw, e, r_t, s, p, ident, valid);
+        float R = r_t;
+        block_merge_pairs(R, s, wp[par], p.c, p.neg, ident);
+        scale_and_store<DT, VPT>(e, r_t, R, s, p, ident, yv + row * p.nvec, valid, vec);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// block per row, rows staged in a shared-memory ring by bulk async copies
+// dynamic shared memory: [nstage][stage_bytes] row buffers | nstage mbarriers (8 B each)
+// ---------------------------------------------------------------------------------------------
+template <int DT, int VPT>
+__global__ void __launch_bounds__(BlockCfg<DT, VPT>::MAX_THREADS, 1)
+block_row_tma_kernel(const Params p, const int nstage, const uint32_t stage_bytes) {
+    constexpr int VE = Traits<DT>::VE;
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ float2 wp[2][32];
+    const int T = blockDim.x, tid = threadIdx.x;
+    const int nvec = static_cast<int>(p.nvec);
+    const uint32_t row_bytes = static_cast<uint32_t>(p.nvec) * 16u;
+    const float ident = ref_identity(p.neg);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + size_t(nstage) * stage_bytes);
+    const char* xb = static_cast<const char*>(p.x);
+    uint4* __restrict__ yv = static_cast<uint4*>(p.y);
+    auto valid = [&](int k) { return tid + k * T < nvec; };
+    auto vec = [&](int k) { return tid + k * T; };
+
+    const int64_t first = blockIdx.x;
+    const int64_t n_my = first < p.rows ? (p.rows - first + gridDim.x - 1) / gridDim.x : 0;
+    if (tid == 0) {
+        for (int s = 0; s < nstage; ++s) mbar_init(smem_u32(&bars[s]), 1);
+        mbar_fence_init();
+        fence_proxy_async_smem();
+        for (int s = 0; s < nstage && s < n_my; ++s)
+            bulk_load_row(smem_u32(smem + size_t(s) * stage_bytes),
+                          xb + (first + int64_t(s) * gridDim.x) * row_bytes, row_bytes, smem_u32(&bars[s]));
+    }
+    __syncthreads();
+
+    int stage = 0;
+    uint32_t phase = 0;
+    bool alive = true;      // false once a bounded wait has expired: later waits are skipped
+    for (int64_t i = 0; i < n_my; ++i) {
+        const int64_t row = first + i * gridDim.x;
+        if (alive) alive = mbar_wait(smem_u32(&bars[stage]), phase, p.status);
+        const uint4* srow = reinterpret_cast<const uint4*>(smem + size_t(stage) * stage_bytes);
+        uint4 raw[VPT];
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            raw[k] = make_uint4(0u, 0u, 0u, 0u);
+            if (valid(k)) raw[k] = srow[vec(k)];
+        }
+        float e[VPT][VE], r_t, s;
+        thread_partial<DT, VPT>(raw, e, r_t, s, p, ident, valid);
+        float R = r_t;
+        // one warp: no __syncthreads inside the merge, so order the stage reads explicitly
+        if (T == 32) __syncwarp();
+        block_merge_pairs(R, s, wp[i & 1], p.c, p.neg, ident);
+        // every thread has read its part of this stage (the merge's barrier): refill it
+        if (tid == 0 && i + nstage < n_my) {
+            fence_proxy_async_smem();
+            bulk_load_row(smem_u32(smem + size_t(stage) * stage_bytes),
+                          xb + (row + int64_t(nstage) * gridDim.x) * row_bytes, row_bytes, smem_u32(&bars[stage]));
+        }
+        scale_and_store<DT, VPT>(e, r_t, R, s, p, ident, yv + row * p.nvec, valid, vec);
+        if (++stage == nstage) { stage = 0; phase ^= 1u; }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// cluster per row: block q of the cluster owns vectors [q*slice, min((q+1)*slice, nvec)) of the row
+// dynamic shared memory: [nstage][stage_bytes] slice buffers | nstage mbarriers
+// static shared memory : warp pairs, and xchg[2][16] where peers deposit their block's pair
+// ---------------------------------------------------------------------------------------------
+template <int DT, int VPT>
+__global__ void __launch_bounds__(BlockCfg<DT, VPT>::MAX_THREADS, 1)
+cluster_row_kernel(const Params p, const int nstage, const uint32_t stage_bytes, const int slice) {
+    constexpr int VE = Traits<DT>::VE;
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ float2 wp[2][32];
+    __shared__ __align__(16) float2 xchg[2][16];
+    const int T = blockDim.x, tid = threadIdx.x, lane = tid & 31;
+    const uint32_t q = cluster_ctarank(), cs = cluster_nctarank();
+    const int64_t ncl = cluster_count_x();             // clusters in the grid
+    const int64_t cid = cluster_id_x();
+    const int nvec = static_cast<int>(p.nvec);
+    const int v0 = min(nvec, static_cast<int>(q) * slice);
+    const int nv = min(nvec, v0 + slice) - v0;         // vectors of this block's slice (may be 0)
+    const uint32_t my_bytes = static_cast<uint32_t>(nv) * 16u;
+    const float ident = ref_identity(p.neg);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + size_t(nstage) * stage_bytes);
+    const char* xb = static_cast<const char*>(p.x);
+    uint4* __restrict__ yv = static_cast<uint4*>(p.y);
+    auto valid = [&](int k) { return tid + k * T < nv; };
+    auto vec = [&](int k) { return v0 + tid + k * T; };
+
+    const int64_t n_my = cid < p.rows ? (p.rows - cid + ncl - 1) / ncl : 0;   // same for the whole cluster
+    const int64_t row_bytes = p.nvec * 16;
+    if (tid == 0) {
+        for (int s = 0; s < nstage; ++s) mbar_init(smem_u32(&bars[s]), 1);
+        mbar_fence_init();
+        fence_proxy_async_smem();
+        if (nv > 0)
+            for (int s = 0; s < nstage && s < n_my; ++s)
+                bulk_load_row(smem_u32(smem + size_t(s) * stage_bytes),
+                              xb + (cid + int64_t(s) * ncl) * row_bytes + int64_t(v0) * 16, my_bytes, smem_u32(&bars[s]));
+    }
+    __syncthreads();
+    // every block of the cluster is resident before anyone writes into a peer's shared memory
+    cluster_arrive_release();
+    cluster_wait_acquire();
+
+    int stage = 0;
+    uint32_t phase = 0;
+    bool alive = true;      // false once a bounded wait has expired: later waits are skipped
+    for (int64_t i = 0; i < n_my; ++i) {
+        const int64_t row = cid + i * ncl;
+        const int par = static_cast<int>(i & 1);
+        uint4 raw[VPT];
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) raw[k] = make_uint4(0u, 0u, 0u, 0u);
+        if (nv > 0) {
+            if (alive) alive = mbar_wait(smem_u32(&bars[stage]), phase, p.status);
+            const uint4* srow = reinterpret_cast<const uint4*>(smem + size_t(stage) * stage_bytes);
+#pragma unroll
+            for (int k = 0; k < VPT; ++k)
+                if (valid(k)) raw[k] = srow[tid + k * T];
+        }
+        float e[VPT][VE], r_t, s;
+        thread_partial<DT, VPT>(raw, e, r_t, s, p, ident, valid);
+        float R = r_t;
+        if (T == 32) __syncwarp();
+        block_merge_pairs(R, s, wp[par], p.c, p.neg, ident);
+        if (tid == 0 && nv > 0 && i + nstage < n_my) {
+            fence_proxy_async_smem();
+            bulk_load_row(smem_u32(smem + size_t(stage) * stage_bytes),
+                          xb + (row + int64_t(nstage) * ncl) * row_bytes + int64_t(v0) * 16, my_bytes, smem_u32(&bars[stage]));
+        }
+        // deposit this block's pair in slot q of every block of the cluster (this one included)
+        if (tid < cs) st_cluster_v2(map_to_rank(smem_u32(&xchg[par][q]), tid), R, s);
+        __syncwarp();
+        cluster_arrive_release();
+        cluster_wait_acquire();
+        R = ident; s = 0.0f;
+        if (lane < static_cast<int>(cs)) ld_shared_v2(smem_u32(&xchg[par][lane]), R, s);
+        warp_merge_pairs(R, s, p.c, p.neg, ident);
+        scale_and_store<DT, VPT>(e, r_t, R, s, p, ident, yv + row * p.nvec, valid, vec);
+        if (++stage == nstage) { stage = 0; phase ^= 1u; }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// generic: any cols, any alignment, element-wise accesses; reads the row twice (the second read
+// normally hits L2). Pass 1 keeps a running (r, s) per thread -- the online update itself.
+// ---------------------------------------------------------------------------------------------
+template <int DT>
+__global__ void __launch_bounds__(1024, 1)
+generic_row_kernel(const Params p) {
+    __shared__ float2 wp[2][32];
+    const int T = blockDim.x, tid = threadIdx.x;
+    const float ident = ref_identity(p.neg);
+    int par = 0;
+    for (int64_t row = blockIdx.x; row < p.rows; row += gridDim.x, par ^= 1) {
+        const int64_t base = row * p.cols;
+        float r = ident, s = 0.0f;
+        for (int64_t j = tid; j < p.cols; j += T) {
+            const float x = load_elem<DT>(p.x, base + j);
+            const float rn = ref_pick(r, x, p.neg);
+            const float ru = (rn == ident) ? 0.0f : rn;
+            s = s * ref_factor(r, rn, p.c, ident) + ex2_noflush((x - ru) * p.c);
+            r = rn;
+        }
+        block_merge_pairs(r, s, wp[par], p.c, p.neg, ident);
+        const float ru = (r == ident) ? 0.0f : r;
+        const float inv = 1.0f / s;
+        for (int64_t j = tid; j < p.cols; j += T) {
+            const float x = load_elem<DT>(p.x, base + j);
+            store_elem<DT>(p.y, base + j, ex2_noflush((x - ru) * p.c) * inv);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// speed-of-light calibration: 16-byte streaming copy, one block per 1024 consecutive vectors
+// (four independent loads in flight per thread), blocks handed out by the hardware scheduler
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+copy_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, const int64_t nvec) {
+    for (int64_t base = int64_t(blockIdx.x) * 1024; base < nvec; base += int64_t(gridDim.x) * 1024) {
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int64_t i = base + u * 256 + threadIdx.x;
+            if (i < nvec) v[u] = ld_stream(x + i);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int64_t i = base + u * 256 + threadIdx.x;
+            if (i < nvec) st_stream(y + i, v[u]);
+        }
+    }
+}
+
+}  // namespace fsm

@@ -1,0 +1,253 @@
+// Shared device helpers for the softmax kernels: 128-bit vector access, dtype unpack/pack,
+// base-2 exponential, (reference, sum) pair algebra, warp reductions, mbarrier + bulk-copy PTX.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace fsm {
+
+enum : int { DT_F32 = 0, DT_BF16 = 1, DT_F16 = 2 };
+
+// Status bits a kernel may OR into the per-device status word.
+enum : int { DEV_TIMEOUT = 1 };
+
+struct Params {
+    const void* x;
+    void* y;
+    int64_t rows;
+    int64_t cols;
+    int64_t nvec;      // 16-byte vectors per row (fast kernels: cols * elem_size / 16)
+    float c;           // scale * log2(e): exponents are taken in base 2
+    int neg;           // c < 0: the row reference is the minimum of x instead of the maximum
+    int* status;       // device status word
+};
+
+template <int DT> struct Traits;
+template <> struct Traits<DT_F32>  { static constexpr int VE = 4; static constexpr int ESZ = 4; };
+template <> struct Traits<DT_BF16> { static constexpr int VE = 8; static constexpr int ESZ = 2; };
+template <> struct Traits<DT_F16>  { static constexpr int VE = 8; static constexpr int ESZ = 2; };
+
+// ---- 128-bit streaming global access (every byte is touched once: evict-first) -------------
+
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};"
+                 :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+
+// ---- dtype unpack / pack of one 16-byte vector ------------------------------------------------
+
+template <int DT>
+__device__ __forceinline__ void unpack(const uint4& v, float (&f)[Traits<DT>::VE]) {
+    if constexpr (DT == DT_F32) {
+        f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
+        f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+    } else if constexpr (DT == DT_BF16) {
+        // bfloat16 is the high half of a binary32 pattern
+        f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);
+        f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xffff0000u);
+        f[4] = __uint_as_float(v.z << 16); f[5] = __uint_as_float(v.z & 0xffff0000u);
+        f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xffff0000u);
+    } else {
+        const __half2* h = reinterpret_cast<const __half2*>(&v);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 t = __half22float2(h[i]);
+            f[2 * i] = t.x; f[2 * i + 1] = t.y;
+        }
+    }
+}
+
+// Round-to-nearest-even to the stored dtype.
+template <int DT>
+__device__ __forceinline__ uint4 pack(const float (&f)[Traits<DT>::VE]) {
+    uint4 v;
+    if constexpr (DT == DT_F32) {
+        v.x = __float_as_uint(f[0]); v.y = __float_as_uint(f[1]);
+        v.z = __float_as_uint(f[2]); v.w = __float_as_uint(f[3]);
+    } else if constexpr (DT == DT_BF16) {
+        __nv_bfloat162 a = __floats2bfloat162_rn(f[0], f[1]);
+        __nv_bfloat162 b = __floats2bfloat162_rn(f[2], f[3]);
+        __nv_bfloat162 c = __floats2bfloat162_rn(f[4], f[5]);
+        __nv_bfloat162 d = __floats2bfloat162_rn(f[6], f[7]);
+        v.x = *reinterpret_cast<uint32_t*>(&a); v.y = *reinterpret_cast<uint32_t*>(&b);
+        v.z = *reinterpret_cast<uint32_t*>(&c); v.w = *reinterpret_cast<uint32_t*>(&d);
+    } else {
+        __half2 a = __floats2half2_rn(f[0], f[1]);
+        __half2 b = __floats2half2_rn(f[2], f[3]);
+        __half2 c = __floats2half2_rn(f[4], f[5]);
+        __half2 d = __floats2half2_rn(f[6], f[7]);
+        v.x = *reinterpret_cast<uint32_t*>(&a); v.y = *reinterpret_cast<uint32_t*>(&b);
+        v.z = *reinterpret_cast<uint32_t*>(&c); v.w = *reinterpret_cast<uint32_t*>(&d);
+    }
+    return v;
+}
+
+template <int DT> __device__ __forceinline__ float load_elem(const void* p, int64_t i) {
+    if constexpr (DT == DT_F32) return static_cast<const float*>(p)[i];
+    else if constexpr (DT == DT_BF16) return __bfloat162float(static_cast<const __nv_bfloat16*>(p)[i]);
+    else return __half2float(static_cast<const __half*>(p)[i]);
+}
+
+template <int DT> __device__ __forceinline__ void store_elem(void* p, int64_t i, float v) {
+    if constexpr (DT == DT_F32) static_cast<float*>(p)[i] = v;
+    else if constexpr (DT == DT_BF16) static_cast<__nv_bfloat16*>(p)[i] = __float2bfloat16_rn(v);
+    else static_cast<__half*>(p)[i] = __float2half_rn(v);
+}
+
+// ---- base-2 exponential on the special-function unit ---------------------------------------
+// bfloat16 shares binary32's exponent range, so a result below 2^-126 is still a representable
+// (subnormal) bf16 value and must not be flushed: bf16 uses the non-flushing form. fp32 results are
+// judged on absolute error and fp16's subnormals are normal binary32 numbers, so they flush.
+template <int DT>
+__device__ __forceinline__ float ex2(float t) {
+    float r;
+    if constexpr (DT == DT_BF16) asm("ex2.approx.f32 %0, %1;" : "=f"(r) : "f"(t));
+    else                         asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(t));
+    return r;
+}
+
+__device__ __forceinline__ float ex2_noflush(float t) {
+    float r;
+    asm("ex2.approx.f32 %0, %1;" : "=f"(r) : "f"(t));
+    return r;
+}
+
+// ---- row reference (max of x, or min when the scale is negative) ----------------------------
+
+__device__ __forceinline__ float ref_identity(int neg) { return neg ? __int_as_float(0x7f800000) : __int_as_float(0xff800000); }
+__device__ __forceinline__ float ref_pick(float a, float b, int neg) { return neg ? fminf(a, b) : fmaxf(a, b); }
+
+// Factor that moves a partial sum taken against reference `r` to the reference `R`
+// (R = pick(r, ...)). A partial whose reference is still the identity has sum 0 (or NaN) and keeps
+// it: returning 1 avoids inf - inf and 0 * inf for rows that are partly or wholly masked.
+__device__ __forceinline__ float ref_factor(float r, float R, float c, float ident) {
+    return (r == R || r == ident) ? 1.0f : ex2_noflush((r - R) * c);
+}
+
+template <int WIDTH>
+__device__ __forceinline__ float warp_pick(float v, int neg) {
+#pragma unroll
+    for (int o = WIDTH / 2; o > 0; o >>= 1) v = ref_pick(v, __shfl_xor_sync(0xffffffffu, v, o), neg);
+    return v;
+}
+
+template <int WIDTH>
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = WIDTH / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Merge (r, s) pairs across the 32 lanes of a warp:
+//   R = pick_l r_l,  S = sum_l s_l * 2^((r_l - R) c)      (online-softmax merge, Milakov-Gimelshein)
+__device__ __forceinline__ void warp_merge_pairs(float& r, float& s, float c, int neg, float ident) {
+    const float R = warp_pick<32>(r, neg);
+    s = warp_sum<32>(s * ref_factor(r, R, c, ident));
+    r = R;
+}
+
+// ---- shared-memory addresses, mbarrier, bulk async copy (non-multicast) ---------------------
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void mbar_fence_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+
+__device__ __forceinline__ void fence_proxy_async_smem() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
+}
+
+// Global -> this block's shared memory, completion counted in bytes on `bar`.
+// dst, src and bytes must be multiples of 16.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+// Arms `bar` for `bytes` and issues the copy in pieces of at most 32 KiB. The expected byte count
+// and the copied byte count come from the same loop.
+__device__ __forceinline__ void bulk_load_row(uint32_t dst, const char* src, uint32_t bytes, uint32_t bar) {
+    mbar_expect_tx(bar, bytes);
+    for (uint32_t off = 0; off < bytes; off += 32768u) {
+        const uint32_t n = min(32768u, bytes - off);
+        bulk_load(dst + off, src + off, n, bar);
+    }
+}
+
+// Bounded wait on an mbarrier phase: at most 2^20 polls, each suspending for up to ~1 us, i.e.
+// about a second. Returns false (and records DEV_TIMEOUT) if the phase did not complete; the
+// caller carries on, skipping further waits, so that every block-wide and cluster-wide barrier is
+// still reached and the kernel ends.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status) {
+    for (int it = 0; it < (1 << 20); ++it) {
+        uint32_t done;
+        asm volatile("{\n\t.reg .pred p;\n\t"
+                     "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+                     "selp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(bar), "r"(parity), "r"(1000u) : "memory");
+        if (done) return true;
+    }
+    atomicOr(status, DEV_TIMEOUT);
+    return false;
+}
+
+// ---- thread-block cluster ------------------------------------------------------------------
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r;
+}
+__device__ __forceinline__ uint32_t cluster_nctarank() {
+    uint32_t r; asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r)); return r;
+}
+__device__ __forceinline__ uint32_t cluster_id_x() {
+    uint32_t r; asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(r)); return r;
+}
+__device__ __forceinline__ uint32_t cluster_count_x() {
+    uint32_t r; asm volatile("mov.u32 %0, %%nclusterid.x;" : "=r"(r)); return r;
+}
+// Address of `local_addr` (a shared::cta address of this block) in block `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t local_addr, uint32_t rank) {
+    uint32_t a; asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"(local_addr), "r"(rank)); return a;
+}
+__device__ __forceinline__ void st_cluster_v2(uint32_t addr, float a, float b) {
+    asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" :: "r"(addr), "f"(a), "f"(b) : "memory");
+}
+__device__ __forceinline__ void ld_shared_v2(uint32_t addr, float& a, float& b) {
+    asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(a), "=f"(b) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void cluster_arrive_release() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait_acquire() {
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+}  // namespace fsm

@@ -1,0 +1,140 @@
+"""Host-side checks that need no GPU: the shared library loads and exports every symbol the header
+declares, argument validation answers before any CUDA call, the dispatcher's table, and the loud
+failure when no device is usable. No compute happens here."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import paper_2607_24762_b200 as fs
+from paper_2607_24762_b200 import _build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "fsoftmax.h")
+
+
+@pytest.fixture(scope="module")
+def lib():
+    _build.build_library()
+    return fs.binding.lib()
+
+
+def declared_functions():
+    text = open(HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(fs_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_header_declares_the_boundary():
+    names = declared_functions()
+    for must in ("fs_softmax", "fs_softmax_ex", "fs_select_kernel", "fs_softmax_host", "fs_copy",
+                 "fs_device_status", "fs_release", "fs_last_cuda_error", "fs_strerror", "fs_kernel_name",
+                 "fs_version"):
+        assert must in names
+
+
+def test_library_exports_every_declared_symbol(lib):
+    raw = ctypes.CDLL(fs.binding.LIB_PATH)
+    for name in declared_functions():
+        assert hasattr(raw, name), f"{name} declared in fsoftmax.h but not exported"
+    assert "sm_100a" in fs.fs_version()
+
+
+def test_binding_mirrors_the_header():
+    for name in declared_functions():
+        assert hasattr(fs, name), f"binding lacks {name}"
+
+
+def test_enums_match_header():
+    text = open(HEADER).read()
+    for name, value in re.findall(r"(FS_[A-Z0-9_]+)\s*=\s*(\d+)", text):
+        assert getattr(fs, name) == int(value), name
+
+
+def test_strings(lib):
+    assert fs.fs_strerror(fs.FS_OK) == "ok"
+    assert "invalid" in fs.fs_strerror(fs.FS_ERR_INVALID_ARG)
+    assert [fs.fs_kernel_name(k) for k in range(6)] == ["auto", "warp", "block", "block_tma", "cluster", "generic"]
+    assert fs.fs_kernel_name(99) == "unknown"
+
+
+def test_invalid_arguments_are_rejected_before_any_launch(lib):
+    a, b = 0x10000, 0x20000000         # never dereferenced: validation fails first
+    bad = fs.FS_ERR_INVALID_ARG
+    st = fs.fs_softmax_status
+    assert st(a, b, -1, 8, fs.FS_DTYPE_FP32) == bad
+    assert st(a, b, 8, -1, fs.FS_DTYPE_FP32) == bad
+    assert st(a, b, 8, 8, 3) == bad
+    assert st(a, b, 8, 8, -1) == bad
+    assert st(0, b, 8, 8, fs.FS_DTYPE_FP32) == bad
+    assert st(a, 0, 8, 8, fs.FS_DTYPE_FP32) == bad
+    assert st(a, b, 8, 8, fs.FS_DTYPE_FP32, float("nan")) == bad
+    assert st(a, b, 8, 8, fs.FS_DTYPE_FP32, float("inf")) == bad
+    assert st(a, a + 16, 8, 8, fs.FS_DTYPE_FP32) == bad            # partial overlap
+    assert st(a + 16, a, 8, 8, fs.FS_DTYPE_BF16) == bad
+    assert st(a, b, 8, 8, fs.FS_DTYPE_FP32, 1.0, None, 6) == bad     # unknown kernel
+    assert st(a, b, 8, 8, fs.FS_DTYPE_FP32, 1.0, None, 0, 0, 17) == bad
+    assert st(a, b, 1 << 41, 8, fs.FS_DTYPE_FP32) == bad
+    # empty problems are fine and launch nothing (null pointers allowed)
+    assert st(0, 0, 0, 8, fs.FS_DTYPE_FP32) == fs.FS_OK
+    assert st(0, 0, 8, 0, fs.FS_DTYPE_FP16) == fs.FS_OK
+    with pytest.raises(fs.FsError):
+        fs.fs_softmax(0, b, 8, 8, fs.FS_DTYPE_FP32)
+    assert lib.fs_copy(a, b, 24, None) == bad
+    assert lib.fs_copy(a + 4, b, 32, None) == bad
+    assert lib.fs_copy(0, 0, 0, None) == fs.FS_OK
+
+
+def test_dispatcher_table(lib):
+    k = fs.fs_select_kernel
+    F32, BF16, F16 = fs.FS_DTYPE_FP32, fs.FS_DTYPE_BF16, fs.FS_DTYPE_FP16
+    # the five benchmark workloads
+    assert k(64, 1000, F32) == fs.FS_KERNEL_WARP
+    assert k(16384, 2048, BF16) in (fs.FS_KERNEL_WARP, fs.FS_KERNEL_BLOCK, fs.FS_KERNEL_BLOCK_TMA)
+    assert k(131072, 128, BF16) == fs.FS_KERNEL_WARP
+    assert k(256, 262144, BF16) == fs.FS_KERNEL_CLUSTER
+    assert k(32768, 32768, F32) in (fs.FS_KERNEL_CLUSTER, fs.FS_KERNEL_BLOCK_TMA)
+    # mid-size rows take a block-per-row kernel
+    assert k(100, 8192, F32) in (fs.FS_KERNEL_BLOCK, fs.FS_KERNEL_BLOCK_TMA)
+    assert k(100, 8192, F16) in (fs.FS_KERNEL_BLOCK, fs.FS_KERNEL_BLOCK_TMA)
+    # ragged rows or misaligned bases take the generic kernel
+    assert k(10, 1001, BF16) == fs.FS_KERNEL_GENERIC
+    assert k(10, 1023, F32) == fs.FS_KERNEL_GENERIC
+    assert k(10, 1024, F32, 4, 16) == fs.FS_KERNEL_GENERIC
+    assert k(10, 1024, F32, 16, 8) == fs.FS_KERNEL_GENERIC
+    # rows beyond what a 16-block cluster holds in registers fall back too
+    assert k(2, 1 << 22, F32) == fs.FS_KERNEL_GENERIC
+    assert k(-1, 8, F32) < 0 and k(8, 8, 7) < 0 and k(8, 8, F32, 0, 16) < 0
+    # monotone in row size: warp -> block -> cluster -> generic
+    order = {fs.FS_KERNEL_WARP: 0, fs.FS_KERNEL_BLOCK: 1, fs.FS_KERNEL_BLOCK_TMA: 1, fs.FS_KERNEL_CLUSTER: 2,
+             fs.FS_KERNEL_GENERIC: 3}
+    for dt, e in ((F32, 4), (BF16, 2)):
+        last = 0
+        for log in range(2, 24):
+            cur = order[k(4, (1 << log) * 16 // e // 4, dt)]
+            assert cur >= last
+            last = cur
+
+
+def test_no_device_fails_loudly(lib):
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a CUDA device is present")
+    x = np.zeros((4, 8), dtype=np.float32)
+    # a valid-looking call without a GPU must report a CUDA error, never compute on the host
+    assert fs.fs_softmax_status(x.ctypes.data, x.ctypes.data, 4, 8, fs.FS_DTYPE_FP32) == fs.FS_ERR_CUDA
+    assert fs.fs_last_cuda_error() != 0
+    y = np.full_like(x, 7.0)
+    with pytest.raises(fs.FsError):
+        fs.fs_softmax_host(x, y, 4, 8, fs.FS_DTYPE_FP32)
+    assert np.all(y == 7.0)
+
+
+def test_missing_library_raises(monkeypatch, tmp_path):
+    from paper_2607_24762_b200 import binding
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
+        binding.lib()
