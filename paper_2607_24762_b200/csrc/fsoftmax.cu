@@ -7,6 +7,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <mutex>
+#include <type_traits>
 #include <unordered_map>
 
 #include "kernels/block_row.cuh"
@@ -109,16 +110,19 @@ constexpr int64_t kWarpMaxRowBytes = 4096;          // (sub-)warp per row up to 
 constexpr int64_t kBlockMaxRowBytes = 32768;        // block per row up to here, cluster beyond
 constexpr int64_t kClusterSliceBytes = 32768;       // target slice per block of a cluster
 constexpr int kMaxCluster = 16;
+constexpr int64_t kTileBytes = 16384;              // rows per bulk copy of the warp-tile kernel
 
 int64_t warp_capacity_vecs(int dtype) { return 32 * int64_t(max_vpt(dtype)); }
 
 struct WarpGeom { int lanes, vpl, r; };
+// Four vectors per lane where the row allows it (few shuffle steps per element, four loads in
+// flight per lane), more lanes per row as rows grow, then more vectors per lane.
 bool warp_geom(int64_t nvec, int dtype, WarpGeom* g) {
     if (nvec < 1 || nvec > warp_capacity_vecs(dtype)) return false;
-    if (nvec <= 32) { g->lanes = next_pow2(nvec); g->vpl = 1; g->r = 4; return true; }
-    g->lanes = 32;
-    g->vpl = next_pow2((nvec + 31) / 32);
-    g->r = g->vpl == 2 ? 2 : 1;
+    if (nvec <= 2) { g->lanes = 1; g->vpl = static_cast<int>(nvec); g->r = 4 / g->vpl; return true; }
+    g->lanes = std::min(32, next_pow2((nvec + 3) / 4));
+    g->vpl = std::max(4, next_pow2((nvec + g->lanes - 1) / g->lanes));
+    g->r = 1;
     return true;
 }
 
@@ -274,37 +278,55 @@ int launch(const void* fn, int64_t grid, int threads, size_t smem, int cs, cudaS
 
 // ---- kernel tables --------------------------------------------------------------------------
 
-template <int DT> const void* warp_fn(const WarpGeom& g) {
-    if (g.vpl == 1) {
+template <int DT, bool NEG> const void* warp_fn(const WarpGeom& g) {
+    if (g.vpl == 1) return (const void*)warp_row_kernel<DT, NEG, 1, 1, 4>;
+    if (g.vpl == 2) return (const void*)warp_row_kernel<DT, NEG, 1, 2, 2>;
+    if (g.vpl == 4) {
         switch (g.lanes) {
-            case 1:  return (const void*)warp_row_kernel<DT, 1, 1, 4>;
-            case 2:  return (const void*)warp_row_kernel<DT, 2, 1, 4>;
-            case 4:  return (const void*)warp_row_kernel<DT, 4, 1, 4>;
-            case 8:  return (const void*)warp_row_kernel<DT, 8, 1, 4>;
-            case 16: return (const void*)warp_row_kernel<DT, 16, 1, 4>;
-            default: return (const void*)warp_row_kernel<DT, 32, 1, 4>;
+            case 1:  return (const void*)warp_row_kernel<DT, NEG, 1, 4, 1>;
+            case 2:  return (const void*)warp_row_kernel<DT, NEG, 2, 4, 1>;
+            case 4:  return (const void*)warp_row_kernel<DT, NEG, 4, 4, 1>;
+            case 8:  return (const void*)warp_row_kernel<DT, NEG, 8, 4, 1>;
+            case 16: return (const void*)warp_row_kernel<DT, NEG, 16, 4, 1>;
+            default: return (const void*)warp_row_kernel<DT, NEG, 32, 4, 1>;
         }
     }
-    switch (g.vpl) {
-        case 2: return (const void*)warp_row_kernel<DT, 32, 2, 2>;
-        case 4: return (const void*)warp_row_kernel<DT, 32, 4, 1>;
-        case 8: return (const void*)warp_row_kernel<DT, 32, 8, 1>;
-        case 16:
-            if constexpr (DT == DT_F32) return (const void*)warp_row_kernel<DT, 32, 16, 1>;
-            else return nullptr;
+    if (g.vpl == 8) return (const void*)warp_row_kernel<DT, NEG, 32, 8, 1>;
+    if constexpr (DT == DT_F32) {
+        if (g.vpl == 16) return (const void*)warp_row_kernel<DT, NEG, 32, 16, 1>;
+    }
+    return nullptr;
+}
+
+template <int DT, bool NEG> const void* warp_tma_fn(const WarpGeom& g) {
+    if (g.vpl == 1) return (const void*)warp_row_tma_kernel<DT, NEG, 1, 1>;
+    if (g.vpl == 2) return (const void*)warp_row_tma_kernel<DT, NEG, 1, 2>;
+    if (g.vpl == 4) {
+        switch (g.lanes) {
+            case 1:  return (const void*)warp_row_tma_kernel<DT, NEG, 1, 4>;
+            case 2:  return (const void*)warp_row_tma_kernel<DT, NEG, 2, 4>;
+            case 4:  return (const void*)warp_row_tma_kernel<DT, NEG, 4, 4>;
+            case 8:  return (const void*)warp_row_tma_kernel<DT, NEG, 8, 4>;
+            case 16: return (const void*)warp_row_tma_kernel<DT, NEG, 16, 4>;
+            default: return (const void*)warp_row_tma_kernel<DT, NEG, 32, 4>;
+        }
+    }
+    if (g.vpl == 8) return (const void*)warp_row_tma_kernel<DT, NEG, 32, 8>;
+    if constexpr (DT == DT_F32) {
+        if (g.vpl == 16) return (const void*)warp_row_tma_kernel<DT, NEG, 32, 16>;
     }
     return nullptr;
 }
 
 #define FS_VPT_TABLE(NAME, KERNEL)                                                          \
-    template <int DT> const void* NAME(int vpt) {                                           \
+    template <int DT, bool NEG> const void* NAME(int vpt) {                                 \
         switch (vpt) {                                                                      \
-            case 1: return (const void*)KERNEL<DT, 1>;                                      \
-            case 2: return (const void*)KERNEL<DT, 2>;                                      \
-            case 4: return (const void*)KERNEL<DT, 4>;                                      \
-            case 8: return (const void*)KERNEL<DT, 8>;                                      \
+            case 1: return (const void*)KERNEL<DT, NEG, 1>;                                 \
+            case 2: return (const void*)KERNEL<DT, NEG, 2>;                                 \
+            case 4: return (const void*)KERNEL<DT, NEG, 4>;                                 \
+            case 8: return (const void*)KERNEL<DT, NEG, 8>;                                 \
             case 16:                                                                        \
-                if constexpr (DT == DT_F32) return (const void*)KERNEL<DT, 16>;             \
+                if constexpr (DT == DT_F32) return (const void*)KERNEL<DT, NEG, 16>;        \
                 else return nullptr;                                                        \
         }                                                                                   \
         return nullptr;                                                                     \
@@ -313,11 +335,15 @@ FS_VPT_TABLE(block_fn, block_row_kernel)
 FS_VPT_TABLE(block_tma_fn, block_row_tma_kernel)
 FS_VPT_TABLE(cluster_fn, cluster_row_kernel)
 
-template <typename F> const void* by_dtype(int dtype, F f) {
+// Calls f(std::integral_constant<int, DT>, std::bool_constant<NEG>) for the run-time dtype and sign.
+template <typename F> const void* by_variant(int dtype, bool neg, F f) {
+    auto with_dt = [&](auto dt) -> const void* {
+        return neg ? f(dt, std::true_type{}) : f(dt, std::false_type{});
+    };
     switch (dtype) {
-        case FS_DTYPE_FP32: return f(std::integral_constant<int, DT_F32>{});
-        case FS_DTYPE_BF16: return f(std::integral_constant<int, DT_BF16>{});
-        default:            return f(std::integral_constant<int, DT_F16>{});
+        case FS_DTYPE_FP32: return with_dt(std::integral_constant<int, DT_F32>{});
+        case FS_DTYPE_BF16: return with_dt(std::integral_constant<int, DT_BF16>{});
+        default:            return with_dt(std::integral_constant<int, DT_F16>{});
     }
 }
 
@@ -353,7 +379,7 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
         case FS_KERNEL_WARP: {
             WarpGeom g;
             if (!warp_geom(p.nvec, dtype, &g)) return FS_ERR_UNSUPPORTED;
-            const void* fn = by_dtype(dtype, [&](auto dt) { return warp_fn<decltype(dt)::value>(g); });
+            const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) { return warp_fn<decltype(dt)::value, decltype(ng)::value>(g); });
             if (!fn) return FS_ERR_UNSUPPORTED;
             const int t = threads ? threads : 128;
             if (t > 256) return FS_ERR_UNSUPPORTED;
@@ -370,7 +396,7 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
         case FS_KERNEL_BLOCK: {
             BlockGeom g;
             if (!block_geom(p.nvec, dtype, threads, &g)) return FS_ERR_UNSUPPORTED;
-            const void* fn = by_dtype(dtype, [&](auto dt) { return block_fn<decltype(dt)::value>(g.vpt); });
+            const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) { return block_fn<decltype(dt)::value, decltype(ng)::value>(g.vpt); });
             if (!fn) return FS_ERR_UNSUPPORTED;
             int64_t grid = std::min<int64_t>(rows, max_grid);
             if (persistent_grids()) {
@@ -381,13 +407,35 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
             return launch(fn, grid, g.threads, 0, 0, st, p);
         }
         case FS_KERNEL_BLOCK_TMA: {
+            const size_t smem_cap = static_cast<size_t>(dev.smem_optin) - 2048;   // room for the static part
+            WarpGeom wg;
+            if (p.nvec * 16 <= kWarpMaxRowBytes && warp_geom(p.nvec, dtype, &wg)) {
+                // short rows: one bulk copy brings a tile of consecutive rows, each (sub-)warp owns rows
+                const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) { return warp_tma_fn<decltype(dt)::value, decltype(ng)::value>(wg); });
+                if (!fn) return FS_ERR_UNSUPPORTED;
+                const int t = threads ? threads : 128;
+                if (t > 256) return FS_ERR_UNSUPPORTED;
+                const int64_t row_bytes = p.nvec * 16;
+                const int rows_per_pass = (t / 32) * (32 / wg.lanes);
+                int64_t tile_rows = std::max<int64_t>(1, kTileBytes / row_bytes);
+                tile_rows = std::max<int64_t>(rows_per_pass, tile_rows / rows_per_pass * rows_per_pass);
+                tile_rows = std::min<int64_t>(tile_rows, (rows + rows_per_pass - 1) / rows_per_pass * rows_per_pass);
+                const size_t tile_bytes = static_cast<size_t>(tile_rows * row_bytes);
+                if (tile_bytes + 8 > smem_cap || tile_bytes > (size_t(1) << 20) - 16) return FS_ERR_UNSUPPORTED;
+                const size_t smem = tile_bytes + 8;
+                int bps = 0;
+                if ((rc = blocks_per_sm(dev, fn, t, smem, &bps)) != FS_OK) return rc;
+                const int64_t tiles = (rows + tile_rows - 1) / tile_rows;
+                int64_t grid = std::min<int64_t>(tiles, max_grid);
+                if (persistent_grids()) grid = std::min<int64_t>(grid, int64_t(dev.sm_count) * bps);
+                return launch(fn, grid, t, smem, 0, st, p, static_cast<int>(tile_rows), static_cast<uint32_t>(tile_bytes));
+            }
             BlockGeom g;
             if (!block_geom(p.nvec, dtype, threads, &g)) return FS_ERR_UNSUPPORTED;
-            const void* fn = by_dtype(dtype, [&](auto dt) { return block_tma_fn<decltype(dt)::value>(g.vpt); });
+            const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) { return block_tma_fn<decltype(dt)::value, decltype(ng)::value>(g.vpt); });
             if (!fn) return FS_ERR_UNSUPPORTED;
             const size_t stage_bytes = static_cast<size_t>(p.nvec) * 16;
             if (stage_bytes > (size_t(1) << 20) - 16) return FS_ERR_UNSUPPORTED;
-            const size_t smem_cap = static_cast<size_t>(dev.smem_optin) - 2048;   // room for the static part
             int nstage = 1;
             if (persistent_grids()) {
                 // aim at ~2048 resident threads per SM, and give each block its share of shared memory
@@ -408,7 +456,7 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
             if (!dev.cluster_ok) return FS_ERR_UNSUPPORTED;
             ClusterGeom g;
             if (!cluster_geom(p.nvec, dtype, threads, cluster, &g)) return FS_ERR_UNSUPPORTED;
-            const void* fn = by_dtype(dtype, [&](auto dt) { return cluster_fn<decltype(dt)::value>(g.b.vpt); });
+            const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) { return cluster_fn<decltype(dt)::value, decltype(ng)::value>(g.b.vpt); });
             if (!fn) return FS_ERR_UNSUPPORTED;
             const size_t stage_bytes = static_cast<size_t>(g.slice) * 16;
             const size_t smem_cap = static_cast<size_t>(dev.smem_optin) - 2048;
@@ -429,7 +477,7 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
                           static_cast<uint32_t>(stage_bytes), g.slice);
         }
         case FS_KERNEL_GENERIC: {
-            const void* fn = by_dtype(dtype, [&](auto dt) { return (const void*)generic_row_kernel<decltype(dt)::value>; });
+            const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) { return (const void*)generic_row_kernel<decltype(dt)::value, decltype(ng)::value>; });
             int t = threads;
             if (t == 0) {
                 t = 32;

@@ -26,28 +26,26 @@ template <int DT, int VPT> struct BlockCfg {
 
 // Per-thread part: e[k][i] = 2^((x - r_use) c), r = own reference, s = sum of e.
 // valid(k) says whether this thread's k-th vector exists.
-template <int DT, int VPT, typename Valid>
+template <int DT, bool NEG, int VPT, typename Valid>
 __device__ __forceinline__ void thread_partial(const uint4 (&raw)[VPT], float (&e)[VPT][Traits<DT>::VE],
-                                               float& r, float& s, const Params& p, float ident, Valid valid) {
+                                               float& r, float& s, float c, Valid valid) {
     constexpr int VE = Traits<DT>::VE;
-    r = ident;
+    RefAcc<DT, NEG> acc;
+    acc.init();
+#pragma unroll
+    for (int k = 0; k < VPT; ++k)
+        if (valid(k)) acc.fold(raw[k]);
+    r = acc.value();
+    // A thread whose elements are all masked (or that has none) subtracts 0 instead of the identity.
+    const float r_use = (r == ref_identity<NEG>()) ? 0.0f : r;
+    s = 0.0f;
 #pragma unroll
     for (int k = 0; k < VPT; ++k) {
         unpack<DT>(raw[k], e[k]);
         if (valid(k)) {
 #pragma unroll
-            for (int i = 0; i < VE; ++i) r = ref_pick(r, e[k][i], p.neg);
-        }
-    }
-    // A thread whose elements are all masked (or that has none) subtracts 0 instead of the identity.
-    const float r_use = (r == ident) ? 0.0f : r;
-    s = 0.0f;
-#pragma unroll
-    for (int k = 0; k < VPT; ++k) {
-        if (valid(k)) {
-#pragma unroll
             for (int i = 0; i < VE; ++i) {
-                e[k][i] = ex2<DT>((e[k][i] - r_use) * p.c);
+                e[k][i] = ex2_elem<DT>(e[k][i] - r_use, c);
                 s += e[k][i];
             }
         }
@@ -56,28 +54,45 @@ __device__ __forceinline__ void thread_partial(const uint4 (&raw)[VPT], float (&
 
 // Block-wide merge of (r, s). `wp` points at 32 float2 slots; the caller alternates between two
 // such arrays from row to row so that one __syncthreads per row is enough.
-__device__ __forceinline__ void block_merge_pairs(float& r, float& s, float2* wp, float c, int neg, float ident) {
+template <bool NEG>
+__device__ __forceinline__ void block_merge_pairs(float& r, float& s, float2* wp, float c) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    warp_merge_pairs(r, s, c, neg, ident);
+    warp_merge_pairs<NEG>(r, s, c);
     if (nwarps == 1) return;
     if (lane == 0) wp[warp] = make_float2(r, s);
     __syncthreads();
-    const float2 v = (lane < nwarps) ? wp[lane] : make_float2(ident, 0.0f);
+    const float2 v = (lane < nwarps) ? wp[lane] : make_float2(ref_identity<NEG>(), 0.0f);
     r = v.x; s = v.y;
-    warp_merge_pairs(r, s, c, neg, ident);
+    warp_merge_pairs<NEG>(r, s, c);
 }
 
-template <int DT, int VPT, typename Valid, typename VecIndex>
+template <int DT, bool NEG, int VPT, typename Valid, typename VecIndex>
 __device__ __forceinline__ void scale_and_store(float (&e)[VPT][Traits<DT>::VE], float r_t, float R, float S,
-                                                const Params& p, float ident, uint4* yrow, Valid valid, VecIndex vec) {
+                                                float c, uint4* yrow, Valid valid, VecIndex vec) {
     constexpr int VE = Traits<DT>::VE;
-    const float f = ref_factor(r_t, R, p.c, ident) * (1.0f / S);
+    const float fac = ref_factor(r_t, R, c, ref_identity<NEG>());
+    const float inv = recip<DT>(S);
+    if (DT != DT_BF16 || fac >= 0x1p-40f || !(fac == fac)) {
+        const float f = fac * inv;
 #pragma unroll
-    for (int k = 0; k < VPT; ++k) {
-        if (valid(k)) {
+        for (int k = 0; k < VPT; ++k) {
+            if (valid(k)) {
 #pragma unroll
-            for (int i = 0; i < VE; ++i) e[k][i] *= f;
-            st_stream(yrow + vec(k), pack<DT>(e[k]));
+                for (int i = 0; i < VE; ++i) e[k][i] *= f;
+                st_stream(yrow + vec(k), pack<DT>(e[k]));
+            }
+        }
+    } else {
+        // bf16 carries a 2^64 bias in e and 2^-64 in inv: with a thread reference far below the
+        // row's, fac * inv would underflow although e * inv * fac is a representable (subnormal)
+        // bf16 value, so the two factors are applied one after the other.
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            if (valid(k)) {
+#pragma unroll
+                for (int i = 0; i < VE; ++i) e[k][i] = (e[k][i] * inv) * fac;
+                st_stream(yrow + vec(k), pack<DT>(e[k]));
+            }
         }
     }
 }
@@ -85,14 +100,13 @@ __device__ __forceinline__ void scale_and_store(float (&e)[VPT][Traits<DT>::VE],
 // ---------------------------------------------------------------------------------------------
 // block per row, direct global loads
 // ---------------------------------------------------------------------------------------------
-template <int DT, int VPT>
+template <int DT, bool NEG, int VPT>
 __global__ void __launch_bounds__(BlockCfg<DT, VPT>::MAX_THREADS, 1)
 block_row_kernel(const Params p) {
     constexpr int VE = Traits<DT>::VE;
     __shared__ float2 wp[2][32];
     const int T = blockDim.x, tid = threadIdx.x;
     const int nvec = static_cast<int>(p.nvec);
-    const float ident = ref_identity(p.neg);
     const uint4* __restrict__ xv = static_cast<const uint4*>(p.x);
     uint4* __restrict__ yv = static_cast<uint4*>(p.y);
     auto valid = [&](int k) { return tid + k * T < nvec; };
@@ -106,10 +120,10 @@ block_row_kernel(const Params p) {
             if (valid(k)) raw[k] = ld_stream(xv + row * p.nvec + vec(k));
         }
         float e[VPT][VE], r_t, s;
-        thread_partial<DT, VPT>(raw, e, r_t, s, p, ident, valid);
+        thread_partial<DT, NEG, VPT>(raw, e, r_t, s, p.c, valid);
         float R = r_t;
-        block_merge_pairs(R, s, wp[par], p.c, p.neg, ident);
-        scale_and_store<DT, VPT>(e, r_t, R, s, p, ident, yv + row * p.nvec, valid, vec);
+        block_merge_pairs<NEG>(R, s, wp[par], p.c);
+        scale_and_store<DT, NEG, VPT>(e, r_t, R, s, p.c, yv + row * p.nvec, valid, vec);
     }
 }
 
@@ -117,7 +131,7 @@ block_row_kernel(const Params p) {
 // block per row, rows staged in a shared-memory ring by bulk async copies
 // dynamic shared memory: [nstage][stage_bytes] row buffers | nstage mbarriers (8 B each)
 // ---------------------------------------------------------------------------------------------
-template <int DT, int VPT>
+template <int DT, bool NEG, int VPT>
 __global__ void __launch_bounds__(BlockCfg<DT, VPT>::MAX_THREADS, 1)
 block_row_tma_kernel(const Params p, const int nstage, const uint32_t stage_bytes) {
     constexpr int VE = Traits<DT>::VE;
@@ -126,7 +140,6 @@ block_row_tma_kernel(const Params p, const int nstage, const uint32_t stage_byte
     const int T = blockDim.x, tid = threadIdx.x;
     const int nvec = static_cast<int>(p.nvec);
     const uint32_t row_bytes = static_cast<uint32_t>(p.nvec) * 16u;
-    const float ident = ref_identity(p.neg);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + size_t(nstage) * stage_bytes);
     const char* xb = static_cast<const char*>(p.x);
     uint4* __restrict__ yv = static_cast<uint4*>(p.y);
@@ -150,7 +163,7 @@ block_row_tma_kernel(const Params p, const int nstage, const uint32_t stage_byte
     bool alive = true;      // false once a bounded wait has expired: later waits are skipped
     for (int64_t i = 0; i < n_my; ++i) {
         const int64_t row = first + i * gridDim.x;
-        if (alive) alive = mbar_wait(smem_u32(&bars[stage]), phase, p.status);
+        if (alive) alive = mbar_wait_warp(smem_u32(&bars[stage]), phase, p.status);
         const uint4* srow = reinterpret_cast<const uint4*>(smem + size_t(stage) * stage_bytes);
         uint4 raw[VPT];
 #pragma unroll
@@ -159,18 +172,17 @@ block_row_tma_kernel(const Params p, const int nstage, const uint32_t stage_byte
             if (valid(k)) raw[k] = srow[vec(k)];
         }
         float e[VPT][VE], r_t, s;
-        thread_partial<DT, VPT>(raw, e, r_t, s, p, ident, valid);
+        thread_partial<DT, NEG, VPT>(raw, e, r_t, s, p.c, valid);
         float R = r_t;
-        // one warp: no __syncthreads inside the merge, so order the stage reads explicitly
-        if (T == 32) __syncwarp();
-        block_merge_pairs(R, s, wp[i & 1], p.c, p.neg, ident);
-        // every thread has read its part of this stage (the merge's barrier): refill it
+        block_merge_pairs<NEG>(R, s, wp[i & 1], p.c);
+        // every thread has read its part of this stage (the merge's barrier, or the shuffles of a
+        // single-warp block): refill it
         if (tid == 0 && i + nstage < n_my) {
             fence_proxy_async_smem();
             bulk_load_row(smem_u32(smem + size_t(stage) * stage_bytes),
                           xb + (row + int64_t(nstage) * gridDim.x) * row_bytes, row_bytes, smem_u32(&bars[stage]));
         }
-        scale_and_store<DT, VPT>(e, r_t, R, s, p, ident, yv + row * p.nvec, valid, vec);
+        scale_and_store<DT, NEG, VPT>(e, r_t, R, s, p.c, yv + row * p.nvec, valid, vec);
         if (++stage == nstage) { stage = 0; phase ^= 1u; }
     }
 }
@@ -178,15 +190,17 @@ block_row_tma_kernel(const Params p, const int nstage, const uint32_t stage_byte
 // ---------------------------------------------------------------------------------------------
 // cluster per row: block q of the cluster owns vectors [q*slice, min((q+1)*slice, nvec)) of the row
 // dynamic shared memory: [nstage][stage_bytes] slice buffers | nstage mbarriers
-// static shared memory : warp pairs, and xchg[2][16] where peers deposit their block's pair
+// static shared memory : warp pairs; xchg[2][16], where peers deposit their block's pair with
+//                        st.async, and xbar[2], the mbarriers that count those deposits
 // ---------------------------------------------------------------------------------------------
-template <int DT, int VPT>
+template <int DT, bool NEG, int VPT>
 __global__ void __launch_bounds__(BlockCfg<DT, VPT>::MAX_THREADS, 1)
 cluster_row_kernel(const Params p, const int nstage, const uint32_t stage_bytes, const int slice) {
     constexpr int VE = Traits<DT>::VE;
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ float2 wp[2][32];
     __shared__ __align__(16) float2 xchg[2][16];
+    __shared__ __align__(8) uint64_t xbar[2];
     const int T = blockDim.x, tid = threadIdx.x, lane = tid & 31;
     const uint32_t q = cluster_ctarank(), cs = cluster_nctarank();
     const int64_t ncl = cluster_count_x();             // clusters in the grid
@@ -195,7 +209,7 @@ cluster_row_kernel(const Params p, const int nstage, const uint32_t stage_bytes,
     const int v0 = min(nvec, static_cast<int>(q) * slice);
     const int nv = min(nvec, v0 + slice) - v0;         // vectors of this block's slice (may be 0)
     const uint32_t my_bytes = static_cast<uint32_t>(nv) * 16u;
-    const float ident = ref_identity(p.neg);
+    const float ident = ref_identity<NEG>();
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + size_t(nstage) * stage_bytes);
     const char* xb = static_cast<const char*>(p.x);
     uint4* __restrict__ yv = static_cast<uint4*>(p.y);
@@ -206,6 +220,8 @@ cluster_row_kernel(const Params p, const int nstage, const uint32_t stage_bytes,
     const int64_t row_bytes = p.nvec * 16;
     if (tid == 0) {
         for (int s = 0; s < nstage; ++s) mbar_init(smem_u32(&bars[s]), 1);
+        mbar_init(smem_u32(&xbar[0]), 1);
+        mbar_init(smem_u32(&xbar[1]), 1);
         mbar_fence_init();
         fence_proxy_async_smem();
         if (nv > 0)
@@ -214,7 +230,8 @@ cluster_row_kernel(const Params p, const int nstage, const uint32_t stage_bytes,
                               xb + (cid + int64_t(s) * ncl) * row_bytes + int64_t(v0) * 16, my_bytes, smem_u32(&bars[s]));
     }
     __syncthreads();
-    // every block of the cluster is resident before anyone writes into a peer's shared memory
+    // every block of the cluster is resident, with its mbarriers initialised, before anyone writes
+    // into a peer's shared memory
     cluster_arrive_release();
     cluster_wait_acquire();
 
@@ -224,35 +241,39 @@ cluster_row_kernel(const Params p, const int nstage, const uint32_t stage_bytes,
     for (int64_t i = 0; i < n_my; ++i) {
         const int64_t row = cid + i * ncl;
         const int par = static_cast<int>(i & 1);
+        const uint32_t xphase = static_cast<uint32_t>(i >> 1) & 1u;
+        // arm this row's exchange barrier: cs deposits of 8 bytes (a deposit may arrive first; the
+        // transaction count is signed)
+        if (tid == 0) mbar_expect_tx(smem_u32(&xbar[par]), cs * 8u);
         uint4 raw[VPT];
 #pragma unroll
         for (int k = 0; k < VPT; ++k) raw[k] = make_uint4(0u, 0u, 0u, 0u);
         if (nv > 0) {
-            if (alive) alive = mbar_wait(smem_u32(&bars[stage]), phase, p.status);
+            if (alive) alive = mbar_wait_warp(smem_u32(&bars[stage]), phase, p.status);
             const uint4* srow = reinterpret_cast<const uint4*>(smem + size_t(stage) * stage_bytes);
 #pragma unroll
             for (int k = 0; k < VPT; ++k)
                 if (valid(k)) raw[k] = srow[tid + k * T];
         }
         float e[VPT][VE], r_t, s;
-        thread_partial<DT, VPT>(raw, e, r_t, s, p, ident, valid);
+        thread_partial<DT, NEG, VPT>(raw, e, r_t, s, p.c, valid);
         float R = r_t;
-        if (T == 32) __syncwarp();
-        block_merge_pairs(R, s, wp[par], p.c, p.neg, ident);
+        block_merge_pairs<NEG>(R, s, wp[par], p.c);
         if (tid == 0 && nv > 0 && i + nstage < n_my) {
             fence_proxy_async_smem();
             bulk_load_row(smem_u32(smem + size_t(stage) * stage_bytes),
                           xb + (row + int64_t(nstage) * ncl) * row_bytes + int64_t(v0) * 16, my_bytes, smem_u32(&bars[stage]));
         }
-        // deposit this block's pair in slot q of every block of the cluster (this one included)
-        if (tid < cs) st_cluster_v2(map_to_rank(smem_u32(&xchg[par][q]), tid), R, s);
-        __syncwarp();
-        cluster_arrive_release();
-        cluster_wait_acquire();
+        // deposit this block's pair in slot q of every block of the cluster (this one included);
+        // rows alternate between two slots/barriers, so a fast peer's next deposit cannot be
+        // counted against this row
+        if (tid < cs)
+            st_async_v2(map_to_rank(smem_u32(&xchg[par][q]), tid), R, s, map_to_rank(smem_u32(&xbar[par]), tid));
+        if (alive) alive = mbar_wait_warp(smem_u32(&xbar[par]), xphase, p.status);
         R = ident; s = 0.0f;
         if (lane < static_cast<int>(cs)) ld_shared_v2(smem_u32(&xchg[par][lane]), R, s);
-        warp_merge_pairs(R, s, p.c, p.neg, ident);
-        scale_and_store<DT, VPT>(e, r_t, R, s, p, ident, yv + row * p.nvec, valid, vec);
+        warp_merge_pairs<NEG>(R, s, p.c);
+        scale_and_store<DT, NEG, VPT>(e, r_t, R, s, p.c, yv + row * p.nvec, valid, vec);
         if (++stage == nstage) { stage = 0; phase ^= 1u; }
     }
 }
@@ -261,24 +282,24 @@ cluster_row_kernel(const Params p, const int nstage, const uint32_t stage_bytes,
 // generic: any cols, any alignment, element-wise accesses; reads the row twice (the second read
 // normally hits L2). Pass 1 keeps a running (r, s) per thread -- the online update itself.
 // ---------------------------------------------------------------------------------------------
-template <int DT>
+template <int DT, bool NEG>
 __global__ void __launch_bounds__(1024, 1)
 generic_row_kernel(const Params p) {
     __shared__ float2 wp[2][32];
     const int T = blockDim.x, tid = threadIdx.x;
-    const float ident = ref_identity(p.neg);
+    const float ident = ref_identity<NEG>();
     int par = 0;
     for (int64_t row = blockIdx.x; row < p.rows; row += gridDim.x, par ^= 1) {
         const int64_t base = row * p.cols;
         float r = ident, s = 0.0f;
         for (int64_t j = tid; j < p.cols; j += T) {
             const float x = load_elem<DT>(p.x, base + j);
-            const float rn = ref_pick(r, x, p.neg);
+            const float rn = ref_pick<NEG>(r, x);
             const float ru = (rn == ident) ? 0.0f : rn;
             s = s * ref_factor(r, rn, p.c, ident) + ex2_noflush((x - ru) * p.c);
             r = rn;
         }
-        block_merge_pairs(r, s, wp[par], p.c, p.neg, ident);
+        block_merge_pairs<NEG>(r, s, wp[par], p.c);
         const float ru = (r == ident) ? 0.0f : r;
         const float inv = 1.0f / s;
         for (int64_t j = tid; j < p.cols; j += T) {

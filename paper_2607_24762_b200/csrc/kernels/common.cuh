@@ -21,7 +21,7 @@ struct Params {
     int64_t cols;
     int64_t nvec;      // 16-byte vectors per row (fast kernels: cols * elem_size / 16)
     float c;           // scale * log2(e): exponents are taken in base 2
-    int neg;           // c < 0: the row reference is the minimum of x instead of the maximum
+    int neg;           // c < 0: the row reference is the minimum of x instead of the maximum (host-side dispatch)
     int* status;       // device status word
 };
 
@@ -112,14 +112,22 @@ template <int DT> __device__ __forceinline__ void store_elem(void* p, int64_t i,
 }
 
 // ---- base-2 exponential on the special-function unit ---------------------------------------
-// bfloat16 shares binary32's exponent range, so a result below 2^-126 is still a representable
-// (subnormal) bf16 value and must not be flushed: bf16 uses the non-flushing form. fp32 results are
-// judged on absolute error and fp16's subnormals are normal binary32 numbers, so they flush.
+// e = 2^t with t = (x - r) * c <= 0 for the row (or thread) reference r. One MUFU.EX2 per element:
+// the flushing form of ex2.approx is a single instruction, the non-flushing one costs three more.
+//
+// bfloat16 shares binary32's exponent range, so an output below 2^-126 is still a representable
+// (subnormal) bf16 value and must not be flushed. bf16 therefore evaluates 2^(t + 64): nothing
+// above 2^-190 is flushed, the common factor 2^64 is carried by the row sum and cancels in the
+// final e * (1/S) product, which is an ordinary (non-flushing) multiply. The bias costs nothing
+// (it is the addend of the fused multiply-add) but rounds t to the spacing of numbers near 64
+// (relative error ~3e-6 on e): harmless at 8 bits of output precision, not at fp32's 1e-6
+// absolute bound, so fp32 and fp16 (whose subnormals are normal binary32 numbers) use t as is.
 template <int DT>
-__device__ __forceinline__ float ex2(float t) {
-    float r;
-    if constexpr (DT == DT_BF16) asm("ex2.approx.f32 %0, %1;" : "=f"(r) : "f"(t));
-    else                         asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(t));
+__device__ __forceinline__ float ex2_elem(float d, float c) {
+    float t, r;
+    if constexpr (DT == DT_BF16) t = fmaf(d, c, 64.0f);
+    else                         t = d * c;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(t));
     return r;
 }
 
@@ -129,10 +137,70 @@ __device__ __forceinline__ float ex2_noflush(float t) {
     return r;
 }
 
+// 1/S. fp32 output: IEEE division. 16-bit output: the special-function unit's reciprocal
+// (1 ulp of binary32, far below half an ulp of the output format).
+template <int DT>
+__device__ __forceinline__ float recip(float s) {
+    if constexpr (DT == DT_F32) return 1.0f / s;
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(s));
+    return r;
+}
+
 // ---- row reference (max of x, or min when the scale is negative) ----------------------------
 
-__device__ __forceinline__ float ref_identity(int neg) { return neg ? __int_as_float(0x7f800000) : __int_as_float(0xff800000); }
-__device__ __forceinline__ float ref_pick(float a, float b, int neg) { return neg ? fminf(a, b) : fmaxf(a, b); }
+template <bool NEG> __device__ __forceinline__ float ref_identity() {
+    return NEG ? __int_as_float(0x7f800000) : __int_as_float(0xff800000);
+}
+template <bool NEG> __device__ __forceinline__ float ref_pick(float a, float b) {
+    return NEG ? fminf(a, b) : fmaxf(a, b);
+}
+
+// Running reference over raw 16-byte vectors. fp32 folds element by element; the 16-bit types
+// fold two elements per instruction with the packed min/max (exact: the max of two bf16/fp16
+// values is one of them; a NaN operand is dropped, as fmaxf does).
+template <int DT, bool NEG> struct RefAcc;
+
+template <bool NEG> struct RefAcc<DT_F32, NEG> {
+    float a;
+    __device__ __forceinline__ void init() { a = ref_identity<NEG>(); }
+    __device__ __forceinline__ void fold(const uint4& v) {
+        a = ref_pick<NEG>(a, __uint_as_float(v.x)); a = ref_pick<NEG>(a, __uint_as_float(v.y));
+        a = ref_pick<NEG>(a, __uint_as_float(v.z)); a = ref_pick<NEG>(a, __uint_as_float(v.w));
+    }
+    __device__ __forceinline__ float value() const { return a; }
+};
+
+template <bool NEG> struct RefAcc<DT_BF16, NEG> {
+    uint32_t a;
+    static __device__ __forceinline__ uint32_t pk(uint32_t x, uint32_t y) {
+        uint32_t r;
+        if constexpr (NEG) asm("min.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(x), "r"(y));
+        else               asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(x), "r"(y));
+        return r;
+    }
+    __device__ __forceinline__ void init() { a = NEG ? 0x7f807f80u : 0xff80ff80u; }
+    __device__ __forceinline__ void fold(const uint4& v) { a = pk(pk(a, v.x), pk(pk(v.y, v.z), v.w)); }
+    __device__ __forceinline__ float value() const {
+        return ref_pick<NEG>(__uint_as_float(a << 16), __uint_as_float(a & 0xffff0000u));
+    }
+};
+
+template <bool NEG> struct RefAcc<DT_F16, NEG> {
+    uint32_t a;
+    static __device__ __forceinline__ uint32_t pk(uint32_t x, uint32_t y) {
+        uint32_t r;
+        if constexpr (NEG) asm("min.f16x2 %0, %1, %2;" : "=r"(r) : "r"(x), "r"(y));
+        else               asm("max.f16x2 %0, %1, %2;" : "=r"(r) : "r"(x), "r"(y));
+        return r;
+    }
+    __device__ __forceinline__ void init() { a = NEG ? 0x7c007c00u : 0xfc00fc00u; }
+    __device__ __forceinline__ void fold(const uint4& v) { a = pk(pk(a, v.x), pk(pk(v.y, v.z), v.w)); }
+    __device__ __forceinline__ float value() const {
+        const float2 t = __half22float2(*reinterpret_cast<const __half2*>(&a));
+        return ref_pick<NEG>(t.x, t.y);
+    }
+};
 
 // Factor that moves a partial sum taken against reference `r` to the reference `R`
 // (R = pick(r, ...)). A partial whose reference is still the identity has sum 0 (or NaN) and keeps
@@ -141,10 +209,10 @@ __device__ __forceinline__ float ref_factor(float r, float R, float c, float ide
     return (r == R || r == ident) ? 1.0f : ex2_noflush((r - R) * c);
 }
 
-template <int WIDTH>
-__device__ __forceinline__ float warp_pick(float v, int neg) {
+template <int WIDTH, bool NEG>
+__device__ __forceinline__ float warp_pick(float v) {
 #pragma unroll
-    for (int o = WIDTH / 2; o > 0; o >>= 1) v = ref_pick(v, __shfl_xor_sync(0xffffffffu, v, o), neg);
+    for (int o = WIDTH / 2; o > 0; o >>= 1) v = ref_pick<NEG>(v, __shfl_xor_sync(0xffffffffu, v, o));
     return v;
 }
 
@@ -157,9 +225,10 @@ __device__ __forceinline__ float warp_sum(float v) {
 
 // Merge (r, s) pairs across the 32 lanes of a warp:
 //   R = pick_l r_l,  S = sum_l s_l * 2^((r_l - R) c)      (online-softmax merge, Milakov-Gimelshein)
-__device__ __forceinline__ void warp_merge_pairs(float& r, float& s, float c, int neg, float ident) {
-    const float R = warp_pick<32>(r, neg);
-    s = warp_sum<32>(s * ref_factor(r, R, c, ident));
+template <bool NEG>
+__device__ __forceinline__ void warp_merge_pairs(float& r, float& s, float c) {
+    const float R = warp_pick<32, NEG>(r);
+    s = warp_sum<32>(s * ref_factor(r, R, c, ref_identity<NEG>()));
     r = R;
 }
 
@@ -219,6 +288,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* st
     return false;
 }
 
+// One lane per warp polls (spinning threads cost issue slots that other blocks' warps need); the
+// result is broadcast so that the whole warp agrees on whether the wait expired.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, int* status) {
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, status) ? 1 : 0;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+
 // ---- thread-block cluster ------------------------------------------------------------------
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -237,8 +314,11 @@ __device__ __forceinline__ uint32_t cluster_count_x() {
 __device__ __forceinline__ uint32_t map_to_rank(uint32_t local_addr, uint32_t rank) {
     uint32_t a; asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"(local_addr), "r"(rank)); return a;
 }
-__device__ __forceinline__ void st_cluster_v2(uint32_t addr, float a, float b) {
-    asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" :: "r"(addr), "f"(a), "f"(b) : "memory");
+// Asynchronous store of two floats into a peer block's shared memory; the 8 bytes are counted as
+// a transaction on the peer's mbarrier `mbar` (both addresses are shared::cluster addresses).
+__device__ __forceinline__ void st_async_v2(uint32_t addr, float a, float b, uint32_t mbar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];"
+                 :: "r"(addr), "f"(a), "f"(b), "r"(mbar) : "memory");
 }
 __device__ __forceinline__ void ld_shared_v2(uint32_t addr, float& a, float& b) {
     asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(a), "=f"(b) : "r"(addr) : "memory");
