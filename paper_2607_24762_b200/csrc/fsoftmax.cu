@@ -12,6 +12,7 @@
 
 #include "kernels/block_row.cuh"
 #include "kernels/common.cuh"
+#include "kernels/smem_row.cuh"
 #include "kernels/warp_row.cuh"
 
 namespace {
@@ -105,12 +106,21 @@ int next_pow2(int64_t v) { int p = 1; while (p < v) p <<= 1; return p; }
 int max_vpt(int dtype) { return dtype == FS_DTYPE_FP32 ? 16 : 8; }
 int max_threads_for(int dtype, int vpt) { return vpt * (dtype == FS_DTYPE_FP32 ? 4 : 8) <= 16 ? 1024 : 512; }
 
-// Row sizes (bytes) at which the dispatcher changes kernel.
-constexpr int64_t kWarpMaxRowBytes = 4096;          // (sub-)warp per row up to here
-constexpr int64_t kBlockMaxRowBytes = 32768;        // block per row up to here, cluster beyond
-constexpr int64_t kClusterSliceBytes = 32768;       // target slice per block of a cluster
+// Row sizes (bytes) at which the dispatcher changes kernel, from sweeps on B200 (256 MiB of
+// traffic per launch, rows from 2 KiB to 1 MiB, against a plain copy of the same bytes).
+//   16-bit: (sub-)warp per row up to 4 KiB, block per row (direct loads) up to 32 KiB, then the
+//           shared-memory-resident split with 32 KiB slices and 128-thread blocks.
+//   fp32:   (sub-)warp per row up to 1 KiB, block per row up to 8 KiB, block per row fed by bulk
+//           copies up to 64 KiB, then the split with 64 KiB slices and 256-thread blocks.
+int64_t warp_max_row_bytes(int dtype) { return dtype == FS_DTYPE_FP32 ? 1024 : 4096; }
+int64_t block_max_row_bytes(int dtype) { return dtype == FS_DTYPE_FP32 ? 8192 : 32768; }
+int64_t block_tma_max_row_bytes(int dtype) { return dtype == FS_DTYPE_FP32 ? 65536 : 32768; }
+int64_t split_slice_bytes(int dtype) { return dtype == FS_DTYPE_FP32 ? 65536 : 32768; }
+int split_threads(int dtype) { return dtype == FS_DTYPE_FP32 ? 256 : 128; }
+constexpr int64_t kWarpTileMaxRowBytes = 4096;      // rows the warp-tile bulk-copy kernel takes
+constexpr int64_t kClusterSliceBytes = 32768;       // register-resident cluster kernel: slice per block
 constexpr int kMaxCluster = 16;
-constexpr int64_t kTileBytes = 16384;              // rows per bulk copy of the warp-tile kernel
+constexpr int64_t kTileBytes = 16384;               // rows per bulk copy of the warp-tile kernel
 
 int64_t warp_capacity_vecs(int dtype) { return 32 * int64_t(max_vpt(dtype)); }
 
@@ -138,8 +148,9 @@ bool block_geom(int64_t nvec, int dtype, int threads, BlockGeom* g) {
         g->threads = threads; g->vpt = vpt;
         return true;
     }
-    int vpt = 1;
-    while (vpt < mv && nvec > 256 * int64_t(vpt)) vpt <<= 1;
+    // at least two loads in flight per thread, 128-thread blocks until the row outgrows them
+    int vpt = 2;
+    while (vpt < mv && nvec > 128 * int64_t(vpt)) vpt <<= 1;
     int64_t t = (nvec + vpt - 1) / vpt;
     t = (t + 31) / 32 * 32;
     if (t > max_threads_for(dtype, vpt)) return false;
@@ -162,6 +173,36 @@ bool cluster_geom(int64_t nvec, int dtype, int threads, int cluster, ClusterGeom
     return block_geom(slice, dtype, threads, &g->b);
 }
 
+// Shared-memory-resident split: slices of about kClusterSliceBytes, up to kMaxCluster blocks; rows
+// beyond that grow the slice up to what one block's shared memory holds.
+struct SmemGeom { int cs, slice, threads, chunk_vecs; };
+constexpr int64_t kSmemSliceMaxBytes = 200 * 1024;
+bool smem_geom(int64_t nvec, int dtype, int threads, int cluster, SmemGeom* g) {
+    if (nvec < 1) return false;
+    int cs = cluster;
+    if (cs == 0) {
+        cs = 1;
+        while (cs < kMaxCluster && (nvec * 16 + cs - 1) / cs > split_slice_bytes(dtype)) cs <<= 1;
+    }
+    if (cs != 1 && cs != 2 && cs != 4 && cs != 8 && cs != 16) return false;
+    const int64_t slice = (nvec + cs - 1) / cs;
+    if (slice * 16 > kSmemSliceMaxBytes) return false;
+    int t = threads;
+    if (t == 0) t = slice * 16 > split_slice_bytes(dtype) ? 256 : (slice >= 256 ? split_threads(dtype) : 64);
+    if (t % 32 || t > 512) return false;
+    // chunks of four vectors per thread; at most kSmemRowMaxChunks of them
+    int64_t cv = int64_t(t) * 4;
+    while ((slice + cv - 1) / cv > kSmemRowMaxChunks) cv += int64_t(t);
+    if (cv * 16 > (int64_t(1) << 20) - 16) return false;
+    g->cs = cs; g->slice = static_cast<int>(slice); g->threads = t; g->chunk_vecs = static_cast<int>(cv);
+    return true;
+}
+
+bool cluster_uses_registers() {
+    static const bool v = [] { const char* e = std::getenv("FS_CLUSTER_REGS"); return e && e[0] == '1'; }();
+    return v;
+}
+
 bool fast_path_ok(int64_t cols, int dtype, int x_align, int y_align) {
     return x_align >= 16 && y_align >= 16 && (cols * elem_size(dtype)) % 16 == 0;
 }
@@ -171,9 +212,11 @@ int select_kernel(int64_t cols, int dtype, int x_align, int y_align) {
     const int64_t row_bytes = cols * elem_size(dtype);
     const int64_t nvec = row_bytes / 16;
     WarpGeom wg; BlockGeom bg; ClusterGeom cg;
-    if (row_bytes <= kWarpMaxRowBytes && warp_geom(nvec, dtype, &wg)) return FS_KERNEL_WARP;
-    if (row_bytes <= kBlockMaxRowBytes && block_geom(nvec, dtype, 0, &bg)) return FS_KERNEL_BLOCK_TMA;
-    if (cluster_geom(nvec, dtype, 0, 0, &cg)) return FS_KERNEL_CLUSTER;
+    if (row_bytes <= warp_max_row_bytes(dtype) && warp_geom(nvec, dtype, &wg)) return FS_KERNEL_WARP;
+    if (row_bytes <= block_max_row_bytes(dtype) && block_geom(nvec, dtype, 0, &bg)) return FS_KERNEL_BLOCK;
+    if (row_bytes <= block_tma_max_row_bytes(dtype) && block_geom(nvec, dtype, 0, &bg)) return FS_KERNEL_BLOCK_TMA;
+    SmemGeom sg;
+    if (smem_geom(nvec, dtype, 0, 0, &sg) || cluster_geom(nvec, dtype, 0, 0, &cg)) return FS_KERNEL_CLUSTER;
     return FS_KERNEL_GENERIC;
 }
 
@@ -409,7 +452,7 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
         case FS_KERNEL_BLOCK_TMA: {
             const size_t smem_cap = static_cast<size_t>(dev.smem_optin) - 2048;   // room for the static part
             WarpGeom wg;
-            if (p.nvec * 16 <= kWarpMaxRowBytes && warp_geom(p.nvec, dtype, &wg)) {
+            if (p.nvec * 16 <= kWarpTileMaxRowBytes && warp_geom(p.nvec, dtype, &wg)) {
                 // short rows: one bulk copy brings a tile of consecutive rows, each (sub-)warp owns rows
                 const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) { return warp_tma_fn<decltype(dt)::value, decltype(ng)::value>(wg); });
                 if (!fn) return FS_ERR_UNSUPPORTED;
@@ -454,6 +497,20 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
         }
         case FS_KERNEL_CLUSTER: {
             if (!dev.cluster_ok) return FS_ERR_UNSUPPORTED;
+            SmemGeom sg;
+            if (!cluster_uses_registers() && smem_geom(p.nvec, dtype, threads, cluster, &sg)) {
+                const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) {
+                    return (const void*)smem_row_kernel<decltype(dt)::value, decltype(ng)::value>; });
+                const size_t stage_bytes = static_cast<size_t>(sg.slice) * 16;
+                const size_t smem = stage_bytes + size_t(kSmemRowMaxChunks) * 8;
+                if (smem > static_cast<size_t>(dev.smem_optin) - 2048) return FS_ERR_UNSUPPORTED;
+                int ncl = 0;
+                if ((rc = active_clusters(dev, fn, sg.threads, smem, sg.cs, &ncl)) != FS_OK) return rc;
+                int64_t clusters = std::min<int64_t>(rows, max_grid / sg.cs);
+                if (persistent_grids()) clusters = std::min<int64_t>(clusters, ncl);
+                return launch(fn, clusters * sg.cs, sg.threads, smem, sg.cs, st, p,
+                              static_cast<uint32_t>(stage_bytes), sg.slice, sg.chunk_vecs);
+            }
             ClusterGeom g;
             if (!cluster_geom(p.nvec, dtype, threads, cluster, &g)) return FS_ERR_UNSUPPORTED;
             const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) { return cluster_fn<decltype(dt)::value, decltype(ng)::value>(g.b.vpt); });

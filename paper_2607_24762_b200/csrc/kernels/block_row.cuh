@@ -232,7 +232,7 @@ cluster_row_kernel(const Params p, const int nstage, const uint32_t stage_bytes,
     __syncthreads();
     // every block of the cluster is resident, with its mbarriers initialised, before anyone writes
     // into a peer's shared memory
-    cluster_arrive_release();
+    cluster_arrive_relaxed();
     cluster_wait_acquire();
 
     int stage = 0;

@@ -323,8 +323,10 @@ __device__ __forceinline__ void st_async_v2(uint32_t addr, float a, float b, uin
 __device__ __forceinline__ void ld_shared_v2(uint32_t addr, float& a, float& b) {
     asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(a), "=f"(b) : "r"(addr) : "memory");
 }
-__device__ __forceinline__ void cluster_arrive_release() {
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+// Start-up rendezvous of a cluster: no data is handed over (mbarrier initialisation is published
+// by fence.mbarrier_init), so the arrive carries no memory fence.
+__device__ __forceinline__ void cluster_arrive_relaxed() {
+    asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void cluster_wait_acquire() {
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
