@@ -109,6 +109,38 @@ int fs_copy(const void* x, void* y, int64_t bytes, void* stream);
  */
 int fs_device_status(void);
 
+/*
+ * fs_softmax_static -- fs_softmax for callers that must not allocate device memory.
+ * (The paper has no counterpart: this entry point exists for the library's users only.)
+ *
+ * Every other compute entry point calls cudaMalloc once per device, on first use, for the status
+ * word its kernels write when a bounded wait expires (fs_softmax_host also for its staging
+ * buffers). Some callers cannot afford that call: a process that has handed all device memory to
+ * its own pool and must not touch the driver's allocator again, a service that has to prove it
+ * cannot run out of memory after start-up, or a latency-critical loop in which the implicit device
+ * synchronisation of an allocation is unacceptable. This entry point makes no cudaMalloc,
+ * cudaFree or other allocating call, ever. It always runs the split-row kernel (FS_KERNEL_CLUSTER's
+ * shared-memory-resident form), whose status word then lives in a 256-byte array that is part of
+ * the library's device code: every GPU that loads the library holds those 256 bytes until the
+ * process exits.
+ *
+ *   x, y, rows, cols, dtype, scale, stream   as for fs_softmax; x and y are DEVICE pointers.
+ *   Limits: x and y 16-byte aligned, row size a multiple of 16 bytes and at most
+ *           FS_STATIC_MAX_ROW_BYTES (what 16 blocks hold in shared memory), rows * blocks-per-row
+ *           below 2^31. Anything else returns FS_ERR_UNSUPPORTED and enqueues nothing; there is no
+ *           silent switch to another kernel.
+ *   First call on a device: looks up the array's device address and raises the kernel's
+ *           shared-memory limit (queries and attribute calls, no allocation). Make that first call
+ *           before starting any stream capture.
+ *   Sharing: all calls on a device share the one array, and it keeps what the last call left
+ *           there. Each call therefore enqueues a 4-byte clear of the status word ahead of its
+ *           kernel on `stream`. Two calls whose work overlaps on the GPU (different streams) race
+ *           on that word: results stay correct, but an expired wait may go unrecorded.
+ *           fs_device_status does not read this word.
+ */
+#define FS_STATIC_MAX_ROW_BYTES (16 * 200 * 1024)
+int fs_softmax_static(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale, void* stream);
+
 /* fs_release -- frees the staging buffers and streams fs_softmax_host created on the current device. */
 int fs_release(void);
 

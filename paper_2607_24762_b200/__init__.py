@@ -9,5 +9,5 @@ from .binding import (  # noqa: F401
     FS_KERNEL_AUTO, FS_KERNEL_BLOCK, FS_KERNEL_BLOCK_TMA, FS_KERNEL_CLUSTER, FS_KERNEL_GENERIC, FS_KERNEL_WARP,
     KERNELS, FsError,
     fs_copy, fs_device_status, fs_kernel_name, fs_last_cuda_error, fs_release, fs_select_kernel,
-    fs_softmax, fs_softmax_ex, fs_softmax_host, fs_softmax_status, fs_strerror, fs_version,
+    fs_softmax, fs_softmax_ex, fs_softmax_host, fs_softmax_static, fs_softmax_status, fs_strerror, fs_version,
 )

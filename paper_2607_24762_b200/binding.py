@@ -51,6 +51,8 @@ def lib() -> ctypes.CDLL:
             L.fs_select_kernel.restype = ci
             L.fs_softmax_host.argtypes = [vp, vp, i64, i64, ci, f32]
             L.fs_softmax_host.restype = ci
+            L.fs_softmax_static.argtypes = [vp, vp, i64, i64, ci, f32, vp]
+            L.fs_softmax_static.restype = ci
             L.fs_copy.argtypes = [vp, vp, i64, vp]
             L.fs_copy.restype = ci
             L.fs_device_status.argtypes = []
@@ -117,6 +119,11 @@ def fs_select_kernel(rows: int, cols: int, dtype: int, x_align: int = 16, y_alig
 
 def fs_softmax_host(x_host, y_host, rows: int, cols: int, dtype: int, scale: float = 1.0) -> None:
     _check(lib().fs_softmax_host(_ptr(x_host), _ptr(y_host), rows, cols, dtype, scale), "fs_softmax_host")
+
+
+def fs_softmax_static(x, y, rows: int, cols: int, dtype: int, scale: float = 1.0, stream=None) -> None:
+    """fs_softmax without any device allocation: split-row kernel, status word in a fixed device array."""
+    _check(lib().fs_softmax_static(_ptr(x), _ptr(y), rows, cols, dtype, scale, _stream(stream)), "fs_softmax_static")
 
 
 def fs_copy(x, y, nbytes: int, stream=None) -> None:

@@ -565,6 +565,33 @@ int validate(const void* x, const void* y, int64_t rows, int64_t cols, int dtype
 
 }  // namespace
 
+// ---------------------------------------------------------------------------------------------
+// fs_softmax_static: the split-row kernel with its scratch in a fixed device array
+// ---------------------------------------------------------------------------------------------
+// The split-row kernel records an expired bounded wait in a status word in global memory. The
+// other entry points keep that word in a buffer obtained with cudaMalloc on first use; this one
+// keeps it in the array below, which is part of the loaded module: 256 bytes on every GPU that
+// loads the library, held until the process exits. Word 0 is the status word, the rest is unused.
+// In host code the array's name is only a handle for the runtime, not a device address: the
+// address a kernel can use comes from cudaGetSymbolAddress, asked once per device with that device
+// current.
+constexpr int kStaticScratchWords = 64;
+static __device__ __align__(256) int fs_static_scratch[kStaticScratchWords];
+
+namespace {
+
+struct StaticDevice {
+    bool ready = false;
+    int smem_optin = 0;
+    int cluster_ok = 0;
+    int* scratch = nullptr;              // device address of fs_static_scratch on this device
+    bool configured[3][2] = {};          // split-row kernel variants whose attributes are set
+};
+StaticDevice g_static[kMaxDevices];
+std::mutex g_static_mu;
+
+}  // namespace
+
 // =============================================================================================
 // C ABI
 // =============================================================================================
@@ -679,6 +706,56 @@ int fs_device_status(void) {
     FS_CUDA(cudaMemcpy(&word, dev->status, sizeof(int), cudaMemcpyDeviceToHost));
     if (word) FS_CUDA(cudaMemset(dev->status, 0, sizeof(int)));
     return (word & DEV_TIMEOUT) ? FS_ERR_DEVICE_TIMEOUT : FS_OK;
+}
+
+int fs_softmax_static(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale, void* stream) {
+    const int v = validate(x, y, rows, cols, dtype, scale);
+    if (v != FS_OK) return v;
+    if (rows == 0 || cols == 0) return FS_OK;
+    if (!fast_path_ok(cols, dtype, ptr_align(x), ptr_align(y))) return FS_ERR_UNSUPPORTED;
+    SmemGeom sg;
+    const int64_t nvec = cols * elem_size(dtype) / 16;
+    if (!smem_geom(nvec, dtype, 0, 0, &sg)) return FS_ERR_UNSUPPORTED;      // row longer than FS_STATIC_MAX_ROW_BYTES
+    if (rows > 0x7fffffff / sg.cs) return FS_ERR_UNSUPPORTED;
+
+    int d = 0;
+    FS_CUDA(cudaGetDevice(&d));
+    if (d < 0 || d >= kMaxDevices) return FS_ERR_UNSUPPORTED;
+    StaticDevice& sd = g_static[d];
+    std::lock_guard<std::mutex> lk(g_static_mu);
+    if (!sd.ready) {                     // first call on this device: no allocation, only queries
+        FS_CUDA(cudaDeviceGetAttribute(&sd.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, d));
+        FS_CUDA(cudaDeviceGetAttribute(&sd.cluster_ok, cudaDevAttrClusterLaunch, d));
+        void* addr = nullptr;
+        FS_CUDA(cudaGetSymbolAddress(&addr, fs_static_scratch));
+        sd.scratch = static_cast<int*>(addr);
+        sd.ready = true;
+    }
+    if (!sd.cluster_ok) return FS_ERR_UNSUPPORTED;
+
+    Params p;
+    p.x = x; p.y = y; p.rows = rows; p.cols = cols; p.nvec = nvec;
+    p.c = static_cast<float>(static_cast<double>(scale) * kLog2e);
+    p.neg = p.c < 0.0f ? 1 : 0;
+    p.status = sd.scratch;
+    const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) {
+        return (const void*)smem_row_kernel<decltype(dt)::value, decltype(ng)::value>; });
+    const size_t stage_bytes = static_cast<size_t>(sg.slice) * 16;
+    const size_t smem = stage_bytes + size_t(kSmemRowMaxChunks) * 8;
+    if (smem > static_cast<size_t>(sd.smem_optin) - 2048) return FS_ERR_UNSUPPORTED;
+    if (!sd.configured[dtype][p.neg]) {
+        cudaFuncAttributes fa;
+        FS_CUDA(cudaFuncGetAttributes(&fa, fn));
+        FS_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     sd.smem_optin - static_cast<int>(fa.sharedSizeBytes)));
+        FS_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+        sd.configured[dtype][p.neg] = true;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the array keeps whatever the last call left: the status word must start at zero
+    FS_CUDA(cudaMemsetAsync(sd.scratch, 0, sizeof(int), st));
+    return launch(fn, rows * sg.cs, sg.threads, smem, sg.cs, st, p,
+                  static_cast<uint32_t>(stage_bytes), sg.slice, sg.chunk_vecs);
 }
 
 int fs_last_cuda_error(void) { return t_last_cuda_error; }
