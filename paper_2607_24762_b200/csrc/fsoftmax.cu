@@ -301,6 +301,13 @@ int active_clusters(Device& dev, const void* fn, int threads, size_t smem, int c
     return FS_OK;
 }
 
+// Programmatic dependent launch (on unless FS_PDL=0): the kernel may be scheduled while the
+// previous kernel of the stream drains; it waits (griddepcontrol.wait) before touching memory.
+bool pdl_enabled() {
+    static const bool v = [] { const char* e = std::getenv("FS_PDL"); return !(e && e[0] == '0'); }();
+    return v;
+}
+
 template <typename... Args>
 int launch(const void* fn, int64_t grid, int threads, size_t smem, int cs, cudaStream_t st, Args... args) {
     void* argv[] = {static_cast<void*>(&args)...};
@@ -309,12 +316,19 @@ int launch(const void* fn, int64_t grid, int threads, size_t smem, int cs, cudaS
     cfg.blockDim = dim3(threads, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
+    unsigned n = 0;
     if (cs > 0) {
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = cs; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr; cfg.numAttrs = 1;
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = cs; attr[n].val.clusterDim.y = 1; attr[n].val.clusterDim.z = 1;
+        ++n;
     }
+    if (pdl_enabled()) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
+    cfg.attrs = n ? attr : nullptr; cfg.numAttrs = n;
     FS_CUDA(cudaLaunchKernelExC(&cfg, fn, argv));
     return FS_OK;
 }

@@ -105,6 +105,7 @@ __global__ void __launch_bounds__(BlockCfg<DT, VPT>::MAX_THREADS, 1)
 block_row_kernel(const Params p) {
     constexpr int VE = Traits<DT>::VE;
     __shared__ float2 wp[2][32];
+    pdl_launch_dependents();
     const int T = blockDim.x, tid = threadIdx.x;
     const int nvec = static_cast<int>(p.nvec);
     const uint4* __restrict__ xv = static_cast<const uint4*>(p.x);
@@ -112,6 +113,7 @@ block_row_kernel(const Params p) {
     auto valid = [&](int k) { return tid + k * T < nvec; };
     auto vec = [&](int k) { return tid + k * T; };
     int par = 0;
+    pdl_wait();
     for (int64_t row = blockIdx.x; row < p.rows; row += gridDim.x, par ^= 1) {
         uint4 raw[VPT];
 #pragma unroll
@@ -135,6 +137,7 @@ template <int DT, bool NEG, int VPT>
 __global__ void __launch_bounds__(BlockCfg<DT, VPT>::MAX_THREADS, 1)
 block_row_tma_kernel(const Params p, const int nstage, const uint32_t stage_bytes) {
     constexpr int VE = Traits<DT>::VE;
+    pdl_launch_dependents();
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ float2 wp[2][32];
     const int T = blockDim.x, tid = threadIdx.x;
@@ -152,11 +155,13 @@ block_row_tma_kernel(const Params p, const int nstage, const uint32_t stage_byte
         for (int s = 0; s < nstage; ++s) mbar_init(smem_u32(&bars[s]), 1);
         mbar_fence_init();
         fence_proxy_async_smem();
+        pdl_wait();
         for (int s = 0; s < nstage && s < n_my; ++s)
             bulk_load_row(smem_u32(smem + size_t(s) * stage_bytes),
                           xb + (first + int64_t(s) * gridDim.x) * row_bytes, row_bytes, smem_u32(&bars[s]));
     }
     __syncthreads();
+    pdl_wait();
 
     int stage = 0;
     uint32_t phase = 0;
@@ -197,6 +202,7 @@ template <int DT, bool NEG, int VPT>
 __global__ void __launch_bounds__(BlockCfg<DT, VPT>::MAX_THREADS, 1)
 cluster_row_kernel(const Params p, const int nstage, const uint32_t stage_bytes, const int slice) {
     constexpr int VE = Traits<DT>::VE;
+    pdl_launch_dependents();
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ float2 wp[2][32];
     __shared__ __align__(16) float2 xchg[2][16];
@@ -224,6 +230,7 @@ cluster_row_kernel(const Params p, const int nstage, const uint32_t stage_bytes,
         mbar_init(smem_u32(&xbar[1]), 1);
         mbar_fence_init();
         fence_proxy_async_smem();
+        pdl_wait();
         if (nv > 0)
             for (int s = 0; s < nstage && s < n_my; ++s)
                 bulk_load_row(smem_u32(smem + size_t(s) * stage_bytes),
@@ -234,6 +241,7 @@ cluster_row_kernel(const Params p, const int nstage, const uint32_t stage_bytes,
     // into a peer's shared memory
     cluster_arrive_relaxed();
     cluster_wait_acquire();
+    pdl_wait();
 
     int stage = 0;
     uint32_t phase = 0;
@@ -286,6 +294,8 @@ template <int DT, bool NEG>
 __global__ void __launch_bounds__(1024, 1)
 generic_row_kernel(const Params p) {
     __shared__ float2 wp[2][32];
+    pdl_launch_dependents();
+    pdl_wait();
     const int T = blockDim.x, tid = threadIdx.x;
     const float ident = ref_identity<NEG>();
     int par = 0;
@@ -315,6 +325,8 @@ generic_row_kernel(const Params p) {
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 copy_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, const int64_t nvec) {
+    pdl_launch_dependents();
+    pdl_wait();
     for (int64_t base = int64_t(blockIdx.x) * 1024; base < nvec; base += int64_t(gridDim.x) * 1024) {
         uint4 v[4];
 #pragma unroll

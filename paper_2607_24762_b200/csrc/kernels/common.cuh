@@ -296,6 +296,14 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, in
     return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
+// ---- programmatic dependent launch ------------------------------------------------------------
+// Every kernel lets the next kernel in the stream be scheduled as soon as all of its own blocks
+// have started (launch_dependents), and touches global memory only after the previous kernel has
+// completed and flushed (wait). With the launch attribute set by the host this overlaps the next
+// launch's latency and prologue with this kernel's tail; without it both are no-ops.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---- thread-block cluster ------------------------------------------------------------------
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {

@@ -27,6 +27,7 @@ __global__ void __launch_bounds__(512, 2)
 smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, const int chunk_vecs) {
     constexpr int VE = Traits<DT>::VE;
     constexpr int U = 4;                                  // vectors a thread handles per step
+    pdl_launch_dependents();
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ float2 wp[2][32];
     __shared__ __align__(16) float2 xchg[2][16];
@@ -62,6 +63,7 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
         mbar_init(smem_u32(&xbar[1]), 1);
         mbar_fence_init();
         fence_proxy_async_smem();
+        pdl_wait();
         if (n_my > 0) issue_row(cid);
     }
     __syncthreads();
@@ -69,6 +71,7 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
         cluster_arrive_relaxed();
         cluster_wait_acquire();
     }
+    pdl_wait();
 
     bool alive = true;      // false once a bounded wait has expired: later waits are skipped
     for (int64_t i = 0; i < n_my; ++i) {

@@ -55,10 +55,17 @@ __device__ __forceinline__ void warp_row_math(const uint4 (&raw)[VPL], float c, 
     }
 }
 
+// Rows that fill 64 payload registers per lane are capped at 85 registers (3 blocks of 256
+// threads per SM) so that enough rows are in flight to cover HBM latency.
+template <int DT, int VPL, int R> struct WarpCfg {
+    static constexpr int MIN_BLOCKS = (VPL * R * Traits<DT>::VE >= 64) ? 3 : 1;
+};
+
 template <int DT, bool NEG, int LANES, int VPL, int R>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, WarpCfg<DT, VPL, R>::MIN_BLOCKS)
 warp_row_kernel(const Params p) {
     constexpr int G = 32 / LANES;
+    pdl_launch_dependents();
     const int lane = threadIdx.x & 31;
     const int sub = lane / LANES;          // which of the warp's G rows
     const int sl = lane % LANES;           // lane within the row's group
@@ -69,6 +76,7 @@ warp_row_kernel(const Params p) {
     uint4* __restrict__ yv = static_cast<uint4*>(p.y);
     const int nvec = static_cast<int>(p.nvec);
     auto live = [&](int k) { return sl + k * LANES < nvec; };
+    pdl_wait();
 
     for (int64_t tile = int64_t(blockIdx.x) * warps + (threadIdx.x >> 5); tile < ntiles;
          tile += int64_t(gridDim.x) * warps) {
@@ -100,6 +108,7 @@ template <int DT, bool NEG, int LANES, int VPL>
 __global__ void __launch_bounds__(256)
 warp_row_tma_kernel(const Params p, const int tile_rows, const uint32_t tile_bytes_max) {
     constexpr int G = 32 / LANES;
+    pdl_launch_dependents();
     extern __shared__ __align__(128) unsigned char smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int sub = lane / LANES, sl = lane % LANES;
@@ -118,6 +127,7 @@ warp_row_tma_kernel(const Params p, const int tile_rows, const uint32_t tile_byt
         fence_proxy_async_smem();
     }
     __syncthreads();
+    pdl_wait();
     uint32_t phase = 0;
     bool alive = true;
     for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
