@@ -107,16 +107,19 @@ int max_vpt(int dtype) { return dtype == FS_DTYPE_FP32 ? 16 : 8; }
 int max_threads_for(int dtype, int vpt) { return vpt * (dtype == FS_DTYPE_FP32 ? 4 : 8) <= 16 ? 1024 : 512; }
 
 // Row sizes (bytes) at which the dispatcher changes kernel, from sweeps on B200 (256 MiB of
-// traffic per launch, rows from 2 KiB to 1 MiB, against a plain copy of the same bytes).
-//   16-bit: (sub-)warp per row up to 4 KiB, block per row (direct loads) up to 32 KiB, then the
-//           shared-memory-resident split with 32 KiB slices and 128-thread blocks.
-//   fp32:   (sub-)warp per row up to 1 KiB, block per row up to 8 KiB, block per row fed by bulk
-//           copies up to 64 KiB, then the split with 64 KiB slices and 256-thread blocks.
-int64_t warp_max_row_bytes(int dtype) { return dtype == FS_DTYPE_FP32 ? 1024 : 4096; }
-int64_t block_max_row_bytes(int dtype) { return dtype == FS_DTYPE_FP32 ? 8192 : 32768; }
-int64_t block_tma_max_row_bytes(int dtype) { return dtype == FS_DTYPE_FP32 ? 65536 : 32768; }
-int64_t split_slice_bytes(int dtype) { return dtype == FS_DTYPE_FP32 ? 65536 : 32768; }
-int split_threads(int dtype) { return dtype == FS_DTYPE_FP32 ? 256 : 128; }
+// traffic per launch, rows from 2 KiB to 1 MiB, every kernel x threads x cluster size, against a
+// plain copy of the same bytes).
+//   16-bit: (sub-)warp per row up to 4 KiB, block per row (direct loads) up to 8 KiB, then the
+//           shared-memory-resident split.
+//   fp32:   (sub-)warp per row up to 2 KiB, block per row up to 8 KiB, block per row fed by bulk
+//           copies up to 32 KiB, then the split.
+//   split:  32 KiB slices and 128-thread blocks (6 blocks per SM), cluster size the next power of
+//           two that reaches that slice; rows beyond 16 x 32 KiB grow the slice, with 256 threads.
+int64_t warp_max_row_bytes(int dtype) { return dtype == FS_DTYPE_FP32 ? 2048 : 4096; }
+int64_t block_max_row_bytes(int) { return 8192; }
+int64_t block_tma_max_row_bytes(int dtype) { return dtype == FS_DTYPE_FP32 ? 32768 : 0; }
+int64_t split_slice_bytes(int) { return 32768; }
+int split_threads(int) { return 128; }
 constexpr int64_t kWarpTileMaxRowBytes = 4096;      // rows the warp-tile bulk-copy kernel takes
 constexpr int64_t kClusterSliceBytes = 32768;       // register-resident cluster kernel: slice per block
 constexpr int kMaxCluster = 16;
@@ -175,7 +178,7 @@ bool cluster_geom(int64_t nvec, int dtype, int threads, int cluster, ClusterGeom
 
 // Shared-memory-resident split: slices of about kClusterSliceBytes, up to kMaxCluster blocks; rows
 // beyond that grow the slice up to what one block's shared memory holds.
-struct SmemGeom { int cs, slice, threads, chunk_vecs; };
+struct SmemGeom { int cs, slice, threads; };
 constexpr int64_t kSmemSliceMaxBytes = 200 * 1024;
 bool smem_geom(int64_t nvec, int dtype, int threads, int cluster, SmemGeom* g) {
     if (nvec < 1) return false;
@@ -187,14 +190,15 @@ bool smem_geom(int64_t nvec, int dtype, int threads, int cluster, SmemGeom* g) {
     if (cs != 1 && cs != 2 && cs != 4 && cs != 8 && cs != 16) return false;
     const int64_t slice = (nvec + cs - 1) / cs;
     if (slice * 16 > kSmemSliceMaxBytes) return false;
+    // a block covers kSmemRowMaxChunks chunks of smem_row_u(dtype) vectors per thread
+    const int64_t per_thread = int64_t(kSmemRowMaxChunks) * smem_row_u(dtype);
     int t = threads;
-    if (t == 0) t = slice * 16 > split_slice_bytes(dtype) ? 256 : (slice >= 256 ? split_threads(dtype) : 64);
-    if (t % 32 || t > 512) return false;
-    // chunks of four vectors per thread; at most kSmemRowMaxChunks of them
-    int64_t cv = int64_t(t) * 4;
-    while ((slice + cv - 1) / cv > kSmemRowMaxChunks) cv += int64_t(t);
-    if (cv * 16 > (int64_t(1) << 20) - 16) return false;
-    g->cs = cs; g->slice = static_cast<int>(slice); g->threads = t; g->chunk_vecs = static_cast<int>(cv);
+    if (t == 0) {
+        t = slice >= 256 ? split_threads(dtype) : 64;
+        while (t < 512 && slice > per_thread * t) t <<= 1;
+    }
+    if (t % 32 || t > 512 || slice > per_thread * t) return false;
+    g->cs = cs; g->slice = static_cast<int>(slice); g->threads = t;
     return true;
 }
 
@@ -404,6 +408,28 @@ template <typename F> const void* by_variant(int dtype, bool neg, F f) {
     }
 }
 
+// The split-row kernel: whether every block's slice is a whole number of chunks, the kernel
+// variant for it, and its dynamic shared memory (slice, chunk mbarriers, per-thread chunk references).
+bool smem_row_full(const SmemGeom& g, int dtype, int64_t nvec) {
+    const int64_t chunk = int64_t(smem_row_u(dtype)) * g.threads;
+    return nvec == int64_t(g.slice) * g.cs && g.slice % chunk == 0;
+}
+int smem_row_nchunk(const SmemGeom& g, int dtype) {
+    const int64_t chunk = int64_t(smem_row_u(dtype)) * g.threads;
+    return static_cast<int>((g.slice + chunk - 1) / chunk);
+}
+const void* smem_row_fn(int dtype, bool neg, const SmemGeom& g, int64_t nvec) {
+    const bool full = smem_row_full(g, dtype, nvec);
+    return by_variant(dtype, neg, [&](auto dt, auto ng) -> const void* {
+        constexpr int DT = decltype(dt)::value;
+        constexpr bool NG = decltype(ng)::value;
+        return full ? (const void*)smem_row_kernel<DT, NG, true> : (const void*)smem_row_kernel<DT, NG, false>;
+    });
+}
+size_t smem_row_bytes(const SmemGeom& g) {
+    return static_cast<size_t>(g.slice) * 16 + size_t(kSmemRowMaxChunks) * 8 + size_t(kSmemRowMaxChunks) * g.threads * 4;
+}
+
 // Shared-memory ring: as many stages as fit in `budget` bytes, between 2 and `max_stages`.
 int ring_stages(size_t stage_bytes, size_t budget, int max_stages) {
     int n = static_cast<int>(budget / (stage_bytes + 8));
@@ -513,17 +539,16 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
             if (!dev.cluster_ok) return FS_ERR_UNSUPPORTED;
             SmemGeom sg;
             if (!cluster_uses_registers() && smem_geom(p.nvec, dtype, threads, cluster, &sg)) {
-                const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) {
-                    return (const void*)smem_row_kernel<decltype(dt)::value, decltype(ng)::value>; });
+                const void* fn = smem_row_fn(dtype, p.neg, sg, p.nvec);
                 const size_t stage_bytes = static_cast<size_t>(sg.slice) * 16;
-                const size_t smem = stage_bytes + size_t(kSmemRowMaxChunks) * 8;
+                const size_t smem = smem_row_bytes(sg);
                 if (smem > static_cast<size_t>(dev.smem_optin) - 2048) return FS_ERR_UNSUPPORTED;
                 int ncl = 0;
                 if ((rc = active_clusters(dev, fn, sg.threads, smem, sg.cs, &ncl)) != FS_OK) return rc;
                 int64_t clusters = std::min<int64_t>(rows, max_grid / sg.cs);
                 if (persistent_grids()) clusters = std::min<int64_t>(clusters, ncl);
                 return launch(fn, clusters * sg.cs, sg.threads, smem, sg.cs, st, p,
-                              static_cast<uint32_t>(stage_bytes), sg.slice, sg.chunk_vecs);
+                              static_cast<uint32_t>(stage_bytes), sg.slice, smem_row_nchunk(sg, dtype));
             }
             ClusterGeom g;
             if (!cluster_geom(p.nvec, dtype, threads, cluster, &g)) return FS_ERR_UNSUPPORTED;
@@ -599,7 +624,7 @@ struct StaticDevice {
     int smem_optin = 0;
     int cluster_ok = 0;
     int* scratch = nullptr;              // device address of fs_static_scratch on this device
-    bool configured[3][2] = {};          // split-row kernel variants whose attributes are set
+    bool configured[3][2][2] = {};       // split-row kernel variants whose attributes are set
 };
 StaticDevice g_static[kMaxDevices];
 std::mutex g_static_mu;
@@ -752,24 +777,24 @@ int fs_softmax_static(const void* x, void* y, int64_t rows, int64_t cols, int dt
     p.c = static_cast<float>(static_cast<double>(scale) * kLog2e);
     p.neg = p.c < 0.0f ? 1 : 0;
     p.status = sd.scratch;
-    const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) {
-        return (const void*)smem_row_kernel<decltype(dt)::value, decltype(ng)::value>; });
+    const void* fn = smem_row_fn(dtype, p.neg, sg, nvec);
     const size_t stage_bytes = static_cast<size_t>(sg.slice) * 16;
-    const size_t smem = stage_bytes + size_t(kSmemRowMaxChunks) * 8;
+    const size_t smem = smem_row_bytes(sg);
     if (smem > static_cast<size_t>(sd.smem_optin) - 2048) return FS_ERR_UNSUPPORTED;
-    if (!sd.configured[dtype][p.neg]) {
+    const bool full_variant = smem_row_full(sg, dtype, nvec);
+    if (!sd.configured[dtype][p.neg][full_variant]) {
         cudaFuncAttributes fa;
         FS_CUDA(cudaFuncGetAttributes(&fa, fn));
         FS_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      sd.smem_optin - static_cast<int>(fa.sharedSizeBytes)));
         FS_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
-        sd.configured[dtype][p.neg] = true;
+        sd.configured[dtype][p.neg][full_variant] = true;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // the array keeps whatever the last call left: the status word must start at zero
     FS_CUDA(cudaMemsetAsync(sd.scratch, 0, sizeof(int), st));
     return launch(fn, rows * sg.cs, sg.threads, smem, sg.cs, st, p,
-                  static_cast<uint32_t>(stage_bytes), sg.slice, sg.chunk_vecs);
+                  static_cast<uint32_t>(stage_bytes), sg.slice, smem_row_nchunk(sg, dtype));
 }
 
 int fs_last_cuda_error(void) { return t_last_cuda_error; }

@@ -271,18 +271,29 @@ __device__ __forceinline__ void bulk_load_row(uint32_t dst, const char* src, uin
     }
 }
 
-// Bounded wait on an mbarrier phase: at most 2^20 polls, each suspending for up to ~1 us, i.e.
-// about a second. Returns false (and records DEV_TIMEOUT) if the phase did not complete; the
-// caller carries on, skipping further waits, so that every block-wide and cluster-wide barrier is
-// still reached and the kernel ends.
+// Bounded wait on an mbarrier phase. A failed try_wait comes back after a short hardware-defined
+// time whatever hint it is given, and a lane that polls back to back burns issue slots the other
+// blocks on the SM need (measured: hundreds of instructions per wait). So the first polls are
+// immediate (later chunks of a row have usually landed) and the following ones are spaced by
+// nanosleep, doubling up to 256 ns. At most 2^23 polls, about two seconds. Returns false (and
+// records DEV_TIMEOUT) if the phase did not complete; the caller carries on, skipping further
+// waits, so that every block-wide and cluster-wide barrier is still reached and the kernel ends.
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done != 0;
+}
+
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status) {
-    for (int it = 0; it < (1 << 20); ++it) {
-        uint32_t done;
-        asm volatile("{\n\t.reg .pred p;\n\t"
-                     "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-                     "selp.u32 %0, 1, 0, p;\n\t}"
-                     : "=r"(done) : "r"(bar), "r"(parity), "r"(1000u) : "memory");
-        if (done) return true;
+    if (mbar_try(bar, parity)) return true;
+    unsigned ns = 32;
+    for (int it = 0; it < (1 << 23); ++it) {
+        __nanosleep(ns);
+        if (mbar_try(bar, parity)) return true;
+        if (ns < 256) ns <<= 1;
     }
     atomicOr(status, DEV_TIMEOUT);
     return false;

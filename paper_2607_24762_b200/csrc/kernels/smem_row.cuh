@@ -1,32 +1,51 @@
 // Split-row softmax with the slice resident in shared memory (long rows: vocabulary-sized, causal
 // attention rows). A row is split over the CS blocks of a thread-block cluster (CS = 1: one block
 // per row). Each block brings its slice into shared memory with bulk async copies, one mbarrier
-// per chunk, and makes two passes over it:
+// per chunk (a chunk = four vectors per thread), and makes two passes over it:
 //
-//   pass 1  as the chunks land: every thread keeps a running (r, s) pair over its vectors, the
-//           online-softmax update (Milakov-Gimelshein): a vector's own reference first, then
-//           s <- s 2^((r - r')c) + sum 2^((x - r')c)
+//   pass 1  as the chunks land: a thread takes its four vectors of the chunk, their reference r_c
+//           first (packed max), then e = 2^((x - r_c)c) for every element: one ex2 per element.
+//           The e are added (fp32, unrounded) to the thread's running (r, s) pair with the
+//           online-softmax merge (Milakov-Gimelshein), and written back IN PLACE over x in the
+//           element's own dtype; r_c stays in a register.
 //   merge   warp shuffles -> block (one __syncthreads) -> cluster: each block deposits its pair
 //           in every peer's shared memory with st.async, counted by an mbarrier there
-//   pass 2  y = 2^((x - R)c) / S from the resident slice, 128-bit streaming stores
+//   pass 2  y = e * 2^((r_c - R)c) / S from the resident slice: no second ex2 per element
+//
+// Storing e rounded to the output dtype costs no accuracy against the stated bar: for fp32 it is
+// exact; for bf16/fp16 it perturbs e, hence y, by at most half a unit in the last place of the
+// output format, so the rounded product can differ from the correctly rounded result by at most
+// one unit (the row sum is taken over the unrounded values).
 //
 // Registers stay low (no per-thread copy of the row), so occupancy is set by shared memory:
-// several blocks per SM in different phases keep HBM busy. Cost: two ex2 per element.
+// several blocks per SM in different phases keep HBM busy.
 #pragma once
 #include "block_row.cuh"
 #include "common.cuh"
 
 namespace fsm {
 
-constexpr int kSmemRowMaxChunks = 16;
+constexpr int kSmemRowMaxChunks = 8;
+// Vectors a thread takes from a chunk: 32 elements per step for every dtype.
+__host__ __device__ constexpr int smem_row_u(int dt) { return dt == DT_F32 ? 8 : 4; }
 
-// Dynamic shared memory: slice (stage_bytes) | kSmemRowMaxChunks chunk mbarriers.
-// chunk_vecs is a multiple of blockDim.x.
-template <int DT, bool NEG>
+__device__ __forceinline__ float ex2_ftz(float t) {
+    float r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(t));
+    return r;
+}
+
+// Dynamic shared memory: slice (stage_bytes) | kSmemRowMaxChunks chunk mbarriers |
+// per-thread chunk references (kSmemRowMaxChunks * blockDim.x floats).
+// The slice must fit in kSmemRowMaxChunks chunks of smem_row_u(DT) * blockDim.x vectors.
+// FULL: every block's slice is exactly nchunk_full chunks (no per-vector bounds checks, no
+// integer division in the prologue).
+// Rows cid, cid + clusters, ... are handled by cluster cid (normally exactly one row).
+template <int DT, bool NEG, bool FULL>
 __global__ void __launch_bounds__(512, 2)
-smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, const int chunk_vecs) {
+smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, const int nchunk_full) {
     constexpr int VE = Traits<DT>::VE;
-    constexpr int U = 4;                                  // vectors a thread handles per step
+    constexpr int U = smem_row_u(DT);
     pdl_launch_dependents();
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ float2 wp[2][32];
@@ -34,25 +53,32 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
     __shared__ __align__(8) uint64_t xbar[2];
     const int T = blockDim.x, tid = threadIdx.x, lane = tid & 31;
     const uint32_t q = cluster_ctarank(), cs = cluster_nctarank();
-    const int64_t ncl = cluster_count_x();
-    const int64_t cid = cluster_id_x();
-    const int nvec = static_cast<int>(p.nvec);
-    const int v0 = min(nvec, static_cast<int>(q) * slice);
-    const int nv = min(nvec, v0 + slice) - v0;            // vectors of this block's slice (may be 0)
-    const int nchunk = (nv + chunk_vecs - 1) / chunk_vecs;
+    const uint32_t ncl = cluster_count_x();
+    const uint32_t cid = cluster_id_x();
+    const int chunk_vecs = U * T;
+    int v0, nv, nchunk;
+    if (FULL) {
+        v0 = static_cast<int>(q) * slice; nv = slice; nchunk = nchunk_full;
+    } else {
+        const int nvec = static_cast<int>(p.nvec);
+        v0 = min(nvec, static_cast<int>(q) * slice);
+        nv = min(nvec, v0 + slice) - v0;                  // vectors of this block's slice (may be 0)
+        nchunk = (nv + chunk_vecs - 1) / chunk_vecs;
+    }
     const float ident = ref_identity<NEG>();
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + stage_bytes);
-    const uint4* sv = reinterpret_cast<const uint4*>(smem);
-    const char* xb = static_cast<const char*>(p.x);
-    uint4* __restrict__ yv = static_cast<uint4*>(p.y);
+    float* rcs = reinterpret_cast<float*>(smem + stage_bytes + kSmemRowMaxChunks * 8) + tid;   // [chunk][thread]
+    uint4* sv = reinterpret_cast<uint4*>(smem) + tid;
+    auto live = [&](int v) { return FULL || v < nv; };
+    const char* xb = static_cast<const char*>(p.x) + int64_t(v0) * 16;
+    uint4* __restrict__ yv = static_cast<uint4*>(p.y) + v0 + tid;
     const int64_t row_bytes = p.nvec * 16;
-    const int64_t n_my = cid < p.rows ? (p.rows - cid + ncl - 1) / ncl : 0;   // same for the whole cluster
 
     auto issue_row = [&](int64_t row) {                    // thread 0: one bulk copy per chunk
         for (int ch = 0; ch < nchunk; ++ch) {
-            const int cv = min(chunk_vecs, nv - ch * chunk_vecs);
+            const int cv = FULL ? chunk_vecs : min(chunk_vecs, nv - ch * chunk_vecs);
             bulk_load_row(smem_u32(smem) + uint32_t(ch) * uint32_t(chunk_vecs) * 16u,
-                          xb + row * row_bytes + (int64_t(v0) + int64_t(ch) * chunk_vecs) * 16,
+                          xb + row * row_bytes + int64_t(ch) * chunk_vecs * 16,
                           uint32_t(cv) * 16u, smem_u32(&bars[ch]));
         }
     };
@@ -64,7 +90,7 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
         mbar_fence_init();
         fence_proxy_async_smem();
         pdl_wait();
-        if (n_my > 0) issue_row(cid);
+        if (cid < p.rows) issue_row(cid);
     }
     __syncthreads();
     if (cs > 1) {   // peers are resident, their mbarriers initialised, before any remote deposit
@@ -74,77 +100,93 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
     pdl_wait();
 
     bool alive = true;      // false once a bounded wait has expired: later waits are skipped
-    for (int64_t i = 0; i < n_my; ++i) {
-        const int64_t row = cid + i * ncl;
-        const int par = static_cast<int>(i & 1);
-        const uint32_t phase = static_cast<uint32_t>(i) & 1u;
+    uint32_t it = 0;
+    for (int64_t row = cid; row < p.rows; row += ncl, ++it) {   // the same trip count for the whole cluster
+        const int par = static_cast<int>(it & 1u);
+        const uint32_t phase = it & 1u;
         if (cs > 1 && tid == 0) mbar_expect_tx(smem_u32(&xbar[par]), cs * 8u);
 
-        // ---- pass 1: running (r, s) over this thread's vectors, chunk by chunk as they land.
-        // A chunk gives a thread U vectors: their common reference first, one rescale of s, then
-        // one ex2 per element.
+        // ---- pass 1
         float r = ident, s = 0.0f;
         for (int ch = 0; ch < nchunk; ++ch) {
-            if (alive) alive = mbar_wait_warp(smem_u32(&bars[ch]), phase, p.status);
-            const int cbeg = ch * chunk_vecs, cend = min(nv, cbeg + chunk_vecs);
-            for (int v0c = cbeg + tid; v0c < cend; v0c += U * T) {
-                uint4 raw[U];
-                RefAcc<DT, NEG> acc;
-                acc.init();
+            // warp 0 polls, the other warps wait at the hardware barrier (no issue slots spent)
+            if (tid < 32 && alive) alive = mbar_wait_warp(smem_u32(&bars[ch]), phase, p.status);
+            if (T > 32) __syncthreads();
+            uint4* sc = sv + ch * chunk_vecs;
+            uint4 raw[U];
+            RefAcc<DT, NEG> acc;
+            acc.init();
 #pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    raw[u] = make_uint4(0u, 0u, 0u, 0u);
-                    if (v0c + u * T < cend) { raw[u] = sv[v0c + u * T]; acc.fold(raw[u]); }
-                }
-                const float rn = ref_pick<NEG>(r, acc.value());
-                if (rn != r) { s *= ref_factor(r, rn, p.c, ident); r = rn; }
-                const float ru = (rn == ident) ? 0.0f : rn;
-                float part = 0.0f;
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    if (v0c + u * T < cend) {
-                        float e[VE];
-                        unpack<DT>(raw[u], e);
-#pragma unroll
-                        for (int k = 0; k < VE; ++k) part += ex2_elem<DT>(e[k] - ru, p.c);
-                    }
-                }
-                s += part;
+            for (int u = 0; u < U; ++u) {
+                if (live(ch * chunk_vecs + tid + u * T)) { raw[u] = sc[u * T]; acc.fold(raw[u]); }
             }
+            const float rc = acc.value();
+            rcs[ch * T] = rc;
+            // all of these elements masked (or none): subtract 0 instead of the identity
+            const float ru = (rc == ident) ? 0.0f : rc;
+            float part = 0.0f;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (live(ch * chunk_vecs + tid + u * T)) {
+                    float e[VE];
+                    unpack<DT>(raw[u], e);
+#pragma unroll
+                    for (int k = 0; k < VE; ++k) { e[k] = ex2_elem<DT>(e[k] - ru, p.c); part += e[k]; }
+                    sc[u * T] = pack<DT>(e);
+                }
+            }
+            // online merge of (rc, part) into (r, s): only the reference left behind is rescaled
+            const float rn = ref_pick<NEG>(r, rc);
+            const bool keep = (rn == r);
+            const float lo = keep ? rc : r;
+            const float f = (lo == ident) ? 1.0f : ex2_ftz((lo - rn) * p.c);
+            s = keep ? fmaf(part, f, s) : fmaf(s, f, part);
+            r = rn;
         }
         float R = r;
         block_merge_pairs<NEG>(R, s, wp[par], p.c);
         if (cs > 1) {
             if (tid < cs)
                 st_async_v2(map_to_rank(smem_u32(&xchg[par][q]), tid), R, s, map_to_rank(smem_u32(&xbar[par]), tid));
-            if (alive) alive = mbar_wait_warp(smem_u32(&xbar[par]), static_cast<uint32_t>(i >> 1) & 1u, p.status);
+            if (tid < 32 && alive) alive = mbar_wait_warp(smem_u32(&xbar[par]), (it >> 1) & 1u, p.status);
+            if (T > 32) __syncthreads();
             R = ident; s = 0.0f;
             if (lane < static_cast<int>(cs)) ld_shared_v2(smem_u32(&xchg[par][lane]), R, s);
             warp_merge_pairs<NEG>(R, s, p.c);
         }
 
-        // ---- pass 2: normalise from the resident slice
+        // ---- pass 2: scale the stored e, chunk by chunk with the chunk's own reference
         const float inv = recip<DT>(s);
-        const float Ru = (R == ident) ? 0.0f : R;
-        uint4* yrow = yv + row * p.nvec + v0;
-        for (int vb = tid; vb < nv; vb += U * T) {
+        uint4* yrow = yv + row * p.nvec;
+        for (int ch = 0; ch < nchunk; ++ch) {
+            const uint4* sc = sv + ch * chunk_vecs;
+            const float rc = rcs[ch * T];
+            const float fac = (rc == ident) ? 1.0f : ex2_noflush((rc - R) * p.c);
+            // bf16: e carries 2^64 and inv 2^-64; a factor this small is applied separately so
+            // that fac * inv cannot underflow before it meets e
+            const bool one_mul = DT != DT_BF16 || fac >= 0x1p-40f || !(fac == fac);
+            const float f1 = one_mul ? fac * inv : inv;
             uint4 raw[U];
 #pragma unroll
             for (int u = 0; u < U; ++u)
-                if (vb + u * T < nv) raw[u] = sv[vb + u * T];
+                if (live(ch * chunk_vecs + tid + u * T)) raw[u] = sc[u * T];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                if (vb + u * T < nv) {
+                if (live(ch * chunk_vecs + tid + u * T)) {
                     float e[VE];
                     unpack<DT>(raw[u], e);
 #pragma unroll
-                    for (int k = 0; k < VE; ++k) e[k] = ex2_elem<DT>(e[k] - Ru, p.c) * inv;
-                    st_stream(yrow + vb + u * T, pack<DT>(e));
+                    for (int k = 0; k < VE; ++k) e[k] *= f1;
+                    if (!one_mul) {
+#pragma unroll
+                        for (int k = 0; k < VE; ++k) e[k] *= fac;
+                    }
+                    st_stream(yrow + ch * chunk_vecs + u * T, pack<DT>(e));
                 }
             }
         }
 
-        if (i + 1 < n_my) {     // resident-grid form: the slice is free once everyone has read it
+        if (row + ncl < p.rows) {     // resident-grid form: the slice is free once everyone has read it
             __syncthreads();
             if (tid == 0) { fence_proxy_async_smem(); issue_row(row + ncl); }
         }

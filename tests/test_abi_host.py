@@ -99,7 +99,8 @@ def test_dispatcher_table(lib):
     assert k(32768, 32768, F32) in (fs.FS_KERNEL_CLUSTER, fs.FS_KERNEL_BLOCK_TMA)
     # mid-size rows take a block-per-row kernel
     assert k(100, 8192, F32) in (fs.FS_KERNEL_BLOCK, fs.FS_KERNEL_BLOCK_TMA)
-    assert k(100, 8192, F16) in (fs.FS_KERNEL_BLOCK, fs.FS_KERNEL_BLOCK_TMA)
+    assert k(100, 4096, F16) in (fs.FS_KERNEL_BLOCK, fs.FS_KERNEL_BLOCK_TMA)
+    assert k(100, 8192, F16) == fs.FS_KERNEL_CLUSTER        # one block per row, row resident in shared memory
     # ragged rows or misaligned bases take the generic kernel
     assert k(10, 1001, BF16) == fs.FS_KERNEL_GENERIC
     assert k(10, 1023, F32) == fs.FS_KERNEL_GENERIC
