@@ -242,7 +242,7 @@ def time_e2e(w: W.Workload, steps: int, warmup: int):
     fs.fs_release()
     return {"value": round(2 * nbytes / dt / 1e9, 2), "unit": UNIT, "ms_per_step": round(dt * 1e3, 4),
             "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": nbytes,
-            "api": "fs_softmax_host (pinned host buffers, 16 MiB chunks pipelined over 3 streams)"}
+            "api": "fs_softmax_host (pinned host buffers, 8 MiB chunks pipelined over copy-in, kernel and copy-out streams)"}
 
 
 # ---------------------------------------------------------------------------------------------

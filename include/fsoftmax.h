@@ -89,9 +89,10 @@ int fs_select_kernel(int64_t rows, int64_t cols, int dtype, int x_align, int y_a
 /*
  * fs_softmax_host -- the same operation on HOST buffers, end to end.
  *   x_host, y_host  host pointers (pinned memory gives full copy bandwidth; pageable works).
- * Splits the rows into chunks and pipelines host->device copy, kernel and device->host copy on
- * internal streams through device staging buffers the library allocates on first use and keeps
- * (grown on demand, released by fs_release). Blocks until y_host is complete.
+ * Splits the rows into chunks of about 8 MiB and pipelines host->device copy, kernel and
+ * device->host copy on three internal streams through four pairs of device staging buffers the
+ * library allocates on first use and keeps (grown on demand, released by fs_release). Blocks until
+ * y_host is complete. Calls on one device are serialised.
  */
 int fs_softmax_host(const void* x_host, void* y_host, int64_t rows, int64_t cols, int dtype, float scale);
 

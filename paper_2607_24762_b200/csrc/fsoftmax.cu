@@ -53,8 +53,9 @@ struct Device {
     std::unordered_map<uint64_t, LaunchInfo> launch_cache;
     std::unordered_map<const void*, bool> configured;   // kernels whose function attributes are set
     // fs_softmax_host staging
-    static constexpr int kSlots = 3;
-    cudaStream_t streams[kSlots] = {};
+    static constexpr int kSlots = 4;
+    cudaStream_t s_in = nullptr, s_run = nullptr, s_out = nullptr;   // copy-in, kernels, copy-out
+    cudaEvent_t ev_in[kSlots] = {}, ev_run[kSlots] = {}, ev_out[kSlots] = {};
     void* dx[kSlots] = {};
     void* dy[kSlots] = {};
     size_t slot_bytes = 0;
@@ -683,7 +684,11 @@ int fs_softmax_host(const void* x_host, void* y_host, int64_t rows, int64_t cols
     std::lock_guard<std::mutex> lk(g_host_mu);
 
     const size_t row_bytes = static_cast<size_t>(cols) * elem_size(dtype);
-    const size_t target = size_t(16) << 20;                       // ~16 MiB per chunk
+    // chunk size: small enough that filling and draining the pipeline costs little, large enough
+    // that the ~10 runtime calls per chunk (20 us of host time) stay hidden behind the copies;
+    // 8 MiB measured best on PCIe Gen5 (FS_HOST_CHUNK_MB overrides, for tuning)
+    static const size_t chunk_mb = [] { const char* e = std::getenv("FS_HOST_CHUNK_MB"); int v = e ? std::atoi(e) : 0; return size_t(v > 0 ? v : 8); }();
+    const size_t target = chunk_mb << 20;
     int64_t chunk_rows = std::max<int64_t>(1, static_cast<int64_t>(target / row_bytes));
     chunk_rows = std::min<int64_t>(chunk_rows, rows);
     const size_t need = (static_cast<size_t>(chunk_rows) * row_bytes + 255) / 256 * 256;
@@ -700,24 +705,43 @@ int fs_softmax_host(const void* x_host, void* y_host, int64_t rows, int64_t cols
         }
         dev.slot_bytes = need;
     }
-    for (int s = 0; s < Device::kSlots; ++s)
-        if (!dev.streams[s]) FS_CUDA(cudaStreamCreateWithFlags(&dev.streams[s], cudaStreamNonBlocking));
+    if (!dev.s_in) {
+        FS_CUDA(cudaStreamCreateWithFlags(&dev.s_in, cudaStreamNonBlocking));
+        FS_CUDA(cudaStreamCreateWithFlags(&dev.s_run, cudaStreamNonBlocking));
+        FS_CUDA(cudaStreamCreateWithFlags(&dev.s_out, cudaStreamNonBlocking));
+        for (int s = 0; s < Device::kSlots; ++s) {
+            FS_CUDA(cudaEventCreateWithFlags(&dev.ev_in[s], cudaEventDisableTiming));
+            FS_CUDA(cudaEventCreateWithFlags(&dev.ev_run[s], cudaEventDisableTiming));
+            FS_CUDA(cudaEventCreateWithFlags(&dev.ev_out[s], cudaEventDisableTiming));
+        }
+    }
 
-    // Each slot's stream runs copy-in -> kernel -> copy-out for its chunk; the slots overlap one
-    // another, so the two copy engines and the SMs work at the same time.
+    // Three streams, one per stage: copies in run back to back on the host-to-device engine,
+    // kernels on the SMs, copies out on the device-to-host engine. Events hand a slot from stage
+    // to stage and back (a slot's input buffer is free once its kernel ran, its output buffer once
+    // it was copied out), so the stages overlap across chunks.
     const char* xin = static_cast<const char*>(x_host);
     char* yout = static_cast<char*>(y_host);
     int slot = 0;
-    for (int64_t r0 = 0; r0 < rows; r0 += chunk_rows, slot = (slot + 1) % Device::kSlots) {
+    int64_t chunk = 0;
+    for (int64_t r0 = 0; r0 < rows; r0 += chunk_rows, slot = (slot + 1) % Device::kSlots, ++chunk) {
         const int64_t nr = std::min<int64_t>(chunk_rows, rows - r0);
         const size_t bytes = static_cast<size_t>(nr) * row_bytes;
-        cudaStream_t st = dev.streams[slot];
-        FS_CUDA(cudaMemcpyAsync(dev.dx[slot], xin + static_cast<size_t>(r0) * row_bytes, bytes, cudaMemcpyHostToDevice, st));
-        rc = run(dev.dx[slot], dev.dy[slot], nr, cols, dtype, scale, st, FS_KERNEL_AUTO, 0, 0);
+        if (chunk >= Device::kSlots) FS_CUDA(cudaStreamWaitEvent(dev.s_in, dev.ev_run[slot], 0));
+        FS_CUDA(cudaMemcpyAsync(dev.dx[slot], xin + static_cast<size_t>(r0) * row_bytes, bytes, cudaMemcpyHostToDevice, dev.s_in));
+        FS_CUDA(cudaEventRecord(dev.ev_in[slot], dev.s_in));
+        FS_CUDA(cudaStreamWaitEvent(dev.s_run, dev.ev_in[slot], 0));
+        if (chunk >= Device::kSlots) FS_CUDA(cudaStreamWaitEvent(dev.s_run, dev.ev_out[slot], 0));
+        rc = run(dev.dx[slot], dev.dy[slot], nr, cols, dtype, scale, dev.s_run, FS_KERNEL_AUTO, 0, 0);
         if (rc != FS_OK) return rc;
-        FS_CUDA(cudaMemcpyAsync(yout + static_cast<size_t>(r0) * row_bytes, dev.dy[slot], bytes, cudaMemcpyDeviceToHost, st));
+        FS_CUDA(cudaEventRecord(dev.ev_run[slot], dev.s_run));
+        FS_CUDA(cudaStreamWaitEvent(dev.s_out, dev.ev_run[slot], 0));
+        FS_CUDA(cudaMemcpyAsync(yout + static_cast<size_t>(r0) * row_bytes, dev.dy[slot], bytes, cudaMemcpyDeviceToHost, dev.s_out));
+        FS_CUDA(cudaEventRecord(dev.ev_out[slot], dev.s_out));
     }
-    for (int s = 0; s < Device::kSlots; ++s) FS_CUDA(cudaStreamSynchronize(dev.streams[s]));
+    FS_CUDA(cudaStreamSynchronize(dev.s_out));
+    FS_CUDA(cudaStreamSynchronize(dev.s_run));
+    FS_CUDA(cudaStreamSynchronize(dev.s_in));
     return FS_OK;
 }
 
@@ -727,8 +751,14 @@ int fs_release(void) {
     if (d < 0 || d >= kMaxDevices) return FS_ERR_UNSUPPORTED;
     std::lock_guard<std::mutex> lk(g_host_mu);
     Device& dev = g_dev[d];
+    cudaStream_t* streams[3] = {&dev.s_in, &dev.s_run, &dev.s_out};
+    for (cudaStream_t* st : streams) {
+        if (*st) { FS_CUDA(cudaStreamSynchronize(*st)); FS_CUDA(cudaStreamDestroy(*st)); *st = nullptr; }
+    }
     for (int s = 0; s < Device::kSlots; ++s) {
-        if (dev.streams[s]) { FS_CUDA(cudaStreamSynchronize(dev.streams[s])); FS_CUDA(cudaStreamDestroy(dev.streams[s])); dev.streams[s] = nullptr; }
+        if (dev.ev_in[s]) { FS_CUDA(cudaEventDestroy(dev.ev_in[s])); dev.ev_in[s] = nullptr; }
+        if (dev.ev_run[s]) { FS_CUDA(cudaEventDestroy(dev.ev_run[s])); dev.ev_run[s] = nullptr; }
+        if (dev.ev_out[s]) { FS_CUDA(cudaEventDestroy(dev.ev_out[s])); dev.ev_out[s] = nullptr; }
         if (dev.dx[s]) { FS_CUDA(cudaFree(dev.dx[s])); dev.dx[s] = nullptr; }
         if (dev.dy[s]) { FS_CUDA(cudaFree(dev.dy[s])); dev.dy[s] = nullptr; }
     }
