@@ -400,12 +400,9 @@ def main():
     l2 = int(getattr(props, "L2_cache_size", 126 << 20))
     sampler = ClockSampler(smi_id(props, local_rank)) if rank == 0 and not args.no_clocks else None
     res = time_device(w, args.steps, args.warmup, l2, sampler=sampler, barrier=barrier, min_clock_samples=8)
-    ms = res["ms_per_step"]
-    if dist:
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    value = world * w.min_bytes / (ms * 1e-3) / 1e9
+    from paper_2607_24762_b200 import sharding
+    ms = sharding.max_over_ranks(res["ms_per_step"], device="cuda")          # as slow as the slowest rank
+    value = sharding.aggregate_throughput(w.min_bytes, ms * 1e-3, world) / 1e9
 
     line = {"metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": round(ms, 6), "higher_is_better": True, "scaling": "weak",
