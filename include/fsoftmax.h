@@ -35,6 +35,9 @@ extern "C" {
 
 typedef enum { FS_DTYPE_FP32 = 0, FS_DTYPE_BF16 = 1, FS_DTYPE_FP16 = 2 } fs_dtype;
 
+/* Longest row (bytes) the split-row kernel holds in the shared memory of a 16-block cluster. */
+#define FS_STATIC_MAX_ROW_BYTES (16 * 192 * 1024)
+
 typedef enum {
     FS_OK = 0,
     FS_ERR_INVALID_ARG = 1,    /* null pointer, negative size, unknown dtype/kernel, non-finite scale, partial overlap */
@@ -77,6 +80,27 @@ int fs_softmax(const void* x, void* y, int64_t rows, int64_t cols, int dtype, fl
  */
 int fs_softmax_ex(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale,
                   void* stream, int kernel, int threads, int cluster);
+
+/*
+ * fs_softmax_causal -- softmax with the causal mask of eager attention applied inside the kernel
+ * (the operator fusion the paper lists among its levers, Sec. II-B; the workloads are the
+ * eager-attention softmax calls of its Table I). Row i keeps columns j <= i + q_offset:
+ *
+ *     y[i][j] = softmax over the kept columns of scale * x[i][.]   for j <= i + q_offset
+ *     y[i][j] = +0                                                   for j >  i + q_offset
+ *
+ * i.e. what fs_softmax returns when every masked x[i][j] holds -inf (for scale > 0), except that
+ * masked inputs are never read, so they may hold anything, and only the kept part of x crosses the
+ * memory bus. q_offset = 0 is the square case (row i sees columns 0..i), q_offset = cols - rows
+ * aligns the last row with the last column (decoding with a key/value cache); q_offset >= cols - 1
+ * masks nothing. A row with no kept column (i + q_offset < 0) is all NaN, like an all -inf row,
+ * and a row made NaN by a kept NaN or +inf is NaN in its masked part too.
+ *   x, y, rows, cols, dtype, scale, stream   as for fs_softmax (x == y allowed).
+ * Vector-aligned tensors with rows up to FS_STATIC_MAX_ROW_BYTES run the split-row kernel, one
+ * cluster per row; everything else the generic kernel.
+ */
+int fs_softmax_causal(const void* x, void* y, int64_t rows, int64_t cols, int64_t q_offset, int dtype, float scale,
+                      void* stream);
 
 /*
  * fs_select_kernel -- the dispatcher's decision, without a launch (no CUDA call is made when the
@@ -128,8 +152,9 @@ int fs_device_status(void);
  *   x, y, rows, cols, dtype, scale, stream   as for fs_softmax; x and y are DEVICE pointers.
  *   Limits: x and y 16-byte aligned, row size a multiple of 16 bytes and at most
  *           FS_STATIC_MAX_ROW_BYTES (what 16 blocks hold in shared memory), rows * blocks-per-row
- *           below 2^31. Anything else returns FS_ERR_UNSUPPORTED and enqueues nothing; there is no
- *           silent switch to another kernel.
+ *           below 2^31; scale == 0 only for rows that split into whole chunks (powers of two do).
+ *           Anything else returns FS_ERR_UNSUPPORTED and enqueues nothing; there is no silent
+ *           switch to another kernel.
  *   First call on a device: looks up the array's device address and raises the kernel's
  *           shared-memory limit (queries and attribute calls, no allocation). Make that first call
  *           before starting any stream capture.
@@ -139,7 +164,6 @@ int fs_device_status(void);
  *           on that word: results stay correct, but an expired wait may go unrecorded.
  *           fs_device_status does not read this word.
  */
-#define FS_STATIC_MAX_ROW_BYTES (16 * 200 * 1024)
 int fs_softmax_static(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale, void* stream);
 
 /* fs_release -- frees the staging buffers and streams fs_softmax_host created on the current device. */

@@ -72,6 +72,8 @@ def _load():
             lib.fso_softmax_f64.restype = None
             lib.fso_softmax_row_f64.argtypes = [vp, ci, i64, f32, vp]
             lib.fso_softmax_row_f64.restype = None
+            lib.fso_softmax_causal_f64.argtypes = [vp, ci, i64, i64, i64, f32, vp]
+            lib.fso_softmax_causal_f64.restype = None
             lib.fso_widen.argtypes = [vp, ci, i64, vp]
             lib.fso_widen.restype = None
             lib.fso_round_from_f64.argtypes = [vp, ci, i64, vp]
@@ -100,6 +102,18 @@ def softmax_f64(x: np.ndarray, dtype: int, scale: float = 1.0) -> np.ndarray:
     y = np.empty((rows, cols), dtype=np.float64)
     if rows and cols:
         _load().fso_softmax_f64(x.ctypes.data, dtype, rows, cols, np.float32(scale), y.ctypes.data)
+    return y
+
+
+def softmax_causal_f64(x: np.ndarray, dtype: int, q_offset: int, scale: float = 1.0) -> np.ndarray:
+    """fp64 causal softmax: row i keeps columns j <= i + q_offset; masked columns give exactly 0."""
+    x = _stored(x, dtype)
+    if x.ndim != 2:
+        raise ValueError("x must be [rows, cols]")
+    rows, cols = x.shape
+    y = np.empty((rows, cols), dtype=np.float64)
+    if rows and cols:
+        _load().fso_softmax_causal_f64(x.ctypes.data, dtype, rows, cols, q_offset, np.float32(scale), y.ctypes.data)
     return y
 
 

@@ -161,6 +161,29 @@ void fso_softmax_f64(const void* x, int dtype, int64_t rows, int64_t cols, float
     }
 }
 
+// Causal variant (the mask eager attention applies before its softmax; fusing it is the "operator
+// fusion" lever of the paper's Sec. II-B): row i keeps columns j <= i + q_offset and the softmax is
+// taken over the kept columns only; a masked column has z = -inf, i.e. y = exactly +0, whatever is
+// stored there (it is never read). A row with no kept column is all NaN, like any row whose
+// entries are all -inf; a row that a kept NaN or +inf makes NaN is NaN in its masked part too.
+void fso_softmax_causal_f64(const void* x, int dtype, int64_t rows, int64_t cols, int64_t q_offset,
+                            float scale, double* y) {
+    const int64_t esz = (dtype == DT_FP32) ? 4 : 2;
+    for (int64_t i = 0; i < rows; ++i) {
+        int64_t keep = i + q_offset + 1;                  // number of leading columns kept
+        if (keep < 0) keep = 0;
+        if (keep > cols) keep = cols;
+        double* yr = y + i * cols;
+        if (keep == 0) {
+            for (int64_t j = 0; j < cols; ++j) yr[j] = std::numeric_limits<double>::quiet_NaN();
+            continue;
+        }
+        fso_softmax_row_f64(static_cast<const char*>(x) + i * cols * esz, dtype, keep, scale, yr);
+        // literally 0 / S: +0, or NaN when a kept NaN or +inf has made the row NaN
+        for (int64_t j = keep; j < cols; ++j) yr[j] = 0.0 * yr[0];
+    }
+}
+
 // Exact widening of stored elements (exposed so tests can pin the decoders).
 void fso_widen(const void* x, int dtype, int64_t n, double* out) {
     for (int64_t i = 0; i < n; ++i) out[i] = widen(x, dtype, i);

@@ -180,7 +180,7 @@ bool cluster_geom(int64_t nvec, int dtype, int threads, int cluster, ClusterGeom
 // Shared-memory-resident split: slices of about kClusterSliceBytes, up to kMaxCluster blocks; rows
 // beyond that grow the slice up to what one block's shared memory holds.
 struct SmemGeom { int cs, slice, threads; };
-constexpr int64_t kSmemSliceMaxBytes = 200 * 1024;
+constexpr int64_t kSmemSliceMaxBytes = 192 * 1024;
 bool smem_geom(int64_t nvec, int dtype, int threads, int cluster, SmemGeom* g) {
     if (nvec < 1) return false;
     int cs = cluster;
@@ -424,11 +424,15 @@ const void* smem_row_fn(int dtype, bool neg, const SmemGeom& g, int64_t nvec) {
     return by_variant(dtype, neg, [&](auto dt, auto ng) -> const void* {
         constexpr int DT = decltype(dt)::value;
         constexpr bool NG = decltype(ng)::value;
-        return full ? (const void*)smem_row_kernel<DT, NG, true> : (const void*)smem_row_kernel<DT, NG, false>;
+        return full ? (const void*)smem_row_kernel<DT, NG, true, false> : (const void*)smem_row_kernel<DT, NG, false, false>;
     });
 }
-size_t smem_row_bytes(const SmemGeom& g) {
-    return static_cast<size_t>(g.slice) * 16 + size_t(kSmemRowMaxChunks) * 8 + size_t(kSmemRowMaxChunks) * g.threads * 4;
+// slice rounded up to whole chunks | chunk mbarriers | per-thread chunk references
+size_t smem_row_stage_bytes(const SmemGeom& g, int dtype) {
+    return static_cast<size_t>(smem_row_nchunk(g, dtype)) * smem_row_u(dtype) * g.threads * 16;
+}
+size_t smem_row_bytes(const SmemGeom& g, int dtype) {
+    return smem_row_stage_bytes(g, dtype) + size_t(kSmemRowMaxChunks) * 8 + size_t(kSmemRowMaxChunks) * g.threads * 4;
 }
 
 // Shared-memory ring: as many stages as fit in `budget` bytes, between 2 and `max_stages`.
@@ -447,7 +451,8 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
 
     const int esz = elem_size(dtype);
     const bool fast = fast_path_ok(cols, dtype, ptr_align(x), ptr_align(y));
-    if (kernel == FS_KERNEL_AUTO) kernel = select_kernel(cols, dtype, ptr_align(x), ptr_align(y));
+    const bool was_auto = kernel == FS_KERNEL_AUTO;
+    if (was_auto) kernel = select_kernel(cols, dtype, ptr_align(x), ptr_align(y));
     if (kernel != FS_KERNEL_GENERIC && !fast) return FS_ERR_UNSUPPORTED;
     if (threads < 0 || threads % 32 || threads > 1024) return FS_ERR_INVALID_ARG;
 
@@ -457,6 +462,7 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
     p.c = static_cast<float>(static_cast<double>(scale) * kLog2e);
     p.neg = p.c < 0.0f ? 1 : 0;
     p.status = dev.status;
+    p.q_offset = 0;
     const int64_t max_grid = 0x7fffffff;
 
     switch (kernel) {
@@ -540,16 +546,23 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
             if (!dev.cluster_ok) return FS_ERR_UNSUPPORTED;
             SmemGeom sg;
             if (!cluster_uses_registers() && smem_geom(p.nvec, dtype, threads, cluster, &sg)) {
-                const void* fn = smem_row_fn(dtype, p.neg, sg, p.nvec);
-                const size_t stage_bytes = static_cast<size_t>(sg.slice) * 16;
-                const size_t smem = smem_row_bytes(sg);
-                if (smem > static_cast<size_t>(dev.smem_optin) - 2048) return FS_ERR_UNSUPPORTED;
-                int ncl = 0;
-                if ((rc = active_clusters(dev, fn, sg.threads, smem, sg.cs, &ncl)) != FS_OK) return rc;
-                int64_t clusters = std::min<int64_t>(rows, max_grid / sg.cs);
-                if (persistent_grids()) clusters = std::min<int64_t>(clusters, ncl);
-                return launch(fn, clusters * sg.cs, sg.threads, smem, sg.cs, st, p,
-                              static_cast<uint32_t>(stage_bytes), sg.slice, smem_row_nchunk(sg, dtype));
+                // a slice that is not a whole number of chunks is padded with -inf, which a zero
+                // scale would turn into NaN: that one case goes to the generic kernel
+                const bool zero_scale_ragged = p.c == 0.0f && !smem_row_full(sg, dtype, p.nvec);
+                if (zero_scale_ragged && !was_auto) return FS_ERR_UNSUPPORTED;
+                if (!zero_scale_ragged) {
+                    const void* fn = smem_row_fn(dtype, p.neg, sg, p.nvec);
+                    const size_t stage_bytes = smem_row_stage_bytes(sg, dtype);
+                    const size_t smem = smem_row_bytes(sg, dtype);
+                    if (smem > static_cast<size_t>(dev.smem_optin) - 2048) return FS_ERR_UNSUPPORTED;
+                    int ncl = 0;
+                    if ((rc = active_clusters(dev, fn, sg.threads, smem, sg.cs, &ncl)) != FS_OK) return rc;
+                    int64_t clusters = std::min<int64_t>(rows, max_grid / sg.cs);
+                    if (persistent_grids()) clusters = std::min<int64_t>(clusters, ncl);
+                    return launch(fn, clusters * sg.cs, sg.threads, smem, sg.cs, st, p,
+                                  static_cast<uint32_t>(stage_bytes), sg.slice, smem_row_nchunk(sg, dtype));
+                }
+                return run(x, y, rows, cols, dtype, scale, st, FS_KERNEL_GENERIC, 0, 0);
             }
             ClusterGeom g;
             if (!cluster_geom(p.nvec, dtype, threads, cluster, &g)) return FS_ERR_UNSUPPORTED;
@@ -574,7 +587,7 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
                           static_cast<uint32_t>(stage_bytes), g.slice);
         }
         case FS_KERNEL_GENERIC: {
-            const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) { return (const void*)generic_row_kernel<decltype(dt)::value, decltype(ng)::value>; });
+            const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) { return (const void*)generic_row_kernel<decltype(dt)::value, decltype(ng)::value, false>; });
             int t = threads;
             if (t == 0) {
                 t = 32;
@@ -586,6 +599,42 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
         default:
             return FS_ERR_INVALID_ARG;
     }
+}
+
+// Causal softmax: the split-row kernel (one cluster per row) when the tensors are vector-aligned
+// and the row fits its shared memory, the generic kernel otherwise.
+int run_causal(const void* x, void* y, int64_t rows, int64_t cols, int64_t q_offset, int dtype, float scale,
+               cudaStream_t st) {
+    Device* devp = nullptr;
+    int rc = get_device(&devp);
+    if (rc != FS_OK) return rc;
+    Device& dev = *devp;
+    const int esz = elem_size(dtype);
+    const bool fast = fast_path_ok(cols, dtype, ptr_align(x), ptr_align(y));
+    Params p;
+    p.x = x; p.y = y; p.rows = rows; p.cols = cols;
+    p.nvec = fast ? cols * esz / 16 : 0;
+    p.c = static_cast<float>(static_cast<double>(scale) * kLog2e);
+    p.neg = p.c < 0.0f ? 1 : 0;
+    p.status = dev.status;
+    p.q_offset = q_offset;
+    SmemGeom sg;
+    // (a zero scale goes to the generic kernel: the split kernel masks with -inf, and 0 * -inf is NaN)
+    if (fast && p.c != 0.0f && dev.cluster_ok && smem_geom(p.nvec, dtype, 0, 0, &sg) && rows <= 0x7fffffff / sg.cs) {
+        const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) -> const void* {
+            return (const void*)smem_row_kernel<decltype(dt)::value, decltype(ng)::value, false, true>; });
+        const size_t smem = smem_row_bytes(sg, dtype);
+        if (smem <= static_cast<size_t>(dev.smem_optin) - 2048) {
+            if ((rc = configure_kernel(dev, fn, true, true)) != FS_OK) return rc;
+            return launch(fn, rows * sg.cs, sg.threads, smem, sg.cs, st, p,
+                          static_cast<uint32_t>(smem_row_stage_bytes(sg, dtype)), sg.slice, smem_row_nchunk(sg, dtype));
+        }
+    }
+    const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) -> const void* {
+        return (const void*)generic_row_kernel<decltype(dt)::value, decltype(ng)::value, true>; });
+    int t = 32;
+    while (t < 1024 && cols > int64_t(t) * 8) t <<= 1;
+    return launch(fn, std::min<int64_t>(rows, 0x7fffffff), t, 0, 0, st, p);
 }
 
 int validate(const void* x, const void* y, int64_t rows, int64_t cols, int dtype, float scale) {
@@ -650,6 +699,15 @@ int fs_softmax_ex(const void* x, void* y, int64_t rows, int64_t cols, int dtype,
 
 int fs_softmax(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale, void* stream) {
     return fs_softmax_ex(x, y, rows, cols, dtype, scale, stream, FS_KERNEL_AUTO, 0, 0);
+}
+
+int fs_softmax_causal(const void* x, void* y, int64_t rows, int64_t cols, int64_t q_offset, int dtype, float scale,
+                      void* stream) {
+    const int v = validate(x, y, rows, cols, dtype, scale);
+    if (v != FS_OK) return v;
+    if (rows == 0 || cols == 0) return FS_OK;
+    if (q_offset > (int64_t(1) << 41) || q_offset < -(int64_t(1) << 41)) return FS_ERR_INVALID_ARG;
+    return run_causal(x, y, rows, cols, q_offset, dtype, scale, static_cast<cudaStream_t>(stream));
 }
 
 int fs_select_kernel(int64_t rows, int64_t cols, int dtype, int x_align, int y_align) {
@@ -807,10 +865,12 @@ int fs_softmax_static(const void* x, void* y, int64_t rows, int64_t cols, int dt
     p.c = static_cast<float>(static_cast<double>(scale) * kLog2e);
     p.neg = p.c < 0.0f ? 1 : 0;
     p.status = sd.scratch;
+    p.q_offset = 0;
     const void* fn = smem_row_fn(dtype, p.neg, sg, nvec);
-    const size_t stage_bytes = static_cast<size_t>(sg.slice) * 16;
-    const size_t smem = smem_row_bytes(sg);
+    const size_t stage_bytes = smem_row_stage_bytes(sg, dtype);
+    const size_t smem = smem_row_bytes(sg, dtype);
     if (smem > static_cast<size_t>(sd.smem_optin) - 2048) return FS_ERR_UNSUPPORTED;
+    if (p.c == 0.0f && !smem_row_full(sg, dtype, nvec)) return FS_ERR_UNSUPPORTED;   // see the header
     const bool full_variant = smem_row_full(sg, dtype, nvec);
     if (!sd.configured[dtype][p.neg][full_variant]) {
         cudaFuncAttributes fa;

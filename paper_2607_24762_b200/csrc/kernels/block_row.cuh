@@ -290,7 +290,7 @@ cluster_row_kernel(const Params p, const int nstage, const uint32_t stage_bytes,
 // generic: any cols, any alignment, element-wise accesses; reads the row twice (the second read
 // normally hits L2). Pass 1 keeps a running (r, s) per thread -- the online update itself.
 // ---------------------------------------------------------------------------------------------
-template <int DT, bool NEG>
+template <int DT, bool NEG, bool CAUSAL>
 __global__ void __launch_bounds__(1024, 1)
 generic_row_kernel(const Params p) {
     __shared__ float2 wp[2][32];
@@ -301,8 +301,10 @@ generic_row_kernel(const Params p) {
     int par = 0;
     for (int64_t row = blockIdx.x; row < p.rows; row += gridDim.x, par ^= 1) {
         const int64_t base = row * p.cols;
+        // causal: only the first `keep` columns enter; the rest is filled with 0 * (1/S)
+        const int64_t keep = CAUSAL ? max(int64_t(0), min(p.cols, row + p.q_offset + 1)) : p.cols;
         float r = ident, s = 0.0f;
-        for (int64_t j = tid; j < p.cols; j += T) {
+        for (int64_t j = tid; j < keep; j += T) {
             const float x = load_elem<DT>(p.x, base + j);
             const float rn = ref_pick<NEG>(r, x);
             const float ru = (rn == ident) ? 0.0f : rn;
@@ -312,9 +314,13 @@ generic_row_kernel(const Params p) {
         block_merge_pairs<NEG>(r, s, wp[par], p.c);
         const float ru = (r == ident) ? 0.0f : r;
         const float inv = 1.0f / s;
-        for (int64_t j = tid; j < p.cols; j += T) {
+        for (int64_t j = tid; j < keep; j += T) {
             const float x = load_elem<DT>(p.x, base + j);
             store_elem<DT>(p.y, base + j, ex2_noflush((x - ru) * p.c) * inv);
+        }
+        if (CAUSAL) {
+            const float fill = 0.0f * inv;
+            for (int64_t j = keep + tid; j < p.cols; j += T) store_elem<DT>(p.y, base + j, fill);
         }
     }
 }

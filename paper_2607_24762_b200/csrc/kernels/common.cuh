@@ -23,6 +23,7 @@ struct Params {
     float c;           // scale * log2(e): exponents are taken in base 2
     int neg;           // c < 0: the row reference is the minimum of x instead of the maximum (host-side dispatch)
     int* status;       // device status word
+    int64_t q_offset;  // causal kernels: row i keeps columns j <= i + q_offset
 };
 
 template <int DT> struct Traits;
@@ -49,6 +50,33 @@ __device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
     return v;
+}
+
+// One 32-bit word of reference identities (one fp32, or two 16-bit elements).
+template <int DT, bool NEG>
+__device__ __forceinline__ uint32_t ident_word() {
+    if constexpr (DT == DT_F32) return NEG ? 0x7f800000u : 0xff800000u;
+    else if constexpr (DT == DT_BF16) return NEG ? 0x7f807f80u : 0xff80ff80u;
+    else return NEG ? 0x7c007c00u : 0xfc00fc00u;
+}
+
+// Causal tail: keep the first `keep` elements (1 .. VE-1) of a vector, set the rest to the
+// reference identity (-inf, or +inf when the reference is a minimum) so that they drop out.
+template <int DT, bool NEG>
+__device__ __forceinline__ void mask_tail(uint4& v, int keep) {
+    uint32_t* w = reinterpret_cast<uint32_t*>(&v);
+    if constexpr (DT == DT_F32) {
+        const uint32_t id = NEG ? 0x7f800000u : 0xff800000u;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) if (k >= keep) w[k] = id;
+    } else {
+        const uint32_t id16 = (DT == DT_BF16) ? (NEG ? 0x7f80u : 0xff80u) : (NEG ? 0x7c00u : 0xfc00u);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            if (2 * k >= keep) w[k] = id16 | (id16 << 16);
+            else if (2 * k + 1 >= keep) w[k] = (w[k] & 0xffffu) | (id16 << 16);
+        }
+    }
 }
 
 // ---- dtype unpack / pack of one 16-byte vector ------------------------------------------------

@@ -35,13 +35,17 @@ __device__ __forceinline__ float ex2_ftz(float t) {
     return r;
 }
 
-// Dynamic shared memory: slice (stage_bytes) | kSmemRowMaxChunks chunk mbarriers |
-// per-thread chunk references (kSmemRowMaxChunks * blockDim.x floats).
+// Dynamic shared memory: slice rounded up to whole chunks (stage_bytes) | kSmemRowMaxChunks chunk
+// mbarriers | per-thread chunk references (kSmemRowMaxChunks * blockDim.x floats).
 // The slice must fit in kSmemRowMaxChunks chunks of smem_row_u(DT) * blockDim.x vectors.
 // FULL: every block's slice is exactly nchunk_full chunks (no per-vector bounds checks, no
 // integer division in the prologue).
 // Rows cid, cid + clusters, ... are handled by cluster cid (normally exactly one row).
-template <int DT, bool NEG, bool FULL>
+// CAUSAL (one cluster per row, not FULL): row i keeps its first min(cols, i + q_offset + 1)
+// columns; only those are fetched, the vector that straddles the boundary gets its masked lanes
+// replaced by the reference identity, and the rest of the row is filled with 0 * (1/S): +0, or NaN
+// for a row that is NaN or has no column left.
+template <int DT, bool NEG, bool FULL, bool CAUSAL>
 __global__ void __launch_bounds__(512, 2)
 smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, const int nchunk_full) {
     constexpr int VE = Traits<DT>::VE;
@@ -57,19 +61,30 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
     const uint32_t cid = cluster_id_x();
     const int chunk_vecs = U * T;
     int v0, nv, nchunk;
+    int nfill = 0;           // causal: masked vectors of this block's slice, to be filled
+    int tail_at = -1;        // causal: local index of the vector that straddles the boundary
+    int tail_keep = 0;       //         and how many of its elements are kept
     if (FULL) {
         v0 = static_cast<int>(q) * slice; nv = slice; nchunk = nchunk_full;
     } else {
         const int nvec = static_cast<int>(p.nvec);
         v0 = min(nvec, static_cast<int>(q) * slice);
         nv = min(nvec, v0 + slice) - v0;                  // vectors of this block's slice (may be 0)
+        if (CAUSAL) {
+            const int64_t keep = max(int64_t(0), min(p.cols, int64_t(cid) + p.q_offset + 1));
+            const int nvv = static_cast<int>((keep + VE - 1) / VE);        // vectors with a kept element
+            const int kept_here = max(0, min(nv, nvv - v0));
+            nfill = nv - kept_here;
+            nv = kept_here;
+            tail_keep = static_cast<int>(keep % VE);
+            if (tail_keep != 0 && nv > 0 && v0 + nv == nvv) tail_at = nv - 1;
+        }
         nchunk = (nv + chunk_vecs - 1) / chunk_vecs;
     }
     const float ident = ref_identity<NEG>();
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + stage_bytes);
     float* rcs = reinterpret_cast<float*>(smem + stage_bytes + kSmemRowMaxChunks * 8) + tid;   // [chunk][thread]
     uint4* sv = reinterpret_cast<uint4*>(smem) + tid;
-    auto live = [&](int v) { return FULL || v < nv; };
     const char* xb = static_cast<const char*>(p.x) + int64_t(v0) * 16;
     uint4* __restrict__ yv = static_cast<uint4*>(p.y) + v0 + tid;
     const int64_t row_bytes = p.nvec * 16;
@@ -99,6 +114,13 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
     }
     pdl_wait();
 
+    if (CAUSAL && nfill > 0 && cid < p.rows) {
+        // masked part of this block's slice: +0, written while the kept part is still on its way
+        const uint4 zv = make_uint4(0u, 0u, 0u, 0u);
+        uint4* yfill = yv - tid + int64_t(cid) * p.nvec;
+        for (int v = nv + tid; v < nv + nfill; v += T) st_stream(yfill + v, zv);
+    }
+
     bool alive = true;      // false once a bounded wait has expired: later waits are skipped
     uint32_t it = 0;
     for (int64_t row = cid; row < p.rows; row += ncl, ++it) {   // the same trip count for the whole cluster
@@ -113,13 +135,28 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
             if (tid < 32 && alive) alive = mbar_wait_warp(smem_u32(&bars[ch]), phase, p.status);
             if (T > 32) __syncthreads();
             uint4* sc = sv + ch * chunk_vecs;
+            const int cbase = ch * chunk_vecs + tid;
+            if (!FULL) {
+                // this thread's vectors of the chunk that lie past the slice's end become identity
+                // vectors, so that the arithmetic below needs no bounds (a zero scale, for which
+                // 2^(-inf * 0) is NaN, never reaches this variant: the host routes it elsewhere)
+                const uint32_t idw = ident_word<DT, NEG>();
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+                    if (cbase + u * T >= nv) sc[u * T] = make_uint4(idw, idw, idw, idw);
+            }
             uint4 raw[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) raw[u] = sc[u * T];
+            if (CAUSAL) {
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+                    if (cbase + u * T == tail_at) mask_tail<DT, NEG>(raw[u], tail_keep);
+            }
             RefAcc<DT, NEG> acc;
             acc.init();
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                if (live(ch * chunk_vecs + tid + u * T)) { raw[u] = sc[u * T]; acc.fold(raw[u]); }
-            }
+            for (int u = 0; u < U; ++u) acc.fold(raw[u]);
             const float rc = acc.value();
             rcs[ch * T] = rc;
             // all of these elements masked (or none): subtract 0 instead of the identity
@@ -127,13 +164,11 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
             float part = 0.0f;
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                if (live(ch * chunk_vecs + tid + u * T)) {
-                    float e[VE];
-                    unpack<DT>(raw[u], e);
+                float e[VE];
+                unpack<DT>(raw[u], e);
 #pragma unroll
-                    for (int k = 0; k < VE; ++k) { e[k] = ex2_elem<DT>(e[k] - ru, p.c); part += e[k]; }
-                    sc[u * T] = pack<DT>(e);
-                }
+                for (int k = 0; k < VE; ++k) { e[k] = ex2_elem<DT>(e[k] - ru, p.c); part += e[k]; }
+                sc[u * T] = pack<DT>(e);
             }
             // online merge of (rc, part) into (r, s): only the reference left behind is rescaled
             const float rn = ref_pick<NEG>(r, rc);
@@ -168,25 +203,32 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
             const float f1 = one_mul ? fac * inv : inv;
             uint4 raw[U];
 #pragma unroll
-            for (int u = 0; u < U; ++u)
-                if (live(ch * chunk_vecs + tid + u * T)) raw[u] = sc[u * T];
+            for (int u = 0; u < U; ++u) raw[u] = sc[u * T];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                if (live(ch * chunk_vecs + tid + u * T)) {
-                    float e[VE];
-                    unpack<DT>(raw[u], e);
+                float e[VE];
+                unpack<DT>(raw[u], e);
 #pragma unroll
-                    for (int k = 0; k < VE; ++k) e[k] *= f1;
-                    if (!one_mul) {
+                for (int k = 0; k < VE; ++k) e[k] *= f1;
+                if (!one_mul) {
 #pragma unroll
-                        for (int k = 0; k < VE; ++k) e[k] *= fac;
-                    }
-                    st_stream(yrow + ch * chunk_vecs + u * T, pack<DT>(e));
+                    for (int k = 0; k < VE; ++k) e[k] *= fac;
                 }
+                if (FULL || ch * chunk_vecs + tid + u * T < nv) st_stream(yrow + ch * chunk_vecs + u * T, pack<DT>(e));
             }
         }
 
-        if (row + ncl < p.rows) {     // resident-grid form: the slice is free once everyone has read it
+        if (CAUSAL && nfill > 0 && !(0.0f * inv == 0.0f)) {
+            // the masked part was filled with +0 up front; a row that turned out NaN (or kept no
+            // column: 1/S is infinite) owes it 0 * (1/S) = NaN instead
+            float z[VE];
+#pragma unroll
+            for (int k = 0; k < VE; ++k) z[k] = 0.0f * inv;
+            const uint4 zv = pack<DT>(z);
+            for (int v = nv + tid; v < nv + nfill; v += T) st_stream(yrow - tid + v, zv);
+        }
+
+        if (!CAUSAL && row + ncl < p.rows) {     // resident-grid form: the slice is free once everyone has read it
             __syncthreads();
             if (tid == 0) { fence_proxy_async_smem(); issue_row(row + ncl); }
         }

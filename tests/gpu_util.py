@@ -29,7 +29,8 @@ def guard_pattern(n: int, np_dtype) -> np.ndarray:
 
 
 def run_softmax(x: np.ndarray, dtype: int, scale: float = 1.0, kernel: int = fs.FS_KERNEL_AUTO, threads: int = 0,
-                cluster: int = 0, offset: int = 0, inplace: bool = False, stream=None, check_guards: bool = True):
+                cluster: int = 0, offset: int = 0, inplace: bool = False, stream=None, check_guards: bool = True,
+                causal_q=None):
     """Runs the library on a copy of x placed `offset` elements past a 256-byte aligned address,
     with guard bands around input and output. Returns (status, y as stored numpy array or None)."""
     rows, cols = x.shape
@@ -50,7 +51,10 @@ def run_softmax(x: np.ndarray, dtype: int, scale: float = 1.0, kernel: int = fs.
     xp = xd.data_ptr() + (GUARD + offset) * esz
     yp = yd.data_ptr() + (GUARD + offset) * esz
     s = stream if stream is not None else torch.cuda.current_stream()
-    status = fs.fs_softmax_status(xp, yp, rows, cols, dtype, scale, s, kernel, threads, cluster)
+    if causal_q is None:
+        status = fs.fs_softmax_status(xp, yp, rows, cols, dtype, scale, s, kernel, threads, cluster)
+    else:
+        status = fs.binding.lib().fs_softmax_causal(xp, yp, rows, cols, causal_q, dtype, scale, int(s.cuda_stream))
     torch.cuda.synchronize()
     if status != fs.FS_OK:
         return status, None

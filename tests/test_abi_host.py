@@ -53,6 +53,12 @@ def test_enums_match_header():
         assert getattr(fs, name) == int(value), name
 
 
+def test_constants_match_header():
+    text = open(HEADER).read()
+    m = re.search(r"#define FS_STATIC_MAX_ROW_BYTES \((\d+) \* (\d+) \* (\d+)\)", text)
+    assert m and int(m.group(1)) * int(m.group(2)) * int(m.group(3)) == fs.FS_STATIC_MAX_ROW_BYTES
+
+
 def test_strings(lib):
     assert fs.fs_strerror(fs.FS_OK) == "ok"
     assert "invalid" in fs.fs_strerror(fs.FS_ERR_INVALID_ARG)

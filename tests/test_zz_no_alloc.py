@@ -54,7 +54,7 @@ def test_static_entry_point_refuses_what_it_cannot_take():
     a = torch.zeros(1 << 22, dtype=torch.float32, device="cuda")
     b = torch.empty_like(a)
     s = torch.cuda.current_stream().cuda_stream
-    big_cols = (16 * 200 * 1024) // 4 + 4                                   # one vector past the limit
+    big_cols = fs.FS_STATIC_MAX_ROW_BYTES // 4 + 4                                   # one vector past the limit
     assert L.fs_softmax_static(a.data_ptr(), b.data_ptr(), 1, big_cols, fs.FS_DTYPE_FP32, 1.0, s) == fs.FS_ERR_UNSUPPORTED
     assert L.fs_softmax_static(a.data_ptr(), b.data_ptr(), 8, 1023, fs.FS_DTYPE_FP32, 1.0, s) == fs.FS_ERR_UNSUPPORTED
     assert L.fs_softmax_static(a.data_ptr() + 4, b.data_ptr(), 8, 1024, fs.FS_DTYPE_FP32, 1.0, s) == fs.FS_ERR_UNSUPPORTED
@@ -63,7 +63,7 @@ def test_static_entry_point_refuses_what_it_cannot_take():
     assert "unsupported" in fs.fs_strerror(fs.FS_ERR_UNSUPPORTED)
     torch.cuda.synchronize()
     # the largest row it does take
-    cols = (16 * 200 * 1024) // 4
+    cols = fs.FS_STATIC_MAX_ROW_BYTES // 4
     x = W.random_case(1, cols, W.FP32, seed=4, sigma=2.0)
     xd = np_to_torch_bits(x).cuda()
     yd = torch.empty_like(xd)
