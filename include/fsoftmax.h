@@ -52,8 +52,9 @@ typedef enum {
     FS_KERNEL_AUTO = 0,
     FS_KERNEL_WARP = 1,       /* (sub-)warp per row, row held in registers */
     FS_KERNEL_BLOCK = 2,      /* block per row, 128-bit global loads, row held in registers */
-    FS_KERNEL_BLOCK_TMA = 3,  /* block per row, rows prefetched into a shared-memory ring by bulk async copies */
-    FS_KERNEL_CLUSTER = 4,    /* thread-block cluster per row, (max,sum) pairs exchanged through distributed shared memory */
+    FS_KERNEL_BLOCK_TMA = 3,  /* block per row (or a tile of short rows per block) staged in shared memory by bulk async copies */
+    FS_KERNEL_CLUSTER = 4,    /* row split over a thread-block cluster of 1..16 blocks, slices resident in shared memory,
+                                 (max,sum) pairs exchanged through distributed shared memory */
     FS_KERNEL_GENERIC = 5     /* any cols, any alignment; reads the row twice */
 } fs_kernel;
 
