@@ -196,9 +196,9 @@ bool smem_geom(int64_t nvec, int dtype, int threads, int cluster, SmemGeom* g) {
     int t = threads;
     if (t == 0) {
         t = slice >= 256 ? split_threads(dtype) : 64;
-        while (t < 512 && slice > per_thread * t) t <<= 1;
+        while (t < 256 && slice > per_thread * t) t <<= 1;
     }
-    if (t % 32 || t > 512 || slice > per_thread * t) return false;
+    if (t % 32 || t > 256 || slice > per_thread * t) return false;
     g->cs = cs; g->slice = static_cast<int>(slice); g->threads = t;
     return true;
 }

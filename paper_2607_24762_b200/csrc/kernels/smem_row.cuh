@@ -26,8 +26,9 @@
 namespace fsm {
 
 constexpr int kSmemRowMaxChunks = 8;
-// Vectors a thread takes from a chunk: 32 elements per step for every dtype.
-__host__ __device__ constexpr int smem_row_u(int dt) { return dt == DT_F32 ? 8 : 4; }
+// Vectors a thread takes from a chunk: 8 (32 fp32 or 64 16-bit elements per step). With blocks of
+// at most 256 threads and a cap of 85 registers, three 256-thread or six 128-thread blocks fit an SM.
+__host__ __device__ constexpr int smem_row_u(int) { return 8; }
 
 __device__ __forceinline__ float ex2_ftz(float t) {
     float r;
@@ -46,7 +47,7 @@ __device__ __forceinline__ float ex2_ftz(float t) {
 // replaced by the reference identity, and the rest of the row is filled with 0 * (1/S): +0, or NaN
 // for a row that is NaN or has no column left.
 template <int DT, bool NEG, bool FULL, bool CAUSAL>
-__global__ void __launch_bounds__(512, 2)
+__global__ void __launch_bounds__(256, 3)
 smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, const int nchunk_full) {
     constexpr int VE = Traits<DT>::VE;
     constexpr int U = smem_row_u(DT);
