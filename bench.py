@@ -225,6 +225,43 @@ def time_device(w: W.Workload, steps: int, warmup: int, l2_bytes: int, sampler: 
     return {"ms_per_step": ms / steps, "n_pairs": n_pairs, "kernel": kernel, "clocks": clocks}
 
 
+def time_router(w: W.Workload, k: int, steps: int, warmup: int, l2_bytes: int):
+    """fs_router_topk on the router workload: reads x once, writes k weights and k columns per row."""
+    import torch
+
+    import paper_2607_24762_b200 as fs
+    alg = w.rows * w.cols * w.elem_size + w.rows * k * 8
+    n_pairs = int(max(1, min(16, math.ceil(4 * l2_bytes / alg))))
+    xs, _ = device_buffers(w, n_pairs, threads=min(8, os.cpu_count() or 1))
+    ws = [torch.empty((w.rows, k), dtype=torch.float32, device="cuda") for _ in range(n_pairs)]
+    ids = [torch.empty((w.rows, k), dtype=torch.int32, device="cuda") for _ in range(n_pairs)]
+    stream = torch.cuda.current_stream()
+    lib = fs.binding.lib()
+
+    def launch(i):
+        j = i % n_pairs
+        st = lib.fs_router_topk(xs[j].data_ptr(), ws[j].data_ptr(), ids[j].data_ptr(), w.rows, w.cols, k, w.dtype,
+                                w.scale_f32, 1, stream.cuda_stream)
+        if st != 0:
+            raise RuntimeError(fs.fs_strerror(st))
+
+    for i in range(max(3, warmup)):
+        launch(i)
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    start.record(stream)
+    for i in range(steps):
+        launch(i)
+    stop.record(stream)
+    torch.cuda.synchronize()
+    ms = start.elapsed_time(stop) / steps
+    peak, _ = measured_peak()
+    gbs = alg / (ms * 1e-3) / 1e9
+    return {"what": f"fs_router_topk(k={k}, renormalize) on cfg3: reads x, writes {k} weights + {k} columns per row",
+            "steps": steps, "ms_per_step": round(ms, 6), "algorithmic_bytes": alg, "GB/s": round(gbs, 1),
+            "rows_per_s": round(w.rows / (ms * 1e-3), 1), "frac_of_measured_copy": round(gbs / peak, 4)}
+
+
 def time_e2e(w: W.Workload, steps: int, warmup: int):
     """The same metric through fs_softmax_host: pinned host buffers in, pinned host buffers out."""
     import torch
@@ -458,6 +495,12 @@ def main():
                                          "frac_of_measured_copy": round(gbs / peak, 4),
                                          "speedup_vs_cfg5": round(others["cfg5"]["ms_per_step"] / r["ms_per_step"], 3)
                                          if "ms_per_step" in others.get("cfg5", {}) else None}
+            # the router step (softmax over experts + top-8, renormalised) on the router workload
+            rw = W.WORKLOADS["cfg3"]
+            try:
+                others["cfg3_router_top8"] = time_router(rw, 8, 500, 10, l2)
+            except Exception as exc:                       # never lose the main line to an extra
+                others["cfg3_router_top8"] = {"error": str(exc)[:200]}
             line["workloads"] = others
         if not args.no_cpu:
             line["cpu_baseline"] = cpu_baseline(w)

@@ -104,6 +104,30 @@ int fs_softmax_causal(const void* x, void* y, int64_t rows, int64_t cols, int64_
                       void* stream);
 
 /*
+ * fs_router_topk -- the router step of a mixture-of-experts layer: softmax over the expert logits
+ * of each token, then the k most probable experts (the softmax of the paper's Qwen 3.5 35B-A3B
+ * workload, Table I, fused with the selection that follows it in such a router; operator fusion
+ * is the lever of Sec. II-B).
+ *
+ *     p = softmax(scale * x[i][.]);   idx[i][0..k) = the k columns with the largest p, largest
+ *     first, equal values in column order;   w[i][j] = p[idx[i][j]], or, with `renormalize`,
+ *     p[idx[i][j]] / sum_j p[idx[i][j]].
+ *
+ *   x     device pointer, rows*cols elements of `dtype`, 16-byte aligned, row size a multiple of
+ *         16 bytes and cols <= 1024 (rows live in the registers of a warp); other shapes return
+ *         FS_ERR_UNSUPPORTED.
+ *   w     device pointer to rows*k floats (fp32 whatever `dtype` is); idx: rows*k int32.
+ *   k     1 <= k <= min(cols, FS_ROUTER_MAX_K).
+ * The selection is made on the inputs (the order of p is the order of scale*x), so it is exact: a
+ * negative scale selects the smallest x, a zero scale the first k columns. NaN inputs count as the
+ * smallest value for the selection; a row with a NaN or +inf (after scaling), or with only -inf,
+ * has NaN weights. Weights meet the fp32 bound of fs_softmax (|error| <= 1e-6).
+ */
+#define FS_ROUTER_MAX_K 64
+int fs_router_topk(const void* x, float* w, int32_t* idx, int64_t rows, int64_t cols, int k, int dtype, float scale,
+                   int renormalize, void* stream);
+
+/*
  * fs_select_kernel -- the dispatcher's decision, without a launch (no CUDA call is made when the
  * device attributes are already cached or `x_align`/`y_align` rule the fast paths out).
  *   x_align, y_align  the largest power of two (<= 16 is enough) dividing each base address.

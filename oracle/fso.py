@@ -74,6 +74,8 @@ def _load():
             lib.fso_softmax_row_f64.restype = None
             lib.fso_softmax_causal_f64.argtypes = [vp, ci, i64, i64, i64, f32, vp]
             lib.fso_softmax_causal_f64.restype = None
+            lib.fso_router_topk_f64.argtypes = [vp, ci, i64, i64, i64, f32, ci, vp, vp]
+            lib.fso_router_topk_f64.restype = None
             lib.fso_widen.argtypes = [vp, ci, i64, vp]
             lib.fso_widen.restype = None
             lib.fso_round_from_f64.argtypes = [vp, ci, i64, vp]
@@ -115,6 +117,20 @@ def softmax_causal_f64(x: np.ndarray, dtype: int, q_offset: int, scale: float = 
     if rows and cols:
         _load().fso_softmax_causal_f64(x.ctypes.data, dtype, rows, cols, q_offset, np.float32(scale), y.ctypes.data)
     return y
+
+
+def router_topk_f64(x: np.ndarray, dtype: int, k: int, scale: float = 1.0, renorm: bool = False):
+    """fp64 router step: (weights [rows, k] float64, indices [rows, k] int32), largest first."""
+    x = _stored(x, dtype)
+    rows, cols = x.shape
+    if not (1 <= k <= cols):
+        raise ValueError("k out of range")
+    w = np.empty((rows, k), dtype=np.float64)
+    idx = np.empty((rows, k), dtype=np.int32)
+    if rows:
+        _load().fso_router_topk_f64(x.ctypes.data, dtype, rows, cols, k, np.float32(scale), int(renorm),
+                                    w.ctypes.data, idx.ctypes.data)
+    return w, idx
 
 
 def widen(x: np.ndarray, dtype: int) -> np.ndarray:

@@ -184,6 +184,45 @@ void fso_softmax_causal_f64(const void* x, int dtype, int64_t rows, int64_t cols
     }
 }
 
+// Router step of a mixture-of-experts layer (the softmax over expert logits of the paper's
+// Qwen 3.5 35B-A3B workload, Table I, followed by the selection every such router makes):
+//   p = softmax(scale * x_row);  take the k largest p, ties going to the lower column;
+//   w_j = p[idx_j], or p[idx_j] / sum of the k selected p when `renorm` is set.
+// The order of p is the order of z = scale * x (exp is increasing), and z is exact in fp64, so
+// the selection is made on z: a stable sort by decreasing z, a NaN z counting as -inf.
+// w: rows*k doubles, idx: rows*k int32, both in selection order (largest first).
+void fso_router_topk_f64(const void* x, int dtype, int64_t rows, int64_t cols, int64_t k, float scale,
+                         int renorm, double* w, int32_t* idx) {
+    const int64_t esz = (dtype == DT_FP32) ? 4 : 2;
+    const double sc = static_cast<double>(scale);
+    double* p = new double[static_cast<size_t>(cols > 0 ? cols : 1)];
+    double* key = new double[static_cast<size_t>(cols > 0 ? cols : 1)];
+    int32_t* order = new int32_t[static_cast<size_t>(cols > 0 ? cols : 1)];
+    for (int64_t i = 0; i < rows; ++i) {
+        const char* row = static_cast<const char*>(x) + i * cols * esz;
+        fso_softmax_row_f64(row, dtype, cols, scale, p);
+        for (int64_t j = 0; j < cols; ++j) {
+            const double z = sc * widen(row, dtype, j);
+            key[j] = std::isnan(z) ? -std::numeric_limits<double>::infinity() : z;
+            order[j] = static_cast<int32_t>(j);
+        }
+        // stable insertion sort by decreasing key (plain and obviously stable; cols is small)
+        for (int64_t a = 1; a < cols; ++a) {
+            const int32_t cur = order[a];
+            int64_t b = a;
+            while (b > 0 && key[order[b - 1]] < key[cur]) { order[b] = order[b - 1]; --b; }
+            order[b] = cur;
+        }
+        double sel = 0.0;
+        for (int64_t j = 0; j < k; ++j) sel += p[order[j]];
+        for (int64_t j = 0; j < k; ++j) {
+            idx[i * k + j] = order[j];
+            w[i * k + j] = renorm ? p[order[j]] / sel : p[order[j]];
+        }
+    }
+    delete[] p; delete[] key; delete[] order;
+}
+
 // Exact widening of stored elements (exposed so tests can pin the decoders).
 void fso_widen(const void* x, int dtype, int64_t n, double* out) {
     for (int64_t i = 0; i < n; ++i) out[i] = widen(x, dtype, i);

@@ -15,6 +15,7 @@ FS_DTYPE_FP32, FS_DTYPE_BF16, FS_DTYPE_FP16 = 0, 1, 2
 FS_OK, FS_ERR_INVALID_ARG, FS_ERR_UNSUPPORTED, FS_ERR_CUDA, FS_ERR_DEVICE_TIMEOUT = 0, 1, 2, 3, 4
 FS_KERNEL_AUTO, FS_KERNEL_WARP, FS_KERNEL_BLOCK, FS_KERNEL_BLOCK_TMA, FS_KERNEL_CLUSTER, FS_KERNEL_GENERIC = range(6)
 FS_STATIC_MAX_ROW_BYTES = 16 * 192 * 1024
+FS_ROUTER_MAX_K = 64
 KERNELS = {"auto": 0, "warp": 1, "block": 2, "block_tma": 3, "cluster": 4, "generic": 5}
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -50,6 +51,8 @@ def lib() -> ctypes.CDLL:
             L.fs_softmax_ex.restype = ci
             L.fs_softmax_causal.argtypes = [vp, vp, i64, i64, i64, ci, f32, vp]
             L.fs_softmax_causal.restype = ci
+            L.fs_router_topk.argtypes = [vp, vp, vp, i64, i64, ci, ci, f32, ci, vp]
+            L.fs_router_topk.restype = ci
             L.fs_select_kernel.argtypes = [i64, i64, ci, ci, ci]
             L.fs_select_kernel.restype = ci
             L.fs_softmax_host.argtypes = [vp, vp, i64, i64, ci, f32]
@@ -120,6 +123,13 @@ def fs_softmax_causal(x, y, rows: int, cols: int, q_offset: int, dtype: int, sca
     """Causal softmax: row i keeps columns j <= i + q_offset; masked inputs are never read."""
     _check(lib().fs_softmax_causal(_ptr(x), _ptr(y), rows, cols, q_offset, dtype, scale, _stream(stream)),
            "fs_softmax_causal")
+
+
+def fs_router_topk(x, w, idx, rows: int, cols: int, k: int, dtype: int, scale: float = 1.0, renormalize: bool = False,
+                   stream=None) -> None:
+    """Softmax over experts + top-k: w [rows, k] float32 and idx [rows, k] int32 device buffers."""
+    _check(lib().fs_router_topk(_ptr(x), _ptr(w), _ptr(idx), rows, cols, k, dtype, scale, int(renormalize),
+                                _stream(stream)), "fs_router_topk")
 
 
 def fs_select_kernel(rows: int, cols: int, dtype: int, x_align: int = 16, y_align: int = 16) -> int:

@@ -3,6 +3,7 @@
 
 #include "../../include/fsoftmax.h"
 
+#include <atomic>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -12,6 +13,7 @@
 
 #include "kernels/block_row.cuh"
 #include "kernels/common.cuh"
+#include "kernels/router_topk.cuh"
 #include "kernels/smem_row.cuh"
 #include "kernels/warp_row.cuh"
 
@@ -45,7 +47,7 @@ struct LaunchInfo {      // cached per (kernel function, threads, dynamic smem, 
 };
 
 struct Device {
-    bool ready = false;
+    std::atomic<bool> ready{false};   // set last, with release order, once the fields below are valid
     int sm_count = 0;
     int smem_optin = 0;      // max dynamic shared memory per block
     int cluster_ok = 0;
@@ -70,15 +72,15 @@ int get_device(Device** out) {
     FS_CUDA(cudaGetDevice(&d));
     if (d < 0 || d >= kMaxDevices) return FS_ERR_UNSUPPORTED;
     Device& dev = g_dev[d];
-    if (!dev.ready) {
+    if (!dev.ready.load(std::memory_order_acquire)) {
         std::lock_guard<std::mutex> lk(g_mu);
-        if (!dev.ready) {
+        if (!dev.ready.load(std::memory_order_relaxed)) {
             FS_CUDA(cudaDeviceGetAttribute(&dev.sm_count, cudaDevAttrMultiProcessorCount, d));
             FS_CUDA(cudaDeviceGetAttribute(&dev.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, d));
             FS_CUDA(cudaDeviceGetAttribute(&dev.cluster_ok, cudaDevAttrClusterLaunch, d));
             FS_CUDA(cudaMalloc(&dev.status, sizeof(int)));
             FS_CUDA(cudaMemset(dev.status, 0, sizeof(int)));
-            dev.ready = true;
+            dev.ready.store(true, std::memory_order_release);
         }
     }
     *out = &dev;
@@ -397,6 +399,25 @@ FS_VPT_TABLE(block_fn, block_row_kernel)
 FS_VPT_TABLE(block_tma_fn, block_row_tma_kernel)
 FS_VPT_TABLE(cluster_fn, cluster_row_kernel)
 
+template <int DT> const void* router_fn(const WarpGeom& g) {
+    if (g.vpl == 1) return (const void*)router_topk_kernel<DT, 1, 1>;
+    if (g.vpl == 2) return (const void*)router_topk_kernel<DT, 1, 2>;
+    if (g.vpl == 4) {
+        switch (g.lanes) {
+            case 1:  return (const void*)router_topk_kernel<DT, 1, 4>;
+            case 2:  return (const void*)router_topk_kernel<DT, 2, 4>;
+            case 4:  return (const void*)router_topk_kernel<DT, 4, 4>;
+            case 8:  return (const void*)router_topk_kernel<DT, 8, 4>;
+            case 16: return (const void*)router_topk_kernel<DT, 16, 4>;
+            default: return (const void*)router_topk_kernel<DT, 32, 4>;
+        }
+    }
+    if constexpr (DT == DT_F32) {
+        if (g.vpl == 8) return (const void*)router_topk_kernel<DT, 32, 8>;
+    }
+    return nullptr;
+}
+
 // Calls f(std::integral_constant<int, DT>, std::bool_constant<NEG>) for the run-time dtype and sign.
 template <typename F> const void* by_variant(int dtype, bool neg, F f) {
     auto with_dt = [&](auto dt) -> const void* {
@@ -708,6 +729,41 @@ int fs_softmax_causal(const void* x, void* y, int64_t rows, int64_t cols, int64_
     if (rows == 0 || cols == 0) return FS_OK;
     if (q_offset > (int64_t(1) << 41) || q_offset < -(int64_t(1) << 41)) return FS_ERR_INVALID_ARG;
     return run_causal(x, y, rows, cols, q_offset, dtype, scale, static_cast<cudaStream_t>(stream));
+}
+
+int fs_router_topk(const void* x, float* w, int32_t* idx, int64_t rows, int64_t cols, int k, int dtype, float scale,
+                   int renormalize, void* stream) {
+    if (rows < 0 || cols < 0) return FS_ERR_INVALID_ARG;
+    if (dtype != FS_DTYPE_FP32 && dtype != FS_DTYPE_BF16 && dtype != FS_DTYPE_FP16) return FS_ERR_INVALID_ARG;
+    if (!std::isfinite(scale)) return FS_ERR_INVALID_ARG;
+    if (rows == 0) return FS_OK;
+    if (k < 1 || k > cols || k > FS_ROUTER_MAX_K) return FS_ERR_INVALID_ARG;
+    if (!x || !w || !idx) return FS_ERR_INVALID_ARG;
+    if (rows > (int64_t(1) << 40)) return FS_ERR_INVALID_ARG;
+    if (ptr_align(x) < 16 || (cols * elem_size(dtype)) % 16 != 0) return FS_ERR_UNSUPPORTED;
+    if (ptr_align(w) < 4 || ptr_align(idx) < 4) return FS_ERR_INVALID_ARG;
+    const int64_t nvec = cols * elem_size(dtype) / 16;
+    WarpGeom g;
+    if (!warp_geom(nvec, dtype, &g) || g.vpl * (dtype == FS_DTYPE_FP32 ? 4 : 8) > 32) return FS_ERR_UNSUPPORTED;
+    Device* dev = nullptr;
+    int rc = get_device(&dev);
+    if (rc != FS_OK) return rc;
+    const void* fn = nullptr;
+    switch (dtype) {
+        case FS_DTYPE_FP32: fn = router_fn<DT_F32>(g); break;
+        case FS_DTYPE_BF16: fn = router_fn<DT_BF16>(g); break;
+        default:            fn = router_fn<DT_F16>(g); break;
+    }
+    if (!fn) return FS_ERR_UNSUPPORTED;
+    RouterParams p;
+    p.x = x; p.w = w; p.idx = idx; p.rows = rows; p.nvec = nvec; p.k = k;
+    p.c = static_cast<float>(static_cast<double>(scale) * kLog2e);
+    p.renorm = renormalize ? 1 : 0;
+    const int t = 128;
+    const size_t smem = static_cast<size_t>(g.vpl) * (dtype == FS_DTYPE_FP32 ? 4 : 8) * t * sizeof(uint32_t);   // <= 16 KiB
+    const int64_t groups = (rows + (32 / g.lanes) - 1) / (32 / g.lanes);
+    const int64_t grid = std::min<int64_t>((groups + (t / 32) - 1) / (t / 32), 0x7fffffff);
+    return launch(fn, grid, t, smem, 0, static_cast<cudaStream_t>(stream), p);
 }
 
 int fs_select_kernel(int64_t rows, int64_t cols, int dtype, int x_align, int y_align) {
