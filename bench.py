@@ -53,7 +53,7 @@ NCU_TRAFFIC_BYTES = {
     "cfg1": 263168,               # profiles/block_row_kernel_cfg1_fp32_64x1000.txt (y stays in L2)
     "cfg2": 85875200,             # profiles/warp_row_kernel_cfg2_bf16_16384x2048.txt (x read once; 0.28 of y written back by kernel end)
     "cfg3": 34245376,             # profiles/warp_row_kernel_cfg3_bf16_131072x128.txt
-    "cfg4": 211956992,            # profiles/smem_row_kernel_cfg4_bf16_256x262144.txt
+    "cfg4": 212063232,            # profiles/smem_row_kernel_cfg4_bf16_256x262144.txt
     "cfg5": 16 * 480043776,       # profiles/smem_row_kernel_cfg5_fp32_2048x32768.txt, scaled from 2048 to 32768 rows
 }
 
@@ -399,6 +399,9 @@ def main():
     ap.add_argument("--all", dest="all_workloads", action="store_true", default=None,
                     help="also time the other workloads (default: on at --gpus 1)")
     ap.add_argument("--no-all", dest="all_workloads", action="store_false")
+    ap.add_argument("--op", default="softmax", choices=["softmax", "causal", "router"],
+                    help="time only fs_softmax_causal (q_offset 0) or fs_router_topk (k=8, renormalised) on the "
+                         "workload and print a short line (profiler captures of those kernels)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the cpu_baseline leg")
     ap.add_argument("--no-e2e", action="store_true", help="skip the end-to-end leg")
     ap.add_argument("--no-clocks", action="store_true", help="do not sample nvidia-smi clocks (profiler captures)")
@@ -442,6 +445,23 @@ def main():
     props = torch.cuda.get_device_properties(local_rank)
     l2 = int(getattr(props, "L2_cache_size", 126 << 20))
     sampler = ClockSampler(smi_id(props, local_rank)) if rank == 0 and not args.no_clocks else None
+    if args.op != "softmax":
+        if args.op == "causal":
+            r = time_device(w, args.steps, args.warmup, l2, causal_q=0)
+            kept = sum(min(w.cols, i + 1) for i in range(w.rows))
+            alg = (kept + w.rows * w.cols) * w.elem_size
+            r = {"ms_per_step": round(r["ms_per_step"], 6), "algorithmic_bytes": alg,
+                 "GB/s": round(alg / (r["ms_per_step"] * 1e-3) / 1e9, 1)}
+        else:
+            r = time_router(w, 8, args.steps, args.warmup, l2)
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "op": args.op, "unit": UNIT, "value": r["GB/s"], "n_gpus": world,
+                              "steps": args.steps, "warmup": max(3, args.warmup), "higher_is_better": True,
+                              "config": {"workload": w.name, "shape": [w.rows, w.cols]}, **r}), flush=True)
+        if dist:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
     res = time_device(w, args.steps, args.warmup, l2, sampler=sampler, barrier=barrier, min_clock_samples=8)
     from paper_2607_24762_b200 import sharding
     ms = sharding.max_over_ranks(res["ms_per_step"], device="cuda")          # as slow as the slowest rank
