@@ -1,0 +1,131 @@
+"""Guarded PyTorch front end of libfsoftmax: the analogue of the paper's guarded dispatch
+(Sec. III-E): per call, the library kernel runs only when it is available and compatible with the
+call; every other call runs the unmodified eager operator, so a patched model keeps running in
+eager mode and never sees a wrong or unsupported kernel.
+
+    from paper_2607_24762_b200 import torch_op
+    y = torch_op.softmax(x, dim=-1)                 # library kernel when the guard admits the call
+    with torch_op.patched():                        # torch.softmax / F.softmax / Tensor.softmax routed
+        out = model(inputs)                         # through the guard for the duration of the block
+    torch_op.stats()                                # how many calls went where, and why not
+
+The guard admits a call when: the tensor is on a CUDA device, dtype fp32/bf16/fp16, the softmax
+dimension is the last one (or the tensor can be seen that way without a copy), the tensor is
+contiguous, no autograd graph is being recorded for it, and no output dtype conversion is asked
+for other than the upcast-and-cast-back pattern of eager attention (``dtype=torch.float32`` on a
+16-bit input followed by ``.to(input dtype)`` cannot be seen from here, so ``dtype=`` calls fall
+back). This module is a convenience layer above the C ABI; the library itself has no fallback.
+"""
+from __future__ import annotations
+
+import contextlib
+import threading
+from collections import Counter
+
+import torch
+
+from . import binding
+
+_DTYPES = {torch.float32: binding.FS_DTYPE_FP32, torch.bfloat16: binding.FS_DTYPE_BF16,
+           torch.float16: binding.FS_DTYPE_FP16}
+_stats = Counter()
+_lock = threading.Lock()
+_eager_softmax = torch.softmax            # the unpatched operators, captured at import
+_eager_F_softmax = torch.nn.functional.softmax
+_eager_T_softmax = torch.Tensor.softmax
+
+
+def _count(key: str) -> None:
+    with _lock:
+        _stats[key] += 1
+
+
+def stats(reset: bool = False) -> dict:
+    """Calls per outcome: 'library', or 'eager:<reason>'."""
+    with _lock:
+        out = dict(_stats)
+        if reset:
+            _stats.clear()
+    return out
+
+
+def why_not(x: torch.Tensor, dim: int, dtype=None) -> str | None:
+    """None when the guard admits the call, else the reason it goes to eager."""
+    if not isinstance(x, torch.Tensor):
+        return "not a tensor"
+    if not x.is_cuda:
+        return "not on a CUDA device"
+    if x.dtype not in _DTYPES:
+        return f"dtype {x.dtype}"
+    if dtype is not None and dtype != x.dtype:
+        return "output dtype conversion requested"
+    if x.dim() == 0:
+        return "0-d tensor"
+    if dim not in (-1, x.dim() - 1):
+        return "softmax dimension is not the last one"
+    if not x.is_contiguous():
+        return "not contiguous"
+    if torch.is_grad_enabled() and x.requires_grad:
+        return "autograd is recording"
+    if x.numel() == 0:
+        return "empty"
+    return None
+
+
+def softmax(x: torch.Tensor, dim: int = -1, dtype=None, scale: float = 1.0, out: torch.Tensor | None = None):
+    """softmax(scale * x) over `dim`: the library kernel when admitted, else eager PyTorch."""
+    reason = why_not(x, dim, dtype)
+    if reason is None and out is not None and (out.shape != x.shape or out.dtype != x.dtype or
+                                                not out.is_contiguous() or out.device != x.device):
+        reason = "incompatible out tensor"
+    if reason is None:
+        try:
+            binding.lib()
+        except RuntimeError:
+            reason = "library not built"
+    if reason is not None:
+        _count("eager:" + reason)
+        xs = x if scale == 1.0 else x * scale
+        y = _eager_softmax(xs, dim, dtype=dtype)
+        if out is not None:
+            out.copy_(y)
+            return out
+        return y
+    cols = x.shape[-1]
+    rows = x.numel() // cols
+    y = out if out is not None else torch.empty_like(x)
+    with torch.cuda.device(x.device):
+        binding.fs_softmax(x, y, rows, cols, _DTYPES[x.dtype], float(scale), torch.cuda.current_stream(x.device))
+    _count("library")
+    return y
+
+
+def _patched_softmax(input, dim=None, *, dtype=None, **kw):        # torch.softmax(input, dim, dtype=None)
+    if kw or dim is None:
+        return _eager_softmax(input, dim, dtype=dtype, **kw)
+    return softmax(input, dim, dtype)
+
+
+def _patched_F_softmax(input, dim=None, _stacklevel=3, dtype=None):
+    if dim is None:
+        return _eager_F_softmax(input, dim, _stacklevel, dtype)
+    return softmax(input, dim, dtype)
+
+
+def _patched_T_softmax(self, dim=None, dtype=None, **kw):
+    if kw or dim is None:
+        return _eager_T_softmax(self, dim, dtype=dtype, **kw)
+    return softmax(self, dim, dtype)
+
+
+@contextlib.contextmanager
+def patched():
+    """Route torch.softmax, torch.nn.functional.softmax and Tensor.softmax through the guard."""
+    saved = (torch.softmax, torch.nn.functional.softmax, torch.Tensor.softmax)
+    torch.softmax = _patched_softmax
+    torch.nn.functional.softmax = _patched_F_softmax
+    torch.Tensor.softmax = _patched_T_softmax
+    try:
+        yield
+    finally:
+        torch.softmax, torch.nn.functional.softmax, torch.Tensor.softmax = saved

@@ -1,0 +1,88 @@
+"""The guarded PyTorch front end (the analogue of the paper's guarded dispatch, Sec. III-E): calls
+the library only when the guard admits them, else eager. CPU part: the guard's reasons, the eager
+route, patch/restore. GPU part: admitted calls against the oracle, a small attention block under
+the patch against its eager self."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_24762_b200 import torch_op
+
+
+def test_guard_reasons_and_eager_route_on_cpu():
+    torch_op.stats(reset=True)
+    x = torch.randn(4, 9)
+    assert torch_op.why_not(x, -1) == "not on a CUDA device"
+    y = torch_op.softmax(x, -1)
+    assert torch.equal(y, torch.softmax(x, -1))
+    y = torch_op.softmax(x, -1, scale=0.5)
+    assert torch.allclose(y, torch.softmax(x * 0.5, -1))
+    out = torch.empty_like(x)
+    assert torch_op.softmax(x, -1, out=out) is out and torch.equal(out, torch.softmax(x, -1))
+    assert torch_op.stats()["eager:not on a CUDA device"] == 3
+    assert torch_op.why_not(torch.zeros(3, dtype=torch.float64), -1) is not None
+    assert torch_op.why_not("x", -1) == "not a tensor"
+
+
+def test_patch_routes_and_restores():
+    before = (torch.softmax, torch.nn.functional.softmax, torch.Tensor.softmax)
+    x = torch.randn(3, 5)
+    torch_op.stats(reset=True)
+    with torch_op.patched():
+        a = torch.softmax(x, -1)
+        b = torch.nn.functional.softmax(x, dim=1)
+        c = x.softmax(-1)
+        d = torch.softmax(x, 0, dtype=torch.float64)
+    assert (torch.softmax, torch.nn.functional.softmax, torch.Tensor.softmax) == before
+    ref = before[0](x, -1)
+    assert torch.equal(a, ref) and torch.equal(b, ref) and torch.equal(c, ref)
+    assert d.dtype == torch.float64
+    assert sum(torch_op.stats().values()) == 4
+
+
+@pytest.mark.gpu
+def test_admitted_calls_match_the_oracle_and_others_fall_back():
+    from oracle import fso
+    from paper_2607_24762_b200 import workloads as W
+    torch_op.stats(reset=True)
+    for tdt, dt in ((torch.float32, W.FP32), (torch.bfloat16, W.BF16), (torch.float16, W.FP16)):
+        x = (torch.randn(2, 4, 33, 2048, device="cuda") * 2).to(tdt)
+        y = torch_op.softmax(x, -1, scale=0.25)
+        assert y.shape == x.shape and y.dtype == x.dtype
+        bits = (lambda t: t.view(torch.int16).cpu().numpy().view(np.uint16)) if dt != W.FP32 else (lambda t: t.cpu().numpy())
+        rep = fso.compare(bits(y).reshape(-1, 2048), dt, fso.softmax_f64(bits(x).reshape(-1, 2048), dt, 0.25))
+        assert rep.ok(dt), rep
+    assert torch_op.stats()["library"] == 3
+    x = torch.randn(8, 64, device="cuda")
+    assert torch_op.why_not(x, 0) == "softmax dimension is not the last one"
+    assert torch.equal(torch_op.softmax(x, 0), torch.softmax(x, 0))
+    xt = x.t()
+    assert torch_op.why_not(xt, -1) == "not contiguous"
+    assert torch.allclose(torch_op.softmax(xt, -1), torch.softmax(xt, -1))
+    xg = x.clone().requires_grad_(True)
+    yg = torch_op.softmax(xg, -1)
+    yg.sum().backward()                                   # eager route keeps autograd working
+    assert xg.grad is not None and torch_op.why_not(xg, -1) == "autograd is recording"
+    with torch.no_grad():
+        assert torch_op.why_not(xg, -1) is None
+    assert torch_op.why_not(x, -1, dtype=torch.float64) == "output dtype conversion requested"
+
+
+@pytest.mark.gpu
+def test_attention_block_under_the_patch_matches_eager():
+    torch.manual_seed(0)
+
+    def attention(q, k, v):                               # eager attention as in the paper's LLM workloads
+        s = torch.matmul(q, k.transpose(-1, -2)) / q.shape[-1] ** 0.5
+        mask = torch.full(s.shape[-2:], float("-inf"), device=s.device, dtype=s.dtype).triu(1)
+        p = torch.nn.functional.softmax(s + mask, dim=-1)
+        return torch.matmul(p, v)
+
+    q, k, v = (torch.randn(1, 8, 256, 64, device="cuda", dtype=torch.bfloat16) for _ in range(3))
+    with torch.no_grad():
+        ref = attention(q, k, v)
+        torch_op.stats(reset=True)
+        with torch_op.patched():
+            got = attention(q, k, v)
+    assert torch_op.stats().get("library", 0) == 1
+    assert torch.allclose(got.float(), ref.float(), atol=2e-2, rtol=2e-2)
