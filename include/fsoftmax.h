@@ -75,7 +75,7 @@ int fs_softmax(const void* x, void* y, int64_t rows, int64_t cols, int dtype, fl
  * fs_softmax_ex -- as fs_softmax, with the kernel and its launch geometry forced (tests, tuning).
  *   kernel   an fs_kernel; FS_KERNEL_AUTO behaves like fs_softmax.
  *   threads  threads per block, 0 = the kernel's own choice. Must be a multiple of 32.
- *   cluster  blocks per cluster for FS_KERNEL_CLUSTER (1, 2, 4, 8 or 16), 0 = the kernel's choice;
+ *   cluster  blocks per cluster for FS_KERNEL_CLUSTER (1 .. 16), 0 = the kernel's choice;
  *            ignored by the other kernels.
  * Returns FS_ERR_UNSUPPORTED when the forced kernel cannot run this shape, alignment or geometry.
  */

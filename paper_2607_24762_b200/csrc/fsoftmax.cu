@@ -116,13 +116,12 @@ int max_threads_for(int dtype, int vpt) { return vpt * (dtype == FS_DTYPE_FP32 ?
 //           shared-memory-resident split.
 //   fp32:   (sub-)warp per row up to 2 KiB, block per row up to 8 KiB, block per row fed by bulk
 //           copies up to 32 KiB, then the split.
-//   split:  32 KiB slices and 128-thread blocks (6 blocks per SM), cluster size the next power of
-//           two that reaches that slice; rows beyond 16 x 32 KiB grow the slice, with 256 threads.
+//   split:  slices of about 32 KiB, cluster and block size chosen per row length (smem_geom);
+//           rows beyond 16 x 32 KiB grow the slice.
 int64_t warp_max_row_bytes(int dtype) { return dtype == FS_DTYPE_FP32 ? 2048 : 4096; }
 int64_t block_max_row_bytes(int) { return 8192; }
 int64_t block_tma_max_row_bytes(int dtype) { return dtype == FS_DTYPE_FP32 ? 32768 : 0; }
 int64_t split_slice_bytes(int) { return 32768; }
-int split_threads(int) { return 128; }
 constexpr int64_t kWarpTileMaxRowBytes = 4096;      // rows the warp-tile bulk-copy kernel takes
 constexpr int64_t kClusterSliceBytes = 32768;       // register-resident cluster kernel: slice per block
 constexpr int kMaxCluster = 16;
@@ -179,30 +178,79 @@ bool cluster_geom(int64_t nvec, int dtype, int threads, int cluster, ClusterGeom
     return block_geom(slice, dtype, threads, &g->b);
 }
 
-// Shared-memory-resident split: slices of about kClusterSliceBytes, up to kMaxCluster blocks; rows
-// beyond that grow the slice up to what one block's shared memory holds.
+// Shared-memory-resident split: which cluster size and block size a row gets.
+//
+// What decides the speed of this kernel is how many bytes of rows an SM holds at a time (blocks per
+// SM x slice), because a block loads, computes and stores one after the other and only the other
+// blocks on the SM keep the memory system busy meanwhile. Measured on B200 over rows from 12 KiB
+// to 1.5 MiB, every cluster size 1..16 and block sizes 64..256: the best geometry has slices of
+// 32 KiB or a little less that are a whole number of chunks (a chunk = 8 vectors per thread, so
+// the block size is chosen to divide the slice), two or three chunks per block, and the smallest
+// cluster that gets there; cluster sizes need not be powers of two. The candidates are scored by a
+// small model of those measurements (mean loss against the best measured geometry: 0.5%).
 struct SmemGeom { int cs, slice, threads; };
 constexpr int64_t kSmemSliceMaxBytes = 192 * 1024;
-bool smem_geom(int64_t nvec, int dtype, int threads, int cluster, SmemGeom* g) {
-    if (nvec < 1) return false;
-    int cs = cluster;
-    if (cs == 0) {
-        cs = 1;
-        while (cs < kMaxCluster && (nvec * 16 + cs - 1) / cs > split_slice_bytes(dtype)) cs <<= 1;
-    }
-    if (cs != 1 && cs != 2 && cs != 4 && cs != 8 && cs != 16) return false;
+constexpr int kSmemPerSm = 228 * 1024;               // shared memory of one SM, 1 KiB reserved per block
+constexpr int kSplitThreadsPerSm = 768;              // the split-row kernel's register cap: 85 per thread
+
+bool smem_geom_fits(int64_t nvec, int dtype, int t, int cs, SmemGeom* g) {
+    if (cs < 1 || cs > kMaxCluster || t < 32 || t % 32 || t > 256) return false;
     const int64_t slice = (nvec + cs - 1) / cs;
     if (slice * 16 > kSmemSliceMaxBytes) return false;
-    // a block covers kSmemRowMaxChunks chunks of smem_row_u(dtype) vectors per thread
-    const int64_t per_thread = int64_t(kSmemRowMaxChunks) * smem_row_u(dtype);
-    int t = threads;
-    if (t == 0) {
-        t = slice >= 256 ? split_threads(dtype) : 64;
-        while (t < 256 && slice > per_thread * t) t <<= 1;
-    }
-    if (t % 32 || t > 256 || slice > per_thread * t) return false;
+    if (slice > int64_t(kSmemRowMaxChunks) * smem_row_u(dtype) * t) return false;
     g->cs = cs; g->slice = static_cast<int>(slice); g->threads = t;
     return true;
+}
+
+double smem_geom_score(int64_t nvec, int dtype, const SmemGeom& g) {
+    const int64_t chunk = int64_t(smem_row_u(dtype)) * g.threads;
+    const int64_t nch = (g.slice + chunk - 1) / chunk;
+    const bool full = nvec == int64_t(g.slice) * g.cs && g.slice % chunk == 0;
+    const double stage = double(nch * chunk * 16);
+    const double smem = stage + kSmemRowMaxChunks * 8 + kSmemRowMaxChunks * 4.0 * g.threads + 1024 + 1024;
+    const int blocks = std::min(std::min(int(kSmemPerSm / smem), kSplitThreadsPerSm / g.threads), 32);
+    if (blocks < 1) return 0.0;
+    const double resident_cap = 184.0 * 1024;
+    double s = std::min(double(blocks) * g.slice * 16, resident_cap) / resident_cap;
+    if (!full) s *= 0.93 * (g.slice * 16 / stage);           // bounds checks, arithmetic on the padding
+    if (nch == 1) s *= 0.92;                                 // nothing to overlap inside the block
+    if (nch > 3) s *= 1.0 - 0.02 * double(nch - 3);
+    const double warps = blocks * g.threads / 32.0;
+    if (warps < 16.0) s *= 1.0 - (dtype == FS_DTYPE_FP32 ? 0.075 : 0.25) * (1.0 - warps / 16.0);
+    // large clusters leave block slots of a GPC unused
+    s *= g.cs <= 4 ? 1.0 : g.cs <= 8 ? 0.97 : g.cs <= 12 ? 0.93 : 0.9;
+    return s;
+}
+
+// threads / cluster == 0: choose. Forced values are honoured (threads a multiple of 32 up to 256,
+// cluster 1..16).
+bool smem_geom(int64_t nvec, int dtype, int threads, int cluster, SmemGeom* g) {
+    if (nvec < 1) return false;
+    const int cs_fit = static_cast<int>(std::min<int64_t>(kMaxCluster, (nvec * 16 + split_slice_bytes(dtype) - 1) / split_slice_bytes(dtype)));
+    const int cs_lo = cluster ? cluster : (cs_fit < kMaxCluster ? std::max(1, cs_fit - 1) : kMaxCluster);
+    const int cs_hi = cluster ? cluster : std::min(kMaxCluster, cs_fit + 1);
+    static const int kThreads[] = {128, 96, 160, 192, 256};     // in order of preference
+    double best = 0.0;
+    bool found = false;
+    // cluster sizes nearest the 32 KiB fit first; a later candidate must be 1% better to win
+    for (int d = 0; d <= 2; ++d) {
+        for (int sgn = 0; sgn < (d ? 2 : 1); ++sgn) {
+            const int cs = cluster ? cluster : cs_fit + (sgn ? d : -d);
+            if (cs < cs_lo || cs > cs_hi || (cluster && d)) continue;
+            for (int ti = 0; ti < (threads ? 1 : 5); ++ti) {
+                SmemGeom c;
+                if (!smem_geom_fits(nvec, dtype, threads ? threads : kThreads[ti], cs, &c)) continue;
+                const double sc = std::max(smem_geom_score(nvec, dtype, c), 1e-9);
+                if (!found || sc > best * 1.01) { best = sc; *g = c; found = true; }
+            }
+        }
+    }
+    if (!found && !threads) {
+        // short slices: fewer threads than the preferred sizes
+        for (int t = 64; t >= 32 && !found; t -= 32)
+            for (int cs = cs_lo; cs <= cs_hi && !found; ++cs) found = smem_geom_fits(nvec, dtype, t, cs, g);
+    }
+    return found;
 }
 
 bool cluster_uses_registers() {
@@ -306,6 +354,18 @@ int active_clusters(Device& dev, const void* fn, int threads, size_t smem, int c
     dev.launch_cache[key] = LaunchInfo{n};
     *out = n;
     return FS_OK;
+}
+
+// Split-row kernel, one-shot grids: a cluster asks L2 for the input of the row that starts about
+// half a generation of resident clusters later, so that DRAM reads run ahead of the blocks that
+// consume them and no longer stop while a block computes. Measured on B200 (384 MiB of bf16 and
+// fp32 rows from 16 KiB to 1 MiB): half a generation brings 16 KiB..512 KiB rows to the speed of
+// a plain copy; a whole generation is too early (up to 20% slower than none: the lines are gone
+// again before they are used), an eighth too late. FS_PREFETCH_PCT (read once) sets the distance
+// in percent of a generation, 0 turns the prefetch off.
+int64_t prefetch_rows(int resident_clusters) {
+    static const int pct = [] { const char* e = std::getenv("FS_PREFETCH_PCT"); return e ? std::max(0, std::atoi(e)) : 50; }();
+    return pct == 0 ? 0 : std::max<int64_t>(1, int64_t(resident_clusters) * pct / 100);
 }
 
 // Programmatic dependent launch (on unless FS_PDL=0): the kernel may be scheduled while the
@@ -484,6 +544,7 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
     p.neg = p.c < 0.0f ? 1 : 0;
     p.status = dev.status;
     p.q_offset = 0;
+    p.pf_rows = 0;
     const int64_t max_grid = 0x7fffffff;
 
     switch (kernel) {
@@ -580,6 +641,7 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
                     if ((rc = active_clusters(dev, fn, sg.threads, smem, sg.cs, &ncl)) != FS_OK) return rc;
                     int64_t clusters = std::min<int64_t>(rows, max_grid / sg.cs);
                     if (persistent_grids()) clusters = std::min<int64_t>(clusters, ncl);
+                    else p.pf_rows = prefetch_rows(ncl);
                     return launch(fn, clusters * sg.cs, sg.threads, smem, sg.cs, st, p,
                                   static_cast<uint32_t>(stage_bytes), sg.slice, smem_row_nchunk(sg, dtype));
                 }
@@ -639,6 +701,7 @@ int run_causal(const void* x, void* y, int64_t rows, int64_t cols, int64_t q_off
     p.neg = p.c < 0.0f ? 1 : 0;
     p.status = dev.status;
     p.q_offset = q_offset;
+    p.pf_rows = 0;
     SmemGeom sg;
     // (a zero scale goes to the generic kernel: the split kernel masks with -inf, and 0 * -inf is NaN)
     if (fast && p.c != 0.0f && dev.cluster_ok && smem_geom(p.nvec, dtype, 0, 0, &sg) && rows <= 0x7fffffff / sg.cs) {
@@ -646,7 +709,9 @@ int run_causal(const void* x, void* y, int64_t rows, int64_t cols, int64_t q_off
             return (const void*)smem_row_kernel<decltype(dt)::value, decltype(ng)::value, false, true>; });
         const size_t smem = smem_row_bytes(sg, dtype);
         if (smem <= static_cast<size_t>(dev.smem_optin) - 2048) {
-            if ((rc = configure_kernel(dev, fn, true, true)) != FS_OK) return rc;
+            int ncl = 0;
+            if ((rc = active_clusters(dev, fn, sg.threads, smem, sg.cs, &ncl)) != FS_OK) return rc;
+            p.pf_rows = prefetch_rows(ncl);
             return launch(fn, rows * sg.cs, sg.threads, smem, sg.cs, st, p,
                           static_cast<uint32_t>(smem_row_stage_bytes(sg, dtype)), sg.slice, smem_row_nchunk(sg, dtype));
         }
@@ -922,6 +987,7 @@ int fs_softmax_static(const void* x, void* y, int64_t rows, int64_t cols, int dt
     p.neg = p.c < 0.0f ? 1 : 0;
     p.status = sd.scratch;
     p.q_offset = 0;
+    p.pf_rows = 0;
     const void* fn = smem_row_fn(dtype, p.neg, sg, nvec);
     const size_t stage_bytes = smem_row_stage_bytes(sg, dtype);
     const size_t smem = smem_row_bytes(sg, dtype);

@@ -24,6 +24,7 @@ struct Params {
     int neg;           // c < 0: the row reference is the minimum of x instead of the maximum (host-side dispatch)
     int* status;       // device status word
     int64_t q_offset;  // causal kernels: row i keeps columns j <= i + q_offset
+    int64_t pf_rows;   // split-row kernel: the cluster of row i asks L2 for row i + pf_rows (0: off)
 };
 
 template <int DT> struct Traits;
@@ -139,6 +140,79 @@ template <int DT> __device__ __forceinline__ void store_elem(void* p, int64_t i,
     else static_cast<__half*>(p)[i] = __float2half_rn(v);
 }
 
+// ---- packed pairs of binary32 -----------------------------------------------------------------
+// sm_100 has two-wide fp32 arithmetic on 64-bit register pairs (add/sub/mul/fma .f32x2): the same
+// IEEE results as the scalar forms, one issue slot for two elements. These kernels are bound by
+// instruction issue long before the fp32 pipe is full, so everything per element that is not the
+// exponential itself goes through the pairs.
+
+typedef uint64_t f32x2;
+
+__device__ __forceinline__ f32x2 pair(float lo, float hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ f32x2 pair_bits(uint32_t lo, uint32_t hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpair(f32x2 v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ void unpair_bits(f32x2 v, uint32_t& lo, uint32_t& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v));
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+    f32x2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ float pair_sum(f32x2 v) {
+    float lo, hi;
+    unpair(v, lo, hi);
+    return lo + hi;
+}
+
+// Two binary32 values to one word of two bf16 / fp16 (round to nearest even), low element first.
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// One word of two 16-bit elements to a pair of binary32.
+template <int DT>
+__device__ __forceinline__ f32x2 widen_word(uint32_t w) {
+    if constexpr (DT == DT_BF16) {
+        return pair_bits(w << 16, w & 0xffff0000u);
+    } else {
+        const float2 t = __half22float2(*reinterpret_cast<const __half2*>(&w));
+        return pair(t.x, t.y);
+    }
+}
+
 // ---- base-2 exponential on the special-function unit ---------------------------------------
 // e = 2^t with t = (x - r) * c <= 0 for the row (or thread) reference r. One MUFU.EX2 per element:
 // the flushing form of ex2.approx is a single instruction, the non-flushing one costs three more.
@@ -157,6 +231,76 @@ __device__ __forceinline__ float ex2_elem(float d, float c) {
     else                         t = d * c;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(t));
     return r;
+}
+
+__device__ __forceinline__ float ex2_ftz(float t) {
+    float r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(t));
+    return r;
+}
+
+// The same for a pair: d = x - r and t = d c (+ 64 for bf16) are two-wide, the exponentials are not.
+template <int DT>
+__device__ __forceinline__ f32x2 ex2_pair(f32x2 x, f32x2 r2, f32x2 c2) {
+    const f32x2 d = sub2(x, r2);
+    f32x2 t;
+    if constexpr (DT == DT_BF16) t = fma2(d, c2, pair(64.0f, 64.0f));
+    else                         t = mul2(d, c2);
+    float lo, hi;
+    unpair(t, lo, hi);
+    return pair(ex2_ftz(lo), ex2_ftz(hi));
+}
+
+// e = 2^((x - r) c) for one 16-byte vector of x: each pair of e is added to its own accumulator
+// (unrounded), and e comes back in the element dtype, rounded to nearest even.
+template <int DT>
+__device__ __forceinline__ uint4 ex2_vec(const uint4& raw, f32x2 r2, f32x2 c2, f32x2 (&acc)[Traits<DT>::VE / 2]) {
+    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+    uint32_t o[4];
+    if constexpr (DT == DT_F32) {
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            const f32x2 e = ex2_pair<DT>(pair_bits(w[2 * k], w[2 * k + 1]), r2, c2);
+            acc[k] = add2(acc[k], e);
+            unpair_bits(e, o[2 * k], o[2 * k + 1]);
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const f32x2 e = ex2_pair<DT>(widen_word<DT>(w[k]), r2, c2);
+            acc[k] = add2(acc[k], e);
+            float lo, hi;
+            unpair(e, lo, hi);
+            o[k] = DT == DT_BF16 ? pack_bf16x2(lo, hi) : pack_f16x2(lo, hi);
+        }
+    }
+    return make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+// y = e * f (TWO: e * f * g, rounded once) for one 16-byte vector of stored e (element dtype),
+// rounded to nearest even.
+template <int DT, bool TWO>
+__device__ __forceinline__ uint4 scale_vec(const uint4& raw, f32x2 f2, f32x2 g2) {
+    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+    uint32_t o[4];
+    if constexpr (DT == DT_F32) {
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            f32x2 v = mul2(pair_bits(w[2 * k], w[2 * k + 1]), f2);
+            if (TWO) v = mul2(v, g2);
+            unpair_bits(v, o[2 * k], o[2 * k + 1]);
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            f32x2 v = mul2(widen_word<DT>(w[k]), f2);
+            if (TWO) v = mul2(v, g2);
+            float lo, hi;
+            unpair(v, lo, hi);
+            o[k] = DT == DT_BF16 ? pack_bf16x2(lo, hi) : pack_f16x2(lo, hi);
+        }
+    }
+    return make_uint4(o[0], o[1], o[2], o[3]);
 }
 
 __device__ __forceinline__ float ex2_noflush(float t) {
@@ -296,6 +440,14 @@ __device__ __forceinline__ void bulk_load_row(uint32_t dst, const char* src, uin
     for (uint32_t off = 0; off < bytes; off += 32768u) {
         const uint32_t n = min(32768u, bytes - off);
         bulk_load(dst + off, src + off, n, bar);
+    }
+}
+
+// Asks the L2 cache for `bytes` (a multiple of 16) at `src`: no destination, nothing to wait for.
+__device__ __forceinline__ void l2_prefetch(const char* src, uint32_t bytes) {
+    for (uint32_t off = 0; off < bytes; off += 32768u) {
+        const uint32_t n = min(32768u, bytes - off);
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" :: "l"(src + off), "r"(n) : "memory");
     }
 }
 

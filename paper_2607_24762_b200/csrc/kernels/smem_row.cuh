@@ -30,12 +30,6 @@ constexpr int kSmemRowMaxChunks = 8;
 // at most 256 threads and a cap of 85 registers, three 256-thread or six 128-thread blocks fit an SM.
 __host__ __device__ constexpr int smem_row_u(int) { return 8; }
 
-__device__ __forceinline__ float ex2_ftz(float t) {
-    float r;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(t));
-    return r;
-}
-
 // Dynamic shared memory: slice rounded up to whole chunks (stage_bytes) | kSmemRowMaxChunks chunk
 // mbarriers | per-thread chunk references (kSmemRowMaxChunks * blockDim.x floats).
 // The slice must fit in kSmemRowMaxChunks chunks of smem_row_u(DT) * blockDim.x vectors.
@@ -57,6 +51,10 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
     __shared__ __align__(16) float2 xchg[2][16];
     __shared__ __align__(8) uint64_t xbar[2];
     const int T = blockDim.x, tid = threadIdx.x, lane = tid & 31;
+    // A warp owns 32 * U consecutive vectors of a chunk and a lane every 32nd of them: accesses
+    // stay coalesced and conflict-free, and the offsets u * US are immediates whatever blockDim is.
+    const int tpos = (tid >> 5) * (32 * U) + lane;
+    constexpr int US = 32;
     const uint32_t q = cluster_ctarank(), cs = cluster_nctarank();
     const uint32_t ncl = cluster_count_x();
     const uint32_t cid = cluster_id_x();
@@ -83,11 +81,12 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
         nchunk = (nv + chunk_vecs - 1) / chunk_vecs;
     }
     const float ident = ref_identity<NEG>();
+    const f32x2 c2 = pair(p.c, p.c);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + stage_bytes);
     float* rcs = reinterpret_cast<float*>(smem + stage_bytes + kSmemRowMaxChunks * 8) + tid;   // [chunk][thread]
-    uint4* sv = reinterpret_cast<uint4*>(smem) + tid;
+    uint4* sv = reinterpret_cast<uint4*>(smem) + tpos;
     const char* xb = static_cast<const char*>(p.x) + int64_t(v0) * 16;
-    uint4* __restrict__ yv = static_cast<uint4*>(p.y) + v0 + tid;
+    uint4* __restrict__ yv = static_cast<uint4*>(p.y) + v0 + tpos;
     const int64_t row_bytes = p.nvec * 16;
 
     auto issue_row = [&](int64_t row) {                    // thread 0: one bulk copy per chunk
@@ -107,6 +106,18 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
         fence_proxy_async_smem();
         pdl_wait();
         if (cid < p.rows) issue_row(cid);
+        // the row that starts about half a generation of resident clusters later: its slice is on
+        // its way to L2 while this one is worked on
+        const int64_t pr = int64_t(cid) + p.pf_rows;
+        if (p.pf_rows > 0 && pr < p.rows) {
+            int pnv = nv;
+            if (CAUSAL) {
+                const int64_t pkeep = max(int64_t(0), min(p.cols, pr + p.q_offset + 1));
+                const int slice_nv = min(static_cast<int>(p.nvec), v0 + slice) - v0;
+                pnv = max(0, min(slice_nv, static_cast<int>((pkeep + VE - 1) / VE) - v0));
+            }
+            if (pnv > 0) l2_prefetch(xb + pr * row_bytes, uint32_t(pnv) * 16u);
+        }
     }
     __syncthreads();
     if (cs > 1) {   // peers are resident, their mbarriers initialised, before any remote deposit
@@ -118,7 +129,7 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
     if (CAUSAL && nfill > 0 && cid < p.rows) {
         // masked part of this block's slice: +0, written while the kept part is still on its way
         const uint4 zv = make_uint4(0u, 0u, 0u, 0u);
-        uint4* yfill = yv - tid + int64_t(cid) * p.nvec;
+        uint4* yfill = yv - tpos + int64_t(cid) * p.nvec;
         for (int v = nv + tid; v < nv + nfill; v += T) st_stream(yfill + v, zv);
     }
 
@@ -136,7 +147,7 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
             if (tid < 32 && alive) alive = mbar_wait_warp(smem_u32(&bars[ch]), phase, p.status);
             if (T > 32) __syncthreads();
             uint4* sc = sv + ch * chunk_vecs;
-            const int cbase = ch * chunk_vecs + tid;
+            const int cbase = ch * chunk_vecs + tpos;
             if (!FULL) {
                 // this thread's vectors of the chunk that lie past the slice's end become identity
                 // vectors, so that the arithmetic below needs no bounds (a zero scale, for which
@@ -144,33 +155,33 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
                 const uint32_t idw = ident_word<DT, NEG>();
 #pragma unroll
                 for (int u = 0; u < U; ++u)
-                    if (cbase + u * T >= nv) sc[u * T] = make_uint4(idw, idw, idw, idw);
+                    if (cbase + u * US >= nv) sc[u * US] = make_uint4(idw, idw, idw, idw);
             }
             uint4 raw[U];
 #pragma unroll
-            for (int u = 0; u < U; ++u) raw[u] = sc[u * T];
+            for (int u = 0; u < U; ++u) raw[u] = sc[u * US];
             if (CAUSAL) {
 #pragma unroll
                 for (int u = 0; u < U; ++u)
-                    if (cbase + u * T == tail_at) mask_tail<DT, NEG>(raw[u], tail_keep);
+                    if (cbase + u * US == tail_at) mask_tail<DT, NEG>(raw[u], tail_keep);
             }
-            RefAcc<DT, NEG> acc;
-            acc.init();
+            RefAcc<DT, NEG> ref;
+            ref.init();
 #pragma unroll
-            for (int u = 0; u < U; ++u) acc.fold(raw[u]);
-            const float rc = acc.value();
+            for (int u = 0; u < U; ++u) ref.fold(raw[u]);
+            const float rc = ref.value();
             rcs[ch * T] = rc;
             // all of these elements masked (or none): subtract 0 instead of the identity
             const float ru = (rc == ident) ? 0.0f : rc;
-            float part = 0.0f;
+            const f32x2 ru2 = pair(ru, ru);
+            f32x2 acc[VE / 2];
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                float e[VE];
-                unpack<DT>(raw[u], e);
+            for (int k = 0; k < VE / 2; ++k) acc[k] = pair(0.0f, 0.0f);
 #pragma unroll
-                for (int k = 0; k < VE; ++k) { e[k] = ex2_elem<DT>(e[k] - ru, p.c); part += e[k]; }
-                sc[u * T] = pack<DT>(e);
-            }
+            for (int u = 0; u < U; ++u) sc[u * US] = ex2_vec<DT>(raw[u], ru2, c2, acc);
+#pragma unroll
+            for (int k = 1; k < VE / 2; ++k) acc[0] = add2(acc[0], acc[k]);
+            const float part = pair_sum(acc[0]);
             // online merge of (rc, part) into (r, s): only the reference left behind is rescaled
             const float rn = ref_pick<NEG>(r, rc);
             const bool keep = (rn == r);
@@ -202,20 +213,22 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
             // that fac * inv cannot underflow before it meets e
             const bool one_mul = DT != DT_BF16 || fac >= 0x1p-40f || !(fac == fac);
             const float f1 = one_mul ? fac * inv : inv;
+            const int cbase = ch * chunk_vecs + tpos;
+            uint4* yc = yrow + ch * chunk_vecs;
             uint4 raw[U];
 #pragma unroll
-            for (int u = 0; u < U; ++u) raw[u] = sc[u * T];
+            for (int u = 0; u < U; ++u) raw[u] = sc[u * US];
+            const f32x2 f2 = pair(f1, f1);
+            if (DT == DT_BF16 && !one_mul) {
+                // rare: both multiplications before the one rounding
+                const f32x2 g2 = pair(fac, fac);
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                float e[VE];
-                unpack<DT>(raw[u], e);
+                for (int u = 0; u < U; ++u)
+                    if (FULL || cbase + u * US < nv) st_stream(yc + u * US, scale_vec<DT, true>(raw[u], f2, g2));
+            } else {
 #pragma unroll
-                for (int k = 0; k < VE; ++k) e[k] *= f1;
-                if (!one_mul) {
-#pragma unroll
-                    for (int k = 0; k < VE; ++k) e[k] *= fac;
-                }
-                if (FULL || ch * chunk_vecs + tid + u * T < nv) st_stream(yrow + ch * chunk_vecs + u * T, pack<DT>(e));
+                for (int u = 0; u < U; ++u)
+                    if (FULL || cbase + u * US < nv) st_stream(yc + u * US, scale_vec<DT, false>(raw[u], f2, f2));
             }
         }
 
@@ -226,7 +239,7 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
 #pragma unroll
             for (int k = 0; k < VE; ++k) z[k] = 0.0f * inv;
             const uint4 zv = pack<DT>(z);
-            for (int v = nv + tid; v < nv + nfill; v += T) st_stream(yrow - tid + v, zv);
+            for (int v = nv + tid; v < nv + nfill; v += T) st_stream(yrow - tpos + v, zv);
         }
 
         if (!CAUSAL && row + ncl < p.rows) {     // resident-grid form: the slice is free once everyone has read it
