@@ -114,11 +114,11 @@ int max_threads_for(int dtype, int vpt) { return vpt * (dtype == FS_DTYPE_FP32 ?
 // plain copy of the same bytes).
 //   16-bit: (sub-)warp per row up to 4 KiB, block per row (direct loads) up to 8 KiB, then the
 //           shared-memory-resident split.
-//   fp32:   (sub-)warp per row up to 2 KiB, block per row up to 8 KiB, block per row fed by bulk
+//   fp32:   (sub-)warp per row up to 3 KiB, block per row up to 8 KiB, block per row fed by bulk
 //           copies up to 32 KiB, then the split.
 //   split:  slices of about 32 KiB, cluster and block size chosen per row length (smem_geom);
 //           rows beyond 16 x 32 KiB grow the slice.
-int64_t warp_max_row_bytes(int dtype) { return dtype == FS_DTYPE_FP32 ? 2048 : 4096; }
+int64_t warp_max_row_bytes(int dtype) { return dtype == FS_DTYPE_FP32 ? 3072 : 4096; }
 int64_t block_max_row_bytes(int) { return 8192; }
 int64_t block_tma_max_row_bytes(int dtype) { return dtype == FS_DTYPE_FP32 ? 32768 : 0; }
 int64_t split_slice_bytes(int) { return 32768; }
@@ -356,15 +356,16 @@ int active_clusters(Device& dev, const void* fn, int threads, size_t smem, int c
     return FS_OK;
 }
 
-// Split-row kernel, one-shot grids: a cluster asks L2 for the input of the row that starts about
-// half a generation of resident clusters later, so that DRAM reads run ahead of the blocks that
-// consume them and no longer stop while a block computes. Measured on B200 (384 MiB of bf16 and
-// fp32 rows from 16 KiB to 1 MiB): half a generation brings 16 KiB..512 KiB rows to the speed of
-// a plain copy; a whole generation is too early (up to 20% slower than none: the lines are gone
-// again before they are used), an eighth too late. FS_PREFETCH_PCT (read once) sets the distance
-// in percent of a generation, 0 turns the prefetch off.
+// One-shot grids of the split-row and block-per-row kernels: a cluster (block) asks L2 for the
+// input of the row that starts about a third of a generation of resident clusters later, so that
+// DRAM reads run ahead of the blocks that consume them and no longer pause while a block computes.
+// Measured on B200 (384 MiB of bf16 and fp32 rows from 6 KiB to 1 MiB): a quarter to a half of a
+// generation brings 6 KiB..512 KiB rows to the speed of a plain copy (before: 0.85-0.98 of it); a
+// whole generation is too early (up to 20% slower than none: the lines are gone again before they
+// are used), an eighth too late; half costs 2% on 4 GiB of 128 KiB rows, a third does not.
+// FS_PREFETCH_PCT (read once) sets the distance in percent of a generation, 0 turns it off.
 int64_t prefetch_rows(int resident_clusters) {
-    static const int pct = [] { const char* e = std::getenv("FS_PREFETCH_PCT"); return e ? std::max(0, std::atoi(e)) : 50; }();
+    static const int pct = [] { const char* e = std::getenv("FS_PREFETCH_PCT"); return e ? std::max(0, std::atoi(e)) : 30; }();
     return pct == 0 ? 0 : std::max<int64_t>(1, int64_t(resident_clusters) * pct / 100);
 }
 
@@ -571,11 +572,10 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
             const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) { return block_fn<decltype(dt)::value, decltype(ng)::value>(g.vpt); });
             if (!fn) return FS_ERR_UNSUPPORTED;
             int64_t grid = std::min<int64_t>(rows, max_grid);
-            if (persistent_grids()) {
-                int bps = 0;
-                if ((rc = blocks_per_sm(dev, fn, g.threads, 0, &bps)) != FS_OK) return rc;
-                grid = std::min<int64_t>(grid, int64_t(dev.sm_count) * bps);
-            }
+            int bps = 0;
+            if ((rc = blocks_per_sm(dev, fn, g.threads, 0, &bps)) != FS_OK) return rc;
+            if (persistent_grids()) grid = std::min<int64_t>(grid, int64_t(dev.sm_count) * bps);
+            else p.pf_rows = prefetch_rows(dev.sm_count * bps);
             return launch(fn, grid, g.threads, 0, 0, st, p);
         }
         case FS_KERNEL_BLOCK_TMA: {

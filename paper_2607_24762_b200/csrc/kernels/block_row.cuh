@@ -121,6 +121,9 @@ block_row_kernel(const Params p) {
             raw[k] = make_uint4(0u, 0u, 0u, 0u);
             if (valid(k)) raw[k] = ld_stream(xv + row * p.nvec + vec(k));
         }
+        // one-shot grids: the row of the block that starts half a generation later goes to L2
+        if (tid == 0 && p.pf_rows > 0 && row + p.pf_rows < p.rows)
+            l2_prefetch(reinterpret_cast<const char*>(xv + (row + p.pf_rows) * p.nvec), uint32_t(nvec) * 16u);
         float e[VPT][VE], r_t, s;
         thread_partial<DT, NEG, VPT>(raw, e, r_t, s, p.c, valid);
         float R = r_t;

@@ -1,24 +1,31 @@
 // Split-row softmax with the slice resident in shared memory (long rows: vocabulary-sized, causal
 // attention rows). A row is split over the CS blocks of a thread-block cluster (CS = 1: one block
-// per row). Each block brings its slice into shared memory with bulk async copies, one mbarrier
-// per chunk (a chunk = four vectors per thread), and makes two passes over it:
+// per row; any size up to 16). Each block brings its slice into shared memory with bulk async
+// copies, one mbarrier per chunk (a chunk = eight vectors per thread), and makes two passes over it:
 //
-//   pass 1  as the chunks land: a thread takes its four vectors of the chunk, their reference r_c
-//           first (packed max), then e = 2^((x - r_c)c) for every element: one ex2 per element.
-//           The e are added (fp32, unrounded) to the thread's running (r, s) pair with the
-//           online-softmax merge (Milakov-Gimelshein), and written back IN PLACE over x in the
-//           element's own dtype; r_c stays in a register.
+//   pass 1  as the chunks land: a thread takes its eight vectors of the chunk, their reference r_c
+//           first (packed max), then e = 2^((x - r_c)c) for every element: one ex2 per element,
+//           the subtraction, the scaling and the summation two elements per instruction
+//           (f32x2). The e are added (fp32, unrounded) to the thread's running (r, s) pair with
+//           the online-softmax merge (Milakov-Gimelshein), and written back IN PLACE over x in
+//           the element's own dtype; r_c goes to a small per-thread table in shared memory.
 //   merge   warp shuffles -> block (one __syncthreads) -> cluster: each block deposits its pair
 //           in every peer's shared memory with st.async, counted by an mbarrier there
 //   pass 2  y = e * 2^((r_c - R)c) / S from the resident slice: no second ex2 per element
 //
-// Storing e rounded to the output dtype costs no accuracy against the stated bar: for fp32 it is
-// exact; for bf16/fp16 it perturbs e, hence y, by at most half a unit in the last place of the
-// output format, so the rounded product can differ from the correctly rounded result by at most
-// one unit (the row sum is taken over the unrounded values).
+// Within a chunk a warp owns 32 * 8 consecutive vectors and a lane every 32nd of them, so the
+// offsets of a thread's eight vectors are compile-time constants (no address arithmetic per
+// access) while every warp-wide access stays contiguous.
+//
+// Storing e rounded to the output dtype keeps the result within the stated bar: for fp32 it is
+// exact; for bf16/fp16 it moves e, hence the unrounded y, by less than one unit in the last place
+// of y (half a unit of e is at most one unit of y = e * f), and two values less than one unit
+// apart round to the same or to adjacent numbers (the row sum is taken over the unrounded e).
 //
 // Registers stay low (no per-thread copy of the row), so occupancy is set by shared memory:
-// several blocks per SM in different phases keep HBM busy.
+// several blocks per SM in different phases keep HBM busy, and thread 0 asks L2 for the slice of a
+// row that starts a fraction of a generation later, so that DRAM reads do not stop while the
+// resident blocks compute.
 #pragma once
 #include "block_row.cuh"
 #include "common.cuh"
