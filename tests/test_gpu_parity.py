@@ -82,7 +82,9 @@ def test_very_long_rows(dtype):
     (fs.FS_KERNEL_BLOCK_TMA, 256, 0), (fs.FS_KERNEL_BLOCK_TMA, 1024, 0),
     (fs.FS_KERNEL_CLUSTER, 0, 1), (fs.FS_KERNEL_CLUSTER, 0, 2), (fs.FS_KERNEL_CLUSTER, 0, 4), (fs.FS_KERNEL_CLUSTER, 0, 8),
     (fs.FS_KERNEL_CLUSTER, 0, 16), (fs.FS_KERNEL_CLUSTER, 128, 4), (fs.FS_KERNEL_CLUSTER, 512, 2),
-    (fs.FS_KERNEL_CLUSTER, 32, 8), (fs.FS_KERNEL_WARP, 128, 0), (fs.FS_KERNEL_WARP, 32, 0),
+    (fs.FS_KERNEL_CLUSTER, 32, 8), (fs.FS_KERNEL_CLUSTER, 0, 3), (fs.FS_KERNEL_CLUSTER, 96, 5), (fs.FS_KERNEL_CLUSTER, 160, 6),
+    (fs.FS_KERNEL_CLUSTER, 0, 7), (fs.FS_KERNEL_CLUSTER, 192, 9), (fs.FS_KERNEL_CLUSTER, 0, 11), (fs.FS_KERNEL_CLUSTER, 224, 12),
+    (fs.FS_KERNEL_CLUSTER, 0, 13), (fs.FS_KERNEL_CLUSTER, 64, 15), (fs.FS_KERNEL_WARP, 128, 0), (fs.FS_KERNEL_WARP, 32, 0),
     (fs.FS_KERNEL_GENERIC, 32, 0), (fs.FS_KERNEL_GENERIC, 1024, 0),
 ])
 def test_every_launch_geometry_the_dispatcher_can_pick(kernel, threads, cluster):
@@ -95,6 +97,19 @@ def test_every_launch_geometry_the_dispatcher_can_pick(kernel, threads, cluster)
                 rep = sweep_case(rows, cols, dtype, kernel, 0.7, seed=77, threads=threads, cluster=cluster)
                 ran += rep is not None
     assert ran > 0
+
+
+@pytest.mark.parametrize("dtype", [FP32, BF16, FP16])
+def test_split_row_geometry_choice_over_row_lengths(dtype):
+    """Row lengths from 8 KiB to 1.5 MiB, multiples of 32 KiB and not: the dispatcher's choice of cluster size
+    (any of 1..16) and block size (96..256 threads) for each, with more rows than resident clusters so
+    that the L2 prefetch of later rows runs."""
+    esz = 4 if dtype == FP32 else 2
+    for kb, rows in ((8, 3000), (12, 2500), (20, 1500), (24, 1200), (40, 900), (48, 800), (62.5, 600), (80, 500), (96, 400),
+                     (100, 400), (160, 260), (192, 230), (250.5, 150), (296.75, 130), (384, 100), (600, 70), (768, 60), (1536, 30)):
+        cols = int(kb * 1024) // esz
+        rep = sweep_case(rows, cols, dtype, fs.FS_KERNEL_AUTO, 1.0, seed=int(kb * 4))
+        assert rep is not None
 
 
 # ---------------------------------------------------------------------------------------------
