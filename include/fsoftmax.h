@@ -128,6 +128,38 @@ int fs_router_topk(const void* x, float* w, int32_t* idx, int64_t rows, int64_t 
                    int renormalize, void* stream);
 
 /*
+ * fs_layer_norm -- layer normalisation over the last dimension, one of the two normalisation
+ * operators the paper reports generated kernels for (Sec. IV-C, Stable Diffusion 3.5 Medium):
+ *
+ *     mu_i = mean_j x[i][j],   var_i = mean_j (x[i][j] - mu_i)^2   (biased),
+ *     y[i][j] = (x[i][j] - mu_i) / sqrt(var_i + eps) * gamma[j] + beta[j]
+ *
+ *   x, y    device pointers, rows*cols elements of `dtype`, row-major, dense; x == y allowed,
+ *           partial overlap is FS_ERR_INVALID_ARG.
+ *   gamma, beta   device pointers to cols elements of `dtype`, or NULL (1 and 0), independently.
+ *   eps     finite, >= 0. Statistics and arithmetic are binary32; the output is rounded once.
+ *   stream  cudaStream_t as void*.
+ * Rows up to 2 KiB stay in the registers of a (sub-)warp; longer rows are split over a cluster of
+ * 1..16 blocks with the slices resident in shared memory (one read and one write of HBM per
+ * element, as for fs_softmax); ragged, misaligned or longer rows take a three-pass kernel.
+ * A NaN or infinity in a row makes the whole row NaN. rows == 0 or cols == 0 launches nothing.
+ */
+int fs_layer_norm(const void* x, const void* gamma, const void* beta, void* y, int64_t rows, int64_t cols, int dtype,
+                  float eps, void* stream);
+
+/*
+ * fs_group_norm -- group normalisation (the paper's largest normalisation result, Sec. IV-C) of a
+ * dense [n, channels, spatial] tensor (NCHW with the spatial dimensions flattened): each
+ * (sample, group) block of channels/groups * spatial contiguous elements is normalised like one
+ * row of fs_layer_norm; gamma and beta (channels elements each, or NULL) are indexed by channel.
+ *   groups  >= 1 and a divisor of channels.
+ * The same kernels as fs_layer_norm run on rows of channels/groups * spatial elements; the fast
+ * path needs spatial * element size to be a multiple of 16 bytes.
+ */
+int fs_group_norm(const void* x, const void* gamma, const void* beta, void* y, int64_t n, int64_t channels, int64_t spatial,
+                  int64_t groups, int dtype, float eps, void* stream);
+
+/*
  * fs_select_kernel -- the dispatcher's decision, without a launch (no CUDA call is made when the
  * device attributes are already cached or `x_align`/`y_align` rule the fast paths out).
  *   x_align, y_align  the largest power of two (<= 16 is enough) dividing each base address.

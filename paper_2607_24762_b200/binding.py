@@ -53,6 +53,10 @@ def lib() -> ctypes.CDLL:
             L.fs_softmax_causal.restype = ci
             L.fs_router_topk.argtypes = [vp, vp, vp, i64, i64, ci, ci, f32, ci, vp]
             L.fs_router_topk.restype = ci
+            L.fs_layer_norm.argtypes = [vp, vp, vp, vp, i64, i64, ci, f32, vp]
+            L.fs_layer_norm.restype = ci
+            L.fs_group_norm.argtypes = [vp, vp, vp, vp, i64, i64, i64, i64, ci, f32, vp]
+            L.fs_group_norm.restype = ci
             L.fs_select_kernel.argtypes = [i64, i64, ci, ci, ci]
             L.fs_select_kernel.restype = ci
             L.fs_softmax_host.argtypes = [vp, vp, i64, i64, ci, f32]
@@ -130,6 +134,19 @@ def fs_router_topk(x, w, idx, rows: int, cols: int, k: int, dtype: int, scale: f
     """Softmax over experts + top-k: w [rows, k] float32 and idx [rows, k] int32 device buffers."""
     _check(lib().fs_router_topk(_ptr(x), _ptr(w), _ptr(idx), rows, cols, k, dtype, scale, int(renormalize),
                                 _stream(stream)), "fs_router_topk")
+
+
+def fs_layer_norm(x, gamma, beta, y, rows: int, cols: int, dtype: int, eps: float = 1e-5, stream=None) -> None:
+    """y = (x - mean) / sqrt(var + eps) * gamma + beta over the last dimension; gamma, beta may be None."""
+    _check(lib().fs_layer_norm(_ptr(x), _ptr(gamma), _ptr(beta), _ptr(y), rows, cols, dtype, eps, _stream(stream)),
+           "fs_layer_norm")
+
+
+def fs_group_norm(x, gamma, beta, y, n: int, channels: int, spatial: int, groups: int, dtype: int, eps: float = 1e-5,
+                  stream=None) -> None:
+    """Group normalisation of a dense [n, channels, spatial] tensor; gamma, beta per channel or None."""
+    _check(lib().fs_group_norm(_ptr(x), _ptr(gamma), _ptr(beta), _ptr(y), n, channels, spatial, groups, dtype, eps,
+                               _stream(stream)), "fs_group_norm")
 
 
 def fs_select_kernel(rows: int, cols: int, dtype: int, x_align: int = 16, y_align: int = 16) -> int:

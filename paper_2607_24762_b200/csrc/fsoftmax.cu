@@ -13,6 +13,7 @@
 
 #include "kernels/block_row.cuh"
 #include "kernels/common.cuh"
+#include "kernels/norm_row.cuh"
 #include "kernels/router_topk.cuh"
 #include "kernels/smem_row.cuh"
 #include "kernels/warp_row.cuh"
@@ -771,6 +772,108 @@ std::mutex g_static_mu;
 // C ABI
 // =============================================================================================
 
+// ---------------------------------------------------------------------------------------------
+// row normalisations
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+template <int DT, int AFF> const void* norm_warp_fn(const WarpGeom& g) {
+    if (g.vpl == 1) return (const void*)norm_warp_kernel<DT, 1, 1, AFF>;
+    if (g.vpl == 2) return (const void*)norm_warp_kernel<DT, 1, 2, AFF>;
+    if (g.vpl != 4) return nullptr;
+    switch (g.lanes) {
+        case 1:  return (const void*)norm_warp_kernel<DT, 1, 4, AFF>;
+        case 2:  return (const void*)norm_warp_kernel<DT, 2, 4, AFF>;
+        case 4:  return (const void*)norm_warp_kernel<DT, 4, 4, AFF>;
+        case 8:  return (const void*)norm_warp_kernel<DT, 8, 4, AFF>;
+        case 16: return (const void*)norm_warp_kernel<DT, 16, 4, AFF>;
+        default: return (const void*)norm_warp_kernel<DT, 32, 4, AFF>;
+    }
+}
+
+template <int DT> const void* norm_smem_fn(bool full, int aff) {
+    if (full) {
+        return aff == 0 ? (const void*)norm_smem_kernel<DT, true, 0> : aff == 1 ? (const void*)norm_smem_kernel<DT, true, 1>
+                                                                                : (const void*)norm_smem_kernel<DT, true, 2>;
+    }
+    return aff == 0 ? (const void*)norm_smem_kernel<DT, false, 0> : aff == 1 ? (const void*)norm_smem_kernel<DT, false, 1>
+                                                                            : (const void*)norm_smem_kernel<DT, false, 2>;
+}
+
+template <typename F> const void* by_dtype(int dtype, F f) {
+    switch (dtype) {
+        case FS_DTYPE_FP32: return f(std::integral_constant<int, DT_F32>{});
+        case FS_DTYPE_BF16: return f(std::integral_constant<int, DT_BF16>{});
+        default:            return f(std::integral_constant<int, DT_F16>{});
+    }
+}
+
+// Rows of `cols` elements; affine parameters per column (aff 1), per run of run_elems elements with
+// aff_rows rows per sample (aff 2), or none (aff 0).
+int run_norm(const void* x, const void* gamma, const void* beta, void* y, int64_t rows, int64_t cols, int dtype,
+             float eps, int aff, int64_t run_elems, int64_t aff_rows, cudaStream_t st) {
+    Device* devp = nullptr;
+    int rc = get_device(&devp);
+    if (rc != FS_OK) return rc;
+    Device& dev = *devp;
+    const int esz = elem_size(dtype);
+    const int ve = 16 / esz;
+    bool fast = fast_path_ok(cols, dtype, ptr_align(x), ptr_align(y));
+    if (aff == 1) fast = fast && (!gamma || ptr_align(gamma) >= 16) && (!beta || ptr_align(beta) >= 16);
+    if (aff == 2) fast = fast && run_elems % ve == 0;
+    NormParams p;
+    p.x = x; p.y = y; p.gamma = gamma; p.beta = beta; p.rows = rows; p.cols = cols;
+    p.nvec = fast ? cols * esz / 16 : 0;
+    p.eps = eps; p.run_elems = run_elems; p.aff_rows = aff_rows;
+    p.status = dev.status; p.pf_rows = 0;
+    WarpGeom wg;
+    if (fast && aff != 2 && p.nvec <= 128 && warp_geom(p.nvec, dtype, &wg) && wg.vpl <= 4) {
+        const void* fn = by_dtype(dtype, [&](auto dt) -> const void* {
+            return aff ? norm_warp_fn<decltype(dt)::value, 1>(wg) : norm_warp_fn<decltype(dt)::value, 0>(wg); });
+        if (fn) {
+            const int t = 128;
+            const int64_t groups = (rows + (32 / wg.lanes) - 1) / (32 / wg.lanes);
+            const int64_t grid = std::min<int64_t>((groups + (t / 32) - 1) / (t / 32), 0x7fffffff);
+            return launch(fn, grid, t, 0, 0, st, p);
+        }
+    }
+    SmemGeom sg;
+    if (fast && dev.cluster_ok && smem_geom(p.nvec, dtype, 0, 0, &sg) && rows <= 0x7fffffff / sg.cs) {
+        const bool full = smem_row_full(sg, dtype, p.nvec);
+        const void* fn = by_dtype(dtype, [&](auto dt) -> const void* { return norm_smem_fn<decltype(dt)::value>(full, aff); });
+        const size_t stage_bytes = smem_row_stage_bytes(sg, dtype);
+        const size_t smem = stage_bytes + size_t(kNormMaxChunks) * 8;
+        if (smem <= static_cast<size_t>(dev.smem_optin) - 2048) {
+            int ncl = 0;
+            if ((rc = active_clusters(dev, fn, sg.threads, smem, sg.cs, &ncl)) != FS_OK) return rc;
+            p.pf_rows = prefetch_rows(ncl);
+            return launch(fn, rows * sg.cs, sg.threads, smem, sg.cs, st, p, static_cast<uint32_t>(stage_bytes), sg.slice,
+                          smem_row_nchunk(sg, dtype));
+        }
+    }
+    const void* fn = by_dtype(dtype, [&](auto dt) -> const void* { return (const void*)norm_generic_kernel<decltype(dt)::value>; });
+    int t = 32;
+    while (t < 1024 && cols > int64_t(t) * 8) t <<= 1;
+    p.nvec = 0;
+    return launch(fn, std::min<int64_t>(rows, 0x7fffffff), t, 0, 0, st, p, aff);
+}
+
+int validate_norm(const void* x, const void* y, int64_t rows, int64_t cols, int dtype, float eps) {
+    if (rows < 0 || cols < 0) return FS_ERR_INVALID_ARG;
+    if (dtype != FS_DTYPE_FP32 && dtype != FS_DTYPE_BF16 && dtype != FS_DTYPE_FP16) return FS_ERR_INVALID_ARG;
+    if (!std::isfinite(eps) || eps < 0.0f) return FS_ERR_INVALID_ARG;
+    if (rows == 0 || cols == 0) return FS_OK;
+    if (!x || !y) return FS_ERR_INVALID_ARG;
+    if (rows > (int64_t(1) << 40) || cols > (int64_t(1) << 40) || rows > (int64_t(1) << 60) / cols) return FS_ERR_INVALID_ARG;
+    const int64_t bytes = rows * cols * elem_size(dtype);
+    const char* xa = static_cast<const char*>(x);
+    const char* ya = static_cast<const char*>(y);
+    if (xa != ya && xa < ya + bytes && ya < xa + bytes) return FS_ERR_INVALID_ARG;      // partial overlap
+    return FS_OK;
+}
+
+}  // namespace
+
 extern "C" {
 
 int fs_softmax_ex(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale,
@@ -829,6 +932,28 @@ int fs_router_topk(const void* x, float* w, int32_t* idx, int64_t rows, int64_t 
     const int64_t groups = (rows + (32 / g.lanes) - 1) / (32 / g.lanes);
     const int64_t grid = std::min<int64_t>((groups + (t / 32) - 1) / (t / 32), 0x7fffffff);
     return launch(fn, grid, t, smem, 0, static_cast<cudaStream_t>(stream), p);
+}
+
+int fs_layer_norm(const void* x, const void* gamma, const void* beta, void* y, int64_t rows, int64_t cols, int dtype,
+                  float eps, void* stream) {
+    const int v = validate_norm(x, y, rows, cols, dtype, eps);
+    if (v != FS_OK || rows == 0 || cols == 0) return v;
+    const int aff = (gamma || beta) ? 1 : 0;
+    return run_norm(x, gamma, beta, y, rows, cols, dtype, eps, aff, 1, 1, static_cast<cudaStream_t>(stream));
+}
+
+int fs_group_norm(const void* x, const void* gamma, const void* beta, void* y, int64_t n, int64_t channels, int64_t spatial,
+                  int64_t groups, int dtype, float eps, void* stream) {
+    if (n < 0 || channels < 0 || spatial < 0 || groups < 1 || channels % groups != 0) return FS_ERR_INVALID_ARG;
+    if (channels > (int64_t(1) << 30) || spatial > (int64_t(1) << 40) || n > (int64_t(1) << 40) / groups) return FS_ERR_INVALID_ARG;
+    const int64_t rows = n * groups;
+    const int64_t cpg = channels / groups;
+    if (cpg > 0 && spatial > (int64_t(1) << 40) / cpg) return FS_ERR_INVALID_ARG;
+    const int64_t cols = cpg * spatial;
+    const int v = validate_norm(x, y, rows, cols, dtype, eps);
+    if (v != FS_OK || rows == 0 || cols == 0) return v;
+    const int aff = (gamma || beta) ? 2 : 0;
+    return run_norm(x, gamma, beta, y, rows, cols, dtype, eps, aff, spatial, groups, static_cast<cudaStream_t>(stream));
 }
 
 int fs_select_kernel(int64_t rows, int64_t cols, int dtype, int x_align, int y_align) {

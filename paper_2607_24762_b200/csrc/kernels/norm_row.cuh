@@ -1,0 +1,407 @@
+// Row normalisations: layer_norm over the last dimension and group_norm over (sample, group)
+// blocks of an [n, channels, spatial] tensor, which is the same computation on rows of
+// channels/groups * spatial elements with the affine parameters indexed by channel:
+//     mu = mean x,  var = mean (x - mu)^2 (biased),  y = (x - mu) / sqrt(var + eps) * gamma + beta
+// The skeleton is the softmax kernels' (load once, reduce, rescale, store once); the reduction
+// item is the triple (n, mean, M2) with Chan's pairwise merge in place of the (reference, sum) pair.
+//
+//   norm_warp_kernel     (sub-)warp per row, the row in registers: exact two-pass statistics
+//   norm_smem_kernel     row split over a cluster of 1..16 blocks, the slice resident in shared
+//                        memory (bulk async copies, one mbarrier per chunk); per chunk a thread
+//                        takes the exact mean and M2 of its own 8 vectors and merges them into
+//                        its running triple; triples merge warp -> block -> cluster (st.async
+//                        deposits counted by an mbarrier); pass 2 normalises from shared memory
+//   norm_generic_kernel  block per row, three passes over global memory (the later ones normally
+//                        from L2): any column count, alignment and row length
+//
+// AFF: 0 no affine parameters, 1 one (gamma, beta) per column (layer_norm: vectors loaded like x),
+//      2 one per run of `run_vecs` vectors (group_norm: a channel's spatial extent).
+#pragma once
+#include "common.cuh"
+
+namespace fsm {
+
+struct NormParams {
+    const void* x;
+    void* y;
+    const void* gamma;     // may be null (1)
+    const void* beta;      // may be null (0)
+    int64_t rows;
+    int64_t cols;
+    int64_t nvec;          // 16-byte vectors per row (fast kernels)
+    float eps;
+    int64_t run_elems;     // AFF 2: elements per affine entry (spatial); 1 otherwise
+    int64_t aff_rows;      // AFF 2: rows per sample (groups): row % aff_rows selects the channel block
+    int* status;
+    int64_t pf_rows;       // one-shot grids: L2 prefetch distance in rows (0: off)
+};
+
+// (count, mean, sum of squared deviations)
+struct Stat { float n, mean, m2; };
+
+__device__ __forceinline__ Stat stat_merge(const Stat& a, const Stat& b) {
+    Stat r;
+    r.n = a.n + b.n;
+    const float w = r.n > 0.0f ? b.n / r.n : 0.0f;
+    const float d = b.mean - a.mean;
+    r.mean = fmaf(d, w, a.mean);
+    r.m2 = a.m2 + b.m2 + d * d * a.n * w;
+    return r;
+}
+
+template <int WIDTH>
+__device__ __forceinline__ Stat warp_merge_stats(Stat s) {
+#pragma unroll
+    for (int o = WIDTH / 2; o > 0; o >>= 1) {
+        Stat t;
+        t.n = __shfl_xor_sync(0xffffffffu, s.n, o);
+        t.mean = __shfl_xor_sync(0xffffffffu, s.mean, o);
+        t.m2 = __shfl_xor_sync(0xffffffffu, s.m2, o);
+        s = stat_merge(s, t);
+    }
+    return s;
+}
+
+__device__ __forceinline__ float rstd_of(float m2, float n, float eps) {
+    return 1.0f / sqrtf(m2 / n + eps);          // IEEE division and square root: once per thread
+}
+
+__device__ __forceinline__ uint4 ld_cached(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+// One vector of x as pairs of binary32.
+template <int DT>
+__device__ __forceinline__ void widen_pairs(const uint4& raw, f32x2 (&x)[Traits<DT>::VE / 2]) {
+    if constexpr (DT == DT_F32) {
+        x[0] = pair_bits(raw.x, raw.y); x[1] = pair_bits(raw.z, raw.w);
+    } else {
+        x[0] = widen_word<DT>(raw.x); x[1] = widen_word<DT>(raw.y);
+        x[2] = widen_word<DT>(raw.z); x[3] = widen_word<DT>(raw.w);
+    }
+}
+template <int DT>
+__device__ __forceinline__ uint4 narrow_pairs(const f32x2 (&x)[Traits<DT>::VE / 2]) {
+    uint4 v;
+    if constexpr (DT == DT_F32) {
+        unpair_bits(x[0], v.x, v.y); unpair_bits(x[1], v.z, v.w);
+    } else {
+        uint32_t o[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            float lo, hi;
+            unpair(x[k], lo, hi);
+            o[k] = DT == DT_BF16 ? pack_bf16x2(lo, hi) : pack_f16x2(lo, hi);
+        }
+        v = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+    return v;
+}
+
+// y = (x - mu) * rstd [* gamma + beta] for one vector.
+//   AFF 1: gv, bv are the column vectors of gamma and beta (null pointers: 1 and 0)
+//   AFF 2: gs, bs are the channel's scalars
+template <int DT, int AFF>
+__device__ __forceinline__ uint4 norm_vec(const uint4& raw, f32x2 mu2, f32x2 r2, const uint4* gv, const uint4* bv,
+                                          float gs, float bs) {
+    constexpr int NP = Traits<DT>::VE / 2;
+    f32x2 x[NP];
+    widen_pairs<DT>(raw, x);
+    if constexpr (AFF == 0) {
+#pragma unroll
+        for (int k = 0; k < NP; ++k) x[k] = mul2(sub2(x[k], mu2), r2);
+    } else if constexpr (AFF == 1) {
+        f32x2 g[NP], b[NP];
+        if (gv) widen_pairs<DT>(ld_cached(gv), g);
+        if (bv) widen_pairs<DT>(ld_cached(bv), b);
+#pragma unroll
+        for (int k = 0; k < NP; ++k) {
+            f32x2 t = mul2(sub2(x[k], mu2), r2);
+            if (gv) t = mul2(t, g[k]);
+            if (bv) t = add2(t, b[k]);
+            x[k] = t;
+        }
+    } else {
+        float rlo, rhi;
+        unpair(r2, rlo, rhi);
+        const f32x2 a2 = pair(rlo * gs, rlo * gs), b2 = pair(bs, bs);
+#pragma unroll
+        for (int k = 0; k < NP; ++k) x[k] = fma2(sub2(x[k], mu2), a2, b2);
+    }
+    return narrow_pairs<DT>(x);
+}
+
+// ---------------------------------------------------------------------------------------------
+// (sub-)warp per row, registers
+// ---------------------------------------------------------------------------------------------
+template <int DT, int LANES, int VPL, int AFF>
+__global__ void __launch_bounds__(256)
+norm_warp_kernel(const NormParams p) {
+    constexpr int VE = Traits<DT>::VE;
+    constexpr int G = 32 / LANES;
+    static_assert(AFF != 2, "per-run affine parameters are handled by the shared-memory kernel");
+    pdl_launch_dependents();
+    const int lane = threadIdx.x & 31;
+    const int sub = lane / LANES, sl = lane % LANES;
+    const int warps = blockDim.x >> 5;
+    const int nvec = static_cast<int>(p.nvec);
+    const uint4* __restrict__ xv = static_cast<const uint4*>(p.x);
+    uint4* __restrict__ yv = static_cast<uint4*>(p.y);
+    const uint4* gv = static_cast<const uint4*>(p.gamma);
+    const uint4* bv = static_cast<const uint4*>(p.beta);
+    const float inv_n = 1.0f / static_cast<float>(p.cols);
+    pdl_wait();
+    const int64_t ngroups = (p.rows + G - 1) / G;
+    for (int64_t grp = int64_t(blockIdx.x) * warps + (threadIdx.x >> 5); grp < ngroups; grp += int64_t(gridDim.x) * warps) {
+        const int64_t row = grp * G + sub;
+        const bool row_ok = row < p.rows;
+        uint4 raw[VPL];
+        float x[VPL][VE];
+        float s = 0.0f;
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+            raw[k] = make_uint4(0u, 0u, 0u, 0u);
+            if (row_ok && sl + k * LANES < nvec) raw[k] = ld_stream(xv + row * p.nvec + sl + k * LANES);
+        }
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+            unpack<DT>(raw[k], x[k]);
+#pragma unroll
+            for (int i = 0; i < VE; ++i) s += x[k][i];                     // absent vectors are zeros
+        }
+        const float mu = warp_sum<LANES>(s) * inv_n;
+        float q = 0.0f;
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+            const bool live = sl + k * LANES < nvec;
+#pragma unroll
+            for (int i = 0; i < VE; ++i) {
+                x[k][i] -= mu;
+                if (live) q = fmaf(x[k][i], x[k][i], q);
+            }
+        }
+        const float rstd = 1.0f / sqrtf(warp_sum<LANES>(q) * inv_n + p.eps);
+        if (row_ok) {
+#pragma unroll
+            for (int k = 0; k < VPL; ++k) {
+                if (sl + k * LANES < nvec) {
+                    float g[VE], b[VE];
+                    if (AFF == 1 && gv) unpack<DT>(ld_cached(gv + sl + k * LANES), g);
+                    if (AFF == 1 && bv) unpack<DT>(ld_cached(bv + sl + k * LANES), b);
+#pragma unroll
+                    for (int i = 0; i < VE; ++i) {
+                        float t = x[k][i] * rstd;
+                        if (AFF == 1 && gv) t *= g[i];
+                        if (AFF == 1 && bv) t += b[i];
+                        x[k][i] = t;
+                    }
+                    st_stream(yv + row * p.nvec + sl + k * LANES, pack<DT>(x[k]));
+                }
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// cluster per row, slices resident in shared memory (one-shot grid: cluster i handles row i)
+// dynamic shared memory: slice rounded up to whole chunks (stage_bytes) | 8 chunk mbarriers
+// FULL: every block's slice is exactly nchunk_full chunks of 8 * blockDim.x vectors.
+// ---------------------------------------------------------------------------------------------
+constexpr int kNormMaxChunks = 8;
+
+template <int DT, bool FULL, int AFF>
+__global__ void __launch_bounds__(256, 3)
+norm_smem_kernel(const NormParams p, const uint32_t stage_bytes, const int slice, const int nchunk_full) {
+    constexpr int VE = Traits<DT>::VE;
+    constexpr int NP = VE / 2;
+    constexpr int U = 8;
+    pdl_launch_dependents();
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ float4 wp[32];
+    __shared__ __align__(16) float4 xchg[16];
+    __shared__ __align__(8) uint64_t xbar;
+    const int T = blockDim.x, tid = threadIdx.x, lane = tid & 31;
+    const int tpos = (tid >> 5) * (32 * U) + lane;     // a warp owns 32 * U consecutive vectors of a chunk
+    const uint32_t q = cluster_ctarank(), cs = cluster_nctarank();
+    const int64_t row = cluster_id_x();
+    const int chunk_vecs = U * T;
+    int v0, nv, nchunk;
+    if (FULL) {
+        v0 = static_cast<int>(q) * slice; nv = slice; nchunk = nchunk_full;
+    } else {
+        const int nvec = static_cast<int>(p.nvec);
+        v0 = min(nvec, static_cast<int>(q) * slice);
+        nv = min(nvec, v0 + slice) - v0;
+        nchunk = (nv + chunk_vecs - 1) / chunk_vecs;
+    }
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + stage_bytes);
+    const uint4* sv = reinterpret_cast<const uint4*>(smem) + tpos;
+    const int64_t row_bytes = p.nvec * 16;
+    const char* xb = static_cast<const char*>(p.x) + int64_t(v0) * 16;
+
+    if (tid == 0) {
+        for (int ch = 0; ch < kNormMaxChunks; ++ch) mbar_init(smem_u32(&bars[ch]), 1);
+        mbar_init(smem_u32(&xbar), 1);
+        mbar_fence_init();
+        fence_proxy_async_smem();
+        pdl_wait();
+        for (int ch = 0; ch < nchunk; ++ch) {
+            const int cv = FULL ? chunk_vecs : min(chunk_vecs, nv - ch * chunk_vecs);
+            bulk_load_row(smem_u32(smem) + uint32_t(ch) * uint32_t(chunk_vecs) * 16u,
+                          xb + row * row_bytes + int64_t(ch) * chunk_vecs * 16, uint32_t(cv) * 16u, smem_u32(&bars[ch]));
+        }
+        if (p.pf_rows > 0 && row + p.pf_rows < p.rows && nv > 0)
+            l2_prefetch(xb + (row + p.pf_rows) * row_bytes, uint32_t(nv) * 16u);
+        if (cs > 1) mbar_expect_tx(smem_u32(&xbar), cs * 16u);
+    }
+    __syncthreads();
+    if (cs > 1) {   // peers are resident, their mbarriers initialised, before any remote deposit
+        cluster_arrive_relaxed();
+        cluster_wait_acquire();
+    }
+    pdl_wait();
+
+    // ---- pass 1: per chunk the exact (count, mean, M2) of this thread's vectors, merged as they land
+    bool alive = true;
+    Stat st = {0.0f, 0.0f, 0.0f};
+    for (int ch = 0; ch < nchunk; ++ch) {
+        if (tid < 32 && alive) alive = mbar_wait_warp(smem_u32(&bars[ch]), 0u, p.status);
+        if (T > 32) __syncthreads();
+        const uint4* sc = sv + ch * chunk_vecs;
+        const int cbase = ch * chunk_vecs + tpos;
+        uint4 raw[U];
+        f32x2 acc[2] = {pair(0.0f, 0.0f), pair(0.0f, 0.0f)};
+        int nvalid = U;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            raw[u] = sc[u * 32];
+            if (!FULL && cbase + u * 32 >= nv) { raw[u] = make_uint4(0u, 0u, 0u, 0u); --nvalid; }   // stale bytes past the slice
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            f32x2 x[NP];
+            widen_pairs<DT>(raw[u], x);
+#pragma unroll
+            for (int k = 0; k < NP; ++k) acc[k & 1] = add2(acc[k & 1], x[k]);
+        }
+        const float cnt = static_cast<float>(nvalid * VE);
+        const float mean_c = nvalid > 0 ? pair_sum(add2(acc[0], acc[1])) / cnt : 0.0f;
+        const f32x2 m2c = pair(mean_c, mean_c);
+        acc[0] = pair(0.0f, 0.0f); acc[1] = pair(0.0f, 0.0f);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (FULL || cbase + u * 32 < nv) {
+                f32x2 x[NP];
+                widen_pairs<DT>(raw[u], x);      // widened again rather than kept: 64 live values would not fit the register cap
+#pragma unroll
+                for (int k = 0; k < NP; ++k) {
+                    const f32x2 d = sub2(x[k], m2c);
+                    acc[k & 1] = fma2(d, d, acc[k & 1]);
+                }
+            }
+        }
+        Stat c;
+        c.n = cnt; c.mean = mean_c; c.m2 = pair_sum(add2(acc[0], acc[1]));
+        st = stat_merge(st, c);
+    }
+    // ---- merge: warp, block, cluster
+    st = warp_merge_stats<32>(st);
+    const int nwarps = T >> 5;
+    if (nwarps > 1) {
+        if (lane == 0) wp[tid >> 5] = make_float4(st.n, st.mean, st.m2, 0.0f);
+        __syncthreads();
+        const float4 v = lane < nwarps ? wp[lane] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        st.n = v.x; st.mean = v.y; st.m2 = v.z;
+        st = warp_merge_stats<32>(st);
+    }
+    if (cs > 1) {
+        if (tid < cs) {
+            const uint32_t dst = map_to_rank(smem_u32(&xchg[q]), tid), bar = map_to_rank(smem_u32(&xbar), tid);
+            st_async_v2(dst, st.n, st.mean, bar);
+            st_async_v2(dst + 8u, st.m2, 0.0f, bar);
+        }
+        if (tid < 32 && alive) alive = mbar_wait_warp(smem_u32(&xbar), 0u, p.status);
+        if (T > 32) __syncthreads();
+        const float4 v = lane < static_cast<int>(cs) ? xchg[lane] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        st.n = v.x; st.mean = v.y; st.m2 = v.z;
+        st = warp_merge_stats<32>(st);
+    }
+    const float rstd = rstd_of(st.m2, st.n, p.eps);
+    const f32x2 mu2 = pair(st.mean, st.mean), r2 = pair(rstd, rstd);
+
+    // ---- pass 2: normalise from the resident slice
+    uint4* __restrict__ yv = static_cast<uint4*>(p.y) + row * p.nvec + v0 + tpos;
+    const uint4* gv = AFF == 1 && p.gamma ? static_cast<const uint4*>(p.gamma) + v0 + tpos : nullptr;
+    const uint4* bv = AFF == 1 && p.beta ? static_cast<const uint4*>(p.beta) + v0 + tpos : nullptr;
+    const int run_vecs = AFF == 2 ? static_cast<int>(p.run_elems / VE) : 1;
+    const int64_t chan0 = AFF == 2 ? (row % p.aff_rows) * (p.nvec / run_vecs) : 0;     // first channel of this row's group
+    for (int ch = 0; ch < nchunk; ++ch) {
+        const uint4* sc = sv + ch * chunk_vecs;
+        const int cbase = ch * chunk_vecs + tpos;
+        uint4 raw[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) raw[u] = sc[u * 32];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (FULL || cbase + u * 32 < nv) {
+                float gs = 1.0f, bs = 0.0f;
+                if (AFF == 2) {
+                    const int64_t c = chan0 + (v0 + cbase + u * 32) / run_vecs;
+                    if (p.gamma) gs = load_elem<DT>(p.gamma, c);
+                    if (p.beta) bs = load_elem<DT>(p.beta, c);
+                }
+                const uint4 o = norm_vec<DT, AFF>(raw[u], mu2, r2, gv ? gv + ch * chunk_vecs + u * 32 : nullptr,
+                                                  bv ? bv + ch * chunk_vecs + u * 32 : nullptr, gs, bs);
+                st_stream(yv + ch * chunk_vecs + u * 32, o);
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// block per row, element-wise accesses, three passes (any shape and alignment)
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float block_sum(float v, float* red) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    v = warp_sum<32>(v);
+    __syncthreads();                       // `red` may still be read from the previous reduction
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    v = lane < nwarps ? red[lane] : 0.0f;
+    return warp_sum<32>(v);
+}
+
+template <int DT>
+__global__ void __launch_bounds__(1024)
+norm_generic_kernel(const NormParams p, const int aff) {
+    __shared__ float red[32];
+    pdl_launch_dependents();
+    pdl_wait();
+    const float inv_n = 1.0f / static_cast<float>(p.cols);
+    for (int64_t row = blockIdx.x; row < p.rows; row += gridDim.x) {
+        const int64_t base = row * p.cols;
+        float s = 0.0f;
+        for (int64_t j = threadIdx.x; j < p.cols; j += blockDim.x) s += load_elem<DT>(p.x, base + j);
+        const float mu = block_sum(s, red) * inv_n;
+        float q = 0.0f;
+        for (int64_t j = threadIdx.x; j < p.cols; j += blockDim.x) {
+            const float d = load_elem<DT>(p.x, base + j) - mu;
+            q = fmaf(d, d, q);
+        }
+        const float rstd = 1.0f / sqrtf(block_sum(q, red) * inv_n + p.eps);
+        const int64_t chan0 = aff == 2 ? (row % p.aff_rows) * (p.cols / p.run_elems) : 0;
+        for (int64_t j = threadIdx.x; j < p.cols; j += blockDim.x) {
+            float t = (load_elem<DT>(p.x, base + j) - mu) * rstd;
+            if (aff) {
+                const int64_t c = aff == 2 ? chan0 + j / p.run_elems : j;
+                if (p.gamma) t *= load_elem<DT>(p.gamma, c);
+                if (p.beta) t += load_elem<DT>(p.beta, c);
+            }
+            store_elem<DT>(p.y, base + j, t);
+        }
+    }
+}
+
+}  // namespace fsm
