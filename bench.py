@@ -262,6 +262,80 @@ def time_router(w: W.Workload, k: int, steps: int, warmup: int, l2_bytes: int):
             "rows_per_s": round(w.rows / (ms * 1e-3), 1), "frac_of_measured_copy": round(gbs / peak, 4)}
 
 
+# Normalisation workloads (synthetic, seeded on the device): the shapes of the two operators the paper
+# reports for Stable Diffusion 3.5 Medium (Sec. IV-C): layer_norm over the transformer's hidden size
+# (1536) for 4 x 4096 tokens, and the VAE decoder's 32-group group_norm at three resolutions.
+NORM_WORKLOADS = {
+    "ln_sd35": ("layer", dict(rows=16384, cols=1536, dtype=W.BF16)),
+    "ln_4096_f32": ("layer", dict(rows=8192, cols=4096, dtype=W.FP32)),
+    "gn_c512_128": ("group", dict(n=1, channels=512, spatial=128 * 128, groups=32, dtype=W.BF16)),
+    "gn_c256_256": ("group", dict(n=1, channels=256, spatial=256 * 256, groups=32, dtype=W.BF16)),
+    "gn_c128_512": ("group", dict(n=1, channels=128, spatial=512 * 512, groups=32, dtype=W.BF16)),
+}
+
+
+def time_norm(name: str, steps: int, warmup: int, l2_bytes: int, eager: bool = True):
+    """fs_layer_norm / fs_group_norm on one NORM_WORKLOADS entry: reads x once, writes y once."""
+    import torch
+
+    import paper_2607_24762_b200 as fs
+    kind, c = NORM_WORKLOADS[name]
+    tdt = {W.FP32: torch.float32, W.BF16: torch.bfloat16, W.FP16: torch.float16}[c["dtype"]]
+    esz = W.ELEM_SIZE[c["dtype"]]
+    shape = (c["rows"], c["cols"]) if kind == "layer" else (c["n"], c["channels"], c["spatial"])
+    nelem = int(np.prod(shape))
+    alg = 2 * nelem * esz
+    n_pairs = int(max(1, min(16, math.ceil(4 * l2_bytes / alg))))
+    g = torch.Generator(device="cuda").manual_seed(1234)
+    xs = [(torch.randn(shape, generator=g, device="cuda") * 1.5 + 0.25).to(tdt) for _ in range(n_pairs)]
+    ys = [torch.empty_like(x) for x in xs]
+    na = c["cols"] if kind == "layer" else c["channels"]
+    gamma = (torch.randn(na, generator=g, device="cuda") * 0.2 + 1.0).to(tdt)
+    beta = (torch.randn(na, generator=g, device="cuda") * 0.1).to(tdt)
+    stream = torch.cuda.current_stream()
+    lib = fs.binding.lib()
+
+    def launch(i):
+        j = i % n_pairs
+        if kind == "layer":
+            st = lib.fs_layer_norm(xs[j].data_ptr(), gamma.data_ptr(), beta.data_ptr(), ys[j].data_ptr(), c["rows"], c["cols"],
+                                   c["dtype"], 1e-5, stream.cuda_stream)
+        else:
+            st = lib.fs_group_norm(xs[j].data_ptr(), gamma.data_ptr(), beta.data_ptr(), ys[j].data_ptr(), c["n"], c["channels"],
+                                   c["spatial"], c["groups"], c["dtype"], 1e-5, stream.cuda_stream)
+        if st != 0:
+            raise RuntimeError(fs.fs_strerror(st))
+
+    def eager_launch(i):
+        j = i % n_pairs
+        if kind == "layer":
+            torch.nn.functional.layer_norm(xs[j], (c["cols"],), gamma, beta, 1e-5)
+        else:
+            torch.nn.functional.group_norm(xs[j], c["groups"], gamma, beta, 1e-5)
+
+    def timed(fn, k):
+        for i in range(max(3, warmup)):
+            fn(i)
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        start.record(stream)
+        for i in range(k):
+            fn(i)
+        stop.record(stream)
+        torch.cuda.synchronize()
+        return start.elapsed_time(stop) / k
+
+    ms = timed(launch, steps)
+    peak, _ = measured_peak()
+    gbs = alg / (ms * 1e-3) / 1e9
+    out = {"what": f"fs_{kind}_norm {name} {list(shape)} {W.DTYPE_NAME[c['dtype']]}, gamma and beta, eps 1e-5", "steps": steps,
+           "ms_per_step": round(ms, 6), "algorithmic_bytes": alg, "GB/s": round(gbs, 1),
+           "frac_of_measured_copy": round(gbs / peak, 4), "n_pairs": n_pairs}
+    if eager:
+        out["torch_eager_ms"] = round(timed(eager_launch, max(5, steps // 4)), 6)
+    return out
+
+
 def time_e2e(w: W.Workload, steps: int, warmup: int):
     """The same metric through fs_softmax_host: pinned host buffers in, pinned host buffers out."""
     import torch
@@ -399,7 +473,8 @@ def main():
     ap.add_argument("--all", dest="all_workloads", action="store_true", default=None,
                     help="also time the other workloads (default: on at --gpus 1)")
     ap.add_argument("--no-all", dest="all_workloads", action="store_false")
-    ap.add_argument("--op", default="softmax", choices=["softmax", "causal", "router"],
+    ap.add_argument("--norm-workload", default="ln_sd35", choices=sorted(NORM_WORKLOADS), help="with --op norm")
+    ap.add_argument("--op", default="softmax", choices=["softmax", "causal", "router", "norm"],
                     help="time only fs_softmax_causal (q_offset 0) or fs_router_topk (k=8, renormalised) on the "
                          "workload and print a short line (profiler captures of those kernels)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the cpu_baseline leg")
@@ -452,6 +527,8 @@ def main():
             alg = (kept + w.rows * w.cols) * w.elem_size
             r = {"ms_per_step": round(r["ms_per_step"], 6), "algorithmic_bytes": alg,
                  "GB/s": round(alg / (r["ms_per_step"] * 1e-3) / 1e9, 1)}
+        elif args.op == "norm":
+            r = time_norm(args.norm_workload, args.steps, args.warmup, l2, eager=not args.no_cpu)
         else:
             r = time_router(w, 8, args.steps, args.warmup, l2)
         if rank == 0:
@@ -521,6 +598,12 @@ def main():
                 others["cfg3_router_top8"] = time_router(rw, 8, 500, 10, l2)
             except Exception as exc:                       # never lose the main line to an extra
                 others["cfg3_router_top8"] = {"error": str(exc)[:200]}
+            # the normalisation entry points on the shapes of the paper's second workload family
+            for nname in NORM_WORKLOADS:
+                try:
+                    others[nname] = time_norm(nname, 200, 10, l2)
+                except Exception as exc:
+                    others[nname] = {"error": str(exc)[:200]}
             line["workloads"] = others
         if not args.no_cpu:
             line["cpu_baseline"] = cpu_baseline(w)

@@ -777,7 +777,30 @@ std::mutex g_static_mu;
 // ---------------------------------------------------------------------------------------------
 namespace {
 
+// Warp-per-row geometry of the normalisation kernels: sub-warp groups with up to four vectors per
+// lane for short rows, whole warps with up to eight (any count, so that no lane idles on rows of
+// 96, 160 or 192 vectors) up to 4 KiB.
+bool norm_warp_geom(int64_t nvec, int dtype, WarpGeom* g) {
+    if (nvec < 1 || nvec > 256) return false;
+    if (nvec <= 64) return warp_geom(nvec, dtype, g) && g->vpl <= 4;
+    g->lanes = 32; g->vpl = static_cast<int>((nvec + 31) / 32); g->r = 1;
+    return true;
+}
+
 template <int DT, int AFF> const void* norm_warp_fn(const WarpGeom& g) {
+    if (g.lanes == 32) {
+        switch (g.vpl) {
+            case 1: return (const void*)norm_warp_kernel<DT, 32, 1, AFF>;
+            case 2: return (const void*)norm_warp_kernel<DT, 32, 2, AFF>;
+            case 3: return (const void*)norm_warp_kernel<DT, 32, 3, AFF>;
+            case 4: return (const void*)norm_warp_kernel<DT, 32, 4, AFF>;
+            case 5: return (const void*)norm_warp_kernel<DT, 32, 5, AFF>;
+            case 6: return (const void*)norm_warp_kernel<DT, 32, 6, AFF>;
+            case 7: return (const void*)norm_warp_kernel<DT, 32, 7, AFF>;
+            case 8: return (const void*)norm_warp_kernel<DT, 32, 8, AFF>;
+            default: return nullptr;
+        }
+    }
     if (g.vpl == 1) return (const void*)norm_warp_kernel<DT, 1, 1, AFF>;
     if (g.vpl == 2) return (const void*)norm_warp_kernel<DT, 1, 2, AFF>;
     if (g.vpl != 4) return nullptr;
@@ -786,9 +809,29 @@ template <int DT, int AFF> const void* norm_warp_fn(const WarpGeom& g) {
         case 2:  return (const void*)norm_warp_kernel<DT, 2, 4, AFF>;
         case 4:  return (const void*)norm_warp_kernel<DT, 4, 4, AFF>;
         case 8:  return (const void*)norm_warp_kernel<DT, 8, 4, AFF>;
-        case 16: return (const void*)norm_warp_kernel<DT, 16, 4, AFF>;
-        default: return (const void*)norm_warp_kernel<DT, 32, 4, AFF>;
+        default: return (const void*)norm_warp_kernel<DT, 16, 4, AFF>;
     }
+}
+
+template <int DT> const void* norm_block_fn(int vpt, int aff) {
+    switch (vpt) {
+        case 1:  return aff ? (const void*)norm_block_kernel<DT, 1, 1> : (const void*)norm_block_kernel<DT, 1, 0>;
+        case 2:  return aff ? (const void*)norm_block_kernel<DT, 2, 1> : (const void*)norm_block_kernel<DT, 2, 0>;
+        default: return aff ? (const void*)norm_block_kernel<DT, 4, 1> : (const void*)norm_block_kernel<DT, 4, 0>;
+    }
+}
+
+// Block-per-row geometry: vectors per thread in {4, 2, 1} and threads a multiple of 32 up to 256,
+// preferring a split that leaves no thread without work.
+bool norm_block_geom(int64_t nvec, int* vpt, int* threads) {
+    if (nvec < 1 || nvec > 1024) return false;
+    for (int v = 4; v >= 1; v >>= 1) {
+        if (nvec % (32 * v) == 0 && nvec / v <= 256) { *vpt = v; *threads = static_cast<int>(nvec / v); return true; }
+    }
+    const int v = nvec > 512 ? 4 : nvec > 128 ? 2 : 1;
+    *vpt = v;
+    *threads = static_cast<int>((nvec + v - 1) / v + 31) / 32 * 32;
+    return *threads <= 256;
 }
 
 template <int DT> const void* norm_smem_fn(bool full, int aff) {
@@ -827,7 +870,7 @@ int run_norm(const void* x, const void* gamma, const void* beta, void* y, int64_
     p.eps = eps; p.run_elems = run_elems; p.aff_rows = aff_rows;
     p.status = dev.status; p.pf_rows = 0;
     WarpGeom wg;
-    if (fast && aff != 2 && p.nvec <= 128 && warp_geom(p.nvec, dtype, &wg) && wg.vpl <= 4) {
+    if (fast && aff != 2 && norm_warp_geom(p.nvec, dtype, &wg)) {
         const void* fn = by_dtype(dtype, [&](auto dt) -> const void* {
             return aff ? norm_warp_fn<decltype(dt)::value, 1>(wg) : norm_warp_fn<decltype(dt)::value, 0>(wg); });
         if (fn) {
@@ -836,6 +879,18 @@ int run_norm(const void* x, const void* gamma, const void* beta, void* y, int64_
             const int64_t grid = std::min<int64_t>((groups + (t / 32) - 1) / (t / 32), 0x7fffffff);
             return launch(fn, grid, t, 0, 0, st, p);
         }
+    }
+    int bvpt = 0, bthreads = 0;
+    // Measured on B200 (256 MiB per direction): the block kernel wins for 16-bit rows of 4-9 KiB; fp32
+    // rows and longer 16-bit rows are faster from shared memory.
+    const int64_t block_max = dtype == FS_DTYPE_FP32 ? 0 : 576;
+    if (fast && aff != 2 && p.nvec <= block_max && norm_block_geom(p.nvec, &bvpt, &bthreads)) {
+        // several rows per block (gamma and beta are loaded once per block), but never so many
+        // that the grid drops below a few waves
+        const int64_t rpb = std::max<int64_t>(1, std::min<int64_t>(8, rows / (int64_t(dev.sm_count) * 32)));
+        const void* fn = by_dtype(dtype, [&](auto dt) -> const void* { return norm_block_fn<decltype(dt)::value>(bvpt, aff); });
+        const int64_t grid = (rows + rpb - 1) / rpb;
+        if (grid <= 0x7fffffff) return launch(fn, grid, bthreads, 0, 0, st, p, static_cast<int>(rpb));
     }
     SmemGeom sg;
     if (fast && dev.cluster_ok && smem_geom(p.nvec, dtype, 0, 0, &sg) && rows <= 0x7fffffff / sg.cs) {

@@ -6,6 +6,8 @@
 // item is the triple (n, mean, M2) with Chan's pairwise merge in place of the (reference, sum) pair.
 //
 //   norm_warp_kernel     (sub-)warp per row, the row in registers: exact two-pass statistics
+//   norm_block_kernel    block per row, the row in registers, several consecutive rows per block
+//                        with gamma and beta kept in registers
 //   norm_smem_kernel     row split over a cluster of 1..16 blocks, the slice resident in shared
 //                        memory (bulk async copies, one mbarrier per chunk); per chunk a thread
 //                        takes the exact mean and M2 of its own 8 vectors and merges them into
@@ -39,10 +41,18 @@ struct NormParams {
 // (count, mean, sum of squared deviations)
 struct Stat { float n, mean, m2; };
 
+// Chan's pairwise merge. The weight b.n / n only positions the merged mean between the two
+// means, so the special-function unit's reciprocal (1 ulp) is enough; an IEEE division would cost
+// more instructions than the rest of the merge.
+__device__ __forceinline__ float fast_rcp(float v) {
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(v));
+    return r;
+}
 __device__ __forceinline__ Stat stat_merge(const Stat& a, const Stat& b) {
     Stat r;
     r.n = a.n + b.n;
-    const float w = r.n > 0.0f ? b.n / r.n : 0.0f;
+    const float w = r.n > 0.0f ? b.n * fast_rcp(r.n) : 0.0f;
     const float d = b.mean - a.mean;
     r.mean = fmaf(d, w, a.mean);
     r.m2 = a.m2 + b.m2 + d * d * a.n * w;
@@ -62,8 +72,15 @@ __device__ __forceinline__ Stat warp_merge_stats(Stat s) {
     return s;
 }
 
-__device__ __forceinline__ float rstd_of(float m2, float n, float eps) {
-    return 1.0f / sqrtf(m2 / n + eps);          // IEEE division and square root: once per thread
+// 1 / sqrt(var + eps): the special-function unit's reciprocal square root (relative error 2^-22)
+// and one Newton step, which brings it to about one unit in the last place.
+__device__ __forceinline__ float rstd_of(float var, float eps) {
+    const float v = var + eps;
+    float r;
+    asm("rsqrt.approx.f32 %0, %1;" : "=f"(r) : "f"(v));
+    const float h = 0.5f * v * r;
+    const float refined = fmaf(r, fmaf(-h, r, 0.5f), r);      // r + r (1/2 - v r^2 / 2)
+    return (v > 0.0f && v < __int_as_float(0x7f800000)) ? refined : r;   // 0, inf, NaN: keep the unit's answer
 }
 
 __device__ __forceinline__ uint4 ld_cached(const uint4* p) {
@@ -100,46 +117,41 @@ __device__ __forceinline__ uint4 narrow_pairs(const f32x2 (&x)[Traits<DT>::VE / 
     return v;
 }
 
-// y = (x - mu) * rstd [* gamma + beta] for one vector.
-//   AFF 1: gv, bv are the column vectors of gamma and beta (null pointers: 1 and 0)
-//   AFF 2: gs, bs are the channel's scalars
-template <int DT, int AFF>
-__device__ __forceinline__ uint4 norm_vec(const uint4& raw, f32x2 mu2, f32x2 r2, const uint4* gv, const uint4* bv,
-                                          float gs, float bs) {
+// Centred pairs d = x - mu of one vector -> d * rstd [* gamma] [+ beta], rounded and stored.
+// Which parameters exist is a compile-time choice here: a run-time "if (gamma)" per element turns
+// into two select instructions per pair, which cost more than the arithmetic.
+template <int DT, bool HG, bool HB>
+__device__ __forceinline__ void affine_store(f32x2 (&d)[Traits<DT>::VE / 2], f32x2 r2, const uint4& graw, const uint4& braw, uint4* dst) {
     constexpr int NP = Traits<DT>::VE / 2;
-    f32x2 x[NP];
-    widen_pairs<DT>(raw, x);
-    if constexpr (AFF == 0) {
+    f32x2 g[NP], b[NP];
+    if (HG) widen_pairs<DT>(graw, g);
+    if (HB) widen_pairs<DT>(braw, b);
 #pragma unroll
-        for (int k = 0; k < NP; ++k) x[k] = mul2(sub2(x[k], mu2), r2);
-    } else if constexpr (AFF == 1) {
-        f32x2 g[NP], b[NP];
-        if (gv) widen_pairs<DT>(ld_cached(gv), g);
-        if (bv) widen_pairs<DT>(ld_cached(bv), b);
-#pragma unroll
-        for (int k = 0; k < NP; ++k) {
-            f32x2 t = mul2(sub2(x[k], mu2), r2);
-            if (gv) t = mul2(t, g[k]);
-            if (bv) t = add2(t, b[k]);
-            x[k] = t;
-        }
-    } else {
-        float rlo, rhi;
-        unpair(r2, rlo, rhi);
-        const f32x2 a2 = pair(rlo * gs, rlo * gs), b2 = pair(bs, bs);
-#pragma unroll
-        for (int k = 0; k < NP; ++k) x[k] = fma2(sub2(x[k], mu2), a2, b2);
+    for (int j = 0; j < NP; ++j) {
+        f32x2 t = mul2(d[j], r2);
+        if (HG && HB) t = fma2(t, g[j], b[j]);
+        else if (HG) t = mul2(t, g[j]);
+        else if (HB) t = add2(t, b[j]);
+        d[j] = t;
     }
-    return narrow_pairs<DT>(x);
+    st_stream(dst, narrow_pairs<DT>(d));
+}
+template <int DT>
+__device__ __forceinline__ void affine_store_any(bool hg, bool hb, f32x2 (&d)[Traits<DT>::VE / 2], f32x2 r2, const uint4& graw,
+                                                 const uint4& braw, uint4* dst) {
+    if (hg && hb) affine_store<DT, true, true>(d, r2, graw, braw, dst);
+    else if (hg)  affine_store<DT, true, false>(d, r2, graw, braw, dst);
+    else if (hb)  affine_store<DT, false, true>(d, r2, graw, braw, dst);
+    else          affine_store<DT, false, false>(d, r2, graw, braw, dst);
 }
 
 // ---------------------------------------------------------------------------------------------
 // (sub-)warp per row, registers
 // ---------------------------------------------------------------------------------------------
 template <int DT, int LANES, int VPL, int AFF>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(128)
 norm_warp_kernel(const NormParams p) {
-    constexpr int VE = Traits<DT>::VE;
+    constexpr int NP = Traits<DT>::VE / 2;
     constexpr int G = 32 / LANES;
     static_assert(AFF != 2, "per-run affine parameters are handled by the shared-memory kernel");
     pdl_launch_dependents();
@@ -149,56 +161,136 @@ norm_warp_kernel(const NormParams p) {
     const int nvec = static_cast<int>(p.nvec);
     const uint4* __restrict__ xv = static_cast<const uint4*>(p.x);
     uint4* __restrict__ yv = static_cast<uint4*>(p.y);
-    const uint4* gv = static_cast<const uint4*>(p.gamma);
-    const uint4* bv = static_cast<const uint4*>(p.beta);
+    const uint4* gv = AFF == 1 && p.gamma ? static_cast<const uint4*>(p.gamma) + sl : nullptr;
+    const uint4* bv = AFF == 1 && p.beta ? static_cast<const uint4*>(p.beta) + sl : nullptr;
     const float inv_n = 1.0f / static_cast<float>(p.cols);
     pdl_wait();
     const int64_t ngroups = (p.rows + G - 1) / G;
     for (int64_t grp = int64_t(blockIdx.x) * warps + (threadIdx.x >> 5); grp < ngroups; grp += int64_t(gridDim.x) * warps) {
         const int64_t row = grp * G + sub;
         const bool row_ok = row < p.rows;
+        const uint4* xr = xv + row * p.nvec + sl;
         uint4 raw[VPL];
-        float x[VPL][VE];
-        float s = 0.0f;
 #pragma unroll
         for (int k = 0; k < VPL; ++k) {
             raw[k] = make_uint4(0u, 0u, 0u, 0u);
-            if (row_ok && sl + k * LANES < nvec) raw[k] = ld_stream(xv + row * p.nvec + sl + k * LANES);
+            if (row_ok && sl + k * LANES < nvec) raw[k] = ld_stream(xr + k * LANES);
         }
+        f32x2 x[VPL][NP];
+        f32x2 acc[2] = {pair(0.0f, 0.0f), pair(0.0f, 0.0f)};
 #pragma unroll
         for (int k = 0; k < VPL; ++k) {
-            unpack<DT>(raw[k], x[k]);
+            widen_pairs<DT>(raw[k], x[k]);                                  // absent vectors are zeros
 #pragma unroll
-            for (int i = 0; i < VE; ++i) s += x[k][i];                     // absent vectors are zeros
+            for (int j = 0; j < NP; ++j) acc[j & 1] = add2(acc[j & 1], x[k][j]);
         }
-        const float mu = warp_sum<LANES>(s) * inv_n;
-        float q = 0.0f;
+        const float mu = warp_sum<LANES>(pair_sum(add2(acc[0], acc[1]))) * inv_n;
+        const f32x2 mu2 = pair(mu, mu);
+        acc[0] = pair(0.0f, 0.0f); acc[1] = pair(0.0f, 0.0f);
 #pragma unroll
         for (int k = 0; k < VPL; ++k) {
-            const bool live = sl + k * LANES < nvec;
+            if (sl + k * LANES < nvec) {
 #pragma unroll
-            for (int i = 0; i < VE; ++i) {
-                x[k][i] -= mu;
-                if (live) q = fmaf(x[k][i], x[k][i], q);
+                for (int j = 0; j < NP; ++j) { x[k][j] = sub2(x[k][j], mu2); acc[j & 1] = fma2(x[k][j], x[k][j], acc[j & 1]); }
             }
         }
-        const float rstd = 1.0f / sqrtf(warp_sum<LANES>(q) * inv_n + p.eps);
+        const float rstd = rstd_of(warp_sum<LANES>(pair_sum(add2(acc[0], acc[1]))) * inv_n, p.eps);
+        const f32x2 r2 = pair(rstd, rstd);
         if (row_ok) {
+            uint4* yr = yv + row * p.nvec + sl;
 #pragma unroll
             for (int k = 0; k < VPL; ++k) {
                 if (sl + k * LANES < nvec) {
-                    float g[VE], b[VE];
-                    if (AFF == 1 && gv) unpack<DT>(ld_cached(gv + sl + k * LANES), g);
-                    if (AFF == 1 && bv) unpack<DT>(ld_cached(bv + sl + k * LANES), b);
-#pragma unroll
-                    for (int i = 0; i < VE; ++i) {
-                        float t = x[k][i] * rstd;
-                        if (AFF == 1 && gv) t *= g[i];
-                        if (AFF == 1 && bv) t += b[i];
-                        x[k][i] = t;
-                    }
-                    st_stream(yv + row * p.nvec + sl + k * LANES, pack<DT>(x[k]));
+                    uint4 graw = make_uint4(0u, 0u, 0u, 0u), braw = make_uint4(0u, 0u, 0u, 0u);
+                    if (gv) graw = ld_cached(gv + k * LANES);
+                    if (bv) braw = ld_cached(bv + k * LANES);
+                    affine_store_any<DT>(gv != nullptr, bv != nullptr, x[k], r2, graw, braw, yr + k * LANES);
                 }
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// block per row, registers; a block takes `rows_per_block` consecutive rows
+// Thread t holds vectors t, t + T, ... of the row, so it meets the same columns in every row:
+// its gamma and beta vectors are loaded once and stay in registers (packed). The next row's
+// vectors are requested before the current row is reduced, so the row-wide barrier does not
+// leave the memory system idle.
+// ---------------------------------------------------------------------------------------------
+template <int DT, int VPT, int AFF>
+__global__ void __launch_bounds__(256)
+norm_block_kernel(const NormParams p, const int rows_per_block) {
+    constexpr int NP = Traits<DT>::VE / 2;
+    static_assert(AFF != 2, "per-run affine parameters are handled by the shared-memory kernel");
+    __shared__ float red[2][2][32];
+    pdl_launch_dependents();
+    const int T = blockDim.x, tid = threadIdx.x, lane = tid & 31, nwarps = T >> 5;
+    const int nvec = static_cast<int>(p.nvec);
+    const uint4* __restrict__ xv = static_cast<const uint4*>(p.x);
+    uint4* __restrict__ yv = static_cast<uint4*>(p.y);
+    const int64_t row0 = int64_t(blockIdx.x) * rows_per_block;
+    const int64_t row_end = min(p.rows, row0 + rows_per_block);
+    const float inv_n = 1.0f / static_cast<float>(p.cols);
+    pdl_wait();
+    uint4 graw[VPT], braw[VPT];
+    const bool hg = AFF == 1 && p.gamma != nullptr, hb = AFF == 1 && p.beta != nullptr;
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+        graw[k] = make_uint4(0u, 0u, 0u, 0u); braw[k] = make_uint4(0u, 0u, 0u, 0u);
+        if (hg && tid + k * T < nvec) graw[k] = ld_cached(static_cast<const uint4*>(p.gamma) + tid + k * T);
+        if (hb && tid + k * T < nvec) braw[k] = ld_cached(static_cast<const uint4*>(p.beta) + tid + k * T);
+    }
+    uint4 next[VPT];
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+        next[k] = make_uint4(0u, 0u, 0u, 0u);
+        if (row0 < row_end && tid + k * T < nvec) next[k] = ld_stream(xv + row0 * p.nvec + tid + k * T);
+    }
+    int par = 0;
+    for (int64_t row = row0; row < row_end; ++row, par ^= 1) {
+        f32x2 x[VPT][NP];
+        f32x2 acc[2] = {pair(0.0f, 0.0f), pair(0.0f, 0.0f)};
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            widen_pairs<DT>(next[k], x[k]);                  // absent vectors are zeros
+#pragma unroll
+            for (int j = 0; j < NP; ++j) acc[j & 1] = add2(acc[j & 1], x[k][j]);
+        }
+        if (row + 1 < row_end) {
+#pragma unroll
+            for (int k = 0; k < VPT; ++k)
+                if (tid + k * T < nvec) next[k] = ld_stream(xv + (row + 1) * p.nvec + tid + k * T);
+        }
+        // exact two-pass statistics: the row sum first, then the squared deviations from the mean
+        float s = warp_sum<32>(pair_sum(add2(acc[0], acc[1])));
+        if (nwarps > 1) {
+            if (lane == 0) red[par][0][tid >> 5] = s;
+            __syncthreads();
+            s = warp_sum<32>(lane < nwarps ? red[par][0][lane] : 0.0f);
+        }
+        const float mu = s * inv_n;
+        const f32x2 mu2 = pair(mu, mu);
+        acc[0] = pair(0.0f, 0.0f); acc[1] = pair(0.0f, 0.0f);
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            if (tid + k * T < nvec) {
+#pragma unroll
+                for (int j = 0; j < NP; ++j) { x[k][j] = sub2(x[k][j], mu2); acc[j & 1] = fma2(x[k][j], x[k][j], acc[j & 1]); }
+            }
+        }
+        float q = warp_sum<32>(pair_sum(add2(acc[0], acc[1])));
+        if (nwarps > 1) {
+            if (lane == 0) red[par][1][tid >> 5] = q;
+            __syncthreads();
+            q = warp_sum<32>(lane < nwarps ? red[par][1][lane] : 0.0f);
+        }
+        const float rstd = rstd_of(q * inv_n, p.eps);
+        const f32x2 r2 = pair(rstd, rstd);
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            if (tid + k * T < nvec) {
+                affine_store_any<DT>(hg, hb, x[k], r2, graw[k], braw[k], yv + row * p.nvec + tid + k * T);
             }
         }
     }
@@ -210,6 +302,70 @@ norm_warp_kernel(const NormParams p) {
 // FULL: every block's slice is exactly nchunk_full chunks of 8 * blockDim.x vectors.
 // ---------------------------------------------------------------------------------------------
 constexpr int kNormMaxChunks = 8;
+
+struct Pass2Ctx {
+    const uint4* sv;       // this thread's first vector of the resident slice
+    uint4* yv;             // and of the output row
+    const uint4* gv;       // AFF 1: gamma / beta at the same column (null: absent)
+    const uint4* bv;
+    f32x2 mu2, r2;
+    int nchunk, chunk_vecs, nv, tpos, v0;
+};
+
+// Pass 2 of the shared-memory kernel. Which affine vectors exist is a template parameter, chosen
+// once per kernel: the loads of a half-chunk (x from shared memory, gamma and beta from L1/L2) are
+// issued together, unconditionally, before any arithmetic.
+template <int DT, bool FULL, int AFF, bool HG, bool HB>
+__device__ __forceinline__ void norm_pass2(const NormParams& p, const Pass2Ctx& c, int64_t row) {
+    constexpr int VE = Traits<DT>::VE;
+    constexpr int NP = VE / 2;
+    constexpr int H = 4;                                   // vectors per batch
+    const int run_vecs = AFF == 2 ? static_cast<int>(p.run_elems / VE) : 1;
+    const int64_t chan0 = AFF == 2 ? (row % p.aff_rows) * (p.nvec / run_vecs) : 0;     // first channel of this row's group
+    for (int ch = 0; ch < c.nchunk; ++ch) {
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            const int off = ch * c.chunk_vecs + half * H * 32;
+            const int cbase = off + c.tpos;
+            uint4 raw[H], graw[H], braw[H];
+#pragma unroll
+            for (int u = 0; u < H; ++u) raw[u] = c.sv[off + u * 32];
+            if (AFF == 1) {
+#pragma unroll
+                for (int u = 0; u < H; ++u) {
+                    const bool in = FULL || cbase + u * 32 < c.nv;      // never read past the end of gamma / beta
+                    graw[u] = make_uint4(0u, 0u, 0u, 0u); braw[u] = make_uint4(0u, 0u, 0u, 0u);
+                    if (HG && in) graw[u] = ld_cached(c.gv + off + u * 32);
+                    if (HB && in) braw[u] = ld_cached(c.bv + off + u * 32);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < H; ++u) {
+                if (FULL || cbase + u * 32 < c.nv) {
+                    f32x2 x[NP];
+                    widen_pairs<DT>(raw[u], x);
+#pragma unroll
+                    for (int k = 0; k < NP; ++k) x[k] = sub2(x[k], c.mu2);
+                    if (AFF == 1) {
+                        affine_store<DT, HG, HB>(x, c.r2, graw[u], braw[u], c.yv + off + u * 32);
+                    } else if (AFF == 2) {
+                        const int64_t chn = chan0 + (c.v0 + cbase + u * 32) / run_vecs;
+                        const float gs = p.gamma ? load_elem<DT>(p.gamma, chn) : 1.0f;
+                        const float bs = p.beta ? load_elem<DT>(p.beta, chn) : 0.0f;
+                        float rlo, rhi;
+                        unpair(c.r2, rlo, rhi);
+                        const f32x2 a2 = pair(rlo * gs, rlo * gs), b2 = pair(bs, bs);
+#pragma unroll
+                        for (int k = 0; k < NP; ++k) x[k] = fma2(x[k], a2, b2);
+                        st_stream(c.yv + off + u * 32, narrow_pairs<DT>(x));
+                    } else {
+                        affine_store<DT, false, false>(x, c.r2, raw[u], raw[u], c.yv + off + u * 32);
+                    }
+                }
+            }
+        }
+    }
+}
 
 template <int DT, bool FULL, int AFF>
 __global__ void __launch_bounds__(256, 3)
@@ -287,7 +443,7 @@ norm_smem_kernel(const NormParams p, const uint32_t stage_bytes, const int slice
             for (int k = 0; k < NP; ++k) acc[k & 1] = add2(acc[k & 1], x[k]);
         }
         const float cnt = static_cast<float>(nvalid * VE);
-        const float mean_c = nvalid > 0 ? pair_sum(add2(acc[0], acc[1])) / cnt : 0.0f;
+        const float mean_c = nvalid > 0 ? pair_sum(add2(acc[0], acc[1])) * fast_rcp(cnt) : 0.0f;
         const f32x2 m2c = pair(mean_c, mean_c);
         acc[0] = pair(0.0f, 0.0f); acc[1] = pair(0.0f, 0.0f);
 #pragma unroll
@@ -328,35 +484,21 @@ norm_smem_kernel(const NormParams p, const uint32_t stage_bytes, const int slice
         st.n = v.x; st.mean = v.y; st.m2 = v.z;
         st = warp_merge_stats<32>(st);
     }
-    const float rstd = rstd_of(st.m2, st.n, p.eps);
+    const float rstd = rstd_of(st.m2 * fast_rcp(st.n), p.eps);
     const f32x2 mu2 = pair(st.mean, st.mean), r2 = pair(rstd, rstd);
 
     // ---- pass 2: normalise from the resident slice
-    uint4* __restrict__ yv = static_cast<uint4*>(p.y) + row * p.nvec + v0 + tpos;
-    const uint4* gv = AFF == 1 && p.gamma ? static_cast<const uint4*>(p.gamma) + v0 + tpos : nullptr;
-    const uint4* bv = AFF == 1 && p.beta ? static_cast<const uint4*>(p.beta) + v0 + tpos : nullptr;
-    const int run_vecs = AFF == 2 ? static_cast<int>(p.run_elems / VE) : 1;
-    const int64_t chan0 = AFF == 2 ? (row % p.aff_rows) * (p.nvec / run_vecs) : 0;     // first channel of this row's group
-    for (int ch = 0; ch < nchunk; ++ch) {
-        const uint4* sc = sv + ch * chunk_vecs;
-        const int cbase = ch * chunk_vecs + tpos;
-        uint4 raw[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) raw[u] = sc[u * 32];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            if (FULL || cbase + u * 32 < nv) {
-                float gs = 1.0f, bs = 0.0f;
-                if (AFF == 2) {
-                    const int64_t c = chan0 + (v0 + cbase + u * 32) / run_vecs;
-                    if (p.gamma) gs = load_elem<DT>(p.gamma, c);
-                    if (p.beta) bs = load_elem<DT>(p.beta, c);
-                }
-                const uint4 o = norm_vec<DT, AFF>(raw[u], mu2, r2, gv ? gv + ch * chunk_vecs + u * 32 : nullptr,
-                                                  bv ? bv + ch * chunk_vecs + u * 32 : nullptr, gs, bs);
-                st_stream(yv + ch * chunk_vecs + u * 32, o);
-            }
-        }
+    Pass2Ctx c2;
+    c2.sv = sv; c2.yv = static_cast<uint4*>(p.y) + row * p.nvec + v0 + tpos;
+    c2.gv = AFF == 1 && p.gamma ? static_cast<const uint4*>(p.gamma) + v0 + tpos : nullptr;
+    c2.bv = AFF == 1 && p.beta ? static_cast<const uint4*>(p.beta) + v0 + tpos : nullptr;
+    c2.mu2 = mu2; c2.r2 = r2; c2.nchunk = nchunk; c2.chunk_vecs = chunk_vecs; c2.nv = nv; c2.tpos = tpos; c2.v0 = v0;
+    if (AFF == 1) {
+        if (c2.gv && c2.bv) norm_pass2<DT, FULL, 1, true, true>(p, c2, row);
+        else if (c2.gv)     norm_pass2<DT, FULL, 1, true, false>(p, c2, row);
+        else                norm_pass2<DT, FULL, 1, false, true>(p, c2, row);
+    } else {
+        norm_pass2<DT, FULL, AFF, false, false>(p, c2, row);
     }
 }
 
@@ -390,7 +532,7 @@ norm_generic_kernel(const NormParams p, const int aff) {
             const float d = load_elem<DT>(p.x, base + j) - mu;
             q = fmaf(d, d, q);
         }
-        const float rstd = 1.0f / sqrtf(block_sum(q, red) * inv_n + p.eps);
+        const float rstd = rstd_of(block_sum(q, red) * inv_n, p.eps);
         const int64_t chan0 = aff == 2 ? (row % p.aff_rows) * (p.cols / p.run_elems) : 0;
         for (int64_t j = threadIdx.x; j < p.cols; j += blockDim.x) {
             float t = (load_elem<DT>(p.x, base + j) - mu) * rstd;

@@ -90,6 +90,28 @@ def test_layer_norm_row_lengths_across_the_split_geometries(dtype):
         check_layer(x, dtype, gamma, beta, 1e-5)
 
 
+@pytest.mark.parametrize("rows,cols,dtype", [(16384, 1536, BF16), (40000, 2304, BF16), (38000, 4096, FP16), (8192, 4096, FP32)])
+def test_layer_norm_at_benchmark_sizes(rows, cols, dtype):
+    """The benchmark's layer_norm shapes, and row counts at which the block kernel takes eight rows per
+    block (gamma and beta kept in registers, next row requested early). Compared in slabs of rows."""
+    from oracle import fso
+    rng = np.random.default_rng(rows + cols)
+    gamma = stored(rng.standard_normal(cols) * 0.2 + 1.0, dtype)
+    beta = stored(rng.standard_normal(cols) * 0.1, dtype)
+    x = np.empty((rows, cols), dtype=W.NP_STORE[dtype])
+    for r0 in range(0, rows, 4096):
+        r1 = min(rows, r0 + 4096)
+        x[r0:r1] = stored(rng.standard_normal((r1 - r0, cols)) * 1.5 + 0.25, dtype)
+    y = run_layer(x, dtype, gamma, beta, 1e-5)
+    g64, b64 = fso.widen(gamma, dtype)[None, :], fso.widen(beta, dtype)[None, :]
+    for r0 in range(0, rows, 4096):
+        r1 = min(rows, r0 + 4096)
+        want = fno.layer_norm_f64(x[r0:r1], dtype, gamma, beta, 1e-5)
+        scale = fno.error_scale(x[r0:r1], dtype, (r1 - r0, cols), g64, b64, 1e-5)
+        rep = fno.compare(y[r0:r1], dtype, want, scale)
+        assert rep.ok(dtype), (r0, rep)
+
+
 @pytest.mark.parametrize("dtype", [FP32, BF16, FP16])
 def test_layer_norm_edge_cases(dtype):
     # constant rows: zero variance, y = beta; eps = 0 with a constant row is 0 * inf = NaN in both
