@@ -843,6 +843,23 @@ template <int DT> const void* norm_smem_fn(bool full, int aff) {
                                                                             : (const void*)norm_smem_kernel<DT, false, 2>;
 }
 
+template <int DT> const void* norm_apply_fn(int aff) {
+    return aff == 0 ? (const void*)norm_apply_kernel<DT, 0> : aff == 1 ? (const void*)norm_apply_kernel<DT, 1>
+                                                                        : (const void*)norm_apply_kernel<DT, 2>;
+}
+
+// FS_NORM_SPLIT=0 / 1 (read once) forces the choice for experiments.
+bool norm_split_wanted(const Device& dev, int64_t rows, int64_t nvec, bool smem_ok, int cs) {
+    static const int forced = [] { const char* e = std::getenv("FS_NORM_SPLIT"); return e ? std::atoi(e) : -1; }();
+    if (forced == 0) return false;
+    if (forced == 1) return true;
+    // Rows that a cluster's shared memory holds stay there: measured on B200 (one image, 32 groups of
+    // 0.5 / 1 / 2 MiB), the cluster kernel takes 12.7 / 21.3 / 43.9 us where the two-kernel form takes
+    // 19.4 / 29.5 / 46.4 (two launches, and the second read does not stay in L2).
+    (void)dev; (void)rows; (void)cs;
+    return !smem_ok && nvec * 16 >= (int64_t(1) << 20);
+}
+
 template <typename F> const void* by_dtype(int dtype, F f) {
     switch (dtype) {
         case FS_DTYPE_FP32: return f(std::integral_constant<int, DT_F32>{});
@@ -893,7 +910,31 @@ int run_norm(const void* x, const void* gamma, const void* beta, void* y, int64_
         if (grid <= 0x7fffffff) return launch(fn, grid, bthreads, 0, 0, st, p, static_cast<int>(rpb));
     }
     SmemGeom sg;
-    if (fast && dev.cluster_ok && smem_geom(p.nvec, dtype, 0, 0, &sg) && rows <= 0x7fffffff / sg.cs) {
+    const bool smem_ok = fast && dev.cluster_ok && smem_geom(p.nvec, dtype, 0, 0, &sg) && rows <= 0x7fffffff / sg.cs;
+    // Few, very long rows (group_norm of a large image): a cluster per row leaves most of the GPU
+    // idle, or the row does not fit a cluster's shared memory at all. Then the rows are cut into
+    // segments over a grid that fills the GPU, with the partial statistics exchanged through a
+    // stream-ordered scratch buffer between two kernels.
+    if (fast && norm_split_wanted(dev, rows, p.nvec, smem_ok, smem_ok ? sg.cs : 0)) {
+        const int t = 256;
+        const int64_t target = int64_t(dev.sm_count) * 8;
+        int64_t nseg = std::max<int64_t>(1, std::min<int64_t>(1024, (target + rows - 1) / rows));
+        int64_t seg_vecs = ((p.nvec + nseg - 1) / nseg + 4 * t - 1) / (4 * t) * (4 * t);
+        nseg = (p.nvec + seg_vecs - 1) / seg_vecs;
+        if (rows * nseg <= 0x7fffffff) {
+            float4* part = nullptr;
+            FS_CUDA(cudaMallocAsync(reinterpret_cast<void**>(&part), static_cast<size_t>(rows * nseg) * sizeof(float4), st));
+            const void* f1 = by_dtype(dtype, [&](auto dt) -> const void* { return (const void*)norm_partial_kernel<decltype(dt)::value>; });
+            const void* f2 = by_dtype(dtype, [&](auto dt) -> const void* { return norm_apply_fn<decltype(dt)::value>(aff); });
+            const float4* cpart = part;
+            rc = launch(f1, rows * nseg, t, 0, 0, st, p, part, static_cast<int>(nseg), static_cast<int>(seg_vecs));
+            if (rc == FS_OK) rc = launch(f2, rows * nseg, t, 0, 0, st, p, cpart, static_cast<int>(nseg), static_cast<int>(seg_vecs));
+            const cudaError_t fe = cudaFreeAsync(part, st);
+            if (rc == FS_OK && fe != cudaSuccess) return cuda_fail(fe);
+            return rc;
+        }
+    }
+    if (smem_ok) {
         const bool full = smem_row_full(sg, dtype, p.nvec);
         const void* fn = by_dtype(dtype, [&](auto dt) -> const void* { return norm_smem_fn<decltype(dt)::value>(full, aff); });
         const size_t stage_bytes = smem_row_stage_bytes(sg, dtype);

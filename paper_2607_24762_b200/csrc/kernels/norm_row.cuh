@@ -13,6 +13,8 @@
 //                        takes the exact mean and M2 of its own 8 vectors and merges them into
 //                        its running triple; triples merge warp -> block -> cluster (st.async
 //                        deposits counted by an mbarrier); pass 2 normalises from shared memory
+//   norm_partial_kernel + norm_apply_kernel   few, very long rows: segments of a row on separate
+//                        blocks, partial triples exchanged through global memory between the two
 //   norm_generic_kernel  block per row, three passes over global memory (the later ones normally
 //                        from L2): any column count, alignment and row length
 //
@@ -499,6 +501,150 @@ norm_smem_kernel(const NormParams p, const uint32_t stage_bytes, const int slice
         else                norm_pass2<DT, FULL, 1, false, true>(p, c2, row);
     } else {
         norm_pass2<DT, FULL, AFF, false, false>(p, c2, row);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// few, very long rows (group_norm of one large image): two kernels over a grid that fills the GPU.
+//   norm_partial_kernel  block (row, b) takes segment b of the row (seg_vecs vectors), reduces it
+//                        to one (n, mean, M2) triple and writes it to part[row * nseg + b]
+//   norm_apply_kernel    the same grid: a block merges its row's nseg triples, then normalises its
+//                        segment, re-reading x -- from L2 when the tensor fits there (the first
+//                        kernel reads with the default policy, this one with evict-first)
+// HBM traffic stays one read and one write per element when x fits L2; otherwise two reads.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint4 ld_keep(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+// (n, mean, M2) of four vectors, exact two-pass in registers; absent vectors (valid < 4) are skipped.
+template <int DT>
+__device__ __forceinline__ Stat stat_of_vectors(const uint4 (&raw)[4], int valid) {
+    constexpr int VE = Traits<DT>::VE;
+    constexpr int NP = VE / 2;
+    f32x2 acc[2] = {pair(0.0f, 0.0f), pair(0.0f, 0.0f)};
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        f32x2 x[NP];
+        widen_pairs<DT>(raw[u], x);                 // absent vectors were loaded as zeros
+#pragma unroll
+        for (int k = 0; k < NP; ++k) acc[k & 1] = add2(acc[k & 1], x[k]);
+    }
+    Stat c;
+    c.n = static_cast<float>(valid * VE);
+    c.mean = valid > 0 ? pair_sum(add2(acc[0], acc[1])) * fast_rcp(c.n) : 0.0f;
+    const f32x2 m2 = pair(c.mean, c.mean);
+    acc[0] = pair(0.0f, 0.0f); acc[1] = pair(0.0f, 0.0f);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        if (u < valid) {
+            f32x2 x[NP];
+            widen_pairs<DT>(raw[u], x);
+#pragma unroll
+            for (int k = 0; k < NP; ++k) { const f32x2 d = sub2(x[k], m2); acc[k & 1] = fma2(d, d, acc[k & 1]); }
+        }
+    }
+    c.m2 = pair_sum(add2(acc[0], acc[1]));
+    return c;
+}
+
+template <int DT>
+__global__ void __launch_bounds__(256)
+norm_partial_kernel(const NormParams p, float4* __restrict__ part, const int nseg, const int seg_vecs) {
+    __shared__ float4 wp[32];
+    pdl_launch_dependents();
+    const int T = blockDim.x, tid = threadIdx.x, lane = tid & 31, nwarps = T >> 5;
+    const int64_t row = blockIdx.x / nseg;
+    const int b = static_cast<int>(blockIdx.x % nseg);
+    const int64_t v0 = int64_t(b) * seg_vecs;
+    const int nv = static_cast<int>(min(int64_t(seg_vecs), p.nvec - v0));
+    const uint4* __restrict__ xv = static_cast<const uint4*>(p.x) + row * p.nvec + v0;
+    pdl_wait();
+    Stat st = {0.0f, 0.0f, 0.0f};
+    for (int base = 0; base < nv; base += 4 * T) {          // a thread takes vectors base + tid + u T
+        uint4 raw[4];
+        int valid = 0;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            raw[u] = make_uint4(0u, 0u, 0u, 0u);
+            if (base + tid + u * T < nv) { raw[u] = ld_keep(xv + base + tid + u * T); valid = u + 1; }
+        }
+        st = stat_merge(st, stat_of_vectors<DT>(raw, valid));
+    }
+    st = warp_merge_stats<32>(st);
+    if (nwarps > 1) {
+        if (lane == 0) wp[tid >> 5] = make_float4(st.n, st.mean, st.m2, 0.0f);
+        __syncthreads();
+        const float4 v = lane < nwarps ? wp[lane] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        st.n = v.x; st.mean = v.y; st.m2 = v.z;
+        st = warp_merge_stats<32>(st);
+    }
+    if (tid == 0) part[blockIdx.x] = make_float4(st.n, st.mean, st.m2, 0.0f);
+}
+
+template <int DT, int AFF>
+__global__ void __launch_bounds__(256)
+norm_apply_kernel(const NormParams p, const float4* __restrict__ part, const int nseg, const int seg_vecs) {
+    constexpr int VE = Traits<DT>::VE;
+    constexpr int NP = VE / 2;
+    pdl_launch_dependents();
+    const int T = blockDim.x, tid = threadIdx.x, lane = tid & 31;
+    const int64_t row = blockIdx.x / nseg;
+    const int b = static_cast<int>(blockIdx.x % nseg);
+    const int64_t v0 = int64_t(b) * seg_vecs;
+    const int nv = static_cast<int>(min(int64_t(seg_vecs), p.nvec - v0));
+    const uint4* __restrict__ xv = static_cast<const uint4*>(p.x) + row * p.nvec + v0;
+    uint4* __restrict__ yv = static_cast<uint4*>(p.y) + row * p.nvec + v0;
+    pdl_wait();
+    // every warp merges the row's partial triples (nseg <= 1024: up to 32 per lane)
+    Stat st = {0.0f, 0.0f, 0.0f};
+    for (int j = lane; j < nseg; j += 32) {
+        const float4 v = part[row * nseg + j];
+        Stat t; t.n = v.x; t.mean = v.y; t.m2 = v.z;
+        st = stat_merge(st, t);
+    }
+    st = warp_merge_stats<32>(st);
+    const float rstd = rstd_of(st.m2 * fast_rcp(st.n), p.eps);
+    const f32x2 mu2 = pair(st.mean, st.mean), r2 = pair(rstd, rstd);
+    const uint4* gv = AFF == 1 && p.gamma ? static_cast<const uint4*>(p.gamma) + v0 : nullptr;
+    const uint4* bv = AFF == 1 && p.beta ? static_cast<const uint4*>(p.beta) + v0 : nullptr;
+    const int run_vecs = AFF == 2 ? static_cast<int>(p.run_elems / VE) : 1;
+    const int64_t chan0 = AFF == 2 ? (row % p.aff_rows) * (p.nvec / run_vecs) : 0;
+    for (int base = 0; base < nv; base += 4 * T) {
+        uint4 raw[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            raw[u] = make_uint4(0u, 0u, 0u, 0u);
+            if (base + tid + u * T < nv) raw[u] = ld_stream(xv + base + tid + u * T);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int v = base + tid + u * T;
+            if (v < nv) {
+                f32x2 x[NP];
+                widen_pairs<DT>(raw[u], x);
+#pragma unroll
+                for (int k = 0; k < NP; ++k) x[k] = sub2(x[k], mu2);
+                if (AFF == 1) {
+                    uint4 graw = make_uint4(0u, 0u, 0u, 0u), braw = make_uint4(0u, 0u, 0u, 0u);
+                    if (gv) graw = ld_cached(gv + v);
+                    if (bv) braw = ld_cached(bv + v);
+                    affine_store_any<DT>(gv != nullptr, bv != nullptr, x, r2, graw, braw, yv + v);
+                } else if (AFF == 2) {
+                    const int64_t chn = chan0 + (v0 + v) / run_vecs;
+                    const float gs = p.gamma ? load_elem<DT>(p.gamma, chn) : 1.0f;
+                    const float bs = p.beta ? load_elem<DT>(p.beta, chn) : 0.0f;
+                    const f32x2 a2 = pair(rstd * gs, rstd * gs), b2 = pair(bs, bs);
+#pragma unroll
+                    for (int k = 0; k < NP; ++k) x[k] = fma2(x[k], a2, b2);
+                    st_stream(yv + v, narrow_pairs<DT>(x));
+                } else {
+                    affine_store<DT, false, false>(x, r2, raw[u], raw[u], yv + v);
+                }
+            }
+        }
     }
 }
 

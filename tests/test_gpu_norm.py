@@ -82,7 +82,7 @@ def test_layer_norm_shape_sweep(dtype):
 def test_layer_norm_row_lengths_across_the_split_geometries(dtype):
     esz = W.ELEM_SIZE[dtype]
     for kb, rows in ((3, 700), (6, 500), (8, 3000), (12, 900), (24, 400), (40, 300), (48, 260), (96, 150), (100, 120), (160, 100),
-                     (250.5, 60), (384, 40), (600, 30), (1024, 12), (2048, 5), (3000, 3)):
+                     (250.5, 60), (384, 40), (600, 30), (1024, 12), (2048, 5), (3000, 3), (5000, 3), (16384, 2)):
         cols = int(kb * 1024) // esz
         x = make_case(rows, cols, dtype, seed=int(kb), offset=0.25)
         gamma = stored(np.random.default_rng(1).standard_normal(cols) * 0.5 + 1.0, dtype)
@@ -165,7 +165,8 @@ def test_group_norm(dtype):
     from oracle import fso
     for ci, (n, ch, sp, groups) in enumerate([(2, 8, 16, 4), (1, 32, 64, 32), (3, 64, 256, 32), (2, 128, 1024, 32), (1, 512, 4096, 32),
                                               (1, 256, 16384, 32), (2, 6, 5, 3), (1, 12, 1000, 4), (1, 4, 100000, 2),
-                                              (1, 128, 65536, 32), (1, 32, 8, 1)]):
+                                              (1, 128, 65536, 32), (1, 32, 8, 1),
+                                              (1, 4, 900000, 2), (2, 2, 1 << 21, 1)]):      # rows beyond a cluster's shared memory: two-kernel path
         rng = np.random.default_rng(40 + ci)
         x64 = rng.standard_normal((n, ch, sp)) * (1 + rng.random((1, ch, 1)) * 2) + rng.standard_normal((1, ch, 1))
         x = stored(x64, dtype)
