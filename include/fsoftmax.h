@@ -1,5 +1,6 @@
 /*
- * libfsoftmax -- last-dimension softmax for NVIDIA B200 (sm_100a), C ABI.
+ * libfsoftmax -- last-dimension softmax for NVIDIA B200 (sm_100a), C ABI, with the operators that
+ * share its row skeleton (causal softmax, router softmax + top-k, layer_norm, group_norm).
  *
  * The operation is the `softmax` operator the paper reports its largest gains on (abstract and
  * Sec. IV-C: Gemma 4 E2B and Qwen 3.5 35B-A3B eager-attention softmax); its semantics are the
@@ -139,9 +140,13 @@ int fs_router_topk(const void* x, float* w, int32_t* idx, int64_t rows, int64_t 
  *   gamma, beta   device pointers to cols elements of `dtype`, or NULL (1 and 0), independently.
  *   eps     finite, >= 0. Statistics and arithmetic are binary32; the output is rounded once.
  *   stream  cudaStream_t as void*.
- * Rows up to 2 KiB stay in the registers of a (sub-)warp; longer rows are split over a cluster of
- * 1..16 blocks with the slices resident in shared memory (one read and one write of HBM per
- * element, as for fs_softmax); ragged, misaligned or longer rows take a three-pass kernel.
+ * Rows up to 4 KiB stay in the registers of a (sub-)warp; 16-bit rows of 4-9 KiB in the registers
+ * of a block (eight rows per block, gamma and beta kept in registers); longer rows are split over
+ * a cluster of 1..16 blocks with the slices resident in shared memory (one read and one write of
+ * HBM per element, as for fs_softmax); rows beyond a cluster's shared memory (about 3 MiB) are
+ * cut into segments over two kernels, whose partial statistics pass through a scratch buffer that
+ * is allocated and freed in stream order (cudaMallocAsync on `stream`); ragged or misaligned
+ * rows take a three-pass kernel.
  * A NaN or infinity in a row makes the whole row NaN. rows == 0 or cols == 0 launches nothing.
  */
 int fs_layer_norm(const void* x, const void* gamma, const void* beta, void* y, int64_t rows, int64_t cols, int dtype,
