@@ -72,6 +72,8 @@ def _load():
             lib.fso_softmax_f64.restype = None
             lib.fso_softmax_row_f64.argtypes = [vp, ci, i64, f32, vp]
             lib.fso_softmax_row_f64.restype = None
+            lib.fso_log_softmax_f64.argtypes = [vp, ci, i64, i64, f32, vp]
+            lib.fso_log_softmax_f64.restype = None
             lib.fso_softmax_causal_f64.argtypes = [vp, ci, i64, i64, i64, f32, vp]
             lib.fso_softmax_causal_f64.restype = None
             lib.fso_router_topk_f64.argtypes = [vp, ci, i64, i64, i64, f32, ci, vp, vp]
@@ -104,6 +106,18 @@ def softmax_f64(x: np.ndarray, dtype: int, scale: float = 1.0) -> np.ndarray:
     y = np.empty((rows, cols), dtype=np.float64)
     if rows and cols:
         _load().fso_softmax_f64(x.ctypes.data, dtype, rows, cols, np.float32(scale), y.ctypes.data)
+    return y
+
+
+def log_softmax_f64(x: np.ndarray, dtype: int, scale: float = 1.0) -> np.ndarray:
+    """fp64 log_softmax over the last axis of a 2-D array of stored elements."""
+    x = _stored(x, dtype)
+    if x.ndim != 2:
+        raise ValueError("x must be [rows, cols]")
+    rows, cols = x.shape
+    y = np.empty((rows, cols), dtype=np.float64)
+    if rows and cols:
+        _load().fso_log_softmax_f64(x.ctypes.data, dtype, rows, cols, np.float32(scale), y.ctypes.data)
     return y
 
 

@@ -161,6 +161,37 @@ void fso_softmax_f64(const void* x, int dtype, int64_t rows, int64_t cols, float
     }
 }
 
+// log_softmax, the logarithm of the same operator (the form language-model heads consume; the
+// paper's harness captures softmax-family operators per model, Sec. III-A):
+//   z_j = scale * x_j;  M = max_j z_j;  S = sum_j exp(z_j - M) (Neumaier);  y_j = (z_j - M) - log(S)
+// A -inf entry beside finite ones gives -inf; a NaN or +inf entry, or a row of only -inf, makes
+// the whole row NaN, as for the softmax.
+void fso_log_softmax_f64(const void* x, int dtype, int64_t rows, int64_t cols, float scale, double* y) {
+    const int64_t esz = (dtype == DT_FP32) ? 4 : 2;
+    const double sc = static_cast<double>(scale);
+    for (int64_t i = 0; i < rows; ++i) {
+        const void* xr = static_cast<const char*>(x) + i * cols * esz;
+        double* yr = y + i * cols;
+        if (cols <= 0) continue;
+        for (int64_t j = 0; j < cols; ++j) yr[j] = sc * widen(xr, dtype, j);
+        double M = yr[0];
+        for (int64_t j = 1; j < cols; ++j) {
+            if (yr[j] > M) M = yr[j];
+        }
+        double S = 0.0, comp = 0.0;
+        for (int64_t j = 0; j < cols; ++j) {
+            const double e = std::exp(yr[j] - M);
+            const double t = S + e;
+            if (std::fabs(S) >= std::fabs(e)) comp += (S - t) + e;
+            else                              comp += (e - t) + S;
+            S = t;
+        }
+        S += comp;
+        const double L = std::log(S);
+        for (int64_t j = 0; j < cols; ++j) yr[j] = (yr[j] - M) - L;
+    }
+}
+
 // Causal variant (the mask eager attention applies before its softmax; fusing it is the "operator
 // fusion" lever of the paper's Sec. II-B): row i keeps columns j <= i + q_offset and the softmax is
 // taken over the kept columns only; a masked column has z = -inf, i.e. y = exactly +0, whatever is
