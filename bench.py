@@ -262,6 +262,49 @@ def time_router(w: W.Workload, k: int, steps: int, warmup: int, l2_bytes: int):
             "rows_per_s": round(w.rows / (ms * 1e-3), 1), "frac_of_measured_copy": round(gbs / peak, 4)}
 
 
+def time_log_softmax(w: W.Workload, steps: int, warmup: int, l2_bytes: int, eager: bool = True):
+    """fs_log_softmax on a softmax workload's data: reads x once, writes y once."""
+    import torch
+
+    import paper_2607_24762_b200 as fs
+    n_pairs = int(max(1, min(16, math.ceil(4 * l2_bytes / w.min_bytes))))
+    xs, ys = device_buffers(w, n_pairs, threads=min(8, os.cpu_count() or 1))
+    stream = torch.cuda.current_stream()
+    lib = fs.binding.lib()
+
+    def launch(i):
+        j = i % n_pairs
+        st = lib.fs_log_softmax(xs[j].data_ptr(), ys[j].data_ptr(), w.rows, w.cols, w.dtype, w.scale_f32, stream.cuda_stream)
+        if st != 0:
+            raise RuntimeError(fs.fs_strerror(st))
+
+    tdt = {W.FP32: torch.float32, W.BF16: torch.bfloat16, W.FP16: torch.float16}[w.dtype]
+
+    def eager_launch(i):
+        torch.log_softmax(xs[i % n_pairs].view(tdt).view(w.rows, w.cols) * w.scale_f32, dim=-1)
+
+    def timed(fn, k):
+        for i in range(max(3, warmup)):
+            fn(i)
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        start.record(stream)
+        for i in range(k):
+            fn(i)
+        stop.record(stream)
+        torch.cuda.synchronize()
+        return start.elapsed_time(stop) / k
+
+    ms = timed(launch, steps)
+    peak, _ = measured_peak()
+    gbs = w.min_bytes / (ms * 1e-3) / 1e9
+    out = {"what": f"fs_log_softmax on {w.name}", "steps": steps, "ms_per_step": round(ms, 6), "algorithmic_bytes": w.min_bytes,
+           "GB/s": round(gbs, 1), "frac_of_measured_copy": round(gbs / peak, 4), "n_pairs": n_pairs}
+    if eager:
+        out["torch_eager_ms"] = round(timed(eager_launch, max(5, steps // 4)), 6)
+    return out
+
+
 # Normalisation workloads (synthetic, seeded on the device): the shapes of the two operators the paper
 # reports for Stable Diffusion 3.5 Medium (Sec. IV-C): layer_norm over the transformer's hidden size
 # (1536) for 4 x 4096 tokens, and the VAE decoder's 32-group group_norm at three resolutions.
@@ -475,7 +518,7 @@ def main():
                     help="also time the other workloads (default: on at --gpus 1)")
     ap.add_argument("--no-all", dest="all_workloads", action="store_false")
     ap.add_argument("--norm-workload", default="ln_sd35", choices=sorted(NORM_WORKLOADS), help="with --op norm")
-    ap.add_argument("--op", default="softmax", choices=["softmax", "causal", "router", "norm"],
+    ap.add_argument("--op", default="softmax", choices=["softmax", "causal", "router", "norm", "log_softmax"],
                     help="time only fs_softmax_causal (q_offset 0) or fs_router_topk (k=8, renormalised) on the "
                          "workload and print a short line (profiler captures of those kernels)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the cpu_baseline leg")
@@ -528,6 +571,8 @@ def main():
             alg = (kept + w.rows * w.cols) * w.elem_size
             r = {"ms_per_step": round(r["ms_per_step"], 6), "algorithmic_bytes": alg,
                  "GB/s": round(alg / (r["ms_per_step"] * 1e-3) / 1e9, 1)}
+        elif args.op == "log_softmax":
+            r = time_log_softmax(w, args.steps, args.warmup, l2, eager=not args.no_cpu)
         elif args.op == "norm":
             r = time_norm(args.norm_workload, args.steps, args.warmup, l2, eager=not args.no_cpu)
         else:
@@ -599,6 +644,12 @@ def main():
                 others["cfg3_router_top8"] = time_router(rw, 8, 500, 10, l2)
             except Exception as exc:                       # never lose the main line to an extra
                 others["cfg3_router_top8"] = {"error": str(exc)[:200]}
+            # log_softmax on the vocabulary-sized and the attention-score workloads
+            for lname in ("cfg4", "cfg2"):
+                try:
+                    others[lname + "_log_softmax"] = time_log_softmax(W.WORKLOADS[lname], 300, 10, l2)
+                except Exception as exc:
+                    others[lname + "_log_softmax"] = {"error": str(exc)[:200]}
             # the normalisation entry points on the shapes of the paper's second workload family
             for nname in NORM_WORKLOADS:
                 try:

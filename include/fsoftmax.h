@@ -129,6 +129,22 @@ int fs_router_topk(const void* x, float* w, int32_t* idx, int64_t rows, int64_t 
                    int renormalize, void* stream);
 
 /*
+ * fs_log_softmax -- the logarithm of the same operator, formed directly (the variant of the softmax
+ * family that language-model heads consume; operator variants are the paper's Sec. III-A):
+ *
+ *     y[i][j] = z[i][j] - max_k z[i][k] - ln sum_k exp(z[i][k] - max_k z[i][k]),   z = scale * x
+ *
+ *   x, y, rows, cols, dtype, scale, stream   as for fs_softmax (x == y allowed; scale may be zero
+ *   or negative). A -inf entry beside finite ones gives -inf; a NaN or +inf entry (after scaling),
+ *   or a row holding only -inf, makes the whole row NaN.
+ * fp32 output is within 1e-6 * max(1, |y|) of the fp64 value, 16-bit output within one unit in the
+ * last place of the correctly rounded fp64 value. Rows up to 4 KiB stay in the registers of a
+ * (sub-)warp, longer rows are split over a cluster with the slices resident in shared memory (one
+ * read and one write of HBM per element), ragged or misaligned rows take a three-pass kernel.
+ */
+int fs_log_softmax(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale, void* stream);
+
+/*
  * fs_layer_norm -- layer normalisation over the last dimension, one of the two normalisation
  * operators the paper reports generated kernels for (Sec. IV-C, Stable Diffusion 3.5 Medium):
  *

@@ -53,6 +53,8 @@ def lib() -> ctypes.CDLL:
             L.fs_softmax_causal.restype = ci
             L.fs_router_topk.argtypes = [vp, vp, vp, i64, i64, ci, ci, f32, ci, vp]
             L.fs_router_topk.restype = ci
+            L.fs_log_softmax.argtypes = [vp, vp, i64, i64, ci, f32, vp]
+            L.fs_log_softmax.restype = ci
             L.fs_layer_norm.argtypes = [vp, vp, vp, vp, i64, i64, ci, f32, vp]
             L.fs_layer_norm.restype = ci
             L.fs_group_norm.argtypes = [vp, vp, vp, vp, i64, i64, i64, i64, ci, f32, vp]
@@ -134,6 +136,11 @@ def fs_router_topk(x, w, idx, rows: int, cols: int, k: int, dtype: int, scale: f
     """Softmax over experts + top-k: w [rows, k] float32 and idx [rows, k] int32 device buffers."""
     _check(lib().fs_router_topk(_ptr(x), _ptr(w), _ptr(idx), rows, cols, k, dtype, scale, int(renormalize),
                                 _stream(stream)), "fs_router_topk")
+
+
+def fs_log_softmax(x, y, rows: int, cols: int, dtype: int, scale: float = 1.0, stream=None) -> None:
+    """y = log_softmax(scale * x) over the last dimension of a [rows, cols] device tensor."""
+    _check(lib().fs_log_softmax(_ptr(x), _ptr(y), rows, cols, dtype, scale, _stream(stream)), "fs_log_softmax")
 
 
 def fs_layer_norm(x, gamma, beta, y, rows: int, cols: int, dtype: int, eps: float = 1e-5, stream=None) -> None:
