@@ -5,7 +5,7 @@ eager mode and never sees a wrong or unsupported kernel.
 
     from paper_2607_24762_b200 import torch_op
     y = torch_op.softmax(x, dim=-1)                 # library kernel when the guard admits the call
-    with torch_op.patched():                        # torch.softmax / F.softmax / Tensor.softmax routed
+    with torch_op.patched():                        # softmax, log_softmax, layer_norm, group_norm routed
         out = model(inputs)                         # through the guard for the duration of the block
     torch_op.stats()                                # how many calls went where, and why not
 
@@ -33,6 +33,10 @@ _lock = threading.Lock()
 _eager_softmax = torch.softmax            # the unpatched operators, captured at import
 _eager_F_softmax = torch.nn.functional.softmax
 _eager_T_softmax = torch.Tensor.softmax
+_eager_log_softmax = torch.log_softmax
+_eager_F_log_softmax = torch.nn.functional.log_softmax
+_eager_F_layer_norm = torch.nn.functional.layer_norm
+_eager_F_group_norm = torch.nn.functional.group_norm
 
 
 def _count(key: str) -> None:
@@ -100,6 +104,80 @@ def softmax(x: torch.Tensor, dim: int = -1, dtype=None, scale: float = 1.0, out:
     return y
 
 
+def log_softmax(x: torch.Tensor, dim: int = -1, dtype=None):
+    """log_softmax over `dim`: the library kernel when admitted, else eager PyTorch."""
+    reason = why_not(x, dim, dtype)
+    if reason is None:
+        try:
+            binding.lib()
+        except RuntimeError:
+            reason = "library not built"
+    if reason is not None:
+        _count("eager:" + reason)
+        return _eager_log_softmax(x, dim, dtype=dtype)
+    cols = x.shape[-1]
+    y = torch.empty_like(x)
+    with torch.cuda.device(x.device):
+        binding.fs_log_softmax(x, y, x.numel() // cols, cols, _DTYPES[x.dtype], 1.0, torch.cuda.current_stream(x.device))
+    _count("library")
+    return y
+
+
+def _affine_ok(x, p, n):
+    return p is None or (isinstance(p, torch.Tensor) and p.is_cuda and p.device == x.device and p.dtype == x.dtype and
+                         p.is_contiguous() and p.numel() == n and not (torch.is_grad_enabled() and p.requires_grad))
+
+
+def layer_norm(x: torch.Tensor, normalized_shape, weight=None, bias=None, eps: float = 1e-5):
+    """layer_norm over the last dimension: the library kernel when admitted, else eager PyTorch."""
+    shape = tuple(normalized_shape) if not isinstance(normalized_shape, int) else (normalized_shape,)
+    reason = why_not(x, -1)
+    if reason is None and (len(shape) != 1 or shape[0] != x.shape[-1]):
+        reason = "normalized_shape is not the last dimension"
+    if reason is None and not (_affine_ok(x, weight, x.shape[-1]) and _affine_ok(x, bias, x.shape[-1])):
+        reason = "incompatible weight or bias"
+    if reason is None:
+        try:
+            binding.lib()
+        except RuntimeError:
+            reason = "library not built"
+    if reason is not None:
+        _count("eager:" + reason)
+        return _eager_F_layer_norm(x, shape, weight, bias, eps)
+    cols = x.shape[-1]
+    y = torch.empty_like(x)
+    with torch.cuda.device(x.device):
+        binding.fs_layer_norm(x, weight, bias, y, x.numel() // cols, cols, _DTYPES[x.dtype], float(eps),
+                              torch.cuda.current_stream(x.device))
+    _count("library")
+    return y
+
+
+def group_norm(x: torch.Tensor, num_groups: int, weight=None, bias=None, eps: float = 1e-5):
+    """group_norm of an [N, C, *] tensor: the library kernel when admitted, else eager PyTorch."""
+    reason = why_not(x, -1)
+    if reason is None and (x.dim() < 2 or num_groups < 1 or x.shape[1] % num_groups):
+        reason = "shape"
+    if reason is None and not (_affine_ok(x, weight, x.shape[1]) and _affine_ok(x, bias, x.shape[1])):
+        reason = "incompatible weight or bias"
+    if reason is None:
+        try:
+            binding.lib()
+        except RuntimeError:
+            reason = "library not built"
+    if reason is not None:
+        _count("eager:" + reason)
+        return _eager_F_group_norm(x, num_groups, weight, bias, eps)
+    n, ch = x.shape[0], x.shape[1]
+    spatial = x.numel() // (n * ch)
+    y = torch.empty_like(x)
+    with torch.cuda.device(x.device):
+        binding.fs_group_norm(x, weight, bias, y, n, ch, spatial, num_groups, _DTYPES[x.dtype], float(eps),
+                              torch.cuda.current_stream(x.device))
+    _count("library")
+    return y
+
+
 def _patched_softmax(input, dim=None, *, dtype=None, **kw):        # torch.softmax(input, dim, dtype=None)
     if kw or dim is None:
         return _eager_softmax(input, dim, dtype=dtype, **kw)
@@ -118,14 +196,32 @@ def _patched_T_softmax(self, dim=None, dtype=None, **kw):
     return softmax(self, dim, dtype)
 
 
+def _patched_F_log_softmax(input, dim=None, _stacklevel=3, dtype=None):
+    if dim is None:
+        return _eager_F_log_softmax(input, dim, _stacklevel, dtype)
+    return log_softmax(input, dim, dtype)
+
+
+def _patched_log_softmax(input, dim=None, *, dtype=None, **kw):
+    if kw or dim is None:
+        return _eager_log_softmax(input, dim, dtype=dtype, **kw)
+    return log_softmax(input, dim, dtype)
+
+
 @contextlib.contextmanager
 def patched():
-    """Route torch.softmax, torch.nn.functional.softmax and Tensor.softmax through the guard."""
-    saved = (torch.softmax, torch.nn.functional.softmax, torch.Tensor.softmax)
+    """Route softmax, log_softmax, layer_norm and group_norm (torch.* and torch.nn.functional.*, and
+    Tensor.softmax) through the guard for the duration of the block."""
+    F = torch.nn.functional
+    saved = (torch.softmax, F.softmax, torch.Tensor.softmax, torch.log_softmax, F.log_softmax, F.layer_norm, F.group_norm)
     torch.softmax = _patched_softmax
-    torch.nn.functional.softmax = _patched_F_softmax
+    F.softmax = _patched_F_softmax
     torch.Tensor.softmax = _patched_T_softmax
+    torch.log_softmax = _patched_log_softmax
+    F.log_softmax = _patched_F_log_softmax
+    F.layer_norm = layer_norm
+    F.group_norm = group_norm
     try:
         yield
     finally:
-        torch.softmax, torch.nn.functional.softmax, torch.Tensor.softmax = saved
+        (torch.softmax, F.softmax, torch.Tensor.softmax, torch.log_softmax, F.log_softmax, F.layer_norm, F.group_norm) = saved

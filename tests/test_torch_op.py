@@ -86,3 +86,50 @@ def test_attention_block_under_the_patch_matches_eager():
             got = attention(q, k, v)
     assert torch_op.stats().get("library", 0) == 1
     assert torch.allclose(got.float(), ref.float(), atol=2e-2, rtol=2e-2)
+
+
+def test_patch_covers_log_softmax_and_norms_on_cpu():
+    F = torch.nn.functional
+    before = (torch.log_softmax, F.log_softmax, F.layer_norm, F.group_norm)
+    x = torch.randn(4, 6, 10)
+    w, b = torch.randn(10), torch.randn(10)
+    torch_op.stats(reset=True)
+    with torch_op.patched():
+        a = F.log_softmax(x, dim=-1)
+        c = torch.log_softmax(x, -1)
+        d = F.layer_norm(x, (10,), w, b, 1e-5)
+        e = F.group_norm(x, 3, None, None, 1e-5)
+        m = torch.nn.LayerNorm(10)(x)                     # modules call F.layer_norm at run time
+    assert (torch.log_softmax, F.log_softmax, F.layer_norm, F.group_norm) == before
+    assert torch.equal(a, before[0](x, -1)) and torch.equal(c, a)
+    assert torch.equal(d, before[2](x, (10,), w, b, 1e-5)) and torch.equal(e, before[3](x, 3, None, None, 1e-5))
+    assert m.shape == x.shape
+    assert sum(torch_op.stats().values()) == 5 and "library" not in torch_op.stats()
+
+
+@pytest.mark.gpu
+def test_log_softmax_and_norms_through_the_guard_on_gpu():
+    F = torch.nn.functional
+    torch.manual_seed(1)
+    torch_op.stats(reset=True)
+    with torch.no_grad():
+        x = torch.randn(3, 50, 1536, device="cuda", dtype=torch.bfloat16)
+        w = torch.randn(1536, device="cuda", dtype=torch.bfloat16)
+        b = torch.randn(1536, device="cuda", dtype=torch.bfloat16)
+        logits = torch.randn(7, 32000, device="cuda", dtype=torch.float32) * 3
+        img = torch.randn(2, 64, 32, 32, device="cuda", dtype=torch.float16)
+        gw = torch.randn(64, device="cuda", dtype=torch.float16)
+        ref = (F.layer_norm(x.float(), (1536,), w.float(), b.float(), 1e-5), torch.log_softmax(logits.double(), -1),
+               F.group_norm(img.float(), 32, gw.float(), None, 1e-5))
+        with torch_op.patched():
+            got = (F.layer_norm(x, (1536,), w, b, 1e-5), torch.log_softmax(logits, -1), F.group_norm(img, 32, gw, None, 1e-5),
+                   torch.nn.LayerNorm(1536, device="cuda", dtype=torch.bfloat16)(x))
+    assert torch_op.stats().get("library", 0) == 4
+    assert torch.allclose(got[0].float(), ref[0], atol=3e-2, rtol=2e-2)
+    assert torch.allclose(got[1].double(), ref[1], atol=1e-5, rtol=1e-6)
+    assert torch.allclose(got[2].float(), ref[2], atol=1e-2, rtol=1e-2)
+    assert got[3].shape == x.shape and torch.isfinite(got[3].float()).all()
+    # guard: a weight on another dtype goes to eager
+    assert torch.allclose(torch_op.layer_norm(x, (1536,), w, b).float(), ref[0], atol=3e-2, rtol=2e-2)
+    y = torch_op.layer_norm(x.float(), (1536,), w.float(), b.float())
+    assert y.dtype == torch.float32
