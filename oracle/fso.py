@@ -74,6 +74,8 @@ def _load():
             lib.fso_softmax_row_f64.restype = None
             lib.fso_log_softmax_f64.argtypes = [vp, ci, i64, i64, f32, vp]
             lib.fso_log_softmax_f64.restype = None
+            lib.fso_softmax_backward_f64.argtypes = [vp, vp, ci, i64, i64, f32, vp]
+            lib.fso_softmax_backward_f64.restype = None
             lib.fso_softmax_causal_f64.argtypes = [vp, ci, i64, i64, i64, f32, vp]
             lib.fso_softmax_causal_f64.restype = None
             lib.fso_router_topk_f64.argtypes = [vp, ci, i64, i64, i64, f32, ci, vp, vp]
@@ -119,6 +121,18 @@ def log_softmax_f64(x: np.ndarray, dtype: int, scale: float = 1.0) -> np.ndarray
     if rows and cols:
         _load().fso_log_softmax_f64(x.ctypes.data, dtype, rows, cols, np.float32(scale), y.ctypes.data)
     return y
+
+
+def softmax_backward_f64(dy: np.ndarray, y: np.ndarray, dtype: int, scale: float = 1.0) -> np.ndarray:
+    """fp64 gradient of softmax(scale * x) with respect to x, from the upstream gradient dy and the output y."""
+    dy, y = _stored(dy, dtype), _stored(y, dtype)
+    if dy.ndim != 2 or dy.shape != y.shape:
+        raise ValueError("dy and y must be [rows, cols] of the same shape")
+    rows, cols = y.shape
+    dx = np.empty((rows, cols), dtype=np.float64)
+    if rows and cols:
+        _load().fso_softmax_backward_f64(dy.ctypes.data, y.ctypes.data, dtype, rows, cols, np.float32(scale), dx.ctypes.data)
+    return dx
 
 
 def softmax_causal_f64(x: np.ndarray, dtype: int, q_offset: int, scale: float = 1.0) -> np.ndarray:

@@ -192,6 +192,28 @@ void fso_log_softmax_f64(const void* x, int dtype, int64_t rows, int64_t cols, f
     }
 }
 
+// Backward of y = softmax(scale * x) (the gradient a training step needs from the same operator):
+//   dx_j = scale * y_j * (dy_j - sum_k dy_k y_k)
+// dy, y: stored elements of `dtype`; dx: doubles. The dot product is a left-to-right Neumaier sum.
+void fso_softmax_backward_f64(const void* dy, const void* y, int dtype, int64_t rows, int64_t cols, float scale, double* dx) {
+    const int64_t esz = (dtype == DT_FP32) ? 4 : 2;
+    const double sc = static_cast<double>(scale);
+    for (int64_t i = 0; i < rows; ++i) {
+        const void* gr = static_cast<const char*>(dy) + i * cols * esz;
+        const void* yr = static_cast<const char*>(y) + i * cols * esz;
+        double S = 0.0, comp = 0.0;
+        for (int64_t j = 0; j < cols; ++j) {
+            const double e = widen(gr, dtype, j) * widen(yr, dtype, j);
+            const double t = S + e;
+            if (std::fabs(S) >= std::fabs(e)) comp += (S - t) + e;
+            else                              comp += (e - t) + S;
+            S = t;
+        }
+        S += comp;
+        for (int64_t j = 0; j < cols; ++j) dx[i * cols + j] = sc * (widen(yr, dtype, j) * (widen(gr, dtype, j) - S));
+    }
+}
+
 // Causal variant (the mask eager attention applies before its softmax; fusing it is the "operator
 // fusion" lever of the paper's Sec. II-B): row i keeps columns j <= i + q_offset and the softmax is
 // taken over the kept columns only; a masked column has z = -inf, i.e. y = exactly +0, whatever is
