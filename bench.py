@@ -305,6 +305,50 @@ def time_log_softmax(w: W.Workload, steps: int, warmup: int, l2_bytes: int, eage
     return out
 
 
+def time_softmax_backward(w: W.Workload, steps: int, warmup: int, l2_bytes: int):
+    """fs_softmax_backward on a softmax workload's shape: y = the library's forward output, dy seeded on
+    the device; reads dy and y once, writes dx once (3 elements of traffic per element)."""
+    import torch
+
+    import paper_2607_24762_b200 as fs
+    alg = 3 * w.rows * w.cols * w.elem_size
+    n_sets = int(max(1, min(12, math.ceil(4 * l2_bytes / alg))))
+    xs, ys = device_buffers(w, n_sets, threads=min(8, os.cpu_count() or 1))
+    stream = torch.cuda.current_stream()
+    lib = fs.binding.lib()
+    tdt = {W.FP32: torch.float32, W.BF16: torch.bfloat16, W.FP16: torch.float16}[w.dtype]
+    g = torch.Generator(device="cuda").manual_seed(99)
+    for j in range(n_sets):                                   # y_j = softmax(x_j); x_j then becomes dy_j
+        st = lib.fs_softmax(xs[j].data_ptr(), ys[j].data_ptr(), w.rows, w.cols, w.dtype, w.scale_f32, stream.cuda_stream)
+        if st != 0:
+            raise RuntimeError(fs.fs_strerror(st))
+        torch.cuda.synchronize()
+        xs[j].view(tdt).copy_(torch.randn((w.rows, w.cols), generator=g, device="cuda", dtype=torch.float32))
+    dxs = [torch.empty_like(x) for x in xs]
+
+    def launch(i):
+        j = i % n_sets
+        st = lib.fs_softmax_backward(xs[j].data_ptr(), ys[j].data_ptr(), dxs[j].data_ptr(), w.rows, w.cols, w.dtype, w.scale_f32,
+                                     stream.cuda_stream)
+        if st != 0:
+            raise RuntimeError(fs.fs_strerror(st))
+
+    for i in range(max(3, warmup)):
+        launch(i)
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    start.record(stream)
+    for i in range(steps):
+        launch(i)
+    stop.record(stream)
+    torch.cuda.synchronize()
+    ms = start.elapsed_time(stop) / steps
+    peak, _ = measured_peak()
+    gbs = alg / (ms * 1e-3) / 1e9
+    return {"what": f"fs_softmax_backward on {w.name}'s shape: reads dy and y, writes dx", "steps": steps, "ms_per_step": round(ms, 6),
+            "algorithmic_bytes": alg, "GB/s": round(gbs, 1), "frac_of_measured_copy": round(gbs / peak, 4), "n_sets": n_sets}
+
+
 # Normalisation workloads (synthetic, seeded on the device): the shapes of the two operators the paper
 # reports for Stable Diffusion 3.5 Medium (Sec. IV-C): layer_norm over the transformer's hidden size
 # (1536) for 4 x 4096 tokens, and the VAE decoder's 32-group group_norm at three resolutions.
@@ -518,7 +562,7 @@ def main():
                     help="also time the other workloads (default: on at --gpus 1)")
     ap.add_argument("--no-all", dest="all_workloads", action="store_false")
     ap.add_argument("--norm-workload", default="ln_sd35", choices=sorted(NORM_WORKLOADS), help="with --op norm")
-    ap.add_argument("--op", default="softmax", choices=["softmax", "causal", "router", "norm", "log_softmax"],
+    ap.add_argument("--op", default="softmax", choices=["softmax", "causal", "router", "norm", "log_softmax", "backward"],
                     help="time only fs_softmax_causal (q_offset 0) or fs_router_topk (k=8, renormalised) on the "
                          "workload and print a short line (profiler captures of those kernels)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the cpu_baseline leg")
@@ -573,6 +617,8 @@ def main():
                  "GB/s": round(alg / (r["ms_per_step"] * 1e-3) / 1e9, 1)}
         elif args.op == "log_softmax":
             r = time_log_softmax(w, args.steps, args.warmup, l2, eager=not args.no_cpu)
+        elif args.op == "backward":
+            r = time_softmax_backward(w, args.steps, args.warmup, l2)
         elif args.op == "norm":
             r = time_norm(args.norm_workload, args.steps, args.warmup, l2, eager=not args.no_cpu)
         else:
@@ -650,6 +696,11 @@ def main():
                     others[lname + "_log_softmax"] = time_log_softmax(W.WORKLOADS[lname], 300, 10, l2)
                 except Exception as exc:
                     others[lname + "_log_softmax"] = {"error": str(exc)[:200]}
+            for bname in ("cfg2", "cfg4"):
+                try:
+                    others[bname + "_backward"] = time_softmax_backward(W.WORKLOADS[bname], 300, 10, l2)
+                except Exception as exc:
+                    others[bname + "_backward"] = {"error": str(exc)[:200]}
             # the normalisation entry points on the shapes of the paper's second workload family
             for nname in NORM_WORKLOADS:
                 try:

@@ -145,6 +145,23 @@ int fs_router_topk(const void* x, float* w, int32_t* idx, int64_t rows, int64_t 
 int fs_log_softmax(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale, void* stream);
 
 /*
+ * fs_softmax_backward -- the gradient of y = softmax(scale * x) with respect to x (what a training
+ * step asks of the same operator):
+ *
+ *     dx[i][j] = scale * y[i][j] * (dy[i][j] - sum_k dy[i][k] * y[i][k])
+ *
+ *   dy, y  device pointers, rows*cols elements of `dtype`: the upstream gradient and the forward output.
+ *   dx     device pointer, rows*cols elements; may be the same buffer as dy or as y (partial overlap
+ *          is FS_ERR_INVALID_ARG).
+ *   scale  the forward call's scale (finite).
+ * Binary32 arithmetic and accumulation; the result is rounded once. Rows up to 4 KiB stay in
+ * registers, longer rows are split over a cluster with both slices resident in shared memory (two
+ * reads and one write of HBM per element), ragged or misaligned rows take a two-pass kernel.
+ */
+int fs_softmax_backward(const void* dy, const void* y, void* dx, int64_t rows, int64_t cols, int dtype, float scale,
+                        void* stream);
+
+/*
  * fs_layer_norm -- layer normalisation over the last dimension, one of the two normalisation
  * operators the paper reports generated kernels for (Sec. IV-C, Stable Diffusion 3.5 Medium):
  *
