@@ -76,6 +76,8 @@ def _load():
             lib.fso_log_softmax_f64.restype = None
             lib.fso_softmax_backward_f64.argtypes = [vp, vp, ci, i64, i64, f32, vp]
             lib.fso_softmax_backward_f64.restype = None
+            lib.fso_softmax_masked_f64.argtypes = [vp, vp, ci, i64, i64, i64, i64, f32, vp]
+            lib.fso_softmax_masked_f64.restype = None
             lib.fso_softmax_causal_f64.argtypes = [vp, ci, i64, i64, i64, f32, vp]
             lib.fso_softmax_causal_f64.restype = None
             lib.fso_router_topk_f64.argtypes = [vp, ci, i64, i64, i64, f32, ci, vp, vp]
@@ -133,6 +135,19 @@ def softmax_backward_f64(dy: np.ndarray, y: np.ndarray, dtype: int, scale: float
     if rows and cols:
         _load().fso_softmax_backward_f64(dy.ctypes.data, y.ctypes.data, dtype, rows, cols, np.float32(scale), dx.ctypes.data)
     return dx
+
+
+def softmax_masked_f64(x: np.ndarray, mask: np.ndarray, dtype: int, q_rows: int, heads: int, scale: float = 1.0) -> np.ndarray:
+    """fp64 softmax(scale * x + mask): x [rows, cols] ordered (batch, head, query), mask [batch * q_rows, cols]."""
+    x, mask = _stored(x, dtype), _stored(mask, dtype)
+    rows, cols = x.shape
+    if q_rows < 1 or heads < 1 or rows % (q_rows * heads) or mask.shape != (rows // heads, cols):
+        raise ValueError("rows must be batch * heads * q_rows and mask [batch * q_rows, cols]")
+    y = np.empty((rows, cols), dtype=np.float64)
+    if rows and cols:
+        _load().fso_softmax_masked_f64(x.ctypes.data, mask.ctypes.data, dtype, rows, cols, q_rows, heads, np.float32(scale),
+                                       y.ctypes.data)
+    return y
 
 
 def softmax_causal_f64(x: np.ndarray, dtype: int, q_offset: int, scale: float = 1.0) -> np.ndarray:

@@ -192,6 +192,40 @@ void fso_log_softmax_f64(const void* x, int dtype, int64_t rows, int64_t cols, f
     }
 }
 
+// Additive-mask variant (the `scores + mask` that eager attention forms before its softmax; fusing
+// the addition is the operator-fusion lever of the paper's Sec. II-B):
+//   z_ij = scale * x_ij + mask[mrow(i)][j],   y_i = softmax(z_i)
+// x: rows ordered (batch, head, query); the mask has one row per (batch, query) and is shared by the
+// heads: mrow(i) = (i / (heads * q_rows)) * q_rows + i % q_rows. The mask is not scaled.
+void fso_softmax_masked_f64(const void* x, const void* mask, int dtype, int64_t rows, int64_t cols, int64_t q_rows,
+                            int64_t heads, float scale, double* y) {
+    const int64_t esz = (dtype == DT_FP32) ? 4 : 2;
+    const double sc = static_cast<double>(scale);
+    for (int64_t i = 0; i < rows; ++i) {
+        const void* xr = static_cast<const char*>(x) + i * cols * esz;
+        const int64_t mrow = (i / (heads * q_rows)) * q_rows + i % q_rows;
+        const void* mr = static_cast<const char*>(mask) + mrow * cols * esz;
+        double* yr = y + i * cols;
+        if (cols <= 0) continue;
+        for (int64_t j = 0; j < cols; ++j) yr[j] = sc * widen(xr, dtype, j) + widen(mr, dtype, j);
+        double M = yr[0];
+        for (int64_t j = 1; j < cols; ++j) {
+            if (yr[j] > M) M = yr[j];
+        }
+        double S = 0.0, comp = 0.0;
+        for (int64_t j = 0; j < cols; ++j) {
+            const double e = std::exp(yr[j] - M);
+            yr[j] = e;
+            const double t = S + e;
+            if (std::fabs(S) >= std::fabs(e)) comp += (S - t) + e;
+            else                              comp += (e - t) + S;
+            S = t;
+        }
+        S += comp;
+        for (int64_t j = 0; j < cols; ++j) yr[j] = yr[j] / S;
+    }
+}
+
 // Backward of y = softmax(scale * x) (the gradient a training step needs from the same operator):
 //   dx_j = scale * y_j * (dy_j - sum_k dy_k y_k)
 // dy, y: stored elements of `dtype`; dx: doubles. The dot product is a left-to-right Neumaier sum.
