@@ -305,6 +305,55 @@ def time_log_softmax(w: W.Workload, steps: int, warmup: int, l2_bytes: int, eage
     return out
 
 
+def time_softmax_masked(w: W.Workload, steps: int, warmup: int, l2_bytes: int, heads: int = 8, eager: bool = True):
+    """fs_softmax_masked on a softmax workload's data viewed as (batch 1, `heads`, rows/heads queries) with a
+    causal mask shared by the heads; algorithmic bytes = x + y + the mask once."""
+    import torch
+
+    import paper_2607_24762_b200 as fs
+    q = w.rows // heads
+    alg = w.min_bytes + q * w.cols * w.elem_size
+    n_pairs = int(max(1, min(16, math.ceil(4 * l2_bytes / alg))))
+    xs, ys = device_buffers(w, n_pairs, threads=min(8, os.cpu_count() or 1))
+    tdt = {W.FP32: torch.float32, W.BF16: torch.bfloat16, W.FP16: torch.float16}[w.dtype]
+    mask = torch.full((q, w.cols), float("-inf"), device="cuda", dtype=torch.float32).triu(1 + w.cols - q).to(tdt).contiguous()
+    stream = torch.cuda.current_stream()
+    lib = fs.binding.lib()
+
+    def launch(i):
+        j = i % n_pairs
+        st = lib.fs_softmax_masked(xs[j].data_ptr(), mask.data_ptr(), ys[j].data_ptr(), w.rows, w.cols, q, heads, w.dtype,
+                                   w.scale_f32, stream.cuda_stream)
+        if st != 0:
+            raise RuntimeError(fs.fs_strerror(st))
+
+    def eager_launch(i):
+        s = xs[i % n_pairs].view(tdt).view(1, heads, q, w.cols)
+        torch.softmax(s * w.scale_f32 + mask, dim=-1)
+
+    def timed(fn, k):
+        for i in range(max(3, warmup)):
+            fn(i)
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        start.record(stream)
+        for i in range(k):
+            fn(i)
+        stop.record(stream)
+        torch.cuda.synchronize()
+        return start.elapsed_time(stop) / k
+
+    ms = timed(launch, steps)
+    peak, _ = measured_peak()
+    gbs = alg / (ms * 1e-3) / 1e9
+    out = {"what": f"fs_softmax_masked on {w.name} as 1 x {heads} x {q} x {w.cols}, causal mask shared by the heads", "steps": steps,
+           "ms_per_step": round(ms, 6), "algorithmic_bytes": alg, "GB/s": round(gbs, 1), "frac_of_measured_copy": round(gbs / peak, 4),
+           "n_pairs": n_pairs}
+    if eager:
+        out["torch_eager_ms"] = round(timed(eager_launch, max(5, steps // 4)), 6)
+    return out
+
+
 def time_softmax_backward(w: W.Workload, steps: int, warmup: int, l2_bytes: int):
     """fs_softmax_backward on a softmax workload's shape: y = the library's forward output, dy seeded on
     the device; reads dy and y once, writes dx once (3 elements of traffic per element)."""
@@ -562,7 +611,7 @@ def main():
                     help="also time the other workloads (default: on at --gpus 1)")
     ap.add_argument("--no-all", dest="all_workloads", action="store_false")
     ap.add_argument("--norm-workload", default="ln_sd35", choices=sorted(NORM_WORKLOADS), help="with --op norm")
-    ap.add_argument("--op", default="softmax", choices=["softmax", "causal", "router", "norm", "log_softmax", "backward"],
+    ap.add_argument("--op", default="softmax", choices=["softmax", "causal", "router", "norm", "log_softmax", "backward", "masked"],
                     help="time only fs_softmax_causal (q_offset 0) or fs_router_topk (k=8, renormalised) on the "
                          "workload and print a short line (profiler captures of those kernels)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the cpu_baseline leg")
@@ -617,6 +666,8 @@ def main():
                  "GB/s": round(alg / (r["ms_per_step"] * 1e-3) / 1e9, 1)}
         elif args.op == "log_softmax":
             r = time_log_softmax(w, args.steps, args.warmup, l2, eager=not args.no_cpu)
+        elif args.op == "masked":
+            r = time_softmax_masked(w, args.steps, args.warmup, l2, eager=not args.no_cpu)
         elif args.op == "backward":
             r = time_softmax_backward(w, args.steps, args.warmup, l2)
         elif args.op == "norm":
@@ -696,6 +747,10 @@ def main():
                     others[lname + "_log_softmax"] = time_log_softmax(W.WORKLOADS[lname], 300, 10, l2)
                 except Exception as exc:
                     others[lname + "_log_softmax"] = {"error": str(exc)[:200]}
+            try:
+                others["cfg2_masked"] = time_softmax_masked(W.WORKLOADS["cfg2"], 300, 10, l2)
+            except Exception as exc:
+                others["cfg2_masked"] = {"error": str(exc)[:200]}
             for bname in ("cfg2", "cfg4"):
                 try:
                     others[bname + "_backward"] = time_softmax_backward(W.WORKLOADS[bname], 300, 10, l2)

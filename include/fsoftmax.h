@@ -145,6 +145,27 @@ int fs_router_topk(const void* x, float* w, int32_t* idx, int64_t rows, int64_t 
 int fs_log_softmax(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale, void* stream);
 
 /*
+ * fs_softmax_masked -- softmax with an additive mask applied inside the kernel, the other half of the
+ * `scores + mask -> softmax` pair of eager attention (operator fusion, the paper's Sec. II-B; the
+ * workloads are the eager-attention softmax calls of its Table I):
+ *
+ *     y[i][j] = softmax over j of ( scale * x[i][j] + mask[mrow(i)][j] )
+ *
+ * The rows of x are ordered (batch, head, query); the mask has one row per (batch, query) and is
+ * shared by the heads: mrow(i) = (i / (heads * q_rows)) * q_rows + i % q_rows. The mask is added
+ * unscaled; -inf entries mask a column (a fully masked row is NaN, like an all -inf row), finite
+ * entries act as a bias.
+ *   x, y    as for fs_softmax (x == y allowed); rows must be a multiple of heads * q_rows.
+ *   mask    device pointer, (rows / heads) * cols elements of `dtype`, dense, never written.
+ * Parity: the exponent scale * x + mask is formed in binary32 before the row maximum is taken off,
+ * so fp32 output is within 1e-6 + 2.5e-7 * Z * y of the fp64 value, Z the largest finite |scale * x
+ * + mask| of the row (1e-6 for |z| up to a few units); 16-bit output within one unit in the last
+ * place of the correctly rounded value.
+ */
+int fs_softmax_masked(const void* x, const void* mask, void* y, int64_t rows, int64_t cols, int64_t q_rows, int64_t heads,
+                      int dtype, float scale, void* stream);
+
+/*
  * fs_softmax_backward -- the gradient of y = softmax(scale * x) with respect to x (what a training
  * step asks of the same operator):
  *

@@ -18,6 +18,7 @@
 #include "kernels/router_topk.cuh"
 #include "kernels/smem_row.cuh"
 #include "kernels/softmax_backward.cuh"
+#include "kernels/softmax_masked.cuh"
 #include "kernels/warp_row.cuh"
 
 namespace {
@@ -1121,6 +1122,81 @@ int run_softmax_backward(const void* dy, const void* y, void* dx, int64_t rows, 
     return launch(fn, std::min<int64_t>(rows, 0x7fffffff), t, 0, 0, st, p);
 }
 
+// ---------------------------------------------------------------------------------------------
+// softmax with an additive mask
+// ---------------------------------------------------------------------------------------------
+template <int DT> const void* masked_warp_fn(const WarpGeom& g) {
+    if (g.lanes == 32) {
+        switch (g.vpl) {
+            case 1: return (const void*)sm_masked_warp_kernel<DT, 32, 1>;
+            case 2: return (const void*)sm_masked_warp_kernel<DT, 32, 2>;
+            case 3: return (const void*)sm_masked_warp_kernel<DT, 32, 3>;
+            case 4: return (const void*)sm_masked_warp_kernel<DT, 32, 4>;
+            case 5: return (const void*)sm_masked_warp_kernel<DT, 32, 5>;
+            case 6: return (const void*)sm_masked_warp_kernel<DT, 32, 6>;
+            case 7: return (const void*)sm_masked_warp_kernel<DT, 32, 7>;
+            case 8: return (const void*)sm_masked_warp_kernel<DT, 32, 8>;
+            default: return nullptr;
+        }
+    }
+    if (g.vpl == 1) return (const void*)sm_masked_warp_kernel<DT, 1, 1>;
+    if (g.vpl == 2) return (const void*)sm_masked_warp_kernel<DT, 1, 2>;
+    if (g.vpl != 4) return nullptr;
+    switch (g.lanes) {
+        case 1:  return (const void*)sm_masked_warp_kernel<DT, 1, 4>;
+        case 2:  return (const void*)sm_masked_warp_kernel<DT, 2, 4>;
+        case 4:  return (const void*)sm_masked_warp_kernel<DT, 4, 4>;
+        case 8:  return (const void*)sm_masked_warp_kernel<DT, 8, 4>;
+        default: return (const void*)sm_masked_warp_kernel<DT, 16, 4>;
+    }
+}
+
+int run_softmax_masked(const void* x, const void* mask, void* y, int64_t rows, int64_t cols, int64_t q_rows, int64_t heads,
+                       int dtype, float scale, cudaStream_t st) {
+    Device* devp = nullptr;
+    int rc = get_device(&devp);
+    if (rc != FS_OK) return rc;
+    Device& dev = *devp;
+    const int esz = elem_size(dtype);
+    const bool fast = fast_path_ok(cols, dtype, ptr_align(x), ptr_align(y)) && ptr_align(mask) >= 16;
+    MaskedParams p;
+    p.x = x; p.mask = mask; p.y = y; p.rows = rows; p.cols = cols;
+    p.nvec = fast ? cols * esz / 16 : 0;
+    p.q_rows = q_rows; p.group = q_rows * heads;
+    p.c = static_cast<float>(static_cast<double>(scale) * kLog2e);
+    p.status = dev.status; p.pf_rows = 0;
+    WarpGeom wg;
+    if (fast && norm_warp_geom(p.nvec, dtype, &wg)) {
+        const void* fn = by_dtype(dtype, [&](auto dt) -> const void* { return masked_warp_fn<decltype(dt)::value>(wg); });
+        if (fn) {
+            const int t = 128;
+            const int64_t groups = (rows + (32 / wg.lanes) - 1) / (32 / wg.lanes);
+            const int64_t grid = std::min<int64_t>((groups + (t / 32) - 1) / (t / 32), 0x7fffffff);
+            return launch(fn, grid, t, 0, 0, st, p);
+        }
+    }
+    SmemGeom sg;
+    if (fast && dev.cluster_ok && smem_geom(p.nvec, dtype, 0, 0, &sg) && rows <= 0x7fffffff / sg.cs) {
+        const bool full = smem_row_full(sg, dtype, p.nvec);
+        const void* fn = by_dtype(dtype, [&](auto dt) -> const void* {
+            constexpr int DT = decltype(dt)::value;
+            return full ? (const void*)sm_masked_smem_kernel<DT, true> : (const void*)sm_masked_smem_kernel<DT, false>; });
+        const size_t stage_bytes = smem_row_stage_bytes(sg, dtype);
+        const size_t smem = stage_bytes + size_t(kNormMaxChunks) * 8 + size_t(2 * kNormMaxChunks) * sg.threads * 4;
+        if (smem <= static_cast<size_t>(dev.smem_optin) - 2048) {
+            int ncl = 0;
+            if ((rc = active_clusters(dev, fn, sg.threads, smem, sg.cs, &ncl)) != FS_OK) return rc;
+            p.pf_rows = prefetch_rows(ncl);
+            return launch(fn, rows * sg.cs, sg.threads, smem, sg.cs, st, p, static_cast<uint32_t>(stage_bytes), sg.slice,
+                          smem_row_nchunk(sg, dtype));
+        }
+    }
+    const void* fn = by_dtype(dtype, [&](auto dt) -> const void* { return (const void*)sm_masked_generic_kernel<decltype(dt)::value>; });
+    int t = 32;
+    while (t < 1024 && cols > int64_t(t) * 8) t <<= 1;
+    return launch(fn, std::min<int64_t>(rows, 0x7fffffff), t, 0, 0, st, p);
+}
+
 }  // namespace
 
 extern "C" {
@@ -1188,6 +1264,17 @@ int fs_log_softmax(const void* x, void* y, int64_t rows, int64_t cols, int dtype
     if (v != FS_OK) return v;
     if (rows == 0 || cols == 0) return FS_OK;
     return run_log_softmax(x, y, rows, cols, dtype, scale, static_cast<cudaStream_t>(stream));
+}
+
+int fs_softmax_masked(const void* x, const void* mask, void* y, int64_t rows, int64_t cols, int64_t q_rows, int64_t heads,
+                      int dtype, float scale, void* stream) {
+    const int v = validate(x, y, rows, cols, dtype, scale);
+    if (v != FS_OK) return v;
+    if (q_rows < 1 || heads < 1 || q_rows > (int64_t(1) << 40) || heads > (int64_t(1) << 20)) return FS_ERR_INVALID_ARG;
+    if (rows % (q_rows * heads) != 0) return FS_ERR_INVALID_ARG;
+    if (rows == 0 || cols == 0) return FS_OK;
+    if (!mask) return FS_ERR_INVALID_ARG;
+    return run_softmax_masked(x, mask, y, rows, cols, q_rows, heads, dtype, scale, static_cast<cudaStream_t>(stream));
 }
 
 int fs_softmax_backward(const void* dy, const void* y, void* dx, int64_t rows, int64_t cols, int dtype, float scale,
