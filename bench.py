@@ -408,6 +408,8 @@ NORM_WORKLOADS = {
     "gn_c256_256": ("group", dict(n=1, channels=256, spatial=256 * 256, groups=32, dtype=W.BF16)),
     "gn_c128_512": ("group", dict(n=1, channels=128, spatial=512 * 512, groups=32, dtype=W.BF16)),
     "gn_c128_1024": ("group", dict(n=1, channels=128, spatial=1024 * 1024, groups=32, dtype=W.BF16)),
+    "gn_c512_128_b8": ("group", dict(n=8, channels=512, spatial=128 * 128, groups=32, dtype=W.BF16)),
+    "gn_c256_256_b8": ("group", dict(n=8, channels=256, spatial=256 * 256, groups=32, dtype=W.BF16)),
 }
 
 

@@ -91,20 +91,27 @@ lsm_warp_kernel(const LsmParams p) {
         }
         const float r = warp_pick<LANES, false>(ref.value());
         const f32x2 r2 = pair(r, r);
-        f32x2 d[VPL][NP];
+        // the row stays packed in registers and is widened where it is used (twice): a widened row
+        // of eight vectors per lane costs 64 more registers and a third of the resident warps
         f32x2 acc[2] = {pair(0.0f, 0.0f), pair(0.0f, 0.0f)};
 #pragma unroll
-        for (int k = 0; k < VPL; ++k)
-            if (sl + k * LANES < nvec) lsm_accumulate<DT>(raw[k], r2, c2, d[k], acc);
+        for (int k = 0; k < VPL; ++k) {
+            if (sl + k * LANES < nvec) {
+                f32x2 d[NP];
+                lsm_accumulate<DT>(raw[k], r2, c2, d, acc);
+            }
+        }
         const float lns = ln_of(warp_sum<LANES>(pair_sum(add2(acc[0], acc[1]))));
         const f32x2 l2 = pair(-lns, -lns);
         if (row_ok) {
 #pragma unroll
             for (int k = 0; k < VPL; ++k) {
                 if (sl + k * LANES < nvec) {
+                    f32x2 d[NP];
+                    widen_pairs<DT>(raw[k], d);
 #pragma unroll
-                    for (int j = 0; j < NP; ++j) d[k][j] = fma2(d[k][j], s2, l2);
-                    st_stream(yv + row * p.nvec + sl + k * LANES, narrow_pairs<DT>(d[k]));
+                    for (int j = 0; j < NP; ++j) d[j] = fma2(sub2(d[j], r2), s2, l2);
+                    st_stream(yv + row * p.nvec + sl + k * LANES, narrow_pairs<DT>(d));
                 }
             }
         }

@@ -61,7 +61,7 @@ __device__ __forceinline__ float masked_exponents(const uint4& xraw, const uint4
 
 // ---------------------------------------------------------------------------------------------
 template <int DT, int LANES, int VPL>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(128, 5)      // 102 registers: five blocks per SM; a tighter cap spills
 sm_masked_warp_kernel(const MaskedParams p) {
     constexpr int NP = Traits<DT>::VE / 2;
     constexpr int G = 32 / LANES;
