@@ -219,6 +219,15 @@ int fs_group_norm(const void* x, const void* gamma, const void* beta, void* y, i
                   int64_t groups, int dtype, float eps, void* stream);
 
 /*
+ * fs_split_geometry -- the launch geometry the dispatcher gives the split-row kernels (softmax,
+ * log_softmax, masked, backward, normalisations) for rows of `cols` elements: blocks per cluster
+ * (1..16), threads per block and the bytes of a row each block holds in shared memory. Pure host
+ * arithmetic, no CUDA call. FS_ERR_UNSUPPORTED when the row size is not a multiple of 16 bytes or
+ * exceeds what a 16-block cluster holds.
+ */
+int fs_split_geometry(int64_t cols, int dtype, int* cluster, int* threads, int64_t* slice_bytes);
+
+/*
  * fs_select_kernel -- the dispatcher's decision, without a launch (no CUDA call is made when the
  * device attributes are already cached or `x_align`/`y_align` rule the fast paths out).
  *   x_align, y_align  the largest power of two (<= 16 is enough) dividing each base address.

@@ -63,6 +63,8 @@ def lib() -> ctypes.CDLL:
             L.fs_layer_norm.restype = ci
             L.fs_group_norm.argtypes = [vp, vp, vp, vp, i64, i64, i64, i64, ci, f32, vp]
             L.fs_group_norm.restype = ci
+            L.fs_split_geometry.argtypes = [i64, ci, ctypes.POINTER(ci), ctypes.POINTER(ci), ctypes.POINTER(i64)]
+            L.fs_split_geometry.restype = ci
             L.fs_select_kernel.argtypes = [i64, i64, ci, ci, ci]
             L.fs_select_kernel.restype = ci
             L.fs_softmax_host.argtypes = [vp, vp, i64, i64, ci, f32]
@@ -171,6 +173,16 @@ def fs_group_norm(x, gamma, beta, y, n: int, channels: int, spatial: int, groups
     """Group normalisation of a dense [n, channels, spatial] tensor; gamma, beta per channel or None."""
     _check(lib().fs_group_norm(_ptr(x), _ptr(gamma), _ptr(beta), _ptr(y), n, channels, spatial, groups, dtype, eps,
                                _stream(stream)), "fs_group_norm")
+
+
+def fs_split_geometry(cols: int, dtype: int):
+    """(cluster size, threads per block, slice bytes) of the split-row kernels for rows of `cols` elements, or None."""
+    cs, t, sl = ctypes.c_int(0), ctypes.c_int(0), ctypes.c_int64(0)
+    st = lib().fs_split_geometry(cols, dtype, ctypes.byref(cs), ctypes.byref(t), ctypes.byref(sl))
+    if st == FS_ERR_UNSUPPORTED:
+        return None
+    _check(st, "fs_split_geometry")
+    return cs.value, t.value, sl.value
 
 
 def fs_select_kernel(rows: int, cols: int, dtype: int, x_align: int = 16, y_align: int = 16) -> int:

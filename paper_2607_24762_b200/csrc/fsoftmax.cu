@@ -211,7 +211,8 @@ double smem_geom_score(int64_t nvec, int dtype, const SmemGeom& g) {
     const int64_t nch = (g.slice + chunk - 1) / chunk;
     const bool full = nvec == int64_t(g.slice) * g.cs && g.slice % chunk == 0;
     const double stage = double(nch * chunk * 16);
-    const double smem = stage + kSmemRowMaxChunks * 8 + kSmemRowMaxChunks * 4.0 * g.threads + 1024 + 1024;
+    // dynamic part + the kernel's static shared memory (896 B) + the 1 KiB the hardware reserves per block
+    const double smem = stage + kSmemRowMaxChunks * 8 + kSmemRowMaxChunks * 4.0 * g.threads + 896 + 1024;
     const int blocks = std::min(std::min(int(kSmemPerSm / smem), kSplitThreadsPerSm / g.threads), 32);
     if (blocks < 1) return 0.0;
     const double resident_cap = 184.0 * 1024;
@@ -1306,6 +1307,16 @@ int fs_group_norm(const void* x, const void* gamma, const void* beta, void* y, i
     if (v != FS_OK || rows == 0 || cols == 0) return v;
     const int aff = (gamma || beta) ? 2 : 0;
     return run_norm(x, gamma, beta, y, rows, cols, dtype, eps, aff, spatial, groups, static_cast<cudaStream_t>(stream));
+}
+
+int fs_split_geometry(int64_t cols, int dtype, int* cluster, int* threads, int64_t* slice_bytes) {
+    if (cols < 1 || !cluster || !threads || !slice_bytes) return FS_ERR_INVALID_ARG;
+    if (dtype != FS_DTYPE_FP32 && dtype != FS_DTYPE_BF16 && dtype != FS_DTYPE_FP16) return FS_ERR_INVALID_ARG;
+    if (cols > (int64_t(1) << 40) || (cols * elem_size(dtype)) % 16 != 0) return FS_ERR_UNSUPPORTED;
+    SmemGeom g;
+    if (!smem_geom(cols * elem_size(dtype) / 16, dtype, 0, 0, &g)) return FS_ERR_UNSUPPORTED;
+    *cluster = g.cs; *threads = g.threads; *slice_bytes = int64_t(g.slice) * 16;
+    return FS_OK;
 }
 
 int fs_select_kernel(int64_t rows, int64_t cols, int dtype, int x_align, int y_align) {

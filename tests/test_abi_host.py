@@ -126,6 +126,34 @@ def test_dispatcher_table(lib):
             last = cur
 
 
+def test_split_geometry_choice(lib):
+    """The split-row geometry: slices of about 32 KiB that are whole chunks (8 vectors per thread), the smallest
+    cluster that gets there, any cluster size 1..16 (values fixed by the sweeps the chooser was fitted to)."""
+    g = fs.fs_split_geometry
+    F32, BF16 = fs.FS_DTYPE_FP32, fs.FS_DTYPE_BF16
+    kib = lambda k, e: int(k * 1024) // e
+    assert g(kib(32, 2), BF16) == (1, 128, 32768)
+    assert g(kib(128, 2), BF16) == (4, 128, 32768)
+    assert g(kib(96, 2), BF16) == (3, 128, 32768)                 # not the next power of two with half-empty slices
+    assert g(kib(160, 4), F32) == (5, 128, 32768)
+    assert g(kib(384, 2), BF16) == (12, 128, 32768)
+    assert g(262144, BF16) == (16, 128, 32768)                     # cfg4
+    assert g(32768, F32) == (4, 128, 32768)                        # cfg5
+    assert g(kib(40, 2), BF16) == (1, 160, 40960)                  # one block, two 20 KiB chunks
+    assert g(kib(1024, 2), BF16) == (16, 256, 65536)
+    for cols, dt, e in ((kib(24, 2), BF16, 2), (kib(48, 4), F32, 4), (kib(250.5, 2), BF16, 2), (kib(600, 4), F32, 4), (100000, BF16, 2)):
+        cs, t, sl = g(cols, dt)
+        assert 1 <= cs <= 16 and t % 32 == 0 and 32 <= t <= 256
+        assert sl * cs >= cols * e and sl <= 8 * 8 * t * 16          # covers the row; at most 8 chunks of 8 vectors per thread
+        assert cs == 16 or sl <= 49152
+    assert g(kib(4096, 2), BF16) is None                           # beyond 16 x 192 KiB
+    assert g(1001, BF16) is None                                   # not a whole number of vectors
+    # every row length the chooser can meet yields a valid geometry
+    for nv in list(range(1, 600)) + [1000, 2047, 2048, 2049, 4096, 10000, 65536, 196608]:
+        r = g(nv * 8, BF16)
+        assert r is not None and r[2] * r[0] >= nv * 16 and r[2] <= 8 * 8 * r[1] * 16, (nv, r)
+
+
 def test_no_device_fails_loudly(lib):
     import torch
     if torch.cuda.is_available():
