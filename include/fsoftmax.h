@@ -231,7 +231,10 @@ int fs_split_geometry(int64_t cols, int dtype, int* cluster, int* threads, int64
  * fs_select_kernel -- the dispatcher's decision, without a launch (no CUDA call is made when the
  * device attributes are already cached or `x_align`/`y_align` rule the fast paths out).
  *   x_align, y_align  the largest power of two (<= 16 is enough) dividing each base address.
- * Returns an fs_kernel (>= 1), or a negative fs_status on invalid arguments.
+ * Returns an fs_kernel (>= 1), or a negative fs_status on invalid arguments. FS_KERNEL_GENERIC
+ * covers two forms: vector-aligned rows of 1 MiB or more that no cluster holds are cut into
+ * segments over two kernels (partial (max, sum) pairs through a scratch buffer allocated and freed
+ * in stream order); everything else runs one block per row.
  */
 int fs_select_kernel(int64_t rows, int64_t cols, int dtype, int x_align, int y_align);
 

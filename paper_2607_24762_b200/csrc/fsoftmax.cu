@@ -19,6 +19,7 @@
 #include "kernels/smem_row.cuh"
 #include "kernels/softmax_backward.cuh"
 #include "kernels/softmax_masked.cuh"
+#include "kernels/softmax_split.cuh"
 #include "kernels/warp_row.cuh"
 
 namespace {
@@ -529,6 +530,39 @@ int ring_stages(size_t stage_bytes, size_t budget, int max_stages) {
     return n;
 }
 
+// Rows longer than a cluster's shared memory: segments over a grid that fills the GPU, the
+// (reference, sum) pairs of the segments exchanged through a stream-ordered scratch buffer.
+int run_softmax_split(Device& dev, const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale, cudaStream_t st) {
+    LsmParams p;
+    p.x = x; p.y = y; p.rows = rows; p.cols = cols;
+    p.nvec = cols * elem_size(dtype) / 16;
+    p.scale = std::fabs(scale);
+    p.c = static_cast<float>(static_cast<double>(p.scale) * kLog2e);
+    p.flip = std::signbit(scale) && scale != 0.0f ? (dtype == FS_DTYPE_FP32 ? 0x80000000u : 0x80008000u) : 0u;
+    p.status = dev.status; p.pf_rows = 0;
+    const int t = 256;
+    const int64_t target = int64_t(dev.sm_count) * 8;
+    int64_t nseg = std::max<int64_t>(1, std::min<int64_t>(1024, (target + rows - 1) / rows));
+    const int64_t seg_vecs = ((p.nvec + nseg - 1) / nseg + 4 * t - 1) / (4 * t) * (4 * t);
+    nseg = (p.nvec + seg_vecs - 1) / seg_vecs;
+    if (rows * nseg > 0x7fffffff || seg_vecs > 0x7fffffff) return FS_ERR_UNSUPPORTED;
+    float2* part = nullptr;
+    FS_CUDA(cudaMallocAsync(reinterpret_cast<void**>(&part), static_cast<size_t>(rows * nseg) * sizeof(float2), st));
+    const void* f1 = nullptr;
+    const void* f2 = nullptr;
+    switch (dtype) {
+        case FS_DTYPE_FP32: f1 = (const void*)sm_partial_kernel<DT_F32>; f2 = (const void*)sm_apply_kernel<DT_F32>; break;
+        case FS_DTYPE_BF16: f1 = (const void*)sm_partial_kernel<DT_BF16>; f2 = (const void*)sm_apply_kernel<DT_BF16>; break;
+        default:            f1 = (const void*)sm_partial_kernel<DT_F16>; f2 = (const void*)sm_apply_kernel<DT_F16>; break;
+    }
+    const float2* cpart = part;
+    int rc = launch(f1, rows * nseg, t, 0, 0, st, p, part, static_cast<int>(nseg), static_cast<int>(seg_vecs));
+    if (rc == FS_OK) rc = launch(f2, rows * nseg, t, 0, 0, st, p, cpart, static_cast<int>(nseg), static_cast<int>(seg_vecs));
+    const cudaError_t fe = cudaFreeAsync(part, st);
+    if (rc == FS_OK && fe != cudaSuccess) return cuda_fail(fe);
+    return rc;
+}
+
 int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale, cudaStream_t st,
         int kernel, int threads, int cluster) {
     Device* devp = nullptr;
@@ -675,6 +709,10 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
                           static_cast<uint32_t>(stage_bytes), g.slice);
         }
         case FS_KERNEL_GENERIC: {
+            // vector-aligned rows that no cluster holds (the dispatcher's own choice only): rows cut
+            // into segments over two kernels instead of one block per row
+            if (was_auto && fast_path_ok(cols, dtype, ptr_align(x), ptr_align(y)) && cols * elem_size(dtype) >= (int64_t(1) << 20))
+                return run_softmax_split(dev, x, y, rows, cols, dtype, scale, st);
             const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) { return (const void*)generic_row_kernel<decltype(dt)::value, decltype(ng)::value, false>; });
             int t = threads;
             if (t == 0) {

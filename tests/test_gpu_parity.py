@@ -76,6 +76,23 @@ def test_very_long_rows(dtype):
         assert sweep_case(rows, cols, dtype, fs.FS_KERNEL_AUTO, 1.0, seed=31) is not None
 
 
+@pytest.mark.parametrize("dtype", [FP32, BF16, FP16])
+def test_rows_beyond_a_cluster_take_the_two_kernel_path(dtype):
+    """Rows of 4-16 MiB (no cluster's shared memory holds them): segments over two kernels, partial pairs through a
+    stream-ordered scratch buffer. Positive, negative and zero scale, -inf entries, a NaN row, in place."""
+    cols = (1 << 21) + 24 if dtype != FP32 else (1 << 20) + 12
+    for rows, scale in ((3, 1.0), (2, -0.5), (1, 0.0)):
+        x = W.random_case(rows, cols, dtype, seed=90 + rows, sigma=3.0, neg_inf_frac=0.02 if scale > 0 else 0.0)
+        status, y = run_softmax(x, dtype, scale)
+        assert status == fs.FS_OK
+        check(x, dtype, scale, y)
+    x = W.random_case(2, cols, dtype, seed=99, sigma=2.0)
+    x[1, 12345] = np.float32(np.nan) if dtype == FP32 else np.uint16(0x7FC0 if dtype == BF16 else 0x7E00)
+    status, y = run_softmax(x, dtype, 1.0, inplace=True)
+    assert status == fs.FS_OK
+    check(x, dtype, 1.0, y)
+
+
 @pytest.mark.parametrize("kernel,threads,cluster", [
     (fs.FS_KERNEL_BLOCK, 32, 0), (fs.FS_KERNEL_BLOCK, 64, 0), (fs.FS_KERNEL_BLOCK, 128, 0), (fs.FS_KERNEL_BLOCK, 512, 0),
     (fs.FS_KERNEL_BLOCK, 1024, 0), (fs.FS_KERNEL_BLOCK_TMA, 32, 0), (fs.FS_KERNEL_BLOCK_TMA, 96, 0),
