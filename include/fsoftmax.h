@@ -194,8 +194,8 @@ int fs_softmax_backward(const void* dy, const void* y, void* dx, int64_t rows, i
  *   gamma, beta   device pointers to cols elements of `dtype`, or NULL (1 and 0), independently.
  *   eps     finite, >= 0. Statistics and arithmetic are binary32; the output is rounded once.
  *   stream  cudaStream_t as void*.
- * Rows up to 4 KiB stay in the registers of a (sub-)warp; 16-bit rows of 4-9 KiB in the registers
- * of a block (eight rows per block, gamma and beta kept in registers); longer rows are split over
+ * Rows up to 4 KiB stay in the registers of a (sub-)warp, 16-bit rows up to 9 KiB too (packed, and
+ * widened where they are used); longer rows are split over
  * a cluster of 1..16 blocks with the slices resident in shared memory (one read and one write of
  * HBM per element, as for fs_softmax); rows beyond a cluster's shared memory (about 3 MiB) are
  * cut into segments over two kernels, whose partial statistics pass through a scratch buffer that

@@ -855,25 +855,15 @@ template <int DT, int AFF> const void* norm_warp_fn(const WarpGeom& g) {
     }
 }
 
-template <int DT> const void* norm_block_fn(int vpt, int aff) {
-    switch (vpt) {
-        case 1:  return aff ? (const void*)norm_block_kernel<DT, 1, 1> : (const void*)norm_block_kernel<DT, 1, 0>;
-        case 2:  return aff ? (const void*)norm_block_kernel<DT, 2, 1> : (const void*)norm_block_kernel<DT, 2, 0>;
-        default: return aff ? (const void*)norm_block_kernel<DT, 4, 1> : (const void*)norm_block_kernel<DT, 4, 0>;
+template <int DT> const void* norm_packed_fn(int vpl, int aff) {
+    switch (vpl) {
+        case 10: return aff ? (const void*)norm_warp_packed_kernel<DT, 10, 1> : (const void*)norm_warp_packed_kernel<DT, 10, 0>;
+        case 12: return aff ? (const void*)norm_warp_packed_kernel<DT, 12, 1> : (const void*)norm_warp_packed_kernel<DT, 12, 0>;
+        case 14: return aff ? (const void*)norm_warp_packed_kernel<DT, 14, 1> : (const void*)norm_warp_packed_kernel<DT, 14, 0>;
+        case 16: return aff ? (const void*)norm_warp_packed_kernel<DT, 16, 1> : (const void*)norm_warp_packed_kernel<DT, 16, 0>;
+        case 18: return aff ? (const void*)norm_warp_packed_kernel<DT, 18, 1> : (const void*)norm_warp_packed_kernel<DT, 18, 0>;
+        default: return nullptr;
     }
-}
-
-// Block-per-row geometry: vectors per thread in {4, 2, 1} and threads a multiple of 32 up to 256,
-// preferring a split that leaves no thread without work.
-bool norm_block_geom(int64_t nvec, int* vpt, int* threads) {
-    if (nvec < 1 || nvec > 1024) return false;
-    for (int v = 4; v >= 1; v >>= 1) {
-        if (nvec % (32 * v) == 0 && nvec / v <= 256) { *vpt = v; *threads = static_cast<int>(nvec / v); return true; }
-    }
-    const int v = nvec > 512 ? 4 : nvec > 128 ? 2 : 1;
-    *vpt = v;
-    *threads = static_cast<int>((nvec + v - 1) / v + 31) / 32 * 32;
-    return *threads <= 256;
 }
 
 template <int DT> const void* norm_smem_fn(bool full, int aff) {
@@ -939,17 +929,17 @@ int run_norm(const void* x, const void* gamma, const void* beta, void* y, int64_
             return launch(fn, grid, t, 0, 0, st, p);
         }
     }
-    int bvpt = 0, bthreads = 0;
-    // Measured on B200 (256 MiB per direction): the block kernel wins for 16-bit rows of 4-9 KiB; fp32
-    // rows and longer 16-bit rows are faster from shared memory.
-    const int64_t block_max = dtype == FS_DTYPE_FP32 ? 0 : 576;
-    if (fast && aff != 2 && p.nvec <= block_max && norm_block_geom(p.nvec, &bvpt, &bthreads)) {
-        // several rows per block (gamma and beta are loaded once per block), but never so many
-        // that the grid drops below a few waves
-        const int64_t rpb = std::max<int64_t>(1, std::min<int64_t>(8, rows / (int64_t(dev.sm_count) * 32)));
-        const void* fn = by_dtype(dtype, [&](auto dt) -> const void* { return norm_block_fn<decltype(dt)::value>(bvpt, aff); });
-        const int64_t grid = (rows + rpb - 1) / rpb;
-        if (grid <= 0x7fffffff) return launch(fn, grid, bthreads, 0, 0, st, p, static_cast<int>(rpb));
+    // 16-bit rows of 4-9 KiB: a warp per row with the row packed in registers. Measured on B200 (256 MiB
+    // per direction, gamma and beta present): 90-106 us where a block per row (two barriers per row) took
+    // 106-131 and the shared-memory kernel 121-174; fp32 rows of this size are faster from shared memory.
+    if (fast && aff != 2 && dtype != FS_DTYPE_FP32 && p.nvec > 256 && p.nvec <= 576) {
+        const int vpl = static_cast<int>((p.nvec + 63) / 64) * 2;          // even, 10..18
+        const void* fn = dtype == FS_DTYPE_BF16 ? norm_packed_fn<DT_BF16>(vpl, aff) : norm_packed_fn<DT_F16>(vpl, aff);
+        if (fn) {
+            const int t = 128;
+            const int64_t grid = std::min<int64_t>((rows + (t / 32) - 1) / (t / 32), 0x7fffffff);
+            return launch(fn, grid, t, 0, 0, st, p);
+        }
     }
     SmemGeom sg;
     const bool smem_ok = fast && dev.cluster_ok && smem_geom(p.nvec, dtype, 0, 0, &sg) && rows <= 0x7fffffff / sg.cs;

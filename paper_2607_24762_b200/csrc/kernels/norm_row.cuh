@@ -6,8 +6,8 @@
 // item is the triple (n, mean, M2) with Chan's pairwise merge in place of the (reference, sum) pair.
 //
 //   norm_warp_kernel     (sub-)warp per row, the row in registers: exact two-pass statistics
-//   norm_block_kernel    block per row, the row in registers, several consecutive rows per block
-//                        with gamma and beta kept in registers
+//   norm_warp_packed_kernel  warp per row for 16-bit rows of 4-9 KiB: the row stays packed in
+//                        registers (10..18 vectors per lane) and is widened where it is used
 //   norm_smem_kernel     row split over a cluster of 1..16 blocks, the slice resident in shared
 //                        memory (bulk async copies, one mbarrier per chunk); per chunk a thread
 //                        takes the exact mean and M2 of its own 8 vectors and merges them into
@@ -214,85 +214,64 @@ norm_warp_kernel(const NormParams p) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// block per row, registers; a block takes `rows_per_block` consecutive rows
-// Thread t holds vectors t, t + T, ... of the row, so it meets the same columns in every row:
-// its gamma and beta vectors are loaded once and stay in registers (packed). The next row's
-// vectors are requested before the current row is reduced, so the row-wide barrier does not
-// leave the memory system idle.
+// warp per row for 16-bit rows of 4-9 KiB: the row stays PACKED in registers (VPL vectors per lane,
+// 10..18) and is widened where it is used, three times; no shared memory, no block barrier.
 // ---------------------------------------------------------------------------------------------
-template <int DT, int VPT, int AFF>
-__global__ void __launch_bounds__(256)
-norm_block_kernel(const NormParams p, const int rows_per_block) {
+template <int DT, int VPL, int AFF>
+__global__ void __launch_bounds__(128, VPL <= 12 ? 4 : 3)
+norm_warp_packed_kernel(const NormParams p) {
     constexpr int NP = Traits<DT>::VE / 2;
-    static_assert(AFF != 2, "per-run affine parameters are handled by the shared-memory kernel");
-    __shared__ float red[2][2][32];
+    static_assert(AFF != 2 && DT != DT_F32, "16-bit rows, column affine parameters");
     pdl_launch_dependents();
-    const int T = blockDim.x, tid = threadIdx.x, lane = tid & 31, nwarps = T >> 5;
+    const int lane = threadIdx.x & 31;
+    const int warps = blockDim.x >> 5;
     const int nvec = static_cast<int>(p.nvec);
-    const uint4* __restrict__ xv = static_cast<const uint4*>(p.x);
-    uint4* __restrict__ yv = static_cast<uint4*>(p.y);
-    const int64_t row0 = int64_t(blockIdx.x) * rows_per_block;
-    const int64_t row_end = min(p.rows, row0 + rows_per_block);
+    const uint4* __restrict__ xv = static_cast<const uint4*>(p.x) + lane;
+    uint4* __restrict__ yv = static_cast<uint4*>(p.y) + lane;
+    const uint4* gv = AFF == 1 && p.gamma ? static_cast<const uint4*>(p.gamma) + lane : nullptr;
+    const uint4* bv = AFF == 1 && p.beta ? static_cast<const uint4*>(p.beta) + lane : nullptr;
     const float inv_n = 1.0f / static_cast<float>(p.cols);
     pdl_wait();
-    uint4 graw[VPT], braw[VPT];
-    const bool hg = AFF == 1 && p.gamma != nullptr, hb = AFF == 1 && p.beta != nullptr;
+    for (int64_t row = int64_t(blockIdx.x) * warps + (threadIdx.x >> 5); row < p.rows; row += int64_t(gridDim.x) * warps) {
+        uint4 raw[VPL];
 #pragma unroll
-    for (int k = 0; k < VPT; ++k) {
-        graw[k] = make_uint4(0u, 0u, 0u, 0u); braw[k] = make_uint4(0u, 0u, 0u, 0u);
-        if (hg && tid + k * T < nvec) graw[k] = ld_cached(static_cast<const uint4*>(p.gamma) + tid + k * T);
-        if (hb && tid + k * T < nvec) braw[k] = ld_cached(static_cast<const uint4*>(p.beta) + tid + k * T);
-    }
-    uint4 next[VPT];
-#pragma unroll
-    for (int k = 0; k < VPT; ++k) {
-        next[k] = make_uint4(0u, 0u, 0u, 0u);
-        if (row0 < row_end && tid + k * T < nvec) next[k] = ld_stream(xv + row0 * p.nvec + tid + k * T);
-    }
-    int par = 0;
-    for (int64_t row = row0; row < row_end; ++row, par ^= 1) {
-        f32x2 x[VPT][NP];
+        for (int k = 0; k < VPL; ++k) {
+            raw[k] = make_uint4(0u, 0u, 0u, 0u);
+            if (lane + k * 32 < nvec) raw[k] = ld_stream(xv + row * p.nvec + k * 32);
+        }
         f32x2 acc[2] = {pair(0.0f, 0.0f), pair(0.0f, 0.0f)};
 #pragma unroll
-        for (int k = 0; k < VPT; ++k) {
-            widen_pairs<DT>(next[k], x[k]);                  // absent vectors are zeros
+        for (int k = 0; k < VPL; ++k) {
+            f32x2 x[NP];
+            widen_pairs<DT>(raw[k], x);                                    // absent vectors are zeros
 #pragma unroll
-            for (int j = 0; j < NP; ++j) acc[j & 1] = add2(acc[j & 1], x[k][j]);
+            for (int j = 0; j < NP; ++j) acc[j & 1] = add2(acc[j & 1], x[j]);
         }
-        if (row + 1 < row_end) {
-#pragma unroll
-            for (int k = 0; k < VPT; ++k)
-                if (tid + k * T < nvec) next[k] = ld_stream(xv + (row + 1) * p.nvec + tid + k * T);
-        }
-        // exact two-pass statistics: the row sum first, then the squared deviations from the mean
-        float s = warp_sum<32>(pair_sum(add2(acc[0], acc[1])));
-        if (nwarps > 1) {
-            if (lane == 0) red[par][0][tid >> 5] = s;
-            __syncthreads();
-            s = warp_sum<32>(lane < nwarps ? red[par][0][lane] : 0.0f);
-        }
-        const float mu = s * inv_n;
+        const float mu = warp_sum<32>(pair_sum(add2(acc[0], acc[1]))) * inv_n;
         const f32x2 mu2 = pair(mu, mu);
         acc[0] = pair(0.0f, 0.0f); acc[1] = pair(0.0f, 0.0f);
 #pragma unroll
-        for (int k = 0; k < VPT; ++k) {
-            if (tid + k * T < nvec) {
+        for (int k = 0; k < VPL; ++k) {
+            if (lane + k * 32 < nvec) {
+                f32x2 x[NP];
+                widen_pairs<DT>(raw[k], x);
 #pragma unroll
-                for (int j = 0; j < NP; ++j) { x[k][j] = sub2(x[k][j], mu2); acc[j & 1] = fma2(x[k][j], x[k][j], acc[j & 1]); }
+                for (int j = 0; j < NP; ++j) { const f32x2 d = sub2(x[j], mu2); acc[j & 1] = fma2(d, d, acc[j & 1]); }
             }
         }
-        float q = warp_sum<32>(pair_sum(add2(acc[0], acc[1])));
-        if (nwarps > 1) {
-            if (lane == 0) red[par][1][tid >> 5] = q;
-            __syncthreads();
-            q = warp_sum<32>(lane < nwarps ? red[par][1][lane] : 0.0f);
-        }
-        const float rstd = rstd_of(q * inv_n, p.eps);
+        const float rstd = rstd_of(warp_sum<32>(pair_sum(add2(acc[0], acc[1]))) * inv_n, p.eps);
         const f32x2 r2 = pair(rstd, rstd);
 #pragma unroll
-        for (int k = 0; k < VPT; ++k) {
-            if (tid + k * T < nvec) {
-                affine_store_any<DT>(hg, hb, x[k], r2, graw[k], braw[k], yv + row * p.nvec + tid + k * T);
+        for (int k = 0; k < VPL; ++k) {
+            if (lane + k * 32 < nvec) {
+                f32x2 x[NP];
+                widen_pairs<DT>(raw[k], x);
+#pragma unroll
+                for (int j = 0; j < NP; ++j) x[j] = sub2(x[j], mu2);
+                uint4 graw = make_uint4(0u, 0u, 0u, 0u), braw = make_uint4(0u, 0u, 0u, 0u);
+                if (gv) graw = ld_cached(gv + k * 32);
+                if (bv) braw = ld_cached(bv + k * 32);
+                affine_store_any<DT>(gv != nullptr, bv != nullptr, x, r2, graw, braw, yv + row * p.nvec + k * 32);
             }
         }
     }
