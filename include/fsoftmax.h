@@ -138,7 +138,7 @@ int fs_router_topk(const void* x, float* w, int32_t* idx, int64_t rows, int64_t 
  *   or negative). A -inf entry beside finite ones gives -inf; a NaN or +inf entry (after scaling),
  *   or a row holding only -inf, makes the whole row NaN.
  * fp32 output is within 1e-6 * max(1, |y|) of the fp64 value, 16-bit output within one unit in the
- * last place of the correctly rounded fp64 value. Rows up to 4 KiB stay in the registers of a
+ * last place of the correctly rounded fp64 value. Rows up to 9 KiB stay in the registers of a
  * (sub-)warp, longer rows are split over a cluster with the slices resident in shared memory (one
  * read and one write of HBM per element), ragged or misaligned rows take a three-pass kernel.
  */

@@ -1014,6 +1014,11 @@ template <int DT> const void* lsm_warp_fn(const WarpGeom& g) {
             case 6: return (const void*)lsm_warp_kernel<DT, 32, 6>;
             case 7: return (const void*)lsm_warp_kernel<DT, 32, 7>;
             case 8: return (const void*)lsm_warp_kernel<DT, 32, 8>;
+            case 10: return (const void*)lsm_warp_kernel<DT, 32, 10>;
+            case 12: return (const void*)lsm_warp_kernel<DT, 32, 12>;
+            case 14: return (const void*)lsm_warp_kernel<DT, 32, 14>;
+            case 16: return (const void*)lsm_warp_kernel<DT, 32, 16>;
+            case 18: return (const void*)lsm_warp_kernel<DT, 32, 18>;
             default: return nullptr;
         }
     }
@@ -1044,7 +1049,15 @@ int run_log_softmax(const void* x, void* y, int64_t rows, int64_t cols, int dtyp
     p.flip = std::signbit(scale) && scale != 0.0f ? (dtype == FS_DTYPE_FP32 ? 0x80000000u : 0x80008000u) : 0u;
     p.status = dev.status; p.pf_rows = 0;
     WarpGeom wg;
-    if (fast && norm_warp_geom(p.nvec, dtype, &wg)) {
+    bool warp_ok = fast && norm_warp_geom(p.nvec, dtype, &wg);
+    if (fast && !warp_ok && p.nvec <= 576) {
+        // rows of 4-9 KiB: still a warp per row (the row stays packed in registers: 10..18 vectors per lane);
+        // the shared-memory kernel has too little to overlap on slices this short (measured 96-137 us
+        // against 80 for a copy on 256 MiB)
+        wg.lanes = 32; wg.vpl = static_cast<int>((p.nvec + 63) / 64) * 2; wg.r = 1;
+        warp_ok = true;
+    }
+    if (warp_ok) {
         const void* fn = by_dtype(dtype, [&](auto dt) -> const void* { return lsm_warp_fn<decltype(dt)::value>(wg); });
         if (fn) {
             const int t = 128;

@@ -6,7 +6,7 @@
 // |scale| is used, which is the same product exactly; the kernels therefore always look for a
 // maximum.
 //
-//   lsm_warp_kernel     (sub-)warp per row in registers (rows up to 4 KiB)
+//   lsm_warp_kernel     (sub-)warp per row, the row packed in registers (rows up to 9 KiB)
 //   lsm_smem_kernel     row split over a cluster of 1..16 blocks, slices resident in shared memory
 //                       (bulk async copies, per-chunk mbarriers, online (max, sum) per thread,
 //                       pairs merged warp -> block -> cluster through st.async); pass 2 reads the
@@ -61,7 +61,7 @@ __device__ __forceinline__ void lsm_accumulate(const uint4& raw, f32x2 r2, f32x2
 
 // ---------------------------------------------------------------------------------------------
 template <int DT, int LANES, int VPL>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(128, VPL <= 8 ? 6 : VPL <= 12 ? 5 : 4)
 lsm_warp_kernel(const LsmParams p) {
     constexpr int NP = Traits<DT>::VE / 2;
     constexpr int G = 32 / LANES;
