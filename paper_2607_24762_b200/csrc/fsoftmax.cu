@@ -1014,11 +1014,11 @@ template <int DT> const void* lsm_warp_fn(const WarpGeom& g) {
             case 6: return (const void*)lsm_warp_kernel<DT, 32, 6>;
             case 7: return (const void*)lsm_warp_kernel<DT, 32, 7>;
             case 8: return (const void*)lsm_warp_kernel<DT, 32, 8>;
-            case 10: return (const void*)lsm_warp_kernel<DT, 32, 10>;
-            case 12: return (const void*)lsm_warp_kernel<DT, 32, 12>;
-            case 14: return (const void*)lsm_warp_kernel<DT, 32, 14>;
-            case 16: return (const void*)lsm_warp_kernel<DT, 32, 16>;
-            case 18: return (const void*)lsm_warp_kernel<DT, 32, 18>;
+            case 10: return (const void*)lsm_warp_long_kernel<DT, 10>;
+            case 12: return (const void*)lsm_warp_long_kernel<DT, 12>;
+            case 14: return (const void*)lsm_warp_long_kernel<DT, 14>;
+            case 16: return (const void*)lsm_warp_long_kernel<DT, 16>;
+            case 18: return (const void*)lsm_warp_long_kernel<DT, 18>;
             default: return nullptr;
         }
     }
@@ -1178,6 +1178,11 @@ template <int DT> const void* masked_warp_fn(const WarpGeom& g) {
             case 6: return (const void*)sm_masked_warp_kernel<DT, 32, 6>;
             case 7: return (const void*)sm_masked_warp_kernel<DT, 32, 7>;
             case 8: return (const void*)sm_masked_warp_kernel<DT, 32, 8>;
+            case 10: return (const void*)sm_masked_warp_long_kernel<DT, 10>;
+            case 12: return (const void*)sm_masked_warp_long_kernel<DT, 12>;
+            case 14: return (const void*)sm_masked_warp_long_kernel<DT, 14>;
+            case 16: return (const void*)sm_masked_warp_long_kernel<DT, 16>;
+            case 18: return (const void*)sm_masked_warp_long_kernel<DT, 18>;
             default: return nullptr;
         }
     }
@@ -1208,7 +1213,12 @@ int run_softmax_masked(const void* x, const void* mask, void* y, int64_t rows, i
     p.c = static_cast<float>(static_cast<double>(scale) * kLog2e);
     p.status = dev.status; p.pf_rows = 0;
     WarpGeom wg;
-    if (fast && norm_warp_geom(p.nvec, dtype, &wg)) {
+    bool warp_ok = fast && norm_warp_geom(p.nvec, dtype, &wg);
+    if (fast && !warp_ok && p.nvec <= 576) {        // rows of 4-9 KiB: still a warp per row, 10..18 packed vectors per lane
+        wg.lanes = 32; wg.vpl = static_cast<int>((p.nvec + 63) / 64) * 2; wg.r = 1;
+        warp_ok = true;
+    }
+    if (warp_ok) {
         const void* fn = by_dtype(dtype, [&](auto dt) -> const void* { return masked_warp_fn<decltype(dt)::value>(wg); });
         if (fn) {
             const int t = 128;

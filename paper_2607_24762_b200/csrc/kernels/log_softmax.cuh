@@ -61,8 +61,7 @@ __device__ __forceinline__ void lsm_accumulate(const uint4& raw, f32x2 r2, f32x2
 
 // ---------------------------------------------------------------------------------------------
 template <int DT, int LANES, int VPL>
-__global__ void __launch_bounds__(128, VPL <= 8 ? 6 : VPL <= 12 ? 5 : 4)
-lsm_warp_kernel(const LsmParams p) {
+__device__ __forceinline__ void lsm_warp_body(const LsmParams& p) {
     constexpr int NP = Traits<DT>::VE / 2;
     constexpr int G = 32 / LANES;
     pdl_launch_dependents();
@@ -116,6 +115,20 @@ lsm_warp_kernel(const LsmParams p) {
             }
         }
     }
+}
+
+// Up to eight vectors per lane the compiler's own register choice is best (an explicit minimum of
+// blocks per SM, even 1, makes it spend registers: measured 88 us against 80 on short rows); the
+// long-row variants are capped so that four or five blocks stay resident.
+template <int DT, int LANES, int VPL>
+__global__ void __launch_bounds__(128)
+lsm_warp_kernel(const LsmParams p) {
+    lsm_warp_body<DT, LANES, VPL>(p);
+}
+template <int DT, int VPL>
+__global__ void __launch_bounds__(128, VPL <= 12 ? 5 : 4)
+lsm_warp_long_kernel(const LsmParams p) {
+    lsm_warp_body<DT, 32, VPL>(p);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -9,7 +9,7 @@
 // both terms), so the exponent carries the binary32 rounding of a number of the size of |z|: the
 // parity bound of this entry point grows with max |z| (see the header).
 //
-//   sm_masked_warp_kernel     (sub-)warp per row in registers (rows up to 4 KiB)
+//   sm_masked_warp_kernel     (sub-)warp per row, the row packed in registers (rows up to 9 KiB)
 //   sm_masked_smem_kernel     the split-row design: x slice resident in shared memory, mask slice
 //                             read from L2 in pass 1 only (e is stored in place, as in smem_row)
 //   sm_masked_generic_kernel  block per row, element-wise, any shape and alignment
@@ -60,9 +60,12 @@ __device__ __forceinline__ float masked_exponents(const uint4& xraw, const uint4
 }
 
 // ---------------------------------------------------------------------------------------------
+// The row stays packed in registers; the mask vectors are not kept but read twice through the
+// read-only path (they are shared by the heads and hit L1/L2). Pass A takes the maximum exponent,
+// pass B forms e = 2^(t - R), adds it up and puts it back in place of x in the element dtype
+// (the in-place store of the split-row kernel, in registers), pass C scales and stores.
 template <int DT, int LANES, int VPL>
-__global__ void __launch_bounds__(128, 5)      // 102 registers: five blocks per SM; a tighter cap spills
-sm_masked_warp_kernel(const MaskedParams p) {
+__device__ __forceinline__ void sm_masked_warp_body(const MaskedParams& p) {
     constexpr int NP = Traits<DT>::VE / 2;
     constexpr int G = 32 / LANES;
     pdl_launch_dependents();
@@ -79,52 +82,62 @@ sm_masked_warp_kernel(const MaskedParams p) {
     for (int64_t grp = int64_t(blockIdx.x) * warps + (threadIdx.x >> 5); grp < ngroups; grp += int64_t(gridDim.x) * warps) {
         const int64_t row = grp * G + sub;
         const bool row_ok = row < p.rows;
-        const int64_t mrow = row_ok ? mask_row_of(p, row) : 0;
-        uint4 xraw[VPL], mraw[VPL];
+        const uint4* mr = mv + (row_ok ? mask_row_of(p, row) : 0) * p.nvec + sl;
+        uint4 xraw[VPL];
 #pragma unroll
         for (int k = 0; k < VPL; ++k) {
-            xraw[k] = make_uint4(0u, 0u, 0u, 0u); mraw[k] = make_uint4(0u, 0u, 0u, 0u);
-            if (row_ok && sl + k * LANES < nvec) {
-                xraw[k] = ld_stream(xv + row * p.nvec + sl + k * LANES);
-                mraw[k] = ld_cached(mv + mrow * p.nvec + sl + k * LANES);
-            }
+            xraw[k] = make_uint4(0u, 0u, 0u, 0u);
+            if (row_ok && sl + k * LANES < nvec) xraw[k] = ld_stream(xv + row * p.nvec + sl + k * LANES);
         }
-        f32x2 t[VPL][NP];
         float r = __int_as_float(0xff800000);
 #pragma unroll
         for (int k = 0; k < VPL; ++k) {
-            const float b = masked_exponents<DT>(xraw[k], mraw[k], c2, t[k]);
-            if (sl + k * LANES < nvec) r = fmaxf(r, b);
+            if (row_ok && sl + k * LANES < nvec) {
+                f32x2 t[NP];
+                r = fmaxf(r, masked_exponents<DT>(xraw[k], ld_cached(mr + k * LANES), c2, t));
+            }
         }
         r = warp_pick<LANES, false>(r);
         const f32x2 r2 = pair(r, r);
         f32x2 acc[2] = {pair(0.0f, 0.0f), pair(0.0f, 0.0f)};
 #pragma unroll
         for (int k = 0; k < VPL; ++k) {
-            if (sl + k * LANES < nvec) {
+            if (row_ok && sl + k * LANES < nvec) {
+                f32x2 t[NP];
+                masked_exponents<DT>(xraw[k], ld_cached(mr + k * LANES), c2, t);
 #pragma unroll
                 for (int j = 0; j < NP; ++j) {
                     float lo, hi;
-                    unpair(sub2(t[k][j], r2), lo, hi);
+                    unpair(sub2(t[j], r2), lo, hi);
                     if (DT == DT_BF16) { lo += 64.0f; hi += 64.0f; }        // keeps subnormal bf16 outputs (see ex2_elem)
-                    t[k][j] = pair(ex2_ftz(lo), ex2_ftz(hi));
-                    acc[j & 1] = add2(acc[j & 1], t[k][j]);
+                    t[j] = pair(ex2_ftz(lo), ex2_ftz(hi));
+                    acc[j & 1] = add2(acc[j & 1], t[j]);
                 }
+                xraw[k] = narrow_pairs<DT>(t);
             }
         }
         const float inv = recip<DT>(warp_sum<LANES>(pair_sum(add2(acc[0], acc[1]))));
         const f32x2 i2 = pair(inv, inv);
         if (row_ok) {
 #pragma unroll
-            for (int k = 0; k < VPL; ++k) {
-                if (sl + k * LANES < nvec) {
-#pragma unroll
-                    for (int j = 0; j < NP; ++j) t[k][j] = mul2(t[k][j], i2);
-                    st_stream(yv + row * p.nvec + sl + k * LANES, narrow_pairs<DT>(t[k]));
-                }
-            }
+            for (int k = 0; k < VPL; ++k)
+                if (sl + k * LANES < nvec) st_stream(yv + row * p.nvec + sl + k * LANES, scale_vec<DT, false>(xraw[k], i2, i2));
         }
     }
+}
+
+// Up to eight vectors per lane the compiler's own register choice is best (an explicit minimum of
+// blocks per SM, even 1, makes it spend registers: measured 88 us against 80 on short rows); the
+// long-row variants are capped so that four or five blocks stay resident.
+template <int DT, int LANES, int VPL>
+__global__ void __launch_bounds__(128)
+sm_masked_warp_kernel(const MaskedParams p) {
+    sm_masked_warp_body<DT, LANES, VPL>(p);
+}
+template <int DT, int VPL>
+__global__ void __launch_bounds__(128, VPL <= 12 ? 5 : 4)
+sm_masked_warp_long_kernel(const MaskedParams p) {
+    sm_masked_warp_body<DT, 32, VPL>(p);
 }
 
 // ---------------------------------------------------------------------------------------------
