@@ -45,7 +45,7 @@ def main() -> int:
             ran += 1
     assert fs.fs_device_status() == fs.FS_OK
     print(f"mode_check ok: {ran} cases, env " +
-          " ".join(f"{k}={os.environ[k]}" for k in ("FS_PERSISTENT", "FS_CLUSTER_REGS", "FS_PDL") if k in os.environ))
+          " ".join(f"{k}={os.environ[k]}" for k in ("FS_PERSISTENT", "FS_CLUSTER_REGS", "FS_PDL", "FS_PREFETCH_PCT") if k in os.environ))
     return 0
 
 
