@@ -305,6 +305,52 @@ def time_log_softmax(w: W.Workload, steps: int, warmup: int, l2_bytes: int, eage
     return out
 
 
+def time_softmax_f32out(w: W.Workload, steps: int, warmup: int, l2_bytes: int, eager: bool = True):
+    """fs_softmax_f32out on a 16-bit softmax workload: reads 2 bytes and writes 4 per element."""
+    import torch
+
+    import paper_2607_24762_b200 as fs
+    if w.dtype == W.FP32:
+        raise ValueError("fs_softmax_f32out takes bf16/fp16 input")
+    alg = w.rows * w.cols * 6
+    n_pairs = int(max(1, min(16, math.ceil(4 * l2_bytes / alg))))
+    xs, _ = device_buffers(w, n_pairs, threads=min(8, os.cpu_count() or 1))
+    ys = [torch.empty((w.rows, w.cols), dtype=torch.float32, device="cuda") for _ in range(n_pairs)]
+    stream = torch.cuda.current_stream()
+    lib = fs.binding.lib()
+    tdt = torch.bfloat16 if w.dtype == W.BF16 else torch.float16
+
+    def launch(i):
+        j = i % n_pairs
+        st = lib.fs_softmax_f32out(xs[j].data_ptr(), ys[j].data_ptr(), w.rows, w.cols, w.dtype, w.scale_f32, stream.cuda_stream)
+        if st != 0:
+            raise RuntimeError(fs.fs_strerror(st))
+
+    def eager_launch(i):
+        torch.softmax(xs[i % n_pairs].view(tdt).view(w.rows, w.cols) * w.scale_f32, dim=-1, dtype=torch.float32)
+
+    def timed(fn, k):
+        for i in range(max(3, warmup)):
+            fn(i)
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        start.record(stream)
+        for i in range(k):
+            fn(i)
+        stop.record(stream)
+        torch.cuda.synchronize()
+        return start.elapsed_time(stop) / k
+
+    ms = timed(launch, steps)
+    peak, _ = measured_peak()
+    gbs = alg / (ms * 1e-3) / 1e9
+    out = {"what": f"fs_softmax_f32out on {w.name}: 16-bit in, float32 out", "steps": steps, "ms_per_step": round(ms, 6),
+           "algorithmic_bytes": alg, "GB/s": round(gbs, 1), "frac_of_measured_copy": round(gbs / peak, 4), "n_pairs": n_pairs}
+    if eager:
+        out["torch_eager_ms"] = round(timed(eager_launch, max(5, steps // 4)), 6)
+    return out
+
+
 def time_softmax_masked(w: W.Workload, steps: int, warmup: int, l2_bytes: int, heads: int = 8, eager: bool = True):
     """fs_softmax_masked on a softmax workload's data viewed as (batch 1, `heads`, rows/heads queries) with a
     causal mask shared by the heads; algorithmic bytes = x + y + the mask once."""
@@ -613,7 +659,7 @@ def main():
                     help="also time the other workloads (default: on at --gpus 1)")
     ap.add_argument("--no-all", dest="all_workloads", action="store_false")
     ap.add_argument("--norm-workload", default="ln_sd35", choices=sorted(NORM_WORKLOADS), help="with --op norm")
-    ap.add_argument("--op", default="softmax", choices=["softmax", "causal", "router", "norm", "log_softmax", "backward", "masked"],
+    ap.add_argument("--op", default="softmax", choices=["softmax", "causal", "router", "norm", "log_softmax", "backward", "masked", "f32out"],
                     help="time only fs_softmax_causal (q_offset 0) or fs_router_topk (k=8, renormalised) on the "
                          "workload and print a short line (profiler captures of those kernels)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the cpu_baseline leg")
@@ -668,6 +714,8 @@ def main():
                  "GB/s": round(alg / (r["ms_per_step"] * 1e-3) / 1e9, 1)}
         elif args.op == "log_softmax":
             r = time_log_softmax(w, args.steps, args.warmup, l2, eager=not args.no_cpu)
+        elif args.op == "f32out":
+            r = time_softmax_f32out(w, args.steps, args.warmup, l2, eager=not args.no_cpu)
         elif args.op == "masked":
             r = time_softmax_masked(w, args.steps, args.warmup, l2, eager=not args.no_cpu)
         elif args.op == "backward":
@@ -749,6 +797,10 @@ def main():
                     others[lname + "_log_softmax"] = time_log_softmax(W.WORKLOADS[lname], 300, 10, l2)
                 except Exception as exc:
                     others[lname + "_log_softmax"] = {"error": str(exc)[:200]}
+            try:
+                others["cfg2_f32out"] = time_softmax_f32out(W.WORKLOADS["cfg2"], 300, 10, l2)
+            except Exception as exc:
+                others["cfg2_f32out"] = {"error": str(exc)[:200]}
             try:
                 others["cfg2_masked"] = time_softmax_masked(W.WORKLOADS["cfg2"], 300, 10, l2)
             except Exception as exc:

@@ -145,6 +145,17 @@ int fs_router_topk(const void* x, float* w, int32_t* idx, int64_t rows, int64_t 
 int fs_log_softmax(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale, void* stream);
 
 /*
+ * fs_softmax_f32out -- softmax of a bf16/fp16 tensor written as binary32: what eager attention asks
+ * for with softmax(scores, dim=-1, dtype=float32) before it casts back (the mixed-dtype variant of
+ * the operator; variants are the paper's Sec. III-A).
+ *   x      device pointer, rows*cols elements of `dtype` (FS_DTYPE_BF16 or FS_DTYPE_FP16 only).
+ *   y      device pointer, rows*cols floats; must not overlap x.
+ * Same formula, special values and scale rules as fs_softmax; every output is within 1e-6 of the
+ * fp64 value. Traffic is 6 bytes per element (2 in, 4 out).
+ */
+int fs_softmax_f32out(const void* x, float* y, int64_t rows, int64_t cols, int dtype, float scale, void* stream);
+
+/*
  * fs_softmax_masked -- softmax with an additive mask applied inside the kernel, the other half of the
  * `scores + mask -> softmax` pair of eager attention (operator fusion, the paper's Sec. II-B; the
  * workloads are the eager-attention softmax calls of its Table I):

@@ -10,5 +10,5 @@ from .binding import (  # noqa: F401
     FS_ROUTER_MAX_K, FS_STATIC_MAX_ROW_BYTES, KERNELS, FsError,
     fs_copy, fs_device_status, fs_group_norm, fs_kernel_name, fs_last_cuda_error, fs_layer_norm, fs_log_softmax, fs_release, fs_router_topk,
     fs_select_kernel, fs_split_geometry,
-    fs_softmax, fs_softmax_backward, fs_softmax_causal, fs_softmax_ex, fs_softmax_host, fs_softmax_masked, fs_softmax_static, fs_softmax_status, fs_strerror, fs_version,
+    fs_softmax, fs_softmax_backward, fs_softmax_causal, fs_softmax_ex, fs_softmax_f32out, fs_softmax_host, fs_softmax_masked, fs_softmax_static, fs_softmax_status, fs_strerror, fs_version,
 )

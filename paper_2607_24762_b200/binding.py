@@ -55,6 +55,8 @@ def lib() -> ctypes.CDLL:
             L.fs_router_topk.restype = ci
             L.fs_log_softmax.argtypes = [vp, vp, i64, i64, ci, f32, vp]
             L.fs_log_softmax.restype = ci
+            L.fs_softmax_f32out.argtypes = [vp, vp, i64, i64, ci, f32, vp]
+            L.fs_softmax_f32out.restype = ci
             L.fs_softmax_masked.argtypes = [vp, vp, vp, i64, i64, i64, i64, ci, f32, vp]
             L.fs_softmax_masked.restype = ci
             L.fs_softmax_backward.argtypes = [vp, vp, vp, i64, i64, ci, f32, vp]
@@ -147,6 +149,11 @@ def fs_router_topk(x, w, idx, rows: int, cols: int, k: int, dtype: int, scale: f
 def fs_log_softmax(x, y, rows: int, cols: int, dtype: int, scale: float = 1.0, stream=None) -> None:
     """y = log_softmax(scale * x) over the last dimension of a [rows, cols] device tensor."""
     _check(lib().fs_log_softmax(_ptr(x), _ptr(y), rows, cols, dtype, scale, _stream(stream)), "fs_log_softmax")
+
+
+def fs_softmax_f32out(x, y, rows: int, cols: int, dtype: int, scale: float = 1.0, stream=None) -> None:
+    """softmax(scale * x) of a bf16/fp16 [rows, cols] device tensor, written as float32."""
+    _check(lib().fs_softmax_f32out(_ptr(x), _ptr(y), rows, cols, dtype, scale, _stream(stream)), "fs_softmax_f32out")
 
 
 def fs_softmax_masked(x, mask, y, rows: int, cols: int, q_rows: int, heads: int, dtype: int, scale: float = 1.0,

@@ -1003,38 +1003,39 @@ int validate_norm(const void* x, const void* y, int64_t rows, int64_t cols, int 
 // ---------------------------------------------------------------------------------------------
 // log_softmax
 // ---------------------------------------------------------------------------------------------
-template <int DT> const void* lsm_warp_fn(const WarpGeom& g) {
+template <int DT, int OUT> const void* lsm_warp_fn(const WarpGeom& g) {
     if (g.lanes == 32) {
         switch (g.vpl) {
-            case 1: return (const void*)lsm_warp_kernel<DT, 32, 1>;
-            case 2: return (const void*)lsm_warp_kernel<DT, 32, 2>;
-            case 3: return (const void*)lsm_warp_kernel<DT, 32, 3>;
-            case 4: return (const void*)lsm_warp_kernel<DT, 32, 4>;
-            case 5: return (const void*)lsm_warp_kernel<DT, 32, 5>;
-            case 6: return (const void*)lsm_warp_kernel<DT, 32, 6>;
-            case 7: return (const void*)lsm_warp_kernel<DT, 32, 7>;
-            case 8: return (const void*)lsm_warp_kernel<DT, 32, 8>;
-            case 10: return (const void*)lsm_warp_long_kernel<DT, 10>;
-            case 12: return (const void*)lsm_warp_long_kernel<DT, 12>;
-            case 14: return (const void*)lsm_warp_long_kernel<DT, 14>;
-            case 16: return (const void*)lsm_warp_long_kernel<DT, 16>;
-            case 18: return (const void*)lsm_warp_long_kernel<DT, 18>;
+            case 1: return (const void*)lsm_warp_kernel<DT, 32, 1, OUT>;
+            case 2: return (const void*)lsm_warp_kernel<DT, 32, 2, OUT>;
+            case 3: return (const void*)lsm_warp_kernel<DT, 32, 3, OUT>;
+            case 4: return (const void*)lsm_warp_kernel<DT, 32, 4, OUT>;
+            case 5: return (const void*)lsm_warp_kernel<DT, 32, 5, OUT>;
+            case 6: return (const void*)lsm_warp_kernel<DT, 32, 6, OUT>;
+            case 7: return (const void*)lsm_warp_kernel<DT, 32, 7, OUT>;
+            case 8: return (const void*)lsm_warp_kernel<DT, 32, 8, OUT>;
+            case 10: return (const void*)lsm_warp_long_kernel<DT, 10, OUT>;
+            case 12: return (const void*)lsm_warp_long_kernel<DT, 12, OUT>;
+            case 14: return (const void*)lsm_warp_long_kernel<DT, 14, OUT>;
+            case 16: return (const void*)lsm_warp_long_kernel<DT, 16, OUT>;
+            case 18: return (const void*)lsm_warp_long_kernel<DT, 18, OUT>;
             default: return nullptr;
         }
     }
-    if (g.vpl == 1) return (const void*)lsm_warp_kernel<DT, 1, 1>;
-    if (g.vpl == 2) return (const void*)lsm_warp_kernel<DT, 1, 2>;
+    if (g.vpl == 1) return (const void*)lsm_warp_kernel<DT, 1, 1, OUT>;
+    if (g.vpl == 2) return (const void*)lsm_warp_kernel<DT, 1, 2, OUT>;
     if (g.vpl != 4) return nullptr;
     switch (g.lanes) {
-        case 1:  return (const void*)lsm_warp_kernel<DT, 1, 4>;
-        case 2:  return (const void*)lsm_warp_kernel<DT, 2, 4>;
-        case 4:  return (const void*)lsm_warp_kernel<DT, 4, 4>;
-        case 8:  return (const void*)lsm_warp_kernel<DT, 8, 4>;
-        default: return (const void*)lsm_warp_kernel<DT, 16, 4>;
+        case 1:  return (const void*)lsm_warp_kernel<DT, 1, 4, OUT>;
+        case 2:  return (const void*)lsm_warp_kernel<DT, 2, 4, OUT>;
+        case 4:  return (const void*)lsm_warp_kernel<DT, 4, 4, OUT>;
+        case 8:  return (const void*)lsm_warp_kernel<DT, 8, 4, OUT>;
+        default: return (const void*)lsm_warp_kernel<DT, 16, 4, OUT>;
     }
 }
 
-int run_log_softmax(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale, cudaStream_t st) {
+// out: OUT_LOG (log_softmax in x's dtype) or OUT_PROB32 (softmax of a 16-bit tensor written as binary32)
+int run_log_softmax(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale, int out, cudaStream_t st) {
     Device* devp = nullptr;
     int rc = get_device(&devp);
     if (rc != FS_OK) return rc;
@@ -1058,7 +1059,10 @@ int run_log_softmax(const void* x, void* y, int64_t rows, int64_t cols, int dtyp
         warp_ok = true;
     }
     if (warp_ok) {
-        const void* fn = by_dtype(dtype, [&](auto dt) -> const void* { return lsm_warp_fn<decltype(dt)::value>(wg); });
+        const void* fn = by_dtype(dtype, [&](auto dt) -> const void* {
+            constexpr int DT = decltype(dt)::value;
+            if constexpr (DT == DT_F32) return out == OUT_LOG ? lsm_warp_fn<DT, OUT_LOG>(wg) : nullptr;
+            else return out == OUT_LOG ? lsm_warp_fn<DT, OUT_LOG>(wg) : lsm_warp_fn<DT, OUT_PROB32>(wg); });
         if (fn) {
             const int t = 128;
             const int64_t groups = (rows + (32 / wg.lanes) - 1) / (32 / wg.lanes);
@@ -1073,7 +1077,12 @@ int run_log_softmax(const void* x, void* y, int64_t rows, int64_t cols, int dtyp
         if (full || p.c != 0.0f) {
             const void* fn = by_dtype(dtype, [&](auto dt) -> const void* {
                 constexpr int DT = decltype(dt)::value;
-                return full ? (const void*)lsm_smem_kernel<DT, true> : (const void*)lsm_smem_kernel<DT, false>; });
+                if constexpr (DT == DT_F32) {
+                    return full ? (const void*)lsm_smem_kernel<DT, true, OUT_LOG> : (const void*)lsm_smem_kernel<DT, false, OUT_LOG>;
+                } else {
+                    if (out == OUT_LOG) return full ? (const void*)lsm_smem_kernel<DT, true, OUT_LOG> : (const void*)lsm_smem_kernel<DT, false, OUT_LOG>;
+                    return full ? (const void*)lsm_smem_kernel<DT, true, OUT_PROB32> : (const void*)lsm_smem_kernel<DT, false, OUT_PROB32>;
+                } });
             const size_t stage_bytes = smem_row_stage_bytes(sg, dtype);
             const size_t smem = stage_bytes + size_t(kNormMaxChunks) * 8;
             if (smem <= static_cast<size_t>(dev.smem_optin) - 2048) {
@@ -1085,7 +1094,10 @@ int run_log_softmax(const void* x, void* y, int64_t rows, int64_t cols, int dtyp
             }
         }
     }
-    const void* fn = by_dtype(dtype, [&](auto dt) -> const void* { return (const void*)lsm_generic_kernel<decltype(dt)::value>; });
+    const void* fn = by_dtype(dtype, [&](auto dt) -> const void* {
+        constexpr int DT = decltype(dt)::value;
+        if constexpr (DT == DT_F32) return (const void*)lsm_generic_kernel<DT, OUT_LOG>;
+        else return out == OUT_LOG ? (const void*)lsm_generic_kernel<DT, OUT_LOG> : (const void*)lsm_generic_kernel<DT, OUT_PROB32>; });
     int t = 32;
     while (t < 1024 && cols > int64_t(t) * 8) t <<= 1;
     return launch(fn, std::min<int64_t>(rows, 0x7fffffff), t, 0, 0, st, p);
@@ -1315,7 +1327,7 @@ int fs_log_softmax(const void* x, void* y, int64_t rows, int64_t cols, int dtype
     const int v = validate(x, y, rows, cols, dtype, scale);
     if (v != FS_OK) return v;
     if (rows == 0 || cols == 0) return FS_OK;
-    return run_log_softmax(x, y, rows, cols, dtype, scale, static_cast<cudaStream_t>(stream));
+    return run_log_softmax(x, y, rows, cols, dtype, scale, OUT_LOG, static_cast<cudaStream_t>(stream));
 }
 
 int fs_softmax_masked(const void* x, const void* mask, void* y, int64_t rows, int64_t cols, int64_t q_rows, int64_t heads,
@@ -1336,6 +1348,19 @@ int fs_softmax_backward(const void* dy, const void* y, void* dx, int64_t rows, i
     if (v != FS_OK) return v;
     if (rows == 0 || cols == 0) return FS_OK;
     return run_softmax_backward(dy, y, dx, rows, cols, dtype, scale, static_cast<cudaStream_t>(stream));
+}
+
+int fs_softmax_f32out(const void* x, float* y, int64_t rows, int64_t cols, int dtype, float scale, void* stream) {
+    if (rows < 0 || cols < 0 || !std::isfinite(scale)) return FS_ERR_INVALID_ARG;
+    if (dtype != FS_DTYPE_BF16 && dtype != FS_DTYPE_FP16) return FS_ERR_INVALID_ARG;
+    if (rows == 0 || cols == 0) return FS_OK;
+    if (!x || !y) return FS_ERR_INVALID_ARG;
+    if (cols > (int64_t(1) << 40) || rows > (int64_t(1) << 40) || rows > (int64_t(1) << 59) / cols) return FS_ERR_INVALID_ARG;
+    if (ptr_align(y) < 4) return FS_ERR_INVALID_ARG;
+    const uintptr_t a = reinterpret_cast<uintptr_t>(x), b = reinterpret_cast<uintptr_t>(y);
+    const uintptr_t na = static_cast<uintptr_t>(rows * cols * 2), nb = static_cast<uintptr_t>(rows * cols * 4);
+    if (a < b + nb && b < a + na) return FS_ERR_INVALID_ARG;          // the tensors differ in size: no overlap at all
+    return run_log_softmax(x, y, rows, cols, dtype, scale, OUT_PROB32, static_cast<cudaStream_t>(stream));
 }
 
 int fs_layer_norm(const void* x, const void* gamma, const void* beta, void* y, int64_t rows, int64_t cols, int dtype,

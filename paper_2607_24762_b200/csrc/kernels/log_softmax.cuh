@@ -1,7 +1,9 @@
-// log_softmax over the last dimension: y = z - max z - ln sum exp(z - max z), z = scale * x.
-// The same skeleton as the softmax kernels (one read, reduce, one write), but the output is formed
-// from x itself, so nothing is written back over the resident row:
-//     d = x - r,  S = sum 2^(d c),  y = d * scale - ln S          (c = scale * log2 e)
+// Kernels that form their output from x itself, so nothing is written back over the resident row:
+//   OUT_LOG    log_softmax: y = z - max z - ln sum exp(z - max z), z = scale * x, in x's dtype
+//                  d = x - r,  S = sum 2^(d c),  y = d * scale - ln S      (c = scale * log2 e)
+//   OUT_PROB32 softmax of a 16-bit tensor written as binary32 (what eager attention asks for with
+//              softmax(..., dtype=float32)): y = 2^(d c) / S, the exponential taken a second time
+// The same skeleton as the softmax kernels (one read, reduce, one write).
 // A negative scale is folded into the data: the sign bit of every element is flipped on load and
 // |scale| is used, which is the same product exactly; the kernels therefore always look for a
 // maximum.
@@ -18,6 +20,8 @@
 #include "norm_row.cuh"
 
 namespace fsm {
+
+enum : int { OUT_LOG = 0, OUT_PROB32 = 1 };
 
 struct LsmParams {
     const void* x;
@@ -59,8 +63,36 @@ __device__ __forceinline__ void lsm_accumulate(const uint4& raw, f32x2 r2, f32x2
     }
 }
 
+// One vector of output from one (sign-adjusted) vector of x. `ybase` is the row's first output
+// element; `v` the vector's index in the row. k2 is -ln S (OUT_LOG) or 1/S (OUT_PROB32).
+template <int DT, int OUT>
+__device__ __forceinline__ void lsm_emit(const uint4& raw, f32x2 r2, f32x2 c2, f32x2 s2, f32x2 k2, void* ybase, int64_t v) {
+    constexpr int NP = Traits<DT>::VE / 2;
+    f32x2 d[NP];
+    widen_pairs<DT>(raw, d);
+    if constexpr (OUT == OUT_LOG) {
+#pragma unroll
+        for (int j = 0; j < NP; ++j) d[j] = fma2(sub2(d[j], r2), s2, k2);
+        st_stream(static_cast<uint4*>(ybase) + v, narrow_pairs<DT>(d));
+    } else {
+        static_assert(OUT == OUT_LOG || DT != DT_F32, "binary32 output is for 16-bit inputs");
+#pragma unroll
+        for (int j = 0; j < NP; ++j) {
+            float lo, hi;
+            unpair(mul2(sub2(d[j], r2), c2), lo, hi);
+            d[j] = mul2(pair(ex2_ftz(lo), ex2_ftz(hi)), k2);
+        }
+        uint4* out = static_cast<uint4*>(ybase) + 2 * v;              // eight floats: two vectors
+        uint4 a, b;
+        unpair_bits(d[0], a.x, a.y); unpair_bits(d[1], a.z, a.w);
+        unpair_bits(d[NP - 2], b.x, b.y); unpair_bits(d[NP - 1], b.z, b.w);
+        st_stream(out, a);
+        st_stream(out + 1, b);
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
-template <int DT, int LANES, int VPL>
+template <int DT, int LANES, int VPL, int OUT>
 __device__ __forceinline__ void lsm_warp_body(const LsmParams& p) {
     constexpr int NP = Traits<DT>::VE / 2;
     constexpr int G = 32 / LANES;
@@ -70,7 +102,7 @@ __device__ __forceinline__ void lsm_warp_body(const LsmParams& p) {
     const int warps = blockDim.x >> 5;
     const int nvec = static_cast<int>(p.nvec);
     const uint4* __restrict__ xv = static_cast<const uint4*>(p.x);
-    uint4* __restrict__ yv = static_cast<uint4*>(p.y);
+    const int64_t ypitch = OUT == OUT_LOG ? p.nvec * 16 : p.cols * 4;      // bytes per output row
     const f32x2 c2 = pair(p.c, p.c), s2 = pair(p.scale, p.scale);
     pdl_wait();
     const int64_t ngroups = (p.rows + G - 1) / G;
@@ -100,19 +132,14 @@ __device__ __forceinline__ void lsm_warp_body(const LsmParams& p) {
                 lsm_accumulate<DT>(raw[k], r2, c2, d, acc);
             }
         }
-        const float lns = ln_of(warp_sum<LANES>(pair_sum(add2(acc[0], acc[1]))));
-        const f32x2 l2 = pair(-lns, -lns);
+        const float ssum = warp_sum<LANES>(pair_sum(add2(acc[0], acc[1])));
+        const float kk = OUT == OUT_LOG ? -ln_of(ssum) : 1.0f / ssum;
+        const f32x2 k2 = pair(kk, kk);
         if (row_ok) {
+            char* yrow = static_cast<char*>(p.y) + row * ypitch;
 #pragma unroll
-            for (int k = 0; k < VPL; ++k) {
-                if (sl + k * LANES < nvec) {
-                    f32x2 d[NP];
-                    widen_pairs<DT>(raw[k], d);
-#pragma unroll
-                    for (int j = 0; j < NP; ++j) d[j] = fma2(sub2(d[j], r2), s2, l2);
-                    st_stream(yv + row * p.nvec + sl + k * LANES, narrow_pairs<DT>(d));
-                }
-            }
+            for (int k = 0; k < VPL; ++k)
+                if (sl + k * LANES < nvec) lsm_emit<DT, OUT>(raw[k], r2, c2, s2, k2, yrow, sl + k * LANES);
         }
     }
 }
@@ -120,22 +147,22 @@ __device__ __forceinline__ void lsm_warp_body(const LsmParams& p) {
 // Up to eight vectors per lane the compiler's own register choice is best (an explicit minimum of
 // blocks per SM, even 1, makes it spend registers: measured 88 us against 80 on short rows); the
 // long-row variants are capped so that four or five blocks stay resident.
-template <int DT, int LANES, int VPL>
+template <int DT, int LANES, int VPL, int OUT>
 __global__ void __launch_bounds__(128)
 lsm_warp_kernel(const LsmParams p) {
-    lsm_warp_body<DT, LANES, VPL>(p);
+    lsm_warp_body<DT, LANES, VPL, OUT>(p);
 }
-template <int DT, int VPL>
+template <int DT, int VPL, int OUT>
 __global__ void __launch_bounds__(128, VPL <= 12 ? 5 : 4)
 lsm_warp_long_kernel(const LsmParams p) {
-    lsm_warp_body<DT, 32, VPL>(p);
+    lsm_warp_body<DT, 32, VPL, OUT>(p);
 }
 
 // ---------------------------------------------------------------------------------------------
 // cluster per row (one-shot grid: cluster i handles row i); dynamic shared memory: slice rounded
 // up to whole chunks (stage_bytes) | 8 chunk mbarriers
 // ---------------------------------------------------------------------------------------------
-template <int DT, bool FULL>
+template <int DT, bool FULL, int OUT>
 __global__ void __launch_bounds__(256, 3)
 lsm_smem_kernel(const LsmParams p, const uint32_t stage_bytes, const int slice, const int nchunk_full) {
     constexpr int VE = Traits<DT>::VE;
@@ -235,11 +262,11 @@ lsm_smem_kernel(const LsmParams p, const uint32_t stage_bytes, const int slice, 
         if (lane < static_cast<int>(cs)) ld_shared_v2(smem_u32(&xchg[lane]), R, s);
         warp_merge_pairs<false>(R, s, p.c);
     }
-    const float lns = ln_of(s);
+    const float kk = OUT == OUT_LOG ? -ln_of(s) : 1.0f / s;
 
-    // ---- pass 2: y = (x - R) * scale - ln S from the resident slice
-    const f32x2 R2 = pair(R, R), s2 = pair(p.scale, p.scale), l2 = pair(-lns, -lns);
-    uint4* __restrict__ yv = static_cast<uint4*>(p.y) + row * p.nvec + v0 + tpos;
+    // ---- pass 2: the output from the resident, untouched slice
+    const f32x2 R2 = pair(R, R), s2 = pair(p.scale, p.scale), k2 = pair(kk, kk);
+    char* yrow = static_cast<char*>(p.y) + row * (OUT == OUT_LOG ? p.nvec * 16 : p.cols * 4);
     for (int ch = 0; ch < nchunk; ++ch) {
         const uint4* sc = sv + ch * chunk_vecs;
         const int cbase = ch * chunk_vecs + tpos;
@@ -248,19 +275,14 @@ lsm_smem_kernel(const LsmParams p, const uint32_t stage_bytes, const int slice, 
         for (int u = 0; u < U; ++u) raw[u] = sc[u * 32];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            if (FULL || cbase + u * 32 < nv) {
-                f32x2 d[NP];
-                widen_pairs<DT>(flip_vec(raw[u], p.flip), d);
-#pragma unroll
-                for (int k = 0; k < NP; ++k) d[k] = fma2(sub2(d[k], R2), s2, l2);
-                st_stream(yv + ch * chunk_vecs + u * 32, narrow_pairs<DT>(d));
-            }
+            if (FULL || cbase + u * 32 < nv)
+                lsm_emit<DT, OUT>(flip_vec(raw[u], p.flip), R2, c2, s2, k2, yrow, int64_t(v0) + cbase + u * 32);
         }
     }
 }
 
 // ---------------------------------------------------------------------------------------------
-template <int DT>
+template <int DT, int OUT>
 __global__ void __launch_bounds__(1024)
 lsm_generic_kernel(const LsmParams p) {
     __shared__ float red[32];
@@ -280,9 +302,16 @@ lsm_generic_kernel(const LsmParams p) {
         float s = 0.0f;
         for (int64_t j = threadIdx.x; j < p.cols; j += blockDim.x)
             s += ex2_ftz((load_elem<DT>(p.x, base + j) * sg - m) * p.c);
-        const float lns = ln_of(block_sum(s, red));
-        for (int64_t j = threadIdx.x; j < p.cols; j += blockDim.x)
-            store_elem<DT>(p.y, base + j, fmaf(load_elem<DT>(p.x, base + j) * sg - m, p.scale, -lns));
+        const float ssum = block_sum(s, red);
+        if (OUT == OUT_LOG) {
+            const float lns = ln_of(ssum);
+            for (int64_t j = threadIdx.x; j < p.cols; j += blockDim.x)
+                store_elem<DT>(p.y, base + j, fmaf(load_elem<DT>(p.x, base + j) * sg - m, p.scale, -lns));
+        } else {
+            const float inv = 1.0f / ssum;
+            for (int64_t j = threadIdx.x; j < p.cols; j += blockDim.x)
+                static_cast<float*>(p.y)[base + j] = ex2_ftz((load_elem<DT>(p.x, base + j) * sg - m) * p.c) * inv;
+        }
     }
 }
 
