@@ -12,9 +12,10 @@ eager mode and never sees a wrong or unsupported kernel.
 The guard admits a call when: the tensor is on a CUDA device, dtype fp32/bf16/fp16, the softmax
 dimension is the last one (or the tensor can be seen that way without a copy), the tensor is
 contiguous, no autograd graph is being recorded for it, and no output dtype conversion is asked
-for other than the upcast-and-cast-back pattern of eager attention (``dtype=torch.float32`` on a
-16-bit input followed by ``.to(input dtype)`` cannot be seen from here, so ``dtype=`` calls fall
-back). This module is a convenience layer above the C ABI; the library itself has no fallback.
+for other than eager attention's ``softmax(scores, dim=-1, dtype=torch.float32)`` on 16-bit scores
+(which runs the library's 16-bit-in, float32-out kernel). log_softmax follows the same guard but
+falls back for any ``dtype=``. This module is a convenience layer above the C ABI; the library
+itself has no fallback.
 """
 from __future__ import annotations
 
@@ -61,7 +62,7 @@ def why_not(x: torch.Tensor, dim: int, dtype=None) -> str | None:
         return "not on a CUDA device"
     if x.dtype not in _DTYPES:
         return f"dtype {x.dtype}"
-    if dtype is not None and dtype != x.dtype:
+    if dtype is not None and dtype != x.dtype and not (dtype == torch.float32 and x.dtype in (torch.bfloat16, torch.float16)):
         return "output dtype conversion requested"
     if x.dim() == 0:
         return "0-d tensor"
@@ -97,6 +98,16 @@ def softmax(x: torch.Tensor, dim: int = -1, dtype=None, scale: float = 1.0, out:
         return y
     cols = x.shape[-1]
     rows = x.numel() // cols
+    if dtype == torch.float32 and x.dtype != torch.float32:
+        # the eager-attention pattern softmax(scores, dim=-1, dtype=float32) on 16-bit scores
+        if out is not None:
+            _count("eager:out tensor with a dtype conversion")
+            return out.copy_(_eager_softmax(x if scale == 1.0 else x * scale, dim, dtype=dtype))
+        y = torch.empty(x.shape, dtype=torch.float32, device=x.device)
+        with torch.cuda.device(x.device):
+            binding.fs_softmax_f32out(x, y, rows, cols, _DTYPES[x.dtype], float(scale), torch.cuda.current_stream(x.device))
+        _count("library")
+        return y
     y = out if out is not None else torch.empty_like(x)
     with torch.cuda.device(x.device):
         binding.fs_softmax(x, y, rows, cols, _DTYPES[x.dtype], float(scale), torch.cuda.current_stream(x.device))
@@ -107,6 +118,8 @@ def softmax(x: torch.Tensor, dim: int = -1, dtype=None, scale: float = 1.0, out:
 def log_softmax(x: torch.Tensor, dim: int = -1, dtype=None):
     """log_softmax over `dim`: the library kernel when admitted, else eager PyTorch."""
     reason = why_not(x, dim, dtype)
+    if reason is None and dtype is not None and isinstance(x, torch.Tensor) and dtype != x.dtype:
+        reason = "output dtype conversion requested"
     if reason is None:
         try:
             binding.lib()

@@ -66,6 +66,13 @@ def test_admitted_calls_match_the_oracle_and_others_fall_back():
     with torch.no_grad():
         assert torch_op.why_not(xg, -1) is None
     assert torch_op.why_not(x, -1, dtype=torch.float64) == "output dtype conversion requested"
+    # eager attention's upcast: 16-bit scores, float32 probabilities, through the mixed-dtype kernel
+    xb = (torch.randn(4, 8, 96, 1024, device="cuda") * 2).to(torch.bfloat16)
+    before = torch_op.stats().get("library", 0)
+    yb = torch_op.softmax(xb, -1, dtype=torch.float32)
+    assert yb.dtype == torch.float32 and torch_op.stats()["library"] == before + 1
+    assert torch.allclose(yb, torch.softmax(xb, -1, dtype=torch.float32), atol=2e-6, rtol=0)
+    assert torch_op.log_softmax(xb, -1, dtype=torch.float32).dtype == torch.float32          # eager route
 
 
 @pytest.mark.gpu
