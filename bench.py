@@ -450,6 +450,7 @@ def time_softmax_backward(w: W.Workload, steps: int, warmup: int, l2_bytes: int)
 NORM_WORKLOADS = {
     "ln_sd35": ("layer", dict(rows=16384, cols=1536, dtype=W.BF16)),
     "ln_4096_f32": ("layer", dict(rows=8192, cols=4096, dtype=W.FP32)),
+    "ln_4096_bf16": ("layer", dict(rows=16384, cols=4096, dtype=W.BF16)),
     "gn_c512_128": ("group", dict(n=1, channels=512, spatial=128 * 128, groups=32, dtype=W.BF16)),
     "gn_c256_256": ("group", dict(n=1, channels=256, spatial=256 * 256, groups=32, dtype=W.BF16)),
     "gn_c128_512": ("group", dict(n=1, channels=128, spatial=512 * 512, groups=32, dtype=W.BF16)),
