@@ -157,9 +157,12 @@ def device_buffers(w: W.Workload, n_pairs: int, threads: int):
 
 
 def time_device(w: W.Workload, steps: int, warmup: int, l2_bytes: int, sampler: ClockSampler | None = None,
-                barrier=None, min_clock_samples: int = 0, causal_q=None):
+                barrier=None, min_clock_samples: int = 0, causal_q=None, extras: bool = False):
     """Times `steps` fs_softmax (or, with causal_q, fs_softmax_causal) launches with CUDA events on
-    the launching stream."""
+    the launching stream: one event pair around the whole train of launches (the steady state).
+    With `extras`, the same buffers are then timed two more ways: the library's own copy kernel over
+    the same bytes (the ceiling this device gives a kernel that only moves the data), and the same
+    launches one at a time, an event pair around each (that figure includes the launch gap)."""
     import torch
 
     import paper_2607_24762_b200 as fs
@@ -220,9 +223,34 @@ def time_device(w: W.Workload, steps: int, warmup: int, l2_bytes: int, sampler: 
     if status != 0:
         raise RuntimeError(f"device status: {fs.fs_strerror(status)}")
     kernel = fs.fs_kernel_name(fs.fs_select_kernel(w.rows, w.cols, w.dtype))
+    extra = {}
+    if extras:
+        nbytes = w.rows * w.cols * w.elem_size
+        if nbytes % 16 == 0:
+            for i in range(3):
+                lib.fs_copy(ptrs[i % n_pairs][0], ptrs[i % n_pairs][1], nbytes, sh)
+            torch.cuda.synchronize()
+            start.record(stream)
+            for i in range(steps):
+                lib.fs_copy(ptrs[i % n_pairs][0], ptrs[i % n_pairs][1], nbytes, sh)
+            stop.record(stream)
+            torch.cuda.synchronize()
+            copy_ms = start.elapsed_time(stop) / steps
+            extra["own_copy"] = {"ms_per_step": round(copy_ms, 6), "GB/s": round(w.min_bytes / (copy_ms * 1e-3) / 1e9, 1),
+                                 "softmax_over_copy_time": round((ms / steps) / copy_ms, 4)}
+        n1 = min(100, steps)
+        pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n1)]
+        for i, (a, b) in enumerate(pairs):
+            a.record(stream)
+            launch(i)
+            b.record(stream)
+        torch.cuda.synchronize()
+        each = sorted(a.elapsed_time(b) for a, b in pairs)
+        extra["single_launch_ms"] = {"median": round(statistics.median(each), 6), "best": round(each[0], 6), "n": n1,
+                                     "note": "event pair around each launch: includes the launch gap"}
     del xs, ys
     torch.cuda.empty_cache()
-    return {"ms_per_step": ms / steps, "n_pairs": n_pairs, "kernel": kernel, "clocks": clocks}
+    return {"ms_per_step": ms / steps, "n_pairs": n_pairs, "kernel": kernel, "clocks": clocks, **extra}
 
 
 def time_router(w: W.Workload, k: int, steps: int, warmup: int, l2_bytes: int):
@@ -733,7 +761,8 @@ def main():
             dist.barrier()
             dist.destroy_process_group()
         return
-    res = time_device(w, args.steps, args.warmup, l2, sampler=sampler, barrier=barrier, min_clock_samples=8)
+    res = time_device(w, args.steps, args.warmup, l2, sampler=sampler, barrier=barrier, min_clock_samples=8,
+                      extras=world == 1)
     from paper_2607_24762_b200 import sharding
     ms = sharding.max_over_ranks(res["ms_per_step"], device="cuda")          # as slow as the slowest rank
     value = sharding.aggregate_throughput(w.min_bytes, ms * 1e-3, world) / 1e9
@@ -750,6 +779,9 @@ def main():
             "roofline": roofline_obj(w, ms, res["kernel"]),
             "gpu_launches": args.steps,
             "clocks": res["clocks"]}
+    for key in ("own_copy", "single_launch_ms"):           # the train above is the headline; these explain it
+        if key in res:
+            line["roofline"][key] = res[key]
 
     if rank == 0 and world == 1:
         if not args.no_e2e:
@@ -764,13 +796,14 @@ def main():
                     others[name] = {"skipped": "not enough free device memory"}
                     continue
                 k = max(20, min(2000, int(0.08 / max(ow.min_bytes / 6.0e12, 4e-6))))
-                r = time_device(ow, k, 10, l2)
+                r = time_device(ow, k, 10, l2, extras=True)
                 gbs = ow.min_bytes / (r["ms_per_step"] * 1e-3) / 1e9
                 peak, which = measured_peak()
                 others[name] = {"what": ow.note, "kernel": r["kernel"], "steps": k, "ms_per_step": round(r["ms_per_step"], 6),
                                 "GB/s": round(gbs, 1), "rows_per_s": round(ow.rows / (r["ms_per_step"] * 1e-3), 1),
                                 "frac_of_measured_copy": round(gbs / peak, 4),
-                                "frac_of_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 4), "n_pairs": r["n_pairs"]}
+                                "frac_of_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 4), "n_pairs": r["n_pairs"],
+                                **{key: r[key] for key in ("own_copy", "single_launch_ms") if key in r}}
             # the causal entry point on the causal workload: the masked half of x is never read
             ow = W.WORKLOADS["cfg5"]
             free, _ = torch.cuda.mem_get_info()

@@ -29,6 +29,9 @@ def test_main_line_has_the_contract_keys():
     r = d["roofline"]
     assert r["bound"] == "hbm" and r["unit"] == "GB/s" and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-3 and r["traffic"] > 0
     assert abs(d["value"] - r["achieved"]) < 1e-6 and d["value"] > 1000
+    # beside the train of launches: the library's own copy over the same buffers, and launches timed one by one
+    assert r["own_copy"]["GB/s"] > 1000 and 0.5 < r["own_copy"]["softmax_over_copy_time"] < 2.0
+    assert r["single_launch_ms"]["best"] <= r["single_launch_ms"]["median"] and r["single_launch_ms"]["n"] == 20
     e = d["e2e"]
     assert e["value"] > 1 and e["h2d_bytes_per_step"] == e["d2h_bytes_per_step"] == 131072 * 128 * 2
     c = d["cpu_baseline"]
