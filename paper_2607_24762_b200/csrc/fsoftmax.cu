@@ -375,6 +375,18 @@ int64_t prefetch_rows(int resident_clusters) {
     return pct == 0 ? 0 : std::max<int64_t>(1, int64_t(resident_clusters) * pct / 100);
 }
 
+// The lag between the clusters of a one-shot grid's first wave (first_wave_lag in common.cuh):
+// the bytes one cluster loads, at FS_LAG_BW bytes per microsecond (read once; default 6500, this
+// part's copy bandwidth; 0 turns the lag off). Measured on B200, 256 rows of 512 KiB bf16: 49.2 us
+// without, 47.2-47.4 with a spread of 3-4 us over the 45 resident clusters (5900-7900 bytes/us),
+// 47.7-48.1 at half or twice that; orders other than the linear one gain less.
+template <class P>
+void set_first_wave_lag(P& p, int resident_clusters, int64_t bytes_per_cluster) {
+    static const int bw = [] { const char* e = std::getenv("FS_LAG_BW"); return e ? std::max(0, std::atoi(e)) : 6500; }();
+    p.lag_rows = resident_clusters;
+    p.lag_ns = bw > 0 ? static_cast<float>(double(bytes_per_cluster) / double(bw)) : 0.0f;
+}
+
 // Programmatic dependent launch (on unless FS_PDL=0): the kernel may be scheduled while the
 // previous kernel of the stream drains; it waits (griddepcontrol.wait) before touching memory.
 bool pdl_enabled() {
@@ -533,7 +545,7 @@ int ring_stages(size_t stage_bytes, size_t budget, int max_stages) {
 // Rows longer than a cluster's shared memory: segments over a grid that fills the GPU, the
 // (reference, sum) pairs of the segments exchanged through a stream-ordered scratch buffer.
 int run_softmax_split(Device& dev, const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale, cudaStream_t st) {
-    LsmParams p;
+    LsmParams p{};
     p.x = x; p.y = y; p.rows = rows; p.cols = cols;
     p.nvec = cols * elem_size(dtype) / 16;
     p.scale = std::fabs(scale);
@@ -577,7 +589,7 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
     if (kernel != FS_KERNEL_GENERIC && !fast) return FS_ERR_UNSUPPORTED;
     if (threads < 0 || threads % 32 || threads > 1024) return FS_ERR_INVALID_ARG;
 
-    Params p;
+    Params p{};
     p.x = x; p.y = y; p.rows = rows; p.cols = cols;
     p.nvec = fast ? cols * esz / 16 : 0;
     p.c = static_cast<float>(static_cast<double>(scale) * kLog2e);
@@ -661,6 +673,7 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
             if ((rc = blocks_per_sm(dev, fn, g.threads, smem, &bps)) != FS_OK) return rc;
             int64_t grid = std::min<int64_t>(rows, max_grid);
             if (persistent_grids()) grid = std::min<int64_t>(grid, int64_t(dev.sm_count) * bps);
+            else set_first_wave_lag(p, dev.sm_count * bps, p.nvec * 16);
             return launch(fn, grid, g.threads, smem, 0, st, p, nstage, static_cast<uint32_t>(stage_bytes));
         }
         case FS_KERNEL_CLUSTER: {
@@ -681,6 +694,7 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
                     int64_t clusters = std::min<int64_t>(rows, max_grid / sg.cs);
                     if (persistent_grids()) clusters = std::min<int64_t>(clusters, ncl);
                     else p.pf_rows = prefetch_rows(ncl);
+                    set_first_wave_lag(p, ncl, p.nvec * 16);
                     return launch(fn, clusters * sg.cs, sg.threads, smem, sg.cs, st, p,
                                   static_cast<uint32_t>(stage_bytes), sg.slice, smem_row_nchunk(sg, dtype));
                 }
@@ -737,7 +751,7 @@ int run_causal(const void* x, void* y, int64_t rows, int64_t cols, int64_t q_off
     Device& dev = *devp;
     const int esz = elem_size(dtype);
     const bool fast = fast_path_ok(cols, dtype, ptr_align(x), ptr_align(y));
-    Params p;
+    Params p{};
     p.x = x; p.y = y; p.rows = rows; p.cols = cols;
     p.nvec = fast ? cols * esz / 16 : 0;
     p.c = static_cast<float>(static_cast<double>(scale) * kLog2e);
@@ -913,7 +927,7 @@ int run_norm(const void* x, const void* gamma, const void* beta, void* y, int64_
     bool fast = fast_path_ok(cols, dtype, ptr_align(x), ptr_align(y));
     if (aff == 1) fast = fast && (!gamma || ptr_align(gamma) >= 16) && (!beta || ptr_align(beta) >= 16);
     if (aff == 2) fast = fast && run_elems % ve == 0;
-    NormParams p;
+    NormParams p{};
     p.x = x; p.y = y; p.gamma = gamma; p.beta = beta; p.rows = rows; p.cols = cols;
     p.nvec = fast ? cols * esz / 16 : 0;
     p.eps = eps; p.run_elems = run_elems; p.aff_rows = aff_rows;
@@ -975,6 +989,7 @@ int run_norm(const void* x, const void* gamma, const void* beta, void* y, int64_
             int ncl = 0;
             if ((rc = active_clusters(dev, fn, sg.threads, smem, sg.cs, &ncl)) != FS_OK) return rc;
             p.pf_rows = prefetch_rows(ncl);
+            set_first_wave_lag(p, ncl, p.nvec * 16);
             return launch(fn, rows * sg.cs, sg.threads, smem, sg.cs, st, p, static_cast<uint32_t>(stage_bytes), sg.slice,
                           smem_row_nchunk(sg, dtype));
         }
@@ -1042,7 +1057,7 @@ int run_log_softmax(const void* x, void* y, int64_t rows, int64_t cols, int dtyp
     Device& dev = *devp;
     const int esz = elem_size(dtype);
     const bool fast = fast_path_ok(cols, dtype, ptr_align(x), ptr_align(y));
-    LsmParams p;
+    LsmParams p{};
     p.x = x; p.y = y; p.rows = rows; p.cols = cols;
     p.nvec = fast ? cols * esz / 16 : 0;
     p.scale = std::fabs(scale);
@@ -1089,6 +1104,7 @@ int run_log_softmax(const void* x, void* y, int64_t rows, int64_t cols, int dtyp
                 int ncl = 0;
                 if ((rc = active_clusters(dev, fn, sg.threads, smem, sg.cs, &ncl)) != FS_OK) return rc;
                 p.pf_rows = prefetch_rows(ncl);
+                set_first_wave_lag(p, ncl, p.nvec * 16);
                 return launch(fn, rows * sg.cs, sg.threads, smem, sg.cs, st, p, static_cast<uint32_t>(stage_bytes), sg.slice,
                               smem_row_nchunk(sg, dtype));
             }
@@ -1140,7 +1156,7 @@ int run_softmax_backward(const void* dy, const void* y, void* dx, int64_t rows, 
     Device& dev = *devp;
     const int esz = elem_size(dtype);
     const bool fast = fast_path_ok(cols, dtype, ptr_align(dy), ptr_align(y)) && ptr_align(dx) >= 16;
-    SmbParams p;
+    SmbParams p{};
     p.dy = dy; p.y = y; p.dx = dx; p.rows = rows; p.cols = cols;
     p.nvec = fast ? cols * esz / 16 : 0;
     p.scale = scale; p.status = dev.status; p.pf_rows = 0;
@@ -1166,6 +1182,7 @@ int run_softmax_backward(const void* dy, const void* y, void* dx, int64_t rows, 
             int ncl = 0;
             if ((rc = active_clusters(dev, fn, sg.threads, smem, sg.cs, &ncl)) != FS_OK) return rc;
             p.pf_rows = prefetch_rows(ncl);
+            set_first_wave_lag(p, ncl, 2 * p.nvec * 16);
             return launch(fn, rows * sg.cs, sg.threads, smem, sg.cs, st, p, static_cast<uint32_t>(stage_bytes), sg.slice,
                           smem_row_nchunk(sg, dtype));
         }
@@ -1218,7 +1235,7 @@ int run_softmax_masked(const void* x, const void* mask, void* y, int64_t rows, i
     Device& dev = *devp;
     const int esz = elem_size(dtype);
     const bool fast = fast_path_ok(cols, dtype, ptr_align(x), ptr_align(y)) && ptr_align(mask) >= 16;
-    MaskedParams p;
+    MaskedParams p{};
     p.x = x; p.mask = mask; p.y = y; p.rows = rows; p.cols = cols;
     p.nvec = fast ? cols * esz / 16 : 0;
     p.q_rows = q_rows; p.group = q_rows * heads;
@@ -1251,6 +1268,7 @@ int run_softmax_masked(const void* x, const void* mask, void* y, int64_t rows, i
             int ncl = 0;
             if ((rc = active_clusters(dev, fn, sg.threads, smem, sg.cs, &ncl)) != FS_OK) return rc;
             p.pf_rows = prefetch_rows(ncl);
+            set_first_wave_lag(p, ncl, p.nvec * 16);
             return launch(fn, rows * sg.cs, sg.threads, smem, sg.cs, st, p, static_cast<uint32_t>(stage_bytes), sg.slice,
                           smem_row_nchunk(sg, dtype));
         }
@@ -1545,7 +1563,7 @@ int fs_softmax_static(const void* x, void* y, int64_t rows, int64_t cols, int dt
     }
     if (!sd.cluster_ok) return FS_ERR_UNSUPPORTED;
 
-    Params p;
+    Params p{};
     p.x = x; p.y = y; p.rows = rows; p.cols = cols; p.nvec = nvec;
     p.c = static_cast<float>(static_cast<double>(scale) * kLog2e);
     p.neg = p.c < 0.0f ? 1 : 0;

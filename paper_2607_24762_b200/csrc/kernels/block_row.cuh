@@ -159,6 +159,7 @@ block_row_tma_kernel(const Params p, const int nstage, const uint32_t stage_byte
         mbar_fence_init();
         fence_proxy_async_smem();
         pdl_wait();
+        first_wave_lag(first, p.lag_ns, p.lag_rows);
         for (int s = 0; s < nstage && s < n_my; ++s)
             bulk_load_row(smem_u32(smem + size_t(s) * stage_bytes),
                           xb + (first + int64_t(s) * gridDim.x) * row_bytes, row_bytes, smem_u32(&bars[s]));

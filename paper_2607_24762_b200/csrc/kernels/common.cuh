@@ -25,6 +25,8 @@ struct Params {
     int* status;       // device status word
     int64_t q_offset;  // causal kernels: row i keeps columns j <= i + q_offset
     int64_t pf_rows;   // split-row kernel: the cluster of row i asks L2 for row i + pf_rows (0: off)
+    float lag_ns;      // one-shot grids: cluster i < lag_rows starts its loads i * lag_ns late (see first_wave_lag)
+    int lag_rows;
 };
 
 template <int DT> struct Traits;
@@ -449,6 +451,16 @@ __device__ __forceinline__ void l2_prefetch(const char* src, uint32_t bytes) {
         const uint32_t n = min(32768u, bytes - off);
         asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" :: "l"(src + off), "r"(n) : "memory");
     }
+}
+
+// The first wave of a one-shot grid starts everywhere at once: every resident cluster loads, then
+// every one computes (DRAM idle), then every one stores, and only later generations drift apart
+// and overlap. Cluster i of that first wave therefore starts its loads i * lag_ns late, lag_ns
+// being the time DRAM needs for one cluster's input: the requests reach DRAM in the order it could
+// serve them anyway (the earlier clusters' rows keep it busy), and the wave comes out of its load
+// phase already spread over one load time. Later clusters (i >= lag_rows) start as slots free up.
+__device__ __forceinline__ void first_wave_lag(int64_t cluster, float lag_ns, int lag_rows) {
+    if (lag_ns > 0.0f && cluster > 0 && cluster < lag_rows) __nanosleep(static_cast<uint32_t>(float(cluster) * lag_ns));
 }
 
 // Bounded wait on an mbarrier phase. A failed try_wait comes back after a short hardware-defined

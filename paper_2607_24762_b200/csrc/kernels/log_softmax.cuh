@@ -34,6 +34,8 @@ struct LsmParams {
     uint32_t flip;      // XOR mask per 32-bit word that negates every element (0 for scale >= 0)
     int* status;
     int64_t pf_rows;
+    float lag_ns;          // first wave of a one-shot grid: cluster i < lag_rows starts i * lag_ns late
+    int lag_rows;
 };
 
 __device__ __forceinline__ float lg2_approx(float v) {
@@ -200,6 +202,7 @@ lsm_smem_kernel(const LsmParams p, const uint32_t stage_bytes, const int slice, 
         mbar_fence_init();
         fence_proxy_async_smem();
         pdl_wait();
+        first_wave_lag(row, p.lag_ns, p.lag_rows);
         for (int ch = 0; ch < nchunk; ++ch) {
             const int cv = FULL ? chunk_vecs : min(chunk_vecs, nv - ch * chunk_vecs);
             bulk_load_row(smem_u32(smem) + uint32_t(ch) * uint32_t(chunk_vecs) * 16u,

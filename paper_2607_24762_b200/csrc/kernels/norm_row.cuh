@@ -38,6 +38,8 @@ struct NormParams {
     int64_t aff_rows;      // AFF 2: rows per sample (groups): row % aff_rows selects the channel block
     int* status;
     int64_t pf_rows;       // one-shot grids: L2 prefetch distance in rows (0: off)
+    float lag_ns;          // first wave of a one-shot grid: cluster i < lag_rows starts i * lag_ns late
+    int lag_rows;
 };
 
 // (count, mean, sum of squared deviations)
@@ -384,6 +386,7 @@ norm_smem_kernel(const NormParams p, const uint32_t stage_bytes, const int slice
         mbar_fence_init();
         fence_proxy_async_smem();
         pdl_wait();
+        first_wave_lag(row, p.lag_ns, p.lag_rows);
         for (int ch = 0; ch < nchunk; ++ch) {
             const int cv = FULL ? chunk_vecs : min(chunk_vecs, nv - ch * chunk_vecs);
             bulk_load_row(smem_u32(smem) + uint32_t(ch) * uint32_t(chunk_vecs) * 16u,

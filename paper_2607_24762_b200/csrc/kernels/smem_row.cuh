@@ -112,6 +112,7 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
         mbar_fence_init();
         fence_proxy_async_smem();
         pdl_wait();
+        first_wave_lag(cid, p.lag_ns, p.lag_rows);
         if (cid < p.rows) issue_row(cid);
         // the row that starts about half a generation of resident clusters later: its slice is on
         // its way to L2 while this one is worked on

@@ -24,6 +24,8 @@ struct SmbParams {
     float scale;
     int* status;
     int64_t pf_rows;
+    float lag_ns;          // first wave of a one-shot grid: cluster i < lag_rows starts i * lag_ns late
+    int lag_rows;
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -126,6 +128,7 @@ smb_smem_kernel(const SmbParams p, const uint32_t stage_bytes, const int slice, 
         mbar_fence_init();
         fence_proxy_async_smem();
         pdl_wait();
+        first_wave_lag(row, p.lag_ns, p.lag_rows);
         for (int ch = 0; ch < nchunk; ++ch) {
             const uint32_t cv = uint32_t(FULL ? chunk_vecs : min(chunk_vecs, nv - ch * chunk_vecs)) * 16u;
             const uint32_t off = uint32_t(ch) * uint32_t(chunk_vecs) * 16u;

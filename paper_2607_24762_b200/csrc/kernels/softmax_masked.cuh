@@ -32,6 +32,8 @@ struct MaskedParams {
     float c;             // scale * log2(e)
     int* status;
     int64_t pf_rows;
+    float lag_ns;          // first wave of a one-shot grid: cluster i < lag_rows starts i * lag_ns late
+    int lag_rows;
 };
 
 __device__ __forceinline__ int64_t mask_row_of(const MaskedParams& p, int64_t row) {
@@ -184,6 +186,7 @@ sm_masked_smem_kernel(const MaskedParams p, const uint32_t stage_bytes, const in
         mbar_fence_init();
         fence_proxy_async_smem();
         pdl_wait();
+        first_wave_lag(row, p.lag_ns, p.lag_rows);
         for (int ch = 0; ch < nchunk; ++ch) {
             const int cv = FULL ? chunk_vecs : min(chunk_vecs, nv - ch * chunk_vecs);
             bulk_load_row(smem_u32(smem) + uint32_t(ch) * uint32_t(chunk_vecs) * 16u,
