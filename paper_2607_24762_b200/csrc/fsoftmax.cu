@@ -869,17 +869,6 @@ template <int DT, int AFF> const void* norm_warp_fn(const WarpGeom& g) {
     }
 }
 
-template <int DT> const void* norm_packed_fn(int vpl, int aff) {
-    switch (vpl) {
-        case 10: return aff ? (const void*)norm_warp_packed_kernel<DT, 10, 1> : (const void*)norm_warp_packed_kernel<DT, 10, 0>;
-        case 12: return aff ? (const void*)norm_warp_packed_kernel<DT, 12, 1> : (const void*)norm_warp_packed_kernel<DT, 12, 0>;
-        case 14: return aff ? (const void*)norm_warp_packed_kernel<DT, 14, 1> : (const void*)norm_warp_packed_kernel<DT, 14, 0>;
-        case 16: return aff ? (const void*)norm_warp_packed_kernel<DT, 16, 1> : (const void*)norm_warp_packed_kernel<DT, 16, 0>;
-        case 18: return aff ? (const void*)norm_warp_packed_kernel<DT, 18, 1> : (const void*)norm_warp_packed_kernel<DT, 18, 0>;
-        default: return nullptr;
-    }
-}
-
 template <int DT> const void* norm_smem_fn(bool full, int aff) {
     if (full) {
         return aff == 0 ? (const void*)norm_smem_kernel<DT, true, 0> : aff == 1 ? (const void*)norm_smem_kernel<DT, true, 1>
@@ -892,6 +881,26 @@ template <int DT> const void* norm_smem_fn(bool full, int aff) {
 template <int DT> const void* norm_apply_fn(int aff) {
     return aff == 0 ? (const void*)norm_apply_kernel<DT, 0> : aff == 1 ? (const void*)norm_apply_kernel<DT, 1>
                                                                         : (const void*)norm_apply_kernel<DT, 2>;
+}
+
+// Rows the warp-per-row-from-shared-memory kernel takes (16-byte vectors per row): 4-11 KiB.
+// Measured on B200 (256 MiB per direction, gamma and beta present, copy = 80 us), against the
+// kernels on either side of the range: bf16 rows of 4 / 5 / 6 / 8 / 10 KiB 83 / 84 / 81 / 82 / 83 us
+// (register-resident warp kernels: 93 / 92 / 90 / 100 / 105), fp32 rows of 6 / 8 / 10 KiB 82 / 83 / 83
+// (split-row kernel: 118 / 98 / 90); from 12 KiB on the split-row kernel is level or ahead, below
+// 4 KiB four rows per block are too few bytes in flight (3 KiB bf16 rows: 97 against 90).
+// FS_NORM_TILE "lo:hi" (read once) overrides the range (lo < vectors <= hi), "0" turns the kernel off.
+bool norm_tile_wanted(int dtype, int64_t nvec) {
+    static const std::pair<int64_t, int64_t> ov = [] {
+        const char* e = std::getenv("FS_NORM_TILE");
+        if (!e) return std::pair<int64_t, int64_t>(-1, -1);
+        long lo = 0, hi = 0;
+        if (std::sscanf(e, "%ld:%ld", &lo, &hi) == 2) return std::pair<int64_t, int64_t>(lo, hi);
+        return std::pair<int64_t, int64_t>(0, 0);
+    }();
+    if (ov.first >= 0) return nvec > ov.first && nvec <= ov.second;
+    (void)dtype;
+    return nvec >= 256 && nvec <= 704;
 }
 
 // FS_NORM_SPLIT=0 / 1 (read once) forces the choice for experiments.
@@ -932,6 +941,21 @@ int run_norm(const void* x, const void* gamma, const void* beta, void* y, int64_
     p.nvec = fast ? cols * esz / 16 : 0;
     p.eps = eps; p.run_elems = run_elems; p.aff_rows = aff_rows;
     p.status = dev.status; p.pf_rows = 0;
+    // rows of 4-11 KiB: a warp per row from shared memory, four rows per block
+    if (fast && aff != 2 && norm_tile_wanted(dtype, p.nvec)) {
+        const void* fn = by_dtype(dtype, [&](auto dt) -> const void* {
+            return aff ? (const void*)norm_tile_kernel<decltype(dt)::value, 1> : (const void*)norm_tile_kernel<decltype(dt)::value, 0>; });
+        const int t = 128;
+        const size_t smem = size_t(t / 32) * size_t(p.nvec) * 16 + size_t(t / 32) * 8;
+        int bps = 0;
+        if ((rc = blocks_per_sm(dev, fn, t, smem, &bps)) != FS_OK) return rc;
+        const int64_t grid = (rows + (t / 32) - 1) / (t / 32);
+        if (grid <= 0x7fffffff) {
+            p.pf_rows = prefetch_rows(dev.sm_count * bps) * (t / 32);
+            set_first_wave_lag(p, dev.sm_count * bps, (t / 32) * p.nvec * 16);
+            return launch(fn, grid, t, smem, 0, st, p);
+        }
+    }
     WarpGeom wg;
     if (fast && aff != 2 && norm_warp_geom(p.nvec, dtype, &wg)) {
         const void* fn = by_dtype(dtype, [&](auto dt) -> const void* {
@@ -940,18 +964,6 @@ int run_norm(const void* x, const void* gamma, const void* beta, void* y, int64_
             const int t = 128;
             const int64_t groups = (rows + (32 / wg.lanes) - 1) / (32 / wg.lanes);
             const int64_t grid = std::min<int64_t>((groups + (t / 32) - 1) / (t / 32), 0x7fffffff);
-            return launch(fn, grid, t, 0, 0, st, p);
-        }
-    }
-    // 16-bit rows of 4-9 KiB: a warp per row with the row packed in registers. Measured on B200 (256 MiB
-    // per direction, gamma and beta present): 90-106 us where a block per row (two barriers per row) took
-    // 106-131 and the shared-memory kernel 121-174; fp32 rows of this size are faster from shared memory.
-    if (fast && aff != 2 && dtype != FS_DTYPE_FP32 && p.nvec > 256 && p.nvec <= 576) {
-        const int vpl = static_cast<int>((p.nvec + 63) / 64) * 2;          // even, 10..18
-        const void* fn = dtype == FS_DTYPE_BF16 ? norm_packed_fn<DT_BF16>(vpl, aff) : norm_packed_fn<DT_F16>(vpl, aff);
-        if (fn) {
-            const int t = 128;
-            const int64_t grid = std::min<int64_t>((rows + (t / 32) - 1) / (t / 32), 0x7fffffff);
             return launch(fn, grid, t, 0, 0, st, p);
         }
     }

@@ -6,8 +6,8 @@
 // item is the triple (n, mean, M2) with Chan's pairwise merge in place of the (reference, sum) pair.
 //
 //   norm_warp_kernel     (sub-)warp per row, the row in registers: exact two-pass statistics
-//   norm_warp_packed_kernel  warp per row for 16-bit rows of 4-9 KiB: the row stays packed in
-//                        registers (10..18 vectors per lane) and is widened where it is used
+//   norm_tile_kernel     rows of 4-11 KiB: four rows per block, each brought to shared memory by a
+//                        bulk copy of its own and worked on by one warp (three reads of shared memory)
 //   norm_smem_kernel     row split over a cluster of 1..16 blocks, the slice resident in shared
 //                        memory (bulk async copies, one mbarrier per chunk); per chunk a thread
 //                        takes the exact mean and M2 of its own 8 vectors and merges them into
@@ -216,64 +216,103 @@ norm_warp_kernel(const NormParams p) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// warp per row for 16-bit rows of 4-9 KiB: the row stays PACKED in registers (VPL vectors per lane,
-// 10..18) and is widened where it is used, three times; no shared memory, no block barrier.
+// warp per row FROM SHARED MEMORY (rows of 4-16 KiB): a block of W warps brings W consecutive rows
+// with one bulk copy each, every copy on an mbarrier of its own, and each warp works on its row
+// alone: three reads of shared memory (sum, squared deviations, output), no block barrier after
+// start-up, and a register footprint that does not grow with the row, so that many warps are
+// resident. One-shot grid: block b handles rows b*W .. b*W+W-1.
+// dynamic shared memory: W rows | W mbarriers
 // ---------------------------------------------------------------------------------------------
-template <int DT, int VPL, int AFF>
-__global__ void __launch_bounds__(128, VPL <= 12 ? 4 : 3)
-norm_warp_packed_kernel(const NormParams p) {
+template <int DT, int AFF>
+__global__ void __launch_bounds__(128)
+norm_tile_kernel(const NormParams p) {
     constexpr int NP = Traits<DT>::VE / 2;
-    static_assert(AFF != 2 && DT != DT_F32, "16-bit rows, column affine parameters");
+    constexpr int H = 4;                                   // vectors per lane and batch
+    static_assert(AFF != 2, "per-run affine parameters are handled by the split-row kernel");
     pdl_launch_dependents();
-    const int lane = threadIdx.x & 31;
-    const int warps = blockDim.x >> 5;
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, W = blockDim.x >> 5;
     const int nvec = static_cast<int>(p.nvec);
-    const uint4* __restrict__ xv = static_cast<const uint4*>(p.x) + lane;
-    uint4* __restrict__ yv = static_cast<uint4*>(p.y) + lane;
+    const int64_t row_bytes = p.nvec * 16;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + size_t(W) * size_t(row_bytes));
+    const int64_t row = int64_t(blockIdx.x) * W + w;
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < W; ++i) mbar_init(smem_u32(&bars[i]), 1);
+        mbar_fence_init();
+        fence_proxy_async_smem();
+    }
+    __syncthreads();
+    pdl_wait();
+    if (row >= p.rows) return;                             // no block-wide barrier follows
+    const char* xb = static_cast<const char*>(p.x);
+    if (lane == 0) {
+        first_wave_lag(blockIdx.x, p.lag_ns, p.lag_rows);
+        bulk_load_row(smem_u32(smem) + uint32_t(w) * uint32_t(row_bytes), xb + row * row_bytes, uint32_t(row_bytes), smem_u32(&bars[w]));
+        if (p.pf_rows > 0 && row + p.pf_rows < p.rows) l2_prefetch(xb + (row + p.pf_rows) * row_bytes, uint32_t(row_bytes));
+    }
+    const uint4* sv = reinterpret_cast<const uint4*>(smem + size_t(w) * size_t(row_bytes)) + lane;
+    uint4* __restrict__ yv = static_cast<uint4*>(p.y) + row * p.nvec + lane;
     const uint4* gv = AFF == 1 && p.gamma ? static_cast<const uint4*>(p.gamma) + lane : nullptr;
     const uint4* bv = AFF == 1 && p.beta ? static_cast<const uint4*>(p.beta) + lane : nullptr;
     const float inv_n = 1.0f / static_cast<float>(p.cols);
-    pdl_wait();
-    for (int64_t row = int64_t(blockIdx.x) * warps + (threadIdx.x >> 5); row < p.rows; row += int64_t(gridDim.x) * warps) {
-        uint4 raw[VPL];
+    mbar_wait_warp(smem_u32(&bars[w]), 0u, p.status);      // on a timeout the status word is set and the row is garbage
+
+    f32x2 acc[2] = {pair(0.0f, 0.0f), pair(0.0f, 0.0f)};
+    for (int k0 = 0; k0 < nvec; k0 += 32 * H) {
+        uint4 raw[H];
 #pragma unroll
-        for (int k = 0; k < VPL; ++k) {
-            raw[k] = make_uint4(0u, 0u, 0u, 0u);
-            if (lane + k * 32 < nvec) raw[k] = ld_stream(xv + row * p.nvec + k * 32);
+        for (int u = 0; u < H; ++u) {
+            raw[u] = make_uint4(0u, 0u, 0u, 0u);           // absent vectors are zeros: they add nothing
+            if (k0 + u * 32 + lane < nvec) raw[u] = sv[k0 + u * 32];
         }
-        f32x2 acc[2] = {pair(0.0f, 0.0f), pair(0.0f, 0.0f)};
 #pragma unroll
-        for (int k = 0; k < VPL; ++k) {
+        for (int u = 0; u < H; ++u) {
             f32x2 x[NP];
-            widen_pairs<DT>(raw[k], x);                                    // absent vectors are zeros
+            widen_pairs<DT>(raw[u], x);
 #pragma unroll
             for (int j = 0; j < NP; ++j) acc[j & 1] = add2(acc[j & 1], x[j]);
         }
-        const float mu = warp_sum<32>(pair_sum(add2(acc[0], acc[1]))) * inv_n;
-        const f32x2 mu2 = pair(mu, mu);
-        acc[0] = pair(0.0f, 0.0f); acc[1] = pair(0.0f, 0.0f);
+    }
+    const float mu = warp_sum<32>(pair_sum(add2(acc[0], acc[1]))) * inv_n;
+    const f32x2 mu2 = pair(mu, mu);
+    acc[0] = pair(0.0f, 0.0f); acc[1] = pair(0.0f, 0.0f);
+    for (int k0 = 0; k0 < nvec; k0 += 32 * H) {
+        uint4 raw[H];
 #pragma unroll
-        for (int k = 0; k < VPL; ++k) {
-            if (lane + k * 32 < nvec) {
+        for (int u = 0; u < H; ++u) {
+            raw[u] = make_uint4(0u, 0u, 0u, 0u);
+            if (k0 + u * 32 + lane < nvec) raw[u] = sv[k0 + u * 32];
+        }
+#pragma unroll
+        for (int u = 0; u < H; ++u) {
+            if (k0 + u * 32 + lane < nvec) {
                 f32x2 x[NP];
-                widen_pairs<DT>(raw[k], x);
+                widen_pairs<DT>(raw[u], x);
 #pragma unroll
                 for (int j = 0; j < NP; ++j) { const f32x2 d = sub2(x[j], mu2); acc[j & 1] = fma2(d, d, acc[j & 1]); }
             }
         }
-        const float rstd = rstd_of(warp_sum<32>(pair_sum(add2(acc[0], acc[1]))) * inv_n, p.eps);
-        const f32x2 r2 = pair(rstd, rstd);
+    }
+    const float rstd = rstd_of(warp_sum<32>(pair_sum(add2(acc[0], acc[1]))) * inv_n, p.eps);
+    const f32x2 r2 = pair(rstd, rstd);
+    for (int k0 = 0; k0 < nvec; k0 += 32 * H) {
+        uint4 raw[H], graw[H], braw[H];
 #pragma unroll
-        for (int k = 0; k < VPL; ++k) {
-            if (lane + k * 32 < nvec) {
+        for (int u = 0; u < H; ++u) {
+            const bool in = k0 + u * 32 + lane < nvec;
+            raw[u] = make_uint4(0u, 0u, 0u, 0u); graw[u] = raw[u]; braw[u] = raw[u];
+            if (in) raw[u] = sv[k0 + u * 32];
+            if (gv && in) graw[u] = ld_cached(gv + k0 + u * 32);
+            if (bv && in) braw[u] = ld_cached(bv + k0 + u * 32);
+        }
+#pragma unroll
+        for (int u = 0; u < H; ++u) {
+            if (k0 + u * 32 + lane < nvec) {
                 f32x2 x[NP];
-                widen_pairs<DT>(raw[k], x);
+                widen_pairs<DT>(raw[u], x);
 #pragma unroll
                 for (int j = 0; j < NP; ++j) x[j] = sub2(x[j], mu2);
-                uint4 graw = make_uint4(0u, 0u, 0u, 0u), braw = make_uint4(0u, 0u, 0u, 0u);
-                if (gv) graw = ld_cached(gv + k * 32);
-                if (bv) braw = ld_cached(bv + k * 32);
-                affine_store_any<DT>(gv != nullptr, bv != nullptr, x, r2, graw, braw, yv + row * p.nvec + k * 32);
+                affine_store_any<DT>(gv != nullptr, bv != nullptr, x, r2, graw[u], braw[u], yv + k0 + u * 32);
             }
         }
     }

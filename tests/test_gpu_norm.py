@@ -90,6 +90,21 @@ def test_layer_norm_row_lengths_across_the_split_geometries(dtype):
         check_layer(x, dtype, gamma, beta, 1e-5)
 
 
+@pytest.mark.parametrize("dtype", [FP32, BF16, FP16])
+def test_layer_norm_rows_around_the_four_rows_per_block_kernel(dtype):
+    """Rows of 256..704 sixteen-byte vectors take the kernel that works on four rows per block from shared
+    memory: both ends of that range and one vector beyond them, row counts that leave a block partly
+    empty, with and without gamma and beta."""
+    ve = 16 // W.ELEM_SIZE[dtype]
+    for k, nvec in enumerate((255, 256, 257, 300, 511, 703, 704, 705)):
+        cols = nvec * ve
+        for rows in (1, 4, 5, 7, 130):
+            x = make_case(rows, cols, dtype, seed=7 * nvec + rows, offset=0.5 * (k % 3), sigma=1.0 + k % 2)
+            gamma = stored(np.random.default_rng(nvec).standard_normal(cols) * 0.5 + 1.0, dtype) if k % 2 == 0 or rows == 5 else None
+            beta = stored(np.random.default_rng(nvec + 1).standard_normal(cols) * 0.2, dtype) if k % 3 != 1 else None
+            check_layer(x, dtype, gamma, beta, 1e-5)
+
+
 @pytest.mark.parametrize("rows,cols,dtype", [(16384, 1536, BF16), (40000, 2304, BF16), (38000, 4096, FP16), (8192, 4096, FP32)])
 def test_layer_norm_at_benchmark_sizes(rows, cols, dtype):
     """The benchmark's layer_norm shapes, and row counts at which the block kernel takes eight rows per
