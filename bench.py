@@ -53,7 +53,7 @@ NCU_TRAFFIC_BYTES = {
     "cfg1": 265472,               # profiles/block_row_kernel_cfg1_fp32_64x1000.txt (y stays in L2)
     "cfg2": 85469440,             # profiles/warp_row_kernel_cfg2_bf16_16384x2048.txt (x read once; 0.28 of y written back by kernel end)
     "cfg3": 34201088,             # profiles/warp_row_kernel_cfg3_bf16_131072x128.txt
-    "cfg4": 212553984,            # profiles/smem_row_kernel_cfg4_bf16_256x262144.txt
+    "cfg4": 212546048,            # profiles/smem_row_kernel_cfg4_bf16_256x262144.txt
     "cfg5": 16 * 479168512,       # profiles/smem_row_kernel_cfg5_fp32_2048x32768.txt, scaled from 2048 to 32768 rows
 }
 
