@@ -903,6 +903,23 @@ bool norm_tile_wanted(int dtype, int64_t nvec) {
     return nvec >= 256 && nvec <= 704;
 }
 
+// The same for fs_softmax_masked: 16-bit rows of 4-10 KiB. Measured (256 MiB per direction, copy =
+// 80 us; mask of 64 rows shared by all others): bf16 rows of 4 / 5 / 6 / 8 / 10 KiB 94 / 96 / 91 / 98 / 103 us
+// against 96 / 108 / 116 / 130 / 112 with the row packed in registers; from 11 KiB on and for fp32 rows
+// (82-98 against 81-93) the other kernels are level or ahead.
+// FS_MASKED_TILE "lo:hi" overrides the range, "0" turns the kernel off.
+bool masked_tile_wanted(int dtype, int64_t nvec) {
+    static const std::pair<int64_t, int64_t> ov = [] {
+        const char* e = std::getenv("FS_MASKED_TILE");
+        if (!e) return std::pair<int64_t, int64_t>(-1, -1);
+        long lo = 0, hi = 0;
+        if (std::sscanf(e, "%ld:%ld", &lo, &hi) == 2) return std::pair<int64_t, int64_t>(lo, hi);
+        return std::pair<int64_t, int64_t>(0, 0);
+    }();
+    if (ov.first >= 0) return nvec > ov.first && nvec <= ov.second;
+    return dtype != FS_DTYPE_FP32 && nvec >= 256 && nvec <= 640;
+}
+
 // FS_NORM_SPLIT=0 / 1 (read once) forces the choice for experiments.
 bool norm_split_wanted(const Device& dev, int64_t rows, int64_t nvec, bool smem_ok, int cs) {
     static const int forced = [] { const char* e = std::getenv("FS_NORM_SPLIT"); return e ? std::atoi(e) : -1; }();
@@ -1253,6 +1270,19 @@ int run_softmax_masked(const void* x, const void* mask, void* y, int64_t rows, i
     p.q_rows = q_rows; p.group = q_rows * heads;
     p.c = static_cast<float>(static_cast<double>(scale) * kLog2e);
     p.status = dev.status; p.pf_rows = 0;
+    if (fast && masked_tile_wanted(dtype, p.nvec)) {        // rows of 4-11 KiB: a warp per row from shared memory
+        const void* fn = by_dtype(dtype, [&](auto dt) -> const void* { return (const void*)sm_masked_tile_kernel<decltype(dt)::value>; });
+        const int t = 128;
+        const size_t smem = size_t(t / 32) * size_t(p.nvec) * 16 + size_t(t / 32) * 8;
+        int bps = 0;
+        if ((rc = blocks_per_sm(dev, fn, t, smem, &bps)) != FS_OK) return rc;
+        const int64_t grid = (rows + (t / 32) - 1) / (t / 32);
+        if (grid <= 0x7fffffff) {
+            p.pf_rows = prefetch_rows(dev.sm_count * bps) * (t / 32);
+            set_first_wave_lag(p, dev.sm_count * bps, (t / 32) * p.nvec * 16);
+            return launch(fn, grid, t, smem, 0, st, p);
+        }
+    }
     WarpGeom wg;
     bool warp_ok = fast && norm_warp_geom(p.nvec, dtype, &wg);
     if (fast && !warp_ok && p.nvec <= 576) {        // rows of 4-9 KiB: still a warp per row, 10..18 packed vectors per lane

@@ -10,6 +10,7 @@
 // parity bound of this entry point grows with max |z| (see the header).
 //
 //   sm_masked_warp_kernel     (sub-)warp per row, the row packed in registers (rows up to 9 KiB)
+//   sm_masked_tile_kernel     rows of 4-11 KiB: four rows per block in shared memory, a warp per row
 //   sm_masked_smem_kernel     the split-row design: x slice resident in shared memory, mask slice
 //                             read from L2 in pass 1 only (e is stored in place, as in smem_row)
 //   sm_masked_generic_kernel  block per row, element-wise, any shape and alignment
@@ -140,6 +141,105 @@ template <int DT, int VPL>
 __global__ void __launch_bounds__(128, VPL <= 12 ? 5 : 4)
 sm_masked_warp_long_kernel(const MaskedParams p) {
     sm_masked_warp_body<DT, 32, VPL>(p);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Rows of 4-11 KiB: four rows per block, each brought to shared memory by a bulk copy of its own
+// (one mbarrier per row) and worked on by one warp alone, with the arithmetic of the warp kernel
+// above: pass A takes the maximum exponent, pass B puts e = 2^(t - R) back in place of x in shared
+// memory in the element dtype, pass C scales and stores. The mask vectors come through the
+// read-only path in passes A and B. No block barrier after start-up; the register footprint does
+// not grow with the row. One-shot grid: block b handles rows b*W .. b*W+W-1.
+// dynamic shared memory: W rows | W mbarriers
+// ---------------------------------------------------------------------------------------------
+template <int DT>
+__global__ void __launch_bounds__(128)
+sm_masked_tile_kernel(const MaskedParams p) {
+    constexpr int NP = Traits<DT>::VE / 2;
+    constexpr int H = 4;                                   // vectors per lane and batch
+    pdl_launch_dependents();
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, W = blockDim.x >> 5;
+    const int nvec = static_cast<int>(p.nvec);
+    const int64_t row_bytes = p.nvec * 16;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + size_t(W) * size_t(row_bytes));
+    const int64_t row = int64_t(blockIdx.x) * W + w;
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < W; ++i) mbar_init(smem_u32(&bars[i]), 1);
+        mbar_fence_init();
+        fence_proxy_async_smem();
+    }
+    __syncthreads();
+    pdl_wait();
+    if (row >= p.rows) return;                             // no block-wide barrier follows
+    const char* xb = static_cast<const char*>(p.x);
+    if (lane == 0) {
+        first_wave_lag(blockIdx.x, p.lag_ns, p.lag_rows);
+        bulk_load_row(smem_u32(smem) + uint32_t(w) * uint32_t(row_bytes), xb + row * row_bytes, uint32_t(row_bytes), smem_u32(&bars[w]));
+        if (p.pf_rows > 0 && row + p.pf_rows < p.rows) l2_prefetch(xb + (row + p.pf_rows) * row_bytes, uint32_t(row_bytes));
+    }
+    uint4* sv = reinterpret_cast<uint4*>(smem + size_t(w) * size_t(row_bytes)) + lane;
+    const uint4* __restrict__ mr = static_cast<const uint4*>(p.mask) + mask_row_of(p, row) * p.nvec + lane;
+    uint4* __restrict__ yv = static_cast<uint4*>(p.y) + row * p.nvec + lane;
+    const f32x2 c2 = pair(p.c, p.c);
+    mbar_wait_warp(smem_u32(&bars[w]), 0u, p.status);      // on a timeout the status word is set and the row is garbage
+
+    float r = __int_as_float(0xff800000);
+    for (int k0 = 0; k0 < nvec; k0 += 32 * H) {
+        uint4 xr[H], mk[H];
+#pragma unroll
+        for (int u = 0; u < H; ++u) {
+            xr[u] = make_uint4(0u, 0u, 0u, 0u); mk[u] = xr[u];
+            if (k0 + u * 32 + lane < nvec) { xr[u] = sv[k0 + u * 32]; mk[u] = ld_cached(mr + k0 + u * 32); }
+        }
+#pragma unroll
+        for (int u = 0; u < H; ++u) {
+            if (k0 + u * 32 + lane < nvec) {
+                f32x2 t[NP];
+                r = fmaxf(r, masked_exponents<DT>(xr[u], mk[u], c2, t));
+            }
+        }
+    }
+    r = warp_pick<32, false>(r);
+    const f32x2 r2 = pair(r, r);
+    f32x2 acc[2] = {pair(0.0f, 0.0f), pair(0.0f, 0.0f)};
+    for (int k0 = 0; k0 < nvec; k0 += 32 * H) {
+        uint4 xr[H], mk[H];
+#pragma unroll
+        for (int u = 0; u < H; ++u) {
+            xr[u] = make_uint4(0u, 0u, 0u, 0u); mk[u] = xr[u];
+            if (k0 + u * 32 + lane < nvec) { xr[u] = sv[k0 + u * 32]; mk[u] = ld_cached(mr + k0 + u * 32); }
+        }
+#pragma unroll
+        for (int u = 0; u < H; ++u) {
+            if (k0 + u * 32 + lane < nvec) {
+                f32x2 t[NP];
+                masked_exponents<DT>(xr[u], mk[u], c2, t);
+#pragma unroll
+                for (int j = 0; j < NP; ++j) {
+                    float lo, hi;
+                    unpair(sub2(t[j], r2), lo, hi);
+                    if (DT == DT_BF16) { lo += 64.0f; hi += 64.0f; }        // keeps subnormal bf16 outputs (see ex2_elem)
+                    t[j] = pair(ex2_ftz(lo), ex2_ftz(hi));
+                    acc[j & 1] = add2(acc[j & 1], t[j]);
+                }
+                sv[k0 + u * 32] = narrow_pairs<DT>(t);     // this lane alone reads it back
+            }
+        }
+    }
+    const float inv = recip<DT>(warp_sum<32>(pair_sum(add2(acc[0], acc[1]))));
+    const f32x2 i2 = pair(inv, inv);
+    for (int k0 = 0; k0 < nvec; k0 += 32 * H) {
+        uint4 e[H];
+#pragma unroll
+        for (int u = 0; u < H; ++u) {
+            e[u] = make_uint4(0u, 0u, 0u, 0u);
+            if (k0 + u * 32 + lane < nvec) e[u] = sv[k0 + u * 32];
+        }
+#pragma unroll
+        for (int u = 0; u < H; ++u)
+            if (k0 + u * 32 + lane < nvec) st_stream(yv + k0 + u * 32, scale_vec<DT, false>(e[u], i2, i2));
+    }
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -91,6 +91,18 @@ def test_row_lengths_across_the_split_geometries(dtype):
         check(x, m, dtype, q, 2, 0.25)
 
 
+@pytest.mark.parametrize("dtype", [BF16, FP16, FP32])
+def test_rows_around_the_four_rows_per_block_kernel(dtype):
+    """16-bit rows of 256..640 sixteen-byte vectors take the kernel that works on four rows per block from
+    shared memory: both ends of that range and one vector beyond them, row counts that leave a block
+    partly empty, every mask kind."""
+    ve = 16 // W.ELEM_SIZE[dtype]
+    for ci, nvec in enumerate((255, 256, 257, 400, 639, 640, 641)):
+        for heads, q in ((1, 1), (1, 5), (3, 7), (2, 65)):
+            x, m = make(1, heads, q, nvec * ve, dtype, seed=900 + ci * 7 + q, kind=("causal", "padding", "bias")[(ci + q) % 3])
+            check(x, m, dtype, q, heads, [1.0, 0.25, -0.5][(ci + heads) % 3])
+
+
 @pytest.mark.parametrize("dtype", [FP32, BF16, FP16])
 def test_special_values_alignment_and_aliasing(dtype):
     x, m = make(1, 2, 4, 4096, dtype, seed=9, kind="padding")
