@@ -497,6 +497,26 @@ template <int DT> const void* router_fn(const WarpGeom& g) {
     return nullptr;
 }
 
+// k <= 8: the sorting-network kernel, same geometries
+template <int DT> const void* router8_fn(const WarpGeom& g) {
+    if (g.vpl == 1) return (const void*)router_top8_kernel<DT, 1, 1>;
+    if (g.vpl == 2) return (const void*)router_top8_kernel<DT, 1, 2>;
+    if (g.vpl == 4) {
+        switch (g.lanes) {
+            case 1:  return (const void*)router_top8_kernel<DT, 1, 4>;
+            case 2:  return (const void*)router_top8_kernel<DT, 2, 4>;
+            case 4:  return (const void*)router_top8_kernel<DT, 4, 4>;
+            case 8:  return (const void*)router_top8_kernel<DT, 8, 4>;
+            case 16: return (const void*)router_top8_kernel<DT, 16, 4>;
+            default: return (const void*)router_top8_kernel<DT, 32, 4>;
+        }
+    }
+    if constexpr (DT == DT_F32) {
+        if (g.vpl == 8) return (const void*)router_top8_kernel<DT, 32, 8>;
+    }
+    return nullptr;
+}
+
 // Calls f(std::integral_constant<int, DT>, std::bool_constant<NEG>) for the run-time dtype and sign.
 template <typename F> const void* by_variant(int dtype, bool neg, F f) {
     auto with_dt = [&](auto dt) -> const void* {
@@ -1365,11 +1385,14 @@ int fs_router_topk(const void* x, float* w, int32_t* idx, int64_t rows, int64_t 
     Device* dev = nullptr;
     int rc = get_device(&dev);
     if (rc != FS_OK) return rc;
+    // k <= 8 selects with sorting networks in registers (FS_ROUTER_ROUNDS=1, read per call, keeps the
+    // kernel that takes one maximum per round, which serves any k)
+    const bool net = k <= 8 && !std::getenv("FS_ROUTER_ROUNDS");
     const void* fn = nullptr;
     switch (dtype) {
-        case FS_DTYPE_FP32: fn = router_fn<DT_F32>(g); break;
-        case FS_DTYPE_BF16: fn = router_fn<DT_BF16>(g); break;
-        default:            fn = router_fn<DT_F16>(g); break;
+        case FS_DTYPE_FP32: fn = net ? router8_fn<DT_F32>(g) : router_fn<DT_F32>(g); break;
+        case FS_DTYPE_BF16: fn = net ? router8_fn<DT_BF16>(g) : router_fn<DT_BF16>(g); break;
+        default:            fn = net ? router8_fn<DT_F16>(g) : router_fn<DT_F16>(g); break;
     }
     if (!fn) return FS_ERR_UNSUPPORTED;
     RouterParams p;
@@ -1377,7 +1400,7 @@ int fs_router_topk(const void* x, float* w, int32_t* idx, int64_t rows, int64_t 
     p.c = static_cast<float>(static_cast<double>(scale) * kLog2e);
     p.renorm = renormalize ? 1 : 0;
     const int t = 128;
-    const size_t smem = static_cast<size_t>(g.vpl) * (dtype == FS_DTYPE_FP32 ? 4 : 8) * t * sizeof(uint32_t);   // <= 16 KiB
+    const size_t smem = net ? 0 : static_cast<size_t>(g.vpl) * (dtype == FS_DTYPE_FP32 ? 4 : 8) * t * sizeof(uint32_t);   // <= 16 KiB
     const int64_t groups = (rows + (32 / g.lanes) - 1) / (32 / g.lanes);
     const int64_t grid = std::min<int64_t>((groups + (t / 32) - 1) / (t / 32), 0x7fffffff);
     return launch(fn, grid, t, smem, 0, static_cast<cudaStream_t>(stream), p);

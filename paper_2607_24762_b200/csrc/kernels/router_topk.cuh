@@ -14,6 +14,8 @@
 // butterfly, and the owner clears that key and refreshes that one vector's maximum.
 // The weight of a selected element is 2^((key - key_0)|c|) over the row sum (or over the sum of
 // the selected ones), which needs no access to the element itself.
+// That kernel serves any k; router_top8_kernel below (k <= 8) selects with sorting networks in
+// registers instead.
 #pragma once
 #include "common.cuh"
 
@@ -148,6 +150,170 @@ router_topk_kernel(const RouterParams p) {
             // 0 * inv_s carries a NaN row into the renormalised weights (inv_s is finite otherwise)
             const float f = 1.0f / sel + 0.0f * inv_s;
             for (int r = 0; r < p.k; ++r) p.w[row * p.k + r] *= f;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// k <= 8: selection by sorting networks in registers, no shared memory and no rounds.
+// An element becomes ONE integer key: the order-preserving image of its value in the high half,
+// the complement of its column in the low half (16 + 16 bits for bf16/fp16 inputs, 32 + 32 for
+// fp32), so that a plain integer maximum picks the larger value and, among equal values, the
+// lower column; 0 marks padding. A lane sorts its elements in groups of eight (19
+// compare-exchanges each) and merges the groups into its own eight best; two sorted lists merge
+// into the eight best of both by c_i = max(a_i, b_{7-i}) (a bitonic sequence) and a 12-exchange
+// bitonic sort. The lanes of a row merge their lists the same way through shuffles (both partners
+// end with the same list), and lane r mod LANES writes entry r.
+// ---------------------------------------------------------------------------------------------
+template <class K> __device__ __forceinline__ void cmpx(K& a, K& b) {       // a >= b afterwards
+    const K hi = max(a, b), lo = min(a, b);
+    a = hi; b = lo;
+}
+template <class K> __device__ __forceinline__ void sort8_desc(K (&a)[8]) {
+    cmpx(a[0], a[1]); cmpx(a[2], a[3]); cmpx(a[4], a[5]); cmpx(a[6], a[7]);
+    cmpx(a[0], a[2]); cmpx(a[1], a[3]); cmpx(a[4], a[6]); cmpx(a[5], a[7]);
+    cmpx(a[1], a[2]); cmpx(a[5], a[6]);
+    cmpx(a[0], a[4]); cmpx(a[1], a[5]); cmpx(a[2], a[6]); cmpx(a[3], a[7]);
+    cmpx(a[2], a[4]); cmpx(a[3], a[5]);
+    cmpx(a[1], a[2]); cmpx(a[3], a[4]); cmpx(a[5], a[6]);
+}
+template <class K> __device__ __forceinline__ void bitonic8_desc(K (&a)[8]) {
+    cmpx(a[0], a[4]); cmpx(a[1], a[5]); cmpx(a[2], a[6]); cmpx(a[3], a[7]);
+    cmpx(a[0], a[2]); cmpx(a[1], a[3]); cmpx(a[4], a[6]); cmpx(a[5], a[7]);
+    cmpx(a[0], a[1]); cmpx(a[2], a[3]); cmpx(a[4], a[5]); cmpx(a[6], a[7]);
+}
+// a, b sorted (descending): a becomes the eight largest of both, sorted
+template <class K> __device__ __forceinline__ void merge8_desc(K (&a)[8], const K (&b)[8]) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) a[i] = max(a[i], b[7 - i]);
+    bitonic8_desc(a);
+}
+
+template <int DT> struct RouterKey {                       // 16-bit inputs: value and column in one word
+    using type = uint32_t;
+    static __device__ __forceinline__ type make(float z, int col) {
+        if (DT == DT_BF16) {       // z is a bf16 value: the high half of its binary32 key is its 16-bit key
+            const uint32_t b = __float_as_uint(z);
+            const uint32_t o = b ^ (static_cast<uint32_t>(static_cast<int32_t>(b) >> 31) | 0x80000000u);
+            return (o & 0xffff0000u) | (0xffffu - static_cast<uint32_t>(col));
+        }
+        const uint32_t h = static_cast<uint32_t>(__half_as_ushort(__float2half_rn(z))); // z is an fp16 value: exact
+        const uint32_t o = (h & 0x8000u) ? (~h & 0xffffu) : (h | 0x8000u);
+        return (o << 16) | (0xffffu - static_cast<uint32_t>(col));
+    }
+    static __device__ __forceinline__ int col(type k) { return static_cast<int>(0xffffu - (k & 0xffffu)); }
+    static __device__ __forceinline__ float value(type k) {
+        const uint32_t o = k >> 16;
+        const uint32_t h = (o & 0x8000u) ? (o & 0x7fffu) : (~o & 0xffffu);
+        if (DT == DT_BF16) return __uint_as_float(h << 16);
+        return __half2float(__ushort_as_half(static_cast<unsigned short>(h)));
+    }
+};
+template <> struct RouterKey<DT_F32> {
+    using type = unsigned long long;
+    static __device__ __forceinline__ type make(float z, int col) {
+        return (static_cast<type>(order_key(z)) << 32) | static_cast<type>(0xffffffffu - static_cast<uint32_t>(col));
+    }
+    static __device__ __forceinline__ int col(type k) { return static_cast<int>(0xffffffffu - static_cast<uint32_t>(k)); }
+    static __device__ __forceinline__ float value(type k) { return order_unkey(static_cast<uint32_t>(k >> 32)); }
+};
+
+template <int DT, int LANES, int VPL>
+__global__ void __launch_bounds__(128)
+router_top8_kernel(const RouterParams p) {
+    constexpr int VE = Traits<DT>::VE;
+    constexpr int G = 32 / LANES;
+    constexpr int E = VPL * VE;                            // elements per lane
+    constexpr int NG = (E + 7) / 8;                        // groups of eight
+    using RK = RouterKey<DT>;
+    using K = typename RK::type;
+    pdl_launch_dependents();
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int sub = lane / LANES, sl = lane % LANES;
+    const int warps = blockDim.x >> 5;
+    const int nvec = static_cast<int>(p.nvec);
+    const uint4* __restrict__ xv = static_cast<const uint4*>(p.x);
+    const float cabs = fabsf(p.c);
+    const float sg = p.c > 0.0f ? 1.0f : (p.c < 0.0f ? -1.0f : 0.0f);
+    pdl_wait();
+
+    const int64_t ngroups = (p.rows + G - 1) / G;
+    for (int64_t grp = int64_t(blockIdx.x) * warps + (tid >> 5); grp < ngroups; grp += int64_t(gridDim.x) * warps) {
+        const int64_t row = grp * G + sub;
+        const bool row_ok = row < p.rows;
+        float z[VPL][VE];
+        bool live[VPL];
+        float top = __int_as_float(0xff800000);
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) {
+            live[v] = row_ok && sl + v * LANES < nvec;
+            uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+            if (live[v]) raw = ld_stream(xv + row * p.nvec + sl + v * LANES);
+            unpack<DT>(raw, z[v]);
+#pragma unroll
+            for (int i = 0; i < VE; ++i) {
+                z[v][i] = fmaf(z[v][i], sg, 0.0f);          // sign of the scale; -0 becomes +0; inf * 0 = NaN
+                if (live[v]) top = fmaxf(top, z[v][i]);     // fmaxf drops NaN
+            }
+        }
+        top = warp_pick<LANES, false>(top);
+        float s = 0.0f;
+#pragma unroll
+        for (int v = 0; v < VPL; ++v)
+#pragma unroll
+            for (int i = 0; i < VE; ++i)
+                if (live[v]) s += ex2_ftz_r((z[v][i] - top) * cabs);
+        s = warp_sum<LANES>(s);
+        const float inv_s = 1.0f / s;                      // NaN when the row is NaN
+
+        // ---- this lane's eight best
+        K best[8];
+#pragma unroll
+        for (int g = 0; g < NG; ++g) {
+            K grp8[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int f = g * 8 + j;                   // flat element of this lane
+                grp8[j] = 0;
+                if (f < E) {
+                    const int v = f / VE, i = f % VE;
+                    const float kz = fmaxf(z[v][i], __int_as_float(0xff800000));       // NaN counts as -inf (fmaxf drops it)
+                    if (live[v]) grp8[j] = RK::make(kz, (v * LANES + sl) * VE + i);
+                }
+            }
+            sort8_desc(grp8);
+            if (g == 0) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) best[j] = grp8[j];
+            } else {
+                merge8_desc(best, grp8);
+            }
+        }
+        // ---- the row's eight best: merge across the lanes of the group
+#pragma unroll
+        for (int o = 1; o < LANES; o <<= 1) {
+            K other[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) other[j] = __shfl_xor_sync(0xffffffffu, best[j], o);
+            merge8_desc(best, other);
+        }
+        // ---- weights and output: entry r by lane r mod LANES
+        const float key0 = RK::value(best[0]);
+        float e[8];
+        float sel = 0.0f;
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+            e[r] = ex2_ftz_r((RK::value(best[r]) - key0) * cabs);
+            if (r < p.k) sel += e[r];
+        }
+        // 0 * inv_s carries a NaN row into the renormalised weights (inv_s is finite otherwise)
+        const float f = p.renorm ? 1.0f / sel + 0.0f * inv_s : inv_s;
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+            if (row_ok && r < p.k && (r % LANES) == sl) {
+                p.idx[row * p.k + r] = RK::col(best[r]);
+                p.w[row * p.k + r] = e[r] * f;
+            }
         }
     }
 }
