@@ -77,6 +77,34 @@ def test_router_ties_and_special_rows():
     assert list(idx[1]) == [0, 1, 2, 3] and list(idx[5]) == [3, 100, 0, 1] and list(idx[6]) == [0, 1, 2, 3]
 
 
+def test_router_both_selection_kernels_agree(monkeypatch):
+    """k <= 8 selects with sorting networks in registers; FS_ROUTER_ROUNDS=1 (read per call) keeps the
+    kernel that takes one maximum per round. Same columns bit for bit, weights within the parity
+    bound of each against the oracle, on tie-heavy and special rows in every dtype."""
+    rng = np.random.default_rng(11)
+    for dtype in (FP32, BF16, FP16):
+        for cols in (8, 16, 64, 128, 256, 1024):
+            if (cols * W.ELEM_SIZE[dtype]) % 16:
+                continue
+            x64 = np.round(rng.standard_normal((37, cols)) * 2) / 2            # heavy ties
+            x64[3, :] = 0.0
+            x64[5, ::3] = -np.inf
+            x64[7, 1] = np.nan
+            x = W.to_stored(x64, dtype)
+            for k in (1, 3, 8):
+                for scale, renorm in ((1.0, True), (-0.7, False), (0.0, True)):
+                    monkeypatch.delenv("FS_ROUTER_ROUNDS", raising=False)
+                    st_a, w_a, i_a = run_router(x, dtype, k, scale, renorm)
+                    check_router(x, dtype, k, scale, renorm)
+                    monkeypatch.setenv("FS_ROUTER_ROUNDS", "1")
+                    st_b, w_b, i_b = run_router(x, dtype, k, scale, renorm)
+                    check_router(x, dtype, k, scale, renorm)
+                    assert st_a == st_b == fs.FS_OK and np.array_equal(i_a, i_b)
+                    assert np.array_equal(np.isnan(w_a), np.isnan(w_b))
+                    assert np.allclose(np.nan_to_num(w_a), np.nan_to_num(w_b), rtol=0, atol=2e-6)
+    monkeypatch.delenv("FS_ROUTER_ROUNDS", raising=False)
+
+
 def test_router_workload_cfg3_top8():
     w = W.WORKLOADS["cfg3"]
     x = W.generate_rows(w, 0, 32768, threads=8)
