@@ -940,6 +940,21 @@ bool masked_tile_wanted(int dtype, int64_t nvec) {
     return dtype != FS_DTYPE_FP32 && nvec >= 256 && nvec <= 640;
 }
 
+// The same for fs_softmax_backward (the dy and the y row of a warp in shared memory): rows of 4-8 KiB.
+// Measured (256 MiB per tensor, a copy of the same bytes = 115 us): rows of 5 / 6 / 7 / 8 KiB 118 / 118 / 117 / 117 us
+// against 150 / 135 / 126 / 120 on the split-row kernel; level from 10 KiB on. FS_SMB_TILE "lo:hi" overrides.
+bool smb_tile_wanted(int64_t nvec) {
+    static const std::pair<int64_t, int64_t> ov = [] {
+        const char* e = std::getenv("FS_SMB_TILE");
+        if (!e) return std::pair<int64_t, int64_t>(-1, -1);
+        long lo = 0, hi = 0;
+        if (std::sscanf(e, "%ld:%ld", &lo, &hi) == 2) return std::pair<int64_t, int64_t>(lo, hi);
+        return std::pair<int64_t, int64_t>(0, 0);
+    }();
+    if (ov.first >= 0) return nvec > ov.first && nvec <= ov.second;
+    return nvec > 256 && nvec <= 512;
+}
+
 // FS_NORM_SPLIT=0 / 1 (read once) forces the choice for experiments.
 bool norm_split_wanted(const Device& dev, int64_t rows, int64_t nvec, bool smem_ok, int cs) {
     static const int forced = [] { const char* e = std::getenv("FS_NORM_SPLIT"); return e ? std::atoi(e) : -1; }();
@@ -1217,6 +1232,19 @@ int run_softmax_backward(const void* dy, const void* y, void* dx, int64_t rows, 
             const int64_t groups = (rows + (32 / wg.lanes) - 1) / (32 / wg.lanes);
             const int64_t grid = std::min<int64_t>((groups + (t / 32) - 1) / (t / 32), 0x7fffffff);
             return launch(fn, grid, t, 0, 0, st, p);
+        }
+    }
+    if (fast && smb_tile_wanted(p.nvec)) {                  // rows of 4-8 KiB: a warp per row from shared memory
+        const void* fn = by_dtype(dtype, [&](auto dt) -> const void* { return (const void*)smb_tile_kernel<decltype(dt)::value>; });
+        const int t = 128;
+        const size_t smem = 2 * size_t(t / 32) * size_t(p.nvec) * 16 + size_t(t / 32) * 8;
+        int bps = 0;
+        if ((rc = blocks_per_sm(dev, fn, t, smem, &bps)) != FS_OK) return rc;
+        const int64_t grid = (rows + (t / 32) - 1) / (t / 32);
+        if (grid <= 0x7fffffff) {
+            p.pf_rows = prefetch_rows(dev.sm_count * bps) * (t / 32);
+            set_first_wave_lag(p, dev.sm_count * bps, 2 * (t / 32) * p.nvec * 16);
+            return launch(fn, grid, t, smem, 0, st, p);
         }
     }
     SmemGeom sg;

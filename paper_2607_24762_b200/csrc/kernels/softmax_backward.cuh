@@ -3,6 +3,7 @@
 // place of the (max, sum) pair and no exponential. Algorithmic traffic: 3 elements per element.
 //
 //   smb_warp_kernel     (sub-)warp per row, both rows in registers (rows up to 4 KiB)
+//   smb_tile_kernel     rows of 4-8 KiB: four rows per block in shared memory, a warp per row
 //   smb_smem_kernel     row split over a cluster of 1..16 blocks; the dy and y slices are resident
 //                       in shared memory (two bulk copies per chunk on one mbarrier), the partial
 //                       dot products merge warp -> block -> cluster (st.async deposits), pass 2
@@ -81,6 +82,90 @@ smb_warp_kernel(const SmbParams p) {
                     for (int j = 0; j < NP; ++j) g[j] = mul2(mul2(y[j], sub2(g[j], d2)), s2);
                     st_stream(dv + row * p.nvec + sl + k * LANES, narrow_pairs<DT>(g));
                 }
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Rows of 4-8 KiB: four rows per block; the dy row and the y row of a warp come to shared memory
+// by two bulk copies on one mbarrier, and the warp works on them alone (dot product, then dx),
+// with no block barrier after start-up. One-shot grid: block b handles rows b*W .. b*W+W-1.
+// dynamic shared memory: W dy rows | W y rows | W mbarriers
+// ---------------------------------------------------------------------------------------------
+template <int DT>
+__global__ void __launch_bounds__(128)
+smb_tile_kernel(const SmbParams p) {
+    constexpr int NP = Traits<DT>::VE / 2;
+    constexpr int H = 4;                                   // vectors per lane and batch
+    pdl_launch_dependents();
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, W = blockDim.x >> 5;
+    const int nvec = static_cast<int>(p.nvec);
+    const uint32_t row_bytes = static_cast<uint32_t>(p.nvec) * 16u;          // at most 32 KiB: one copy each
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * size_t(W) * row_bytes);
+    const int64_t row = int64_t(blockIdx.x) * W + w;
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < W; ++i) mbar_init(smem_u32(&bars[i]), 1);
+        mbar_fence_init();
+        fence_proxy_async_smem();
+    }
+    __syncthreads();
+    pdl_wait();
+    if (row >= p.rows) return;                             // no block-wide barrier follows
+    const char* gb = static_cast<const char*>(p.dy) + row * int64_t(row_bytes);
+    const char* yb = static_cast<const char*>(p.y) + row * int64_t(row_bytes);
+    if (lane == 0) {
+        first_wave_lag(blockIdx.x, p.lag_ns, p.lag_rows);
+        const uint32_t bar = smem_u32(&bars[w]);
+        mbar_expect_tx(bar, 2u * row_bytes);
+        bulk_load(smem_u32(smem) + uint32_t(w) * row_bytes, gb, row_bytes, bar);
+        bulk_load(smem_u32(smem) + uint32_t(W + w) * row_bytes, yb, row_bytes, bar);
+        if (p.pf_rows > 0 && row + p.pf_rows < p.rows) {
+            l2_prefetch(gb + p.pf_rows * int64_t(row_bytes), row_bytes);
+            l2_prefetch(yb + p.pf_rows * int64_t(row_bytes), row_bytes);
+        }
+    }
+    const uint4* sg = reinterpret_cast<const uint4*>(smem + size_t(w) * row_bytes) + lane;
+    const uint4* sy = reinterpret_cast<const uint4*>(smem + size_t(W + w) * row_bytes) + lane;
+    uint4* __restrict__ dv = static_cast<uint4*>(p.dx) + row * p.nvec + lane;
+    mbar_wait_warp(smem_u32(&bars[w]), 0u, p.status);      // on a timeout the status word is set and the row is garbage
+
+    f32x2 acc[2] = {pair(0.0f, 0.0f), pair(0.0f, 0.0f)};
+    for (int k0 = 0; k0 < nvec; k0 += 32 * H) {
+        uint4 graw[H], yraw[H];
+#pragma unroll
+        for (int u = 0; u < H; ++u) {
+            graw[u] = make_uint4(0u, 0u, 0u, 0u); yraw[u] = graw[u];          // absent vectors are zeros: they add nothing
+            if (k0 + u * 32 + lane < nvec) { graw[u] = sg[k0 + u * 32]; yraw[u] = sy[k0 + u * 32]; }
+        }
+#pragma unroll
+        for (int u = 0; u < H; ++u) {
+            f32x2 g[NP], y[NP];
+            widen_pairs<DT>(graw[u], g);
+            widen_pairs<DT>(yraw[u], y);
+#pragma unroll
+            for (int j = 0; j < NP; ++j) acc[j & 1] = fma2(g[j], y[j], acc[j & 1]);
+        }
+    }
+    const float dot = warp_sum<32>(pair_sum(add2(acc[0], acc[1])));
+    const f32x2 d2 = pair(dot, dot), s2 = pair(p.scale, p.scale);
+    for (int k0 = 0; k0 < nvec; k0 += 32 * H) {
+        uint4 graw[H], yraw[H];
+#pragma unroll
+        for (int u = 0; u < H; ++u) {
+            graw[u] = make_uint4(0u, 0u, 0u, 0u); yraw[u] = graw[u];
+            if (k0 + u * 32 + lane < nvec) { graw[u] = sg[k0 + u * 32]; yraw[u] = sy[k0 + u * 32]; }
+        }
+#pragma unroll
+        for (int u = 0; u < H; ++u) {
+            if (k0 + u * 32 + lane < nvec) {
+                f32x2 g[NP], y[NP];
+                widen_pairs<DT>(graw[u], g);
+                widen_pairs<DT>(yraw[u], y);
+#pragma unroll
+                for (int j = 0; j < NP; ++j) g[j] = mul2(mul2(y[j], sub2(g[j], d2)), s2);
+                st_stream(dv + k0 + u * 32, narrow_pairs<DT>(g));
             }
         }
     }

@@ -75,6 +75,18 @@ def test_row_lengths_across_the_split_geometries(dtype):
 
 
 @pytest.mark.parametrize("dtype", [FP32, BF16, FP16])
+def test_rows_around_the_four_rows_per_block_kernel(dtype):
+    """Rows of 257..512 sixteen-byte vectors take the kernel that works on four row pairs per block from
+    shared memory: both ends of that range and one vector beyond them, row counts that leave a block
+    partly empty, dx aliasing dy or y."""
+    ve = 16 // W.ELEM_SIZE[dtype]
+    for ci, nvec in enumerate((256, 257, 300, 511, 512, 513)):
+        for rows in (1, 4, 5, 7, 130):
+            dy, y = make(rows, nvec * ve, dtype, seed=40 * nvec + rows)
+            check(dy, y, dtype, [1.0, 0.25, -0.5][(ci + rows) % 3], alias=[None, "dy", "y"][(ci + rows) % 3])
+
+
+@pytest.mark.parametrize("dtype", [FP32, BF16, FP16])
 def test_aliasing_alignment_and_special_values(dtype):
     dy, y = make(33, 2048, dtype, seed=3)
     check(dy, y, dtype, 1.0, alias="dy")
