@@ -955,6 +955,23 @@ bool smb_tile_wanted(int64_t nvec) {
     return nvec > 256 && nvec <= 512;
 }
 
+// The same for fs_log_softmax and fs_softmax_f32out: rows of 4-12 KiB. Measured (256 MiB per direction,
+// copy = 80 us): bf16 rows of 5 / 6 / 7 / 8 / 10 / 12 KiB 82 / 82 / 82 / 81 / 82 / 82 us against 88 / 83 / 89 / 86 / 93 / 83
+// with the row packed in registers or split over a block; fp32 rows of 8 / 10 KiB 81 / 81 against 83 / 88;
+// from 14 KiB on the split-row kernel is ahead (bf16 86 / 79 against 91 / 90). FS_LSM_TILE "lo:hi" overrides.
+bool lsm_tile_wanted(int dtype, int64_t nvec) {
+    static const std::pair<int64_t, int64_t> ov = [] {
+        const char* e = std::getenv("FS_LSM_TILE");
+        if (!e) return std::pair<int64_t, int64_t>(-1, -1);
+        long lo = 0, hi = 0;
+        if (std::sscanf(e, "%ld:%ld", &lo, &hi) == 2) return std::pair<int64_t, int64_t>(lo, hi);
+        return std::pair<int64_t, int64_t>(0, 0);
+    }();
+    if (ov.first >= 0) return nvec > ov.first && nvec <= ov.second;
+    (void)dtype;
+    return nvec > 256 && nvec <= 768;
+}
+
 // FS_NORM_SPLIT=0 / 1 (read once) forces the choice for experiments.
 bool norm_split_wanted(const Device& dev, int64_t rows, int64_t nvec, bool smem_ok, int cs) {
     static const int forced = [] { const char* e = std::getenv("FS_NORM_SPLIT"); return e ? std::atoi(e) : -1; }();
@@ -1128,6 +1145,22 @@ int run_log_softmax(const void* x, void* y, int64_t rows, int64_t cols, int dtyp
     p.c = static_cast<float>(static_cast<double>(p.scale) * kLog2e);
     p.flip = std::signbit(scale) && scale != 0.0f ? (dtype == FS_DTYPE_FP32 ? 0x80000000u : 0x80008000u) : 0u;
     p.status = dev.status; p.pf_rows = 0;
+    if (fast && lsm_tile_wanted(dtype, p.nvec) && (out == OUT_LOG || dtype != FS_DTYPE_FP32)) {   // a warp per row from shared memory
+        const void* fn = by_dtype(dtype, [&](auto dt) -> const void* {
+            constexpr int DT = decltype(dt)::value;
+            if constexpr (DT == DT_F32) return (const void*)lsm_tile_kernel<DT, OUT_LOG>;
+            else return out == OUT_LOG ? (const void*)lsm_tile_kernel<DT, OUT_LOG> : (const void*)lsm_tile_kernel<DT, OUT_PROB32>; });
+        const int t = 128;
+        const size_t smem = size_t(t / 32) * size_t(p.nvec) * 16 + size_t(t / 32) * 8;
+        int bps = 0;
+        if ((rc = blocks_per_sm(dev, fn, t, smem, &bps)) != FS_OK) return rc;
+        const int64_t grid = (rows + (t / 32) - 1) / (t / 32);
+        if (grid <= 0x7fffffff) {
+            p.pf_rows = prefetch_rows(dev.sm_count * bps) * (t / 32);
+            set_first_wave_lag(p, dev.sm_count * bps, (t / 32) * p.nvec * 16);
+            return launch(fn, grid, t, smem, 0, st, p);
+        }
+    }
     WarpGeom wg;
     bool warp_ok = fast && norm_warp_geom(p.nvec, dtype, &wg);
     if (fast && !warp_ok && p.nvec <= 576) {

@@ -9,6 +9,7 @@
 // maximum.
 //
 //   lsm_warp_kernel     (sub-)warp per row, the row packed in registers (rows up to 9 KiB)
+//   lsm_tile_kernel     rows of 4-12 KiB: four rows per block in shared memory, a warp per row
 //   lsm_smem_kernel     row split over a cluster of 1..16 blocks, slices resident in shared memory
 //                       (bulk async copies, per-chunk mbarriers, online (max, sum) per thread,
 //                       pairs merged warp -> block -> cluster through st.async); pass 2 reads the
@@ -158,6 +159,85 @@ template <int DT, int VPL, int OUT>
 __global__ void __launch_bounds__(128, VPL <= 12 ? 5 : 4)
 lsm_warp_long_kernel(const LsmParams p) {
     lsm_warp_body<DT, 32, VPL, OUT>(p);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Rows of 4-11 KiB: four rows per block, each brought to shared memory by a bulk copy of its own
+// (one mbarrier per row) and worked on by one warp alone with the arithmetic of the warp kernel
+// above (three reads of shared memory: reference, sum, output); no block barrier after start-up.
+// One-shot grid: block b handles rows b*W .. b*W+W-1. dynamic shared memory: W rows | W mbarriers
+// ---------------------------------------------------------------------------------------------
+template <int DT, int OUT>
+__global__ void __launch_bounds__(128)
+lsm_tile_kernel(const LsmParams p) {
+    constexpr int NP = Traits<DT>::VE / 2;
+    constexpr int H = 4;                                   // vectors per lane and batch
+    pdl_launch_dependents();
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, W = blockDim.x >> 5;
+    const int nvec = static_cast<int>(p.nvec);
+    const int64_t row_bytes = p.nvec * 16;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + size_t(W) * size_t(row_bytes));
+    const int64_t row = int64_t(blockIdx.x) * W + w;
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < W; ++i) mbar_init(smem_u32(&bars[i]), 1);
+        mbar_fence_init();
+        fence_proxy_async_smem();
+    }
+    __syncthreads();
+    pdl_wait();
+    if (row >= p.rows) return;                             // no block-wide barrier follows
+    const char* xb = static_cast<const char*>(p.x);
+    if (lane == 0) {
+        first_wave_lag(blockIdx.x, p.lag_ns, p.lag_rows);
+        bulk_load_row(smem_u32(smem) + uint32_t(w) * uint32_t(row_bytes), xb + row * row_bytes, uint32_t(row_bytes), smem_u32(&bars[w]));
+        if (p.pf_rows > 0 && row + p.pf_rows < p.rows) l2_prefetch(xb + (row + p.pf_rows) * row_bytes, uint32_t(row_bytes));
+    }
+    const uint4* sv = reinterpret_cast<const uint4*>(smem + size_t(w) * size_t(row_bytes)) + lane;
+    const int64_t ypitch = OUT == OUT_LOG ? p.nvec * 16 : p.cols * 4;      // bytes per output row
+    char* yrow = static_cast<char*>(p.y) + row * ypitch;
+    const f32x2 c2 = pair(p.c, p.c), s2 = pair(p.scale, p.scale);
+    mbar_wait_warp(smem_u32(&bars[w]), 0u, p.status);      // on a timeout the status word is set and the row is garbage
+
+    RefAcc<DT, false> ref;
+    ref.init();
+    for (int k0 = 0; k0 < nvec; k0 += 32 * H) {
+#pragma unroll
+        for (int u = 0; u < H; ++u)
+            if (k0 + u * 32 + lane < nvec) ref.fold(flip_vec(sv[k0 + u * 32], p.flip));
+    }
+    const float r = warp_pick<32, false>(ref.value());
+    const f32x2 r2 = pair(r, r);
+    f32x2 acc[2] = {pair(0.0f, 0.0f), pair(0.0f, 0.0f)};
+    for (int k0 = 0; k0 < nvec; k0 += 32 * H) {
+        uint4 raw[H];
+#pragma unroll
+        for (int u = 0; u < H; ++u) {
+            raw[u] = make_uint4(0u, 0u, 0u, 0u);
+            if (k0 + u * 32 + lane < nvec) raw[u] = flip_vec(sv[k0 + u * 32], p.flip);
+        }
+#pragma unroll
+        for (int u = 0; u < H; ++u) {
+            if (k0 + u * 32 + lane < nvec) {
+                f32x2 d[NP];
+                lsm_accumulate<DT>(raw[u], r2, c2, d, acc);
+            }
+        }
+    }
+    const float ssum = warp_sum<32>(pair_sum(add2(acc[0], acc[1])));
+    const float kk = OUT == OUT_LOG ? -ln_of(ssum) : 1.0f / ssum;
+    const f32x2 k2 = pair(kk, kk);
+    for (int k0 = 0; k0 < nvec; k0 += 32 * H) {
+        uint4 raw[H];
+#pragma unroll
+        for (int u = 0; u < H; ++u) {
+            raw[u] = make_uint4(0u, 0u, 0u, 0u);
+            if (k0 + u * 32 + lane < nvec) raw[u] = flip_vec(sv[k0 + u * 32], p.flip);
+        }
+#pragma unroll
+        for (int u = 0; u < H; ++u)
+            if (k0 + u * 32 + lane < nvec) lsm_emit<DT, OUT>(raw[u], r2, c2, s2, k2, yrow, k0 + u * 32 + lane);
+    }
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -68,6 +68,19 @@ def test_row_lengths_across_the_split_geometries(dtype):
 
 
 @pytest.mark.parametrize("dtype", [FP32, BF16, FP16])
+def test_rows_around_the_four_rows_per_block_kernel(dtype):
+    """Rows of 257..768 sixteen-byte vectors take the kernel that works on four rows per block from shared
+    memory: both ends of that range and one vector beyond them, row counts that leave a block partly
+    empty, positive, negative and zero scale, in place."""
+    ve = 16 // W.ELEM_SIZE[dtype]
+    for ci, nvec in enumerate((256, 257, 400, 767, 768, 769)):
+        for rows in (1, 4, 5, 7, 130):
+            scale = [1.0, 0.25, -0.5, 0.0][(ci + rows) % 4]
+            x = W.random_case(rows, nvec * ve, dtype, seed=50 * nvec + rows, sigma=2.0, neg_inf_frac=0.03 if scale > 0 else 0.0)
+            check(x, dtype, scale, inplace=(rows == 5))
+
+
+@pytest.mark.parametrize("dtype", [FP32, BF16, FP16])
 def test_special_values_alignment_and_aliasing(dtype):
     x = W.random_case(6, 4096, dtype, seed=5, sigma=2.0)
     nan_bits = np.float32(np.nan) if dtype == FP32 else np.uint16(0x7FC0 if dtype == BF16 else 0x7E00)
