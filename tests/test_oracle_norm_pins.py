@@ -183,3 +183,77 @@ def test_comparator_rules():
     assert not fno.compare(off2s, BF16, want, scale).ok(BF16)
     big = np.array([4000.0, 4000.0, 4000.0, 4000.0])   # cancellation: a large scale excuses a small result's ulps
     assert fno.compare(off2s, BF16, want, big).ok(BF16)
+
+
+# ---------------------------------------------------------------------------------------------
+# error_scale: the magnitude the binary32 tolerance of the normalisation parity tests multiplies
+# ---------------------------------------------------------------------------------------------
+
+def test_error_scale_hand_computed_rows():
+    """|gamma| (|x - mu| + mean|x|) / sqrt(var + eps) + |beta| worked out by hand."""
+    x = np.array([[1.0, 3.0], [0.0, 4.0]], dtype=np.float32)
+    # row 0: mu 2, var 1, mean|x| 2 -> (1 + 2) / 1 = 3; row 1: mu 2, var 4, mean|x| 2 -> (2 + 2) / 2 = 2
+    s = fno.error_scale(x, FP32, x.shape, None, None, 0.0)
+    assert np.array_equal(s, [[3.0, 3.0], [2.0, 2.0]])
+    gamma = np.array([[2.0, -3.0]])
+    beta = np.array([[0.5, -1.0]])
+    s = fno.error_scale(x, FP32, x.shape, gamma, beta, 0.0)
+    assert np.array_equal(s, [[6.5, 10.0], [4.5, 7.0]])
+    assert np.array_equal(fno.error_scale(x, FP32, x.shape, gamma, None, 0.0), [[6.0, 9.0], [4.0, 6.0]])
+    assert np.array_equal(fno.error_scale(x, FP32, x.shape, None, beta, 0.0), [[3.5, 4.0], [2.5, 3.0]])
+    # eps sits under the root, next to the variance: var 1, eps 3 -> divisor 2
+    assert np.array_equal(fno.error_scale(x[:1], FP32, (1, 2), None, None, 3.0), [[1.5, 1.5]])
+    # a row far from zero: the mean term dominates (mu 1000, |d| 1, var 1)
+    far = np.array([[999.0, 1001.0]], dtype=np.float32)
+    assert np.array_equal(fno.error_scale(far, FP32, (1, 2), None, None, 0.0), [[1001.0, 1001.0]])
+    # the view: six elements as 2 x 3 and as 3 x 2 are different rows
+    six = np.array([0, 3, 6, 1, 1, 1], dtype=np.float32)
+    s23 = fno.error_scale(six, FP32, (2, 3), None, None, 0.0)
+    assert s23.shape == (2, 3) and np.allclose(s23[0], [(3 + 3) / math.sqrt(6), 3 / math.sqrt(6), (3 + 3) / math.sqrt(6)])
+
+
+def _layer_norm_binary32(x, gamma, beta, eps, order):
+    """layer_norm carried out in binary32, one rounding per operation, sums taken in `order`."""
+    out = np.empty_like(x)
+    one, n = np.float32(1), np.float32(x.shape[1])
+    for i, row in enumerate(x):
+        s = np.float32(0)
+        for j in order:
+            s = np.float32(s + row[j])
+        mu = np.float32(s / n)
+        d = (row - mu).astype(np.float32)
+        q = np.float32(0)
+        for j in order:
+            q = np.float32(q + np.float32(d[j] * d[j]))
+        rstd = np.float32(one / np.sqrt(np.float32(np.float32(q / n) + np.float32(eps))))
+        out[i] = ((d * rstd).astype(np.float32) * gamma).astype(np.float32) + beta
+    return out
+
+
+def test_error_scale_brackets_a_binary32_evaluation():
+    """The error of a plain binary32 layer_norm, measured against 60-digit arithmetic, is a fixed small multiple
+    of error_scale whatever the row length, offset, spread or summation order: between 5e-8 and 1e-6 of it
+    (binary32's unit roundoff is 6e-8; the parity tests allow 2e-6). A scale that is ten times too large or too
+    small, or that drops the mean, gamma or beta term, leaves that band on at least one case."""
+    import mpmath as mp
+    rng = np.random.default_rng(7)
+    with mp.workdps(60):
+        for rows, cols, offset, spread, gscale, bscale in ((4, 257, 0.0, 1.0, 0.5, 1.0), (4, 64, 5.0, 0.5, 0.5, 1.0),
+                                                           (3, 1000, -2.0, 3.0, 0.5, 1.0), (3, 96, 40.0, 1.0, 1.0, 0.0),
+                                                           (3, 96, 0.0, 1.0, 20.0, 0.0), (3, 96, 0.0, 1.0, 0.01, 30.0)):
+            x = (rng.standard_normal((rows, cols)) * spread + offset).astype(np.float32)
+            gamma = (rng.standard_normal(cols) * gscale + gscale).astype(np.float32)
+            beta = (rng.standard_normal(cols) * bscale).astype(np.float32)
+            eps = 1e-5
+            want = np.empty((rows, cols))
+            for i in range(rows):
+                xs = [mp.mpf(float(v)) for v in x[i]]
+                mu = mp.fsum(xs) / cols
+                sd = mp.sqrt(mp.fsum([(v - mu) ** 2 for v in xs]) / cols + mp.mpf(float(np.float32(eps))))
+                want[i] = [float((v - mu) / sd * mp.mpf(float(gamma[j])) + mp.mpf(float(beta[j]))) for j, v in enumerate(xs)]
+            scale = fno.error_scale(x, FP32, x.shape, gamma.astype(np.float64)[None, :], beta.astype(np.float64)[None, :], eps)
+            worst = 0.0
+            for order in (range(cols), range(cols - 1, -1, -1), np.random.default_rng(cols).permutation(cols)):
+                got = _layer_norm_binary32(x, gamma, beta, eps, list(order))
+                worst = max(worst, float(np.max(np.abs(got - want) / scale)))
+            assert 5e-8 <= worst <= 1e-6, (rows, cols, offset, spread, gscale, bscale, worst)

@@ -386,6 +386,34 @@ def test_comparator_applies_the_stated_tolerances():
     assert fso.compare(np.array([5, 0x0200], dtype=np.uint16), FP16, w16).max_ulp == 2
 
 
+def test_comparator_fp32_exact_zero_and_sign_rules():
+    """fp32 results: an oracle value of exactly +0 (a -inf input) must be met by the +0 bit pattern, and a
+    softmax output never carries a sign; each of these fails the bar even where |delta| is far below 1e-6."""
+    want = np.array([0.25, 0.0, 0.5, 0.0, 0.25])
+    exact = want.astype(np.float32)
+    rep = fso.compare(exact, FP32, want)
+    assert rep.ok(FP32) and rep.zero_mismatch == 0 and rep.negative == 0 and rep.n_compared == 5
+    tiny = exact.copy(); tiny[1] = np.float32(1e-45)             # the smallest subnormal is not +0
+    rep = fso.compare(tiny, FP32, want)
+    assert rep.zero_mismatch == 1 and rep.negative == 0 and rep.max_abs_err < 1e-44 and not rep.ok(FP32)
+    mz = exact.copy(); mz[3] = np.float32(-0.0)                  # -0: wrong bit pattern, but no magnitude
+    rep = fso.compare(mz, FP32, want)
+    assert rep.zero_mismatch == 1 and rep.negative == 0 and rep.max_abs_err == 0.0 and not rep.ok(FP32)
+    neg0 = exact.copy(); neg0[1] = np.float32(-1e-30)            # negative where the oracle has +0: both rules
+    rep = fso.compare(neg0, FP32, want)
+    assert rep.zero_mismatch == 1 and rep.negative == 1 and not rep.ok(FP32)
+    neg = exact.copy(); neg[0] = np.float32(-1e-30)              # negative where the oracle is positive
+    wneg = want.copy(); wneg[0] = 1e-30
+    rep = fso.compare(neg, FP32, wneg)
+    assert rep.negative == 1 and rep.zero_mismatch == 0 and rep.max_abs_err < 1e-6 and not rep.ok(FP32)
+    both = exact.copy(); both[1] = np.float32(1e-45); both[3] = np.float32(-0.0); both[4] = np.float32(-0.25)
+    rep = fso.compare(both, FP32, want)
+    assert rep.zero_mismatch == 2 and rep.negative == 1
+    # the same rules leave a correct result alone when the oracle value is tiny but not zero
+    wt = np.array([1e-300, 0.5])
+    assert fso.compare(np.array([0.0, 0.5], dtype=np.float32), FP32, wt).ok(FP32)
+
+
 # ---------------------------------------------------------------------------------------------
 # workload structure seen through the oracle
 # ---------------------------------------------------------------------------------------------
