@@ -23,6 +23,18 @@
  *   - The library works on the calling thread's current CUDA device. One GPU; no host fallback:
  *     without a usable CUDA device every compute entry point returns FS_ERR_CUDA.
  *   - Thread-safe. Per-device attributes are cached on first use.
+ *   - Device memory: no entry point allocates per call. On first use per device the library
+ *     allocates a 4-byte status word; the two-kernel path of very long rows (fs_softmax,
+ *     fs_layer_norm, fs_group_norm on rows beyond FS_STATIC_MAX_ROW_BYTES) keeps one scratch buffer
+ *     per device, allocated when first needed, grown when a call needs more, and fs_softmax_host
+ *     keeps its staging buffers; fs_release frees the last two. fs_softmax_static allocates nothing.
+ *   - Environment switches (each read once per process): FS_LOG=1 prints one line per call with the
+ *     dispatcher's decision and launch geometry on stderr; FS_FORCE_KERNEL=warp|block|block_tma|
+ *     cluster|generic replaces the choice of fs_softmax's dispatcher (a shape that kernel cannot run
+ *     returns FS_ERR_UNSUPPORTED); FS_CHECK=1 validates every tensor pointer with
+ *     cudaPointerGetAttributes (memory the current device cannot address is FS_ERR_INVALID_ARG);
+ *     FS_SIM_NO_CLUSTER=1 and FS_SIM_SMEM_OPTIN=<bytes> make the library behave as on a device
+ *     without cluster launch / with less shared memory, so that its downgrade paths can be tested.
  */
 #ifndef FSOFTMAX_H_
 #define FSOFTMAX_H_
@@ -38,6 +50,10 @@ typedef enum { FS_DTYPE_FP32 = 0, FS_DTYPE_BF16 = 1, FS_DTYPE_FP16 = 2 } fs_dtyp
 
 /* Longest row (bytes) the split-row kernel holds in the shared memory of a 16-block cluster. */
 #define FS_STATIC_MAX_ROW_BYTES (16 * 192 * 1024)
+/* fs_softmax_static: size of the fixed device array every GPU holds, and the number of per-segment
+ * (max, sum) pairs of its long-row path that fit behind the array's 256-byte header. */
+#define FS_STATIC_SCRATCH_BYTES 65536
+#define FS_STATIC_MAX_PAIRS ((FS_STATIC_SCRATCH_BYTES - 256) / 8)
 
 typedef enum {
     FS_OK = 0,
@@ -209,9 +225,10 @@ int fs_softmax_backward(const void* dy, const void* y, void* dx, int64_t rows, i
  * widened where they are used); longer rows are split over
  * a cluster of 1..16 blocks with the slices resident in shared memory (one read and one write of
  * HBM per element, as for fs_softmax); rows beyond a cluster's shared memory (about 3 MiB) are
- * cut into segments over two kernels, whose partial statistics pass through a scratch buffer that
- * is allocated and freed in stream order (cudaMallocAsync on `stream`); ragged or misaligned
- * rows take a three-pass kernel.
+ * cut into segments over two kernels, whose partial statistics pass through the library's
+ * per-device scratch buffer (16 bytes per segment; see "Device memory" above: a call allocates
+ * only when the buffer has to grow, which it cannot do inside a stream capture); ragged or
+ * misaligned rows take a three-pass kernel.
  * A NaN or infinity in a row makes the whole row NaN. rows == 0 or cols == 0 launches nothing.
  */
 int fs_layer_norm(const void* x, const void* gamma, const void* beta, void* y, int64_t rows, int64_t cols, int dtype,
@@ -244,8 +261,13 @@ int fs_split_geometry(int64_t cols, int dtype, int* cluster, int* threads, int64
  *   x_align, y_align  the largest power of two (<= 16 is enough) dividing each base address.
  * Returns an fs_kernel (>= 1), or a negative fs_status on invalid arguments. FS_KERNEL_GENERIC
  * covers two forms: vector-aligned rows of 1 MiB or more that no cluster holds are cut into
- * segments over two kernels (partial (max, sum) pairs through a scratch buffer allocated and freed
- * in stream order); everything else runs one block per row.
+ * segments over two kernels (partial (max, sum) pairs, 8 bytes per segment, through the library's
+ * per-device scratch buffer; calls that use it are ordered on the device by an event, whatever
+ * their streams; inside a stream capture the buffer cannot grow, so the first such call should
+ * come before the capture); everything else runs one block per row.
+ * On a device without cluster launch, or with too little shared memory for the split-row kernel,
+ * fs_softmax runs FS_KERNEL_CLUSTER's one-block form where the row fits one block and the generic
+ * forms otherwise; fs_softmax_ex with a forced kernel returns FS_ERR_UNSUPPORTED instead.
  */
 int fs_select_kernel(int64_t rows, int64_t cols, int dtype, int x_align, int y_align);
 
@@ -277,35 +299,74 @@ int fs_device_status(void);
  * fs_softmax_static -- fs_softmax for callers that must not allocate device memory.
  * (The paper has no counterpart: this entry point exists for the library's users only.)
  *
- * Every other compute entry point calls cudaMalloc once per device, on first use, for the status
- * word its kernels write when a bounded wait expires (fs_softmax_host also for its staging
- * buffers). Some callers cannot afford that call: a process that has handed all device memory to
- * its own pool and must not touch the driver's allocator again, a service that has to prove it
- * cannot run out of memory after start-up, or a latency-critical loop in which the implicit device
- * synchronisation of an allocation is unacceptable. This entry point makes no cudaMalloc,
- * cudaFree or other allocating call, ever. It always runs the split-row kernel (FS_KERNEL_CLUSTER's
- * shared-memory-resident form), whose status word then lives in a 256-byte array that is part of
- * the library's device code: every GPU that loads the library holds those 256 bytes until the
- * process exits.
+ * Every other compute entry point calls cudaMalloc on its first use per device (the status buffer
+ * its kernels write when a bounded wait expires), the long-row path of fs_softmax again whenever
+ * its scratch buffer must grow, fs_softmax_host for its staging buffers. Some callers cannot afford
+ * such a call: a process that has handed all device memory to its own pool and must not touch the
+ * driver's allocator again, a service that has to prove it cannot run out of memory after start-up,
+ * or a latency-critical loop in which the implicit device synchronisation of an allocation is
+ * unacceptable. This entry point makes no cudaMalloc, cudaFree or other allocating call, ever.
+ * What the other paths keep in allocated memory lives in one array of FS_STATIC_SCRATCH_BYTES that
+ * is part of the library's device code: every GPU that loads the library holds those bytes until the
+ * process exits. The array carries the status buffer and the scratch of the long-row path:
+ *   - rows up to FS_STATIC_MAX_ROW_BYTES run the split-row kernel (FS_KERNEL_CLUSTER's
+ *     shared-memory-resident form), which needs the status buffer only;
+ *   - longer rows are cut into segments over two kernels, as in fs_softmax; the first writes one
+ *     (max, sum) pair per row and segment into the array, the second reads them back. rows times
+ *     segments per row (about 8 * SM count / rows, at least 1, at most 1024) must not exceed
+ *     FS_STATIC_MAX_PAIRS: FS_ERR_UNSUPPORTED otherwise.
  *
  *   x, y, rows, cols, dtype, scale, stream   as for fs_softmax; x and y are DEVICE pointers.
- *   Limits: x and y 16-byte aligned, row size a multiple of 16 bytes and at most
- *           FS_STATIC_MAX_ROW_BYTES (what 16 blocks hold in shared memory), rows * blocks-per-row
- *           below 2^31; scale == 0 only for rows that split into whole chunks (powers of two do).
- *           Anything else returns FS_ERR_UNSUPPORTED and enqueues nothing; there is no silent
- *           switch to another kernel.
- *   First call on a device: looks up the array's device address and raises the kernel's
- *           shared-memory limit (queries and attribute calls, no allocation). Make that first call
- *           before starting any stream capture.
+ *   Limits: x and y 16-byte aligned, row size a multiple of 16 bytes, rows * blocks-per-row
+ *           below 2^31; scale == 0 only for rows that split into whole chunks (powers of two do)
+ *           or that take the long-row path. Anything else returns FS_ERR_UNSUPPORTED and enqueues
+ *           nothing; there is no silent switch to a path that allocates.
+ *   First call on a device: looks up the array's device address (cudaGetSymbolAddress, with that
+ *           device current) and raises the kernel's shared-memory limit: queries and attribute
+ *           calls, no allocation. Make that first call before starting any stream capture.
  *   Sharing: all calls on a device share the one array, and it keeps what the last call left
- *           there. Each call therefore enqueues a 4-byte clear of the status word ahead of its
- *           kernel on `stream`. Two calls whose work overlaps on the GPU (different streams) race
- *           on that word: results stay correct, but an expired wait may go unrecorded.
- *           fs_device_status does not read this word.
+ *           there. Nothing in it has to start at zero except the status word, which is cleared when
+ *           fs_static_status reads it: the pairs are all written by a call's first kernel before
+ *           its second kernel reads them. Two long-row calls whose work overlaps on the GPU
+ *           (different streams, no event between them) race on the pairs and produce wrong
+ *           results: keep such calls on one stream or order them yourself. Calls on the split-row
+ *           kernel only OR bits into the status word and may overlap freely.
  */
 int fs_softmax_static(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale, void* stream);
 
-/* fs_release -- frees the staging buffers and streams fs_softmax_host created on the current device. */
+/*
+ * fs_static_status -- fs_device_status for fs_softmax_static: synchronises the device, reads the
+ * status word of the fixed array and clears it if set. Allocates nothing (a copy from the address
+ * cudaGetSymbolAddress gave). FS_OK, or FS_ERR_DEVICE_TIMEOUT if a bounded wait expired inside a
+ * kernel launched by fs_softmax_static since the last call.
+ * (The paper has no counterpart.)
+ */
+int fs_static_status(void);
+
+/*
+ * Self-tests of the bounded device-side waits (the paper's validator watches for launches that do not
+ * come back, Sec. III-C; these calls let a test see the library's own guard work without any fault).
+ * Every wait on an async copy polls at most N times (2^23, about two seconds); a wait that runs out
+ * sets a status bit, the kernel carries on without waiting again and returns, and fs_device_status
+ * reports FS_ERR_DEVICE_TIMEOUT once.
+ *   fs_debug_set_wait_polls(polls)  sets N for the two calls below and for FS_KERNEL_CLUSTER launches
+ *           of fs_softmax / fs_softmax_ex on the current device (polls <= 0 restores 2^23); the
+ *           other kernels keep 2^23.
+ *   fs_debug_wait_probe(stream)     launches one block that arms a barrier for 16 bytes nobody
+ *           copies and waits for it: the wait must run out. Touches no tensor.
+ *   fs_debug_softmax_expire(...)    fs_softmax_ex(..., FS_KERNEL_CLUSTER, threads, cluster) with every
+ *           chunk barrier armed for 16 bytes more than are copied: the copies complete, the waits
+ *           run out, every warp gives up once and finishes the row. Call it with a small poll cap
+ *           (a few thousand: long enough for the copies to land) and restore the default after.
+ *           y receives the normal result when the cap was long enough for the data to arrive.
+ */
+int fs_debug_set_wait_polls(int polls);
+int fs_debug_wait_probe(void* stream);
+int fs_debug_softmax_expire(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale, void* stream,
+                            int threads, int cluster);
+
+/* fs_release -- frees the staging buffers and streams fs_softmax_host created on the current device and the
+ * scratch buffer of the two-kernel long-row paths (synchronises the device if there is one to free). */
 int fs_release(void);
 
 /* The cudaError_t behind the last FS_ERR_CUDA returned on this thread (0 if none). */

@@ -15,6 +15,8 @@ FS_DTYPE_FP32, FS_DTYPE_BF16, FS_DTYPE_FP16 = 0, 1, 2
 FS_OK, FS_ERR_INVALID_ARG, FS_ERR_UNSUPPORTED, FS_ERR_CUDA, FS_ERR_DEVICE_TIMEOUT = 0, 1, 2, 3, 4
 FS_KERNEL_AUTO, FS_KERNEL_WARP, FS_KERNEL_BLOCK, FS_KERNEL_BLOCK_TMA, FS_KERNEL_CLUSTER, FS_KERNEL_GENERIC = range(6)
 FS_STATIC_MAX_ROW_BYTES = 16 * 192 * 1024
+FS_STATIC_SCRATCH_BYTES = 65536
+FS_STATIC_MAX_PAIRS = (FS_STATIC_SCRATCH_BYTES - 256) // 8
 FS_ROUTER_MAX_K = 64
 KERNELS = {"auto": 0, "warp": 1, "block": 2, "block_tma": 3, "cluster": 4, "generic": 5}
 
@@ -73,6 +75,14 @@ def lib() -> ctypes.CDLL:
             L.fs_softmax_host.restype = ci
             L.fs_softmax_static.argtypes = [vp, vp, i64, i64, ci, f32, vp]
             L.fs_softmax_static.restype = ci
+            L.fs_static_status.argtypes = []
+            L.fs_static_status.restype = ci
+            L.fs_debug_set_wait_polls.argtypes = [ci]
+            L.fs_debug_set_wait_polls.restype = ci
+            L.fs_debug_wait_probe.argtypes = [vp]
+            L.fs_debug_wait_probe.restype = ci
+            L.fs_debug_softmax_expire.argtypes = [vp, vp, i64, i64, ci, f32, vp, ci, ci]
+            L.fs_debug_softmax_expire.restype = ci
             L.fs_copy.argtypes = [vp, vp, i64, vp]
             L.fs_copy.restype = ci
             L.fs_device_status.argtypes = []
@@ -201,8 +211,29 @@ def fs_softmax_host(x_host, y_host, rows: int, cols: int, dtype: int, scale: flo
 
 
 def fs_softmax_static(x, y, rows: int, cols: int, dtype: int, scale: float = 1.0, stream=None) -> None:
-    """fs_softmax without any device allocation: split-row kernel, status word in a fixed device array."""
+    """fs_softmax without any device allocation: status buffer and long-row scratch in a fixed device array."""
     _check(lib().fs_softmax_static(_ptr(x), _ptr(y), rows, cols, dtype, scale, _stream(stream)), "fs_softmax_static")
+
+
+def fs_static_status() -> int:
+    """Reads and clears the status word of fs_softmax_static's fixed array (synchronises; allocates nothing)."""
+    return lib().fs_static_status()
+
+
+def fs_debug_set_wait_polls(polls: int) -> None:
+    """Poll cap of the bounded device-side waits on the current device (<= 0 restores the default)."""
+    _check(lib().fs_debug_set_wait_polls(polls), "fs_debug_set_wait_polls")
+
+
+def fs_debug_wait_probe(stream=None) -> None:
+    """One block that waits for 16 bytes nobody copies: its bounded wait must run out."""
+    _check(lib().fs_debug_wait_probe(_stream(stream)), "fs_debug_wait_probe")
+
+
+def fs_debug_softmax_expire(x, y, rows: int, cols: int, dtype: int, scale: float = 1.0, stream=None, threads: int = 0,
+                            cluster: int = 0) -> int:
+    """The split-row kernel with every chunk barrier armed for 16 bytes too many; returns the raw status."""
+    return lib().fs_debug_softmax_expire(_ptr(x), _ptr(y), rows, cols, dtype, scale, _stream(stream), threads, cluster)
 
 
 def fs_copy(x, y, nbytes: int, stream=None) -> None:

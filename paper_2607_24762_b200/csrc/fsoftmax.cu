@@ -7,6 +7,8 @@
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
+#include <cstring>
+#include <initializer_list>
 #include <mutex>
 #include <type_traits>
 #include <unordered_map>
@@ -57,6 +59,13 @@ struct Device {
     int smem_optin = 0;      // max dynamic shared memory per block
     int cluster_ok = 0;
     int* status = nullptr;   // device status word
+    std::atomic<int> wait_polls{kDefaultWaitPolls};   // poll cap handed to the split-row kernel (lowered by the self-test only)
+    // scratch of the two-kernel paths (rows beyond a cluster's shared memory): grown on demand, kept,
+    // handed from call to call in stream order through scratch_ev, freed by fs_release
+    void* scratch = nullptr;
+    size_t scratch_bytes = 0;
+    cudaEvent_t scratch_ev = nullptr;
+    bool scratch_used = false;
     std::unordered_map<uint64_t, LaunchInfo> launch_cache;
     std::unordered_map<const void*, bool> configured;   // kernels whose function attributes are set
     // fs_softmax_host staging
@@ -71,6 +80,23 @@ struct Device {
 Device g_dev[kMaxDevices];
 std::mutex g_mu;          // guards g_dev[*].ready transitions and launch caches
 std::mutex g_host_mu;     // serialises fs_softmax_host / fs_release
+std::mutex g_scratch_mu;  // serialises the users of Device::scratch from acquire to event record
+
+// Environment switches, each read once per process.
+//   FS_LOG=1             one line per call on stderr: the dispatcher's decision and launch geometry
+//   FS_FORCE_KERNEL=name the kernel fs_softmax's dispatcher picks (warp, block, block_tma, cluster,
+//                        generic); a shape the forced kernel cannot run returns FS_ERR_UNSUPPORTED
+//   FS_CHECK=1           slow argument validation: every tensor pointer must be device-accessible
+//                        memory of the current device (cudaPointerGetAttributes)
+//   FS_SIM_NO_CLUSTER=1  behave as on a device without cluster launch (downgrade paths, tests)
+//   FS_SIM_SMEM_OPTIN=n  behave as on a device with n bytes of opt-in shared memory per block
+int env_int(const char* name, int dflt) {
+    const char* e = std::getenv(name);
+    return e && e[0] ? std::atoi(e) : dflt;
+}
+bool log_enabled() { static const bool v = env_int("FS_LOG", 0) != 0; return v; }
+bool check_enabled() { static const bool v = env_int("FS_CHECK", 0) != 0; return v; }
+#define FS_LOGF(...) do { if (log_enabled()) { std::fprintf(stderr, "[fsoftmax] " __VA_ARGS__); std::fputc('\n', stderr); } } while (0)
 
 int get_device(Device** out) {
     int d = 0;
@@ -83,8 +109,13 @@ int get_device(Device** out) {
             FS_CUDA(cudaDeviceGetAttribute(&dev.sm_count, cudaDevAttrMultiProcessorCount, d));
             FS_CUDA(cudaDeviceGetAttribute(&dev.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, d));
             FS_CUDA(cudaDeviceGetAttribute(&dev.cluster_ok, cudaDevAttrClusterLaunch, d));
+            if (env_int("FS_SIM_NO_CLUSTER", 0)) dev.cluster_ok = 0;
+            const int sim_smem = env_int("FS_SIM_SMEM_OPTIN", 0);
+            if (sim_smem > 0) dev.smem_optin = std::min(dev.smem_optin, std::max(sim_smem, 16 * 1024));
             FS_CUDA(cudaMalloc(&dev.status, sizeof(int)));
             FS_CUDA(cudaMemset(dev.status, 0, sizeof(int)));
+            FS_LOGF("device %d: %d SMs, %d B opt-in shared memory per block, cluster launch %s", d, dev.sm_count,
+                    dev.smem_optin, dev.cluster_ok ? "yes" : "no");
             dev.ready.store(true, std::memory_order_release);
         }
     }
@@ -94,15 +125,10 @@ int get_device(Device** out) {
 
 int elem_size(int dtype) { return dtype == FS_DTYPE_FP32 ? 4 : 2; }
 
-// Grid policy. The default is one block (or cluster) per unit of work, handed out by the hardware
-// block scheduler: measured on B200 a plain copy written that way runs ~10% faster than the same
-// copy with one resident block per slot looping over a fixed share of the data, because the
-// scheduler balances SMs that see different memory latencies. FS_PERSISTENT=1 (read once) selects
-// the resident-grid form, whose blocks prefetch their next rows through the shared-memory ring.
-bool persistent_grids() {
-    static const bool v = [] { const char* e = std::getenv("FS_PERSISTENT"); return e && e[0] == '1'; }();
-    return v;
-}
+// Grid policy: one block (or cluster) per unit of work, handed out by the hardware block scheduler.
+// Measured on B200, a plain copy written that way runs ~10% faster than the same copy with one
+// resident block per slot looping over a fixed share of the data, because the scheduler balances
+// SMs that see different memory latencies; the resident-grid forms of these kernels lost the same way.
 
 // ---------------------------------------------------------------------------------------------
 // shape -> kernel geometry (pure host arithmetic, no CUDA calls)
@@ -128,8 +154,8 @@ int64_t block_max_row_bytes(int) { return 8192; }
 int64_t block_tma_max_row_bytes(int dtype) { return dtype == FS_DTYPE_FP32 ? 32768 : 0; }
 int64_t split_slice_bytes(int) { return 32768; }
 constexpr int64_t kWarpTileMaxRowBytes = 4096;      // rows the warp-tile bulk-copy kernel takes
-constexpr int64_t kClusterSliceBytes = 32768;       // register-resident cluster kernel: slice per block
 constexpr int kMaxCluster = 16;
+constexpr int kSplitThreads = 256;                   // block size of the two-kernel (segment) path
 constexpr int64_t kTileBytes = 16384;               // rows per bulk copy of the warp-tile kernel
 
 int64_t warp_capacity_vecs(int dtype) { return 32 * int64_t(max_vpt(dtype)); }
@@ -168,21 +194,6 @@ bool block_geom(int64_t nvec, int dtype, int threads, BlockGeom* g) {
     return true;
 }
 
-struct ClusterGeom { int cs, slice; BlockGeom b; };
-bool cluster_geom(int64_t nvec, int dtype, int threads, int cluster, ClusterGeom* g) {
-    if (nvec < 1) return false;
-    int cs = cluster;
-    if (cs == 0) {
-        cs = 1;
-        while (cs < kMaxCluster && (nvec * 16 + cs - 1) / cs > kClusterSliceBytes) cs <<= 1;
-    }
-    if (cs != 1 && cs != 2 && cs != 4 && cs != 8 && cs != 16) return false;
-    const int64_t slice = (nvec + cs - 1) / cs;
-    if (slice > (int64_t(1) << 20) / 16 - 1) return false;   // mbarrier transaction-count range
-    g->cs = cs; g->slice = static_cast<int>(slice);
-    return block_geom(slice, dtype, threads, &g->b);
-}
-
 // Shared-memory-resident split: which cluster size and block size a row gets.
 //
 // What decides the speed of this kernel is how many bytes of rows an SM holds at a time (blocks per
@@ -213,7 +224,7 @@ double smem_geom_score(int64_t nvec, int dtype, const SmemGeom& g) {
     const bool full = nvec == int64_t(g.slice) * g.cs && g.slice % chunk == 0;
     const double stage = double(nch * chunk * 16);
     // dynamic part + the kernel's static shared memory (896 B) + the 1 KiB the hardware reserves per block
-    const double smem = stage + kSmemRowMaxChunks * 8 + kSmemRowMaxChunks * 4.0 * g.threads + 896 + 1024;
+    const double smem = stage + smem_row_tail_bytes(g.threads, int(nch)) + 896 + 1024;
     const int blocks = std::min(std::min(int(kSmemPerSm / smem), kSplitThreadsPerSm / g.threads), 32);
     if (blocks < 1) return 0.0;
     const double resident_cap = 184.0 * 1024;
@@ -259,11 +270,6 @@ bool smem_geom(int64_t nvec, int dtype, int threads, int cluster, SmemGeom* g) {
     return found;
 }
 
-bool cluster_uses_registers() {
-    static const bool v = [] { const char* e = std::getenv("FS_CLUSTER_REGS"); return e && e[0] == '1'; }();
-    return v;
-}
-
 bool fast_path_ok(int64_t cols, int dtype, int x_align, int y_align) {
     return x_align >= 16 && y_align >= 16 && (cols * elem_size(dtype)) % 16 == 0;
 }
@@ -272,12 +278,12 @@ int select_kernel(int64_t cols, int dtype, int x_align, int y_align) {
     if (!fast_path_ok(cols, dtype, x_align, y_align)) return FS_KERNEL_GENERIC;
     const int64_t row_bytes = cols * elem_size(dtype);
     const int64_t nvec = row_bytes / 16;
-    WarpGeom wg; BlockGeom bg; ClusterGeom cg;
+    WarpGeom wg; BlockGeom bg;
     if (row_bytes <= warp_max_row_bytes(dtype) && warp_geom(nvec, dtype, &wg)) return FS_KERNEL_WARP;
     if (row_bytes <= block_max_row_bytes(dtype) && block_geom(nvec, dtype, 0, &bg)) return FS_KERNEL_BLOCK;
     if (row_bytes <= block_tma_max_row_bytes(dtype) && block_geom(nvec, dtype, 0, &bg)) return FS_KERNEL_BLOCK_TMA;
     SmemGeom sg;
-    if (smem_geom(nvec, dtype, 0, 0, &sg) || cluster_geom(nvec, dtype, 0, 0, &cg)) return FS_KERNEL_CLUSTER;
+    if (smem_geom(nvec, dtype, 0, 0, &sg)) return FS_KERNEL_CLUSTER;
     return FS_KERNEL_GENERIC;
 }
 
@@ -419,6 +425,43 @@ int launch(const void* fn, int64_t grid, int threads, size_t smem, int cs, cudaS
     return FS_OK;
 }
 
+// ---- per-device scratch of the two-kernel paths ----------------------------------------------
+// The caller holds g_scratch_mu from scratch_acquire until scratch_done. The buffer is allocated on
+// first need and grown (never shrunk) when a call needs more; a call that fits allocates nothing.
+// Successive users are ordered on the device by an event: the next user's stream waits for the
+// previous user's last kernel. Inside a stream capture no event is waited for or recorded (the
+// captured work is ordered by the capture itself) and the buffer cannot grow: such a call returns
+// FS_ERR_UNSUPPORTED unless an earlier call outside the capture has already sized the buffer.
+int scratch_acquire(Device& dev, size_t bytes, cudaStream_t st, void** out, bool* capturing) {
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    FS_CUDA(cudaStreamIsCapturing(st, &cap));
+    *capturing = cap != cudaStreamCaptureStatusNone;
+    if (bytes > dev.scratch_bytes) {
+        if (*capturing) return FS_ERR_UNSUPPORTED;
+        if (dev.scratch) {
+            FS_CUDA(cudaDeviceSynchronize());          // earlier users have finished with the old buffer
+            FS_CUDA(cudaFree(dev.scratch));
+            dev.scratch = nullptr; dev.scratch_bytes = 0; dev.scratch_used = false;
+        }
+        const size_t want = (std::max<size_t>(bytes, size_t(1) << 20) + 0xfffff) & ~size_t(0xfffff);
+        FS_CUDA(cudaMalloc(&dev.scratch, want));
+        dev.scratch_bytes = want;
+        FS_LOGF("scratch buffer grown to %zu bytes", want);
+        if (!dev.scratch_ev) FS_CUDA(cudaEventCreateWithFlags(&dev.scratch_ev, cudaEventDisableTiming));
+    } else if (!*capturing && dev.scratch_used) {
+        FS_CUDA(cudaStreamWaitEvent(st, dev.scratch_ev, 0));
+    }
+    *out = dev.scratch;
+    return FS_OK;
+}
+
+int scratch_done(Device& dev, cudaStream_t st, bool capturing) {
+    if (capturing) return FS_OK;
+    FS_CUDA(cudaEventRecord(dev.scratch_ev, st));
+    dev.scratch_used = true;
+    return FS_OK;
+}
+
 // ---- kernel tables --------------------------------------------------------------------------
 
 template <int DT, bool NEG> const void* warp_fn(const WarpGeom& g) {
@@ -476,7 +519,6 @@ template <int DT, bool NEG> const void* warp_tma_fn(const WarpGeom& g) {
     }
 FS_VPT_TABLE(block_fn, block_row_kernel)
 FS_VPT_TABLE(block_tma_fn, block_row_tma_kernel)
-FS_VPT_TABLE(cluster_fn, cluster_row_kernel)
 
 template <int DT> const void* router_fn(const WarpGeom& g) {
     if (g.vpl == 1) return (const void*)router_topk_kernel<DT, 1, 1>;
@@ -547,39 +589,53 @@ const void* smem_row_fn(int dtype, bool neg, const SmemGeom& g, int64_t nvec) {
         return full ? (const void*)smem_row_kernel<DT, NG, true, false> : (const void*)smem_row_kernel<DT, NG, false, false>;
     });
 }
-// slice rounded up to whole chunks | chunk mbarriers | per-thread chunk references
+// slice rounded up to whole chunks | (warp, chunk) mbarriers | per-thread chunk references
 size_t smem_row_stage_bytes(const SmemGeom& g, int dtype) {
     return static_cast<size_t>(smem_row_nchunk(g, dtype)) * smem_row_u(dtype) * g.threads * 16;
 }
 size_t smem_row_bytes(const SmemGeom& g, int dtype) {
-    return smem_row_stage_bytes(g, dtype) + size_t(kSmemRowMaxChunks) * 8 + size_t(kSmemRowMaxChunks) * g.threads * 4;
+    return smem_row_stage_bytes(g, dtype) + smem_row_tail_bytes(g.threads, smem_row_nchunk(g, dtype));
 }
 
-// Shared-memory ring: as many stages as fit in `budget` bytes, between 2 and `max_stages`.
-int ring_stages(size_t stage_bytes, size_t budget, int max_stages) {
-    int n = static_cast<int>(budget / (stage_bytes + 8));
-    if (n > max_stages) n = max_stages;
-    return n;
+// FS_FORCE_KERNEL (read once): a kernel name or number that replaces the dispatcher's choice.
+int forced_kernel() {
+    static const int v = [] {
+        const char* e = std::getenv("FS_FORCE_KERNEL");
+        if (!e || !e[0]) return int(FS_KERNEL_AUTO);
+        static const char* names[] = {"auto", "warp", "block", "block_tma", "cluster", "generic"};
+        for (int k = 0; k <= FS_KERNEL_GENERIC; ++k)
+            if (std::strcmp(e, names[k]) == 0) return k;
+        const int k = std::atoi(e);
+        return k >= FS_KERNEL_AUTO && k <= FS_KERNEL_GENERIC ? k : int(FS_KERNEL_AUTO);
+    }();
+    return v;
 }
 
 // Rows longer than a cluster's shared memory: segments over a grid that fills the GPU, the
-// (reference, sum) pairs of the segments exchanged through a stream-ordered scratch buffer.
-int run_softmax_split(Device& dev, const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale, cudaStream_t st) {
+// (reference, sum) pairs of the segments exchanged through the per-device scratch buffer.
+struct SplitPlan { LsmParams p; int64_t nseg, seg_vecs; };
+bool softmax_split_plan(int sm_count, int* status, const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale,
+                        SplitPlan* out) {
     LsmParams p{};
     p.x = x; p.y = y; p.rows = rows; p.cols = cols;
     p.nvec = cols * elem_size(dtype) / 16;
     p.scale = std::fabs(scale);
     p.c = static_cast<float>(static_cast<double>(p.scale) * kLog2e);
     p.flip = std::signbit(scale) && scale != 0.0f ? (dtype == FS_DTYPE_FP32 ? 0x80000000u : 0x80008000u) : 0u;
-    p.status = dev.status; p.pf_rows = 0;
-    const int t = 256;
-    const int64_t target = int64_t(dev.sm_count) * 8;
+    p.status = status; p.pf_rows = 0;
+    const int t = kSplitThreads;
+    const int64_t target = int64_t(sm_count) * 8;
     int64_t nseg = std::max<int64_t>(1, std::min<int64_t>(1024, (target + rows - 1) / rows));
     const int64_t seg_vecs = ((p.nvec + nseg - 1) / nseg + 4 * t - 1) / (4 * t) * (4 * t);
     nseg = (p.nvec + seg_vecs - 1) / seg_vecs;
-    if (rows * nseg > 0x7fffffff || seg_vecs > 0x7fffffff) return FS_ERR_UNSUPPORTED;
-    float2* part = nullptr;
-    FS_CUDA(cudaMallocAsync(reinterpret_cast<void**>(&part), static_cast<size_t>(rows * nseg) * sizeof(float2), st));
+    if (rows * nseg > 0x7fffffff || seg_vecs > 0x7fffffff) return false;
+    out->p = p; out->nseg = nseg; out->seg_vecs = seg_vecs;
+    return true;
+}
+
+// The two launches; `part` holds rows * nseg (reference, sum) pairs, every one written by the first
+// kernel before the second reads it.
+int softmax_split_launch(const SplitPlan& sp, int dtype, float2* part, cudaStream_t st) {
     const void* f1 = nullptr;
     const void* f2 = nullptr;
     switch (dtype) {
@@ -588,15 +644,29 @@ int run_softmax_split(Device& dev, const void* x, void* y, int64_t rows, int64_t
         default:            f1 = (const void*)sm_partial_kernel<DT_F16>; f2 = (const void*)sm_apply_kernel<DT_F16>; break;
     }
     const float2* cpart = part;
-    int rc = launch(f1, rows * nseg, t, 0, 0, st, p, part, static_cast<int>(nseg), static_cast<int>(seg_vecs));
-    if (rc == FS_OK) rc = launch(f2, rows * nseg, t, 0, 0, st, p, cpart, static_cast<int>(nseg), static_cast<int>(seg_vecs));
-    const cudaError_t fe = cudaFreeAsync(part, st);
-    if (rc == FS_OK && fe != cudaSuccess) return cuda_fail(fe);
+    FS_LOGF("softmax %lld x %lld dtype %d: two kernels over %lld segments of %lld vectors per row", (long long)sp.p.rows,
+            (long long)sp.p.cols, dtype, (long long)sp.nseg, (long long)sp.seg_vecs);
+    int rc = launch(f1, sp.p.rows * sp.nseg, kSplitThreads, 0, 0, st, sp.p, part, static_cast<int>(sp.nseg), static_cast<int>(sp.seg_vecs));
+    if (rc == FS_OK)
+        rc = launch(f2, sp.p.rows * sp.nseg, kSplitThreads, 0, 0, st, sp.p, cpart, static_cast<int>(sp.nseg), static_cast<int>(sp.seg_vecs));
     return rc;
 }
 
+int run_softmax_split(Device& dev, const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale, cudaStream_t st) {
+    SplitPlan sp;
+    if (!softmax_split_plan(dev.sm_count, dev.status, x, y, rows, cols, dtype, scale, &sp)) return FS_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lk(g_scratch_mu);
+    void* buf = nullptr;
+    bool capturing = false;
+    int rc = scratch_acquire(dev, static_cast<size_t>(rows * sp.nseg) * sizeof(float2), st, &buf, &capturing);
+    if (rc != FS_OK) return rc;
+    rc = softmax_split_launch(sp, dtype, static_cast<float2*>(buf), st);
+    const int rd = scratch_done(dev, st, capturing);
+    return rc != FS_OK ? rc : rd;
+}
+
 int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale, cudaStream_t st,
-        int kernel, int threads, int cluster) {
+        int kernel, int threads, int cluster, uint32_t dbg_extra_tx = 0u) {
     Device* devp = nullptr;
     int rc = get_device(&devp);
     if (rc != FS_OK) return rc;
@@ -604,8 +674,14 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
 
     const int esz = elem_size(dtype);
     const bool fast = fast_path_ok(cols, dtype, ptr_align(x), ptr_align(y));
-    const bool was_auto = kernel == FS_KERNEL_AUTO;
-    if (was_auto) kernel = select_kernel(cols, dtype, ptr_align(x), ptr_align(y));
+    // The dispatcher's own choice may be downgraded when the device cannot run it (no cluster launch,
+    // too little shared memory); a kernel forced by the caller or by FS_FORCE_KERNEL never is.
+    bool was_auto = kernel == FS_KERNEL_AUTO;
+    if (was_auto) {
+        const int forced = forced_kernel();
+        if (forced != FS_KERNEL_AUTO) { kernel = forced; was_auto = false; }
+        else kernel = select_kernel(cols, dtype, ptr_align(x), ptr_align(y));
+    }
     if (kernel != FS_KERNEL_GENERIC && !fast) return FS_ERR_UNSUPPORTED;
     if (threads < 0 || threads % 32 || threads > 1024) return FS_ERR_INVALID_ARG;
 
@@ -617,7 +693,22 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
     p.status = dev.status;
     p.q_offset = 0;
     p.pf_rows = 0;
+    p.dbg_extra_tx = dbg_extra_tx;
+    p.wait_polls = dev.wait_polls.load(std::memory_order_relaxed);
     const int64_t max_grid = 0x7fffffff;
+
+    // One block per row with element-wise accesses; vector-aligned rows of 1 MiB or more that no
+    // cluster holds (the dispatcher's own choice only) are cut into segments over two kernels instead.
+    const auto run_generic = [&](bool allow_split, int t) -> int {
+        if (allow_split && fast && cols * esz >= (int64_t(1) << 20)) return run_softmax_split(dev, x, y, rows, cols, dtype, scale, st);
+        const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) { return (const void*)generic_row_kernel<decltype(dt)::value, decltype(ng)::value, false>; });
+        if (t == 0) {
+            t = 32;
+            while (t < 1024 && cols > int64_t(t) * 8) t <<= 1;
+        }
+        FS_LOGF("softmax %lld x %lld dtype %d: generic kernel, %d threads per row", (long long)rows, (long long)cols, dtype, t);
+        return launch(fn, std::min<int64_t>(rows, max_grid), t, 0, 0, st, p);
+    };
 
     switch (kernel) {
         case FS_KERNEL_WARP: {
@@ -629,12 +720,9 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
             if (t > 256) return FS_ERR_UNSUPPORTED;
             const int64_t rows_per_tile = int64_t(32 / g.lanes) * g.r;
             const int64_t tiles = (rows + rows_per_tile - 1) / rows_per_tile;
-            int64_t grid = std::min<int64_t>((tiles + (t / 32) - 1) / (t / 32), max_grid);
-            if (persistent_grids()) {
-                int bps = 0;
-                if ((rc = blocks_per_sm(dev, fn, t, 0, &bps)) != FS_OK) return rc;
-                grid = std::min<int64_t>(grid, int64_t(dev.sm_count) * bps);
-            }
+            const int64_t grid = std::min<int64_t>((tiles + (t / 32) - 1) / (t / 32), max_grid);
+            FS_LOGF("softmax %lld x %lld dtype %d: warp kernel, %d lanes x %d vectors per row, %d rows per group, grid %lld x %d",
+                    (long long)rows, (long long)cols, dtype, g.lanes, g.vpl, g.r, (long long)grid, t);
             return launch(fn, grid, t, 0, 0, st, p);
         }
         case FS_KERNEL_BLOCK: {
@@ -642,11 +730,12 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
             if (!block_geom(p.nvec, dtype, threads, &g)) return FS_ERR_UNSUPPORTED;
             const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) { return block_fn<decltype(dt)::value, decltype(ng)::value>(g.vpt); });
             if (!fn) return FS_ERR_UNSUPPORTED;
-            int64_t grid = std::min<int64_t>(rows, max_grid);
+            const int64_t grid = std::min<int64_t>(rows, max_grid);
             int bps = 0;
             if ((rc = blocks_per_sm(dev, fn, g.threads, 0, &bps)) != FS_OK) return rc;
-            if (persistent_grids()) grid = std::min<int64_t>(grid, int64_t(dev.sm_count) * bps);
-            else p.pf_rows = prefetch_rows(dev.sm_count * bps);
+            p.pf_rows = prefetch_rows(dev.sm_count * bps);
+            FS_LOGF("softmax %lld x %lld dtype %d: block kernel, %d threads x %d vectors, %d blocks per SM", (long long)rows,
+                    (long long)cols, dtype, g.threads, g.vpt, bps);
             return launch(fn, grid, g.threads, 0, 0, st, p);
         }
         case FS_KERNEL_BLOCK_TMA: {
@@ -669,8 +758,9 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
                 int bps = 0;
                 if ((rc = blocks_per_sm(dev, fn, t, smem, &bps)) != FS_OK) return rc;
                 const int64_t tiles = (rows + tile_rows - 1) / tile_rows;
-                int64_t grid = std::min<int64_t>(tiles, max_grid);
-                if (persistent_grids()) grid = std::min<int64_t>(grid, int64_t(dev.sm_count) * bps);
+                const int64_t grid = std::min<int64_t>(tiles, max_grid);
+                FS_LOGF("softmax %lld x %lld dtype %d: warp kernel fed by bulk copies, tiles of %lld rows", (long long)rows,
+                        (long long)cols, dtype, (long long)tile_rows);
                 return launch(fn, grid, t, smem, 0, st, p, static_cast<int>(tile_rows), static_cast<uint32_t>(tile_bytes));
             }
             BlockGeom g;
@@ -679,27 +769,31 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
             if (!fn) return FS_ERR_UNSUPPORTED;
             const size_t stage_bytes = static_cast<size_t>(p.nvec) * 16;
             if (stage_bytes > (size_t(1) << 20) - 16) return FS_ERR_UNSUPPORTED;
-            int nstage = 1;
-            if (persistent_grids()) {
-                // aim at ~2048 resident threads per SM, and give each block its share of shared memory
-                const int want_bps = std::max(1, 2048 / g.threads);
-                const size_t budget = std::min<size_t>(smem_cap, (size_t(dev.smem_optin) + 1024) / want_bps - 2048);
-                nstage = ring_stages(stage_bytes, budget, 8);
-                if (nstage < 2) nstage = ring_stages(stage_bytes, smem_cap, 2);
+            const int nstage = 1;                   // one row per block: a single stage
+            if (stage_bytes + 8 > smem_cap) {
+                if (!was_auto) return FS_ERR_UNSUPPORTED;
+                FS_LOGF("softmax: a %zu B row exceeds the device's shared memory per block: generic path", stage_bytes);
+                return run_generic(false, 0);
             }
-            if (stage_bytes + 8 > smem_cap) return FS_ERR_UNSUPPORTED;
             const size_t smem = nstage * stage_bytes + size_t(nstage) * 8;
             int bps = 0;
             if ((rc = blocks_per_sm(dev, fn, g.threads, smem, &bps)) != FS_OK) return rc;
-            int64_t grid = std::min<int64_t>(rows, max_grid);
-            if (persistent_grids()) grid = std::min<int64_t>(grid, int64_t(dev.sm_count) * bps);
-            else set_first_wave_lag(p, dev.sm_count * bps, p.nvec * 16);
+            const int64_t grid = std::min<int64_t>(rows, max_grid);
+            set_first_wave_lag(p, dev.sm_count * bps, p.nvec * 16);
+            FS_LOGF("softmax %lld x %lld dtype %d: block kernel fed by bulk copies, %d threads x %d vectors, %d blocks per SM",
+                    (long long)rows, (long long)cols, dtype, g.threads, g.vpt, bps);
             return launch(fn, grid, g.threads, smem, 0, st, p, nstage, static_cast<uint32_t>(stage_bytes));
         }
         case FS_KERNEL_CLUSTER: {
-            if (!dev.cluster_ok) return FS_ERR_UNSUPPORTED;
+            // A device without cluster launch still runs the one-block form (cluster size 1) on rows
+            // that fit one block's shared memory; the dispatcher sends everything else to the generic
+            // kernels then, and does the same when the device's shared memory is too small.
+            if (!dev.cluster_ok) {
+                if (cluster > 1 || (!was_auto && cluster == 0)) return FS_ERR_UNSUPPORTED;
+                cluster = 1;
+            }
             SmemGeom sg;
-            if (!cluster_uses_registers() && smem_geom(p.nvec, dtype, threads, cluster, &sg)) {
+            if (smem_geom(p.nvec, dtype, threads, cluster, &sg)) {
                 // a slice that is not a whole number of chunks is padded with -inf, which a zero
                 // scale would turn into NaN: that one case goes to the generic kernel
                 const bool zero_scale_ragged = p.c == 0.0f && !smem_row_full(sg, dtype, p.nvec);
@@ -708,54 +802,37 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
                     const void* fn = smem_row_fn(dtype, p.neg, sg, p.nvec);
                     const size_t stage_bytes = smem_row_stage_bytes(sg, dtype);
                     const size_t smem = smem_row_bytes(sg, dtype);
-                    if (smem > static_cast<size_t>(dev.smem_optin) - 2048) return FS_ERR_UNSUPPORTED;
+                    if (smem > static_cast<size_t>(dev.smem_optin) - 2048) {
+                        if (!was_auto) return FS_ERR_UNSUPPORTED;
+                        FS_LOGF("softmax: %zu B of shared memory per block exceed the device's limit: generic path", smem);
+                        return run_generic(true, 0);
+                    }
                     int ncl = 0;
-                    if ((rc = active_clusters(dev, fn, sg.threads, smem, sg.cs, &ncl)) != FS_OK) return rc;
-                    int64_t clusters = std::min<int64_t>(rows, max_grid / sg.cs);
-                    if (persistent_grids()) clusters = std::min<int64_t>(clusters, ncl);
-                    else p.pf_rows = prefetch_rows(ncl);
+                    if (dev.cluster_ok) {
+                        if ((rc = active_clusters(dev, fn, sg.threads, smem, sg.cs, &ncl)) != FS_OK) return rc;
+                    } else {                       // plain launch of the one-block form
+                        if ((rc = blocks_per_sm(dev, fn, sg.threads, smem, &ncl)) != FS_OK) return rc;
+                        ncl *= dev.sm_count;
+                    }
+                    const int64_t clusters = std::min<int64_t>(rows, max_grid / sg.cs);
+                    p.pf_rows = prefetch_rows(ncl);
                     set_first_wave_lag(p, ncl, p.nvec * 16);
-                    return launch(fn, clusters * sg.cs, sg.threads, smem, sg.cs, st, p,
+                    FS_LOGF("softmax %lld x %lld dtype %d: split-row kernel, %d blocks per row x %d threads, slice %d B, %zu B shared, "
+                            "%d resident clusters", (long long)rows, (long long)cols, dtype, sg.cs, sg.threads, sg.slice * 16, smem, ncl);
+                    return launch(fn, clusters * sg.cs, sg.threads, smem, dev.cluster_ok ? sg.cs : 0, st, p,
                                   static_cast<uint32_t>(stage_bytes), sg.slice, smem_row_nchunk(sg, dtype));
                 }
-                return run(x, y, rows, cols, dtype, scale, st, FS_KERNEL_GENERIC, 0, 0);
+                return run_generic(false, 0);
             }
-            ClusterGeom g;
-            if (!cluster_geom(p.nvec, dtype, threads, cluster, &g)) return FS_ERR_UNSUPPORTED;
-            const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) { return cluster_fn<decltype(dt)::value, decltype(ng)::value>(g.b.vpt); });
-            if (!fn) return FS_ERR_UNSUPPORTED;
-            const size_t stage_bytes = static_cast<size_t>(g.slice) * 16;
-            const size_t smem_cap = static_cast<size_t>(dev.smem_optin) - 2048;
-            int nstage = 1;
-            if (persistent_grids()) {
-                const int want_bps = std::max(1, 2048 / g.b.threads);
-                const size_t budget = std::min<size_t>(smem_cap, (size_t(dev.smem_optin) + 1024) / want_bps - 2048);
-                nstage = ring_stages(stage_bytes, budget, 4);
-                if (nstage < 2) nstage = ring_stages(stage_bytes, smem_cap, 2);
+            if (!dev.cluster_ok) {
+                if (!was_auto) return FS_ERR_UNSUPPORTED;
+                FS_LOGF("softmax: no cluster launch on this device and the row does not fit one block: generic path");
+                return run_generic(true, 0);
             }
-            if (stage_bytes + 8 > smem_cap) return FS_ERR_UNSUPPORTED;
-            const size_t smem = nstage * stage_bytes + size_t(nstage) * 8;
-            int ncl = 0;
-            if ((rc = active_clusters(dev, fn, g.b.threads, smem, g.cs, &ncl)) != FS_OK) return rc;
-            int64_t clusters = std::min<int64_t>(rows, max_grid / g.cs);
-            if (persistent_grids()) clusters = std::min<int64_t>(clusters, ncl);
-            return launch(fn, clusters * g.cs, g.b.threads, smem, g.cs, st, p, nstage,
-                          static_cast<uint32_t>(stage_bytes), g.slice);
+            return FS_ERR_UNSUPPORTED;           // no geometry holds this row in a cluster's shared memory
         }
-        case FS_KERNEL_GENERIC: {
-            // vector-aligned rows that no cluster holds (the dispatcher's own choice only): rows cut
-            // into segments over two kernels instead of one block per row
-            if (was_auto && fast_path_ok(cols, dtype, ptr_align(x), ptr_align(y)) && cols * elem_size(dtype) >= (int64_t(1) << 20))
-                return run_softmax_split(dev, x, y, rows, cols, dtype, scale, st);
-            const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) { return (const void*)generic_row_kernel<decltype(dt)::value, decltype(ng)::value, false>; });
-            int t = threads;
-            if (t == 0) {
-                t = 32;
-                while (t < 1024 && cols > int64_t(t) * 8) t <<= 1;
-            }
-            const int64_t grid = std::min<int64_t>(rows, max_grid);
-            return launch(fn, grid, t, 0, 0, st, p);
-        }
+        case FS_KERNEL_GENERIC:
+            return run_generic(was_auto, threads);
         default:
             return FS_ERR_INVALID_ARG;
     }
@@ -779,6 +856,7 @@ int run_causal(const void* x, void* y, int64_t rows, int64_t cols, int64_t q_off
     p.status = dev.status;
     p.q_offset = q_offset;
     p.pf_rows = 0;
+    p.wait_polls = kDefaultWaitPolls;
     SmemGeom sg;
     // (a zero scale goes to the generic kernel: the split kernel masks with -inf, and 0 * -inf is NaN)
     if (fast && p.c != 0.0f && dev.cluster_ok && smem_geom(p.nvec, dtype, 0, 0, &sg) && rows <= 0x7fffffff / sg.cs) {
@@ -815,25 +893,48 @@ int validate(const void* x, const void* y, int64_t rows, int64_t cols, int dtype
     return FS_OK;
 }
 
+// FS_CHECK=1: every tensor pointer must be memory the current device can address (device or managed
+// memory of this device, or mapped pinned host memory). One driver query per pointer: slow, off by default.
+int check_ptrs(std::initializer_list<const void*> ptrs) {
+    if (!check_enabled()) return FS_OK;
+    int d = 0;
+    FS_CUDA(cudaGetDevice(&d));
+    for (const void* q : ptrs) {
+        if (!q) continue;
+        cudaPointerAttributes a{};
+        FS_CUDA(cudaPointerGetAttributes(&a, q));
+        const bool ok = (a.type == cudaMemoryTypeDevice && a.device == d) || a.type == cudaMemoryTypeManaged ||
+                        (a.type == cudaMemoryTypeHost && a.devicePointer != nullptr);
+        if (!ok) {
+            FS_LOGF("FS_CHECK: %p is not addressable by device %d (memory type %d, device %d)", q, d, int(a.type), a.device);
+            return FS_ERR_INVALID_ARG;
+        }
+    }
+    return FS_OK;
+}
+#define FS_CHECK_PTRS(...) do { const int c__ = check_ptrs({__VA_ARGS__}); if (c__ != FS_OK) return c__; } while (0)
+
 }  // namespace
 
 // ---------------------------------------------------------------------------------------------
-// fs_softmax_static: the split-row kernel with its scratch in a fixed device array
+// fs_softmax_static: scratch in a fixed device array instead of allocated memory
 // ---------------------------------------------------------------------------------------------
-// The split-row kernel records an expired bounded wait in a status word in global memory. The
-// other entry points keep that word in a buffer obtained with cudaMalloc on first use; this one
-// keeps it in the array below, which is part of the loaded module: 256 bytes on every GPU that
-// loads the library, held until the process exits. Word 0 is the status word, the rest is unused.
-// In host code the array's name is only a handle for the runtime, not a device address: the
-// address a kernel can use comes from cudaGetSymbolAddress, asked once per device with that device
-// current.
-constexpr int kStaticScratchWords = 64;
+// Two things the other entry points keep in memory from cudaMalloc live in the array below, which is
+// part of the loaded module (FS_STATIC_SCRATCH_BYTES on every GPU that loads the library, held until
+// the process exits): the status word of the bounded waits (word 0), and, from byte 256 on, the
+// (reference, sum) pairs that the two kernels of the long-row path hand to each other. In host code the array's name is only a handle for the runtime, not a device
+// address: the address a kernel can use comes from cudaGetSymbolAddress, asked once per device with
+// that device current.
+constexpr int kStaticScratchWords = FS_STATIC_SCRATCH_BYTES / 4;
+constexpr int kStaticPairOffsetWords = 64;                       // pairs start 256 bytes in
+static_assert((kStaticScratchWords - kStaticPairOffsetWords) / 2 == FS_STATIC_MAX_PAIRS, "header and array disagree");
 static __device__ __align__(256) int fs_static_scratch[kStaticScratchWords];
 
 namespace {
 
 struct StaticDevice {
     bool ready = false;
+    int sm_count = 0;
     int smem_optin = 0;
     int cluster_ok = 0;
     int* scratch = nullptr;              // device address of fs_static_scratch on this device
@@ -841,6 +942,25 @@ struct StaticDevice {
 };
 StaticDevice g_static[kMaxDevices];
 std::mutex g_static_mu;
+
+// First use on a device: queries and the symbol's address, no allocation.
+int get_static_device(StaticDevice** out) {
+    int d = 0;
+    FS_CUDA(cudaGetDevice(&d));
+    if (d < 0 || d >= kMaxDevices) return FS_ERR_UNSUPPORTED;
+    StaticDevice& sd = g_static[d];
+    if (!sd.ready) {
+        FS_CUDA(cudaDeviceGetAttribute(&sd.sm_count, cudaDevAttrMultiProcessorCount, d));
+        FS_CUDA(cudaDeviceGetAttribute(&sd.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, d));
+        FS_CUDA(cudaDeviceGetAttribute(&sd.cluster_ok, cudaDevAttrClusterLaunch, d));
+        void* addr = nullptr;
+        FS_CUDA(cudaGetSymbolAddress(&addr, fs_static_scratch));
+        sd.scratch = static_cast<int*>(addr);
+        sd.ready = true;
+    }
+    *out = &sd;
+    return FS_OK;
+}
 
 }  // namespace
 
@@ -1040,8 +1160,8 @@ int run_norm(const void* x, const void* gamma, const void* beta, void* y, int64_
     const bool smem_ok = fast && dev.cluster_ok && smem_geom(p.nvec, dtype, 0, 0, &sg) && rows <= 0x7fffffff / sg.cs;
     // Few, very long rows (group_norm of a large image): a cluster per row leaves most of the GPU
     // idle, or the row does not fit a cluster's shared memory at all. Then the rows are cut into
-    // segments over a grid that fills the GPU, with the partial statistics exchanged through a
-    // stream-ordered scratch buffer between two kernels.
+    // segments over a grid that fills the GPU, with the partial statistics exchanged through the
+    // per-device scratch buffer between two kernels.
     if (fast && norm_split_wanted(dev, rows, p.nvec, smem_ok, smem_ok ? sg.cs : 0)) {
         const int t = 256;
         const int64_t target = int64_t(dev.sm_count) * 8;
@@ -1049,16 +1169,18 @@ int run_norm(const void* x, const void* gamma, const void* beta, void* y, int64_
         int64_t seg_vecs = ((p.nvec + nseg - 1) / nseg + 4 * t - 1) / (4 * t) * (4 * t);
         nseg = (p.nvec + seg_vecs - 1) / seg_vecs;
         if (rows * nseg <= 0x7fffffff) {
-            float4* part = nullptr;
-            FS_CUDA(cudaMallocAsync(reinterpret_cast<void**>(&part), static_cast<size_t>(rows * nseg) * sizeof(float4), st));
+            std::lock_guard<std::mutex> lk(g_scratch_mu);
+            void* buf = nullptr;
+            bool capturing = false;
+            if ((rc = scratch_acquire(dev, static_cast<size_t>(rows * nseg) * sizeof(float4), st, &buf, &capturing)) != FS_OK) return rc;
+            float4* part = static_cast<float4*>(buf);
             const void* f1 = by_dtype(dtype, [&](auto dt) -> const void* { return (const void*)norm_partial_kernel<decltype(dt)::value>; });
             const void* f2 = by_dtype(dtype, [&](auto dt) -> const void* { return norm_apply_fn<decltype(dt)::value>(aff); });
             const float4* cpart = part;
             rc = launch(f1, rows * nseg, t, 0, 0, st, p, part, static_cast<int>(nseg), static_cast<int>(seg_vecs));
             if (rc == FS_OK) rc = launch(f2, rows * nseg, t, 0, 0, st, p, cpart, static_cast<int>(nseg), static_cast<int>(seg_vecs));
-            const cudaError_t fe = cudaFreeAsync(part, st);
-            if (rc == FS_OK && fe != cudaSuccess) return cuda_fail(fe);
-            return rc;
+            const int rd = scratch_done(dev, st, capturing);
+            return rc != FS_OK ? rc : rd;
         }
     }
     if (smem_ok) {
@@ -1413,6 +1535,7 @@ int fs_softmax_ex(const void* x, void* y, int64_t rows, int64_t cols, int dtype,
     if (kernel < FS_KERNEL_AUTO || kernel > FS_KERNEL_GENERIC) return FS_ERR_INVALID_ARG;
     if (cluster < 0 || cluster > kMaxCluster) return FS_ERR_INVALID_ARG;
     if (rows == 0 || cols == 0) return FS_OK;
+    FS_CHECK_PTRS(x, y);
     return run(x, y, rows, cols, dtype, scale, static_cast<cudaStream_t>(stream), kernel, threads, cluster);
 }
 
@@ -1426,6 +1549,7 @@ int fs_softmax_causal(const void* x, void* y, int64_t rows, int64_t cols, int64_
     if (v != FS_OK) return v;
     if (rows == 0 || cols == 0) return FS_OK;
     if (q_offset > (int64_t(1) << 41) || q_offset < -(int64_t(1) << 41)) return FS_ERR_INVALID_ARG;
+    FS_CHECK_PTRS(x, y);
     return run_causal(x, y, rows, cols, q_offset, dtype, scale, static_cast<cudaStream_t>(stream));
 }
 
@@ -1440,15 +1564,17 @@ int fs_router_topk(const void* x, float* w, int32_t* idx, int64_t rows, int64_t 
     if (rows > (int64_t(1) << 40)) return FS_ERR_INVALID_ARG;
     if (ptr_align(x) < 16 || (cols * elem_size(dtype)) % 16 != 0) return FS_ERR_UNSUPPORTED;
     if (ptr_align(w) < 4 || ptr_align(idx) < 4) return FS_ERR_INVALID_ARG;
+    FS_CHECK_PTRS(x, w, idx);
     const int64_t nvec = cols * elem_size(dtype) / 16;
     WarpGeom g;
     if (!warp_geom(nvec, dtype, &g) || g.vpl * (dtype == FS_DTYPE_FP32 ? 4 : 8) > 32) return FS_ERR_UNSUPPORTED;
     Device* dev = nullptr;
     int rc = get_device(&dev);
     if (rc != FS_OK) return rc;
-    // k <= 8 selects with sorting networks in registers (FS_ROUTER_ROUNDS=1, read per call, keeps the
+    // k <= 8 selects with sorting networks in registers (FS_ROUTER_ROUNDS=1, read once, keeps the
     // kernel that takes one maximum per round, which serves any k)
-    const bool net = k <= 8 && !std::getenv("FS_ROUTER_ROUNDS");
+    static const bool rounds_only = env_int("FS_ROUTER_ROUNDS", 0) != 0;
+    const bool net = k <= 8 && !rounds_only;
     const void* fn = nullptr;
     switch (dtype) {
         case FS_DTYPE_FP32: fn = net ? router8_fn<DT_F32>(g) : router_fn<DT_F32>(g); break;
@@ -1471,6 +1597,7 @@ int fs_log_softmax(const void* x, void* y, int64_t rows, int64_t cols, int dtype
     const int v = validate(x, y, rows, cols, dtype, scale);
     if (v != FS_OK) return v;
     if (rows == 0 || cols == 0) return FS_OK;
+    FS_CHECK_PTRS(x, y);
     return run_log_softmax(x, y, rows, cols, dtype, scale, OUT_LOG, static_cast<cudaStream_t>(stream));
 }
 
@@ -1482,6 +1609,7 @@ int fs_softmax_masked(const void* x, const void* mask, void* y, int64_t rows, in
     if (rows % (q_rows * heads) != 0) return FS_ERR_INVALID_ARG;
     if (rows == 0 || cols == 0) return FS_OK;
     if (!mask) return FS_ERR_INVALID_ARG;
+    FS_CHECK_PTRS(x, mask, y);
     return run_softmax_masked(x, mask, y, rows, cols, q_rows, heads, dtype, scale, static_cast<cudaStream_t>(stream));
 }
 
@@ -1491,6 +1619,7 @@ int fs_softmax_backward(const void* dy, const void* y, void* dx, int64_t rows, i
     if (v == FS_OK) v = validate(y, dx, rows, cols, dtype, scale);
     if (v != FS_OK) return v;
     if (rows == 0 || cols == 0) return FS_OK;
+    FS_CHECK_PTRS(dy, y, dx);
     return run_softmax_backward(dy, y, dx, rows, cols, dtype, scale, static_cast<cudaStream_t>(stream));
 }
 
@@ -1504,6 +1633,7 @@ int fs_softmax_f32out(const void* x, float* y, int64_t rows, int64_t cols, int d
     const uintptr_t a = reinterpret_cast<uintptr_t>(x), b = reinterpret_cast<uintptr_t>(y);
     const uintptr_t na = static_cast<uintptr_t>(rows * cols * 2), nb = static_cast<uintptr_t>(rows * cols * 4);
     if (a < b + nb && b < a + na) return FS_ERR_INVALID_ARG;          // the tensors differ in size: no overlap at all
+    FS_CHECK_PTRS(x, y);
     return run_log_softmax(x, y, rows, cols, dtype, scale, OUT_PROB32, static_cast<cudaStream_t>(stream));
 }
 
@@ -1512,6 +1642,7 @@ int fs_layer_norm(const void* x, const void* gamma, const void* beta, void* y, i
     const int v = validate_norm(x, y, rows, cols, dtype, eps);
     if (v != FS_OK || rows == 0 || cols == 0) return v;
     const int aff = (gamma || beta) ? 1 : 0;
+    FS_CHECK_PTRS(x, gamma, beta, y);
     return run_norm(x, gamma, beta, y, rows, cols, dtype, eps, aff, 1, 1, static_cast<cudaStream_t>(stream));
 }
 
@@ -1526,6 +1657,7 @@ int fs_group_norm(const void* x, const void* gamma, const void* beta, void* y, i
     const int v = validate_norm(x, y, rows, cols, dtype, eps);
     if (v != FS_OK || rows == 0 || cols == 0) return v;
     const int aff = (gamma || beta) ? 2 : 0;
+    FS_CHECK_PTRS(x, gamma, beta, y);
     return run_norm(x, gamma, beta, y, rows, cols, dtype, eps, aff, spatial, groups, static_cast<cudaStream_t>(stream));
 }
 
@@ -1549,6 +1681,7 @@ int fs_copy(const void* x, void* y, int64_t bytes, void* stream) {
     if (bytes < 0 || bytes % 16) return FS_ERR_INVALID_ARG;
     if (bytes == 0) return FS_OK;
     if (!x || !y || ptr_align(x) < 16 || ptr_align(y) < 16) return FS_ERR_INVALID_ARG;
+    FS_CHECK_PTRS(x, y);
     Device* dev = nullptr;
     int rc = get_device(&dev);
     if (rc != FS_OK) return rc;
@@ -1650,6 +1783,15 @@ int fs_release(void) {
         if (dev.dy[s]) { FS_CUDA(cudaFree(dev.dy[s])); dev.dy[s] = nullptr; }
     }
     dev.slot_bytes = 0;
+    {
+        std::lock_guard<std::mutex> sl(g_scratch_mu);
+        if (dev.scratch) {
+            FS_CUDA(cudaDeviceSynchronize());
+            FS_CUDA(cudaFree(dev.scratch));
+            dev.scratch = nullptr; dev.scratch_bytes = 0; dev.scratch_used = false;
+        }
+        if (dev.scratch_ev) { FS_CUDA(cudaEventDestroy(dev.scratch_ev)); dev.scratch_ev = nullptr; }
+    }
     return FS_OK;
 }
 
@@ -1669,24 +1811,23 @@ int fs_softmax_static(const void* x, void* y, int64_t rows, int64_t cols, int dt
     if (v != FS_OK) return v;
     if (rows == 0 || cols == 0) return FS_OK;
     if (!fast_path_ok(cols, dtype, ptr_align(x), ptr_align(y))) return FS_ERR_UNSUPPORTED;
-    SmemGeom sg;
     const int64_t nvec = cols * elem_size(dtype) / 16;
-    if (!smem_geom(nvec, dtype, 0, 0, &sg)) return FS_ERR_UNSUPPORTED;      // row longer than FS_STATIC_MAX_ROW_BYTES
-    if (rows > 0x7fffffff / sg.cs) return FS_ERR_UNSUPPORTED;
-
-    int d = 0;
-    FS_CUDA(cudaGetDevice(&d));
-    if (d < 0 || d >= kMaxDevices) return FS_ERR_UNSUPPORTED;
-    StaticDevice& sd = g_static[d];
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
     std::lock_guard<std::mutex> lk(g_static_mu);
-    if (!sd.ready) {                     // first call on this device: no allocation, only queries
-        FS_CUDA(cudaDeviceGetAttribute(&sd.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, d));
-        FS_CUDA(cudaDeviceGetAttribute(&sd.cluster_ok, cudaDevAttrClusterLaunch, d));
-        void* addr = nullptr;
-        FS_CUDA(cudaGetSymbolAddress(&addr, fs_static_scratch));
-        sd.scratch = static_cast<int*>(addr);
-        sd.ready = true;
+    StaticDevice* sdp = nullptr;
+    int rc = get_static_device(&sdp);
+    if (rc != FS_OK) return rc;
+    StaticDevice& sd = *sdp;
+
+    SmemGeom sg;
+    if (!smem_geom(nvec, dtype, 0, 0, &sg)) {
+        // rows beyond FS_STATIC_MAX_ROW_BYTES: the two-kernel path, its pairs in the array
+        SplitPlan sp;
+        if (!softmax_split_plan(sd.sm_count, sd.scratch, x, y, rows, cols, dtype, scale, &sp)) return FS_ERR_UNSUPPORTED;
+        if (rows * sp.nseg > FS_STATIC_MAX_PAIRS) return FS_ERR_UNSUPPORTED;      // more pairs than the array holds
+        return softmax_split_launch(sp, dtype, reinterpret_cast<float2*>(sd.scratch + kStaticPairOffsetWords), st);
     }
+    if (rows > 0x7fffffff / sg.cs) return FS_ERR_UNSUPPORTED;
     if (!sd.cluster_ok) return FS_ERR_UNSUPPORTED;
 
     Params p{};
@@ -1696,6 +1837,7 @@ int fs_softmax_static(const void* x, void* y, int64_t rows, int64_t cols, int dt
     p.status = sd.scratch;
     p.q_offset = 0;
     p.pf_rows = 0;
+    p.wait_polls = kDefaultWaitPolls;
     const void* fn = smem_row_fn(dtype, p.neg, sg, nvec);
     const size_t stage_bytes = smem_row_stage_bytes(sg, dtype);
     const size_t smem = smem_row_bytes(sg, dtype);
@@ -1710,11 +1852,48 @@ int fs_softmax_static(const void* x, void* y, int64_t rows, int64_t cols, int dt
         FS_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
         sd.configured[dtype][p.neg][full_variant] = true;
     }
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // the array keeps whatever the last call left: the status word must start at zero
-    FS_CUDA(cudaMemsetAsync(sd.scratch, 0, sizeof(int), st));
     return launch(fn, rows * sg.cs, sg.threads, smem, sg.cs, st, p,
                   static_cast<uint32_t>(stage_bytes), sg.slice, smem_row_nchunk(sg, dtype));
+}
+
+int fs_static_status(void) {
+    std::lock_guard<std::mutex> lk(g_static_mu);
+    StaticDevice* sd = nullptr;
+    int rc = get_static_device(&sd);
+    if (rc != FS_OK) return rc;
+    int word = 0;
+    FS_CUDA(cudaDeviceSynchronize());
+    FS_CUDA(cudaMemcpy(&word, sd->scratch, sizeof(int), cudaMemcpyDeviceToHost));
+    if (word) FS_CUDA(cudaMemset(sd->scratch, 0, sizeof(int)));
+    return (word & DEV_TIMEOUT) ? FS_ERR_DEVICE_TIMEOUT : FS_OK;
+}
+
+// ---- self-tests of the bounded waits (nothing here can fault or hang a device) -------------------
+
+int fs_debug_set_wait_polls(int polls) {
+    Device* dev = nullptr;
+    int rc = get_device(&dev);
+    if (rc != FS_OK) return rc;
+    dev->wait_polls.store(polls > 0 ? polls : kDefaultWaitPolls, std::memory_order_relaxed);
+    return FS_OK;
+}
+
+int fs_debug_wait_probe(void* stream) {
+    Device* dev = nullptr;
+    int rc = get_device(&dev);
+    if (rc != FS_OK) return rc;
+    return launch((const void*)wait_probe_kernel, 1, 64, 0, 0, static_cast<cudaStream_t>(stream), dev->status,
+                  dev->wait_polls.load(std::memory_order_relaxed));
+}
+
+int fs_debug_softmax_expire(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale, void* stream,
+                            int threads, int cluster) {
+    const int v = validate(x, y, rows, cols, dtype, scale);
+    if (v != FS_OK) return v;
+    if (cluster < 0 || cluster > kMaxCluster) return FS_ERR_INVALID_ARG;
+    if (rows == 0 || cols == 0) return FS_OK;
+    // every chunk barrier of the split-row kernel is armed for 16 bytes more than are copied
+    return run(x, y, rows, cols, dtype, scale, static_cast<cudaStream_t>(stream), FS_KERNEL_CLUSTER, threads, cluster, 16u);
 }
 
 int fs_last_cuda_error(void) { return t_last_cuda_error; }

@@ -1,18 +1,16 @@
-// Block-per-row and cluster-per-row softmax kernels. One pass over the data: every thread keeps
+// Block-per-row softmax kernels. One pass over the data: every thread keeps
 // its share of the row in registers as 2^((x - r_t) c) against its OWN reference r_t (the max of
 // its elements), so each element costs one ex2; the (r, s) partial pairs are then merged with the
 // online-softmax rule (Milakov-Gimelshein)
 //     (r, s) (+) (r', s') = (R = max(r, r'),  s 2^((r-R)c) + s' 2^((r'-R)c))
-// across the warp (shuffles), the block (shared memory, one __syncthreads per row) and, for the
-// split-row kernel, the thread-block cluster (distributed shared memory, one cluster barrier per
-// row). The output is e * 2^((r_t - R)c) / S.
+// across the warp (shuffles) and the block (shared memory, one __syncthreads per row). The output
+// is e * 2^((r_t - R)c) / S. (Rows split over a thread-block cluster are in smem_row.cuh, which
+// shares block_merge_pairs.)
 //
-// Three front ends share that arithmetic:
+// Two front ends share that arithmetic:
 //   block_row_kernel      128-bit global loads straight into registers
-//   block_row_tma_kernel  rows prefetched into a shared-memory ring by cp.async.bulk (no multicast),
-//                         completion tracked per stage by an mbarrier
-//   cluster_row_kernel    a row split over the blocks of a cluster, each block prefetching its
-//                         own slice like block_row_tma_kernel
+//   block_row_tma_kernel  the row brought into shared memory by cp.async.bulk (no multicast),
+//                         completion tracked by an mbarrier
 #pragma once
 #include "common.cuh"
 
@@ -191,100 +189,6 @@ block_row_tma_kernel(const Params p, const int nstage, const uint32_t stage_byte
             bulk_load_row(smem_u32(smem + size_t(stage) * stage_bytes),
                           xb + (row + int64_t(nstage) * gridDim.x) * row_bytes, row_bytes, smem_u32(&bars[stage]));
         }
-        scale_and_store<DT, NEG, VPT>(e, r_t, R, s, p.c, yv + row * p.nvec, valid, vec);
-        if (++stage == nstage) { stage = 0; phase ^= 1u; }
-    }
-}
-
-// ---------------------------------------------------------------------------------------------
-// cluster per row: block q of the cluster owns vectors [q*slice, min((q+1)*slice, nvec)) of the row
-// dynamic shared memory: [nstage][stage_bytes] slice buffers | nstage mbarriers
-// static shared memory : warp pairs; xchg[2][16], where peers deposit their block's pair with
-//                        st.async, and xbar[2], the mbarriers that count those deposits
-// ---------------------------------------------------------------------------------------------
-template <int DT, bool NEG, int VPT>
-__global__ void __launch_bounds__(BlockCfg<DT, VPT>::MAX_THREADS, 1)
-cluster_row_kernel(const Params p, const int nstage, const uint32_t stage_bytes, const int slice) {
-    constexpr int VE = Traits<DT>::VE;
-    pdl_launch_dependents();
-    extern __shared__ __align__(128) unsigned char smem[];
-    __shared__ float2 wp[2][32];
-    __shared__ __align__(16) float2 xchg[2][16];
-    __shared__ __align__(8) uint64_t xbar[2];
-    const int T = blockDim.x, tid = threadIdx.x, lane = tid & 31;
-    const uint32_t q = cluster_ctarank(), cs = cluster_nctarank();
-    const int64_t ncl = cluster_count_x();             // clusters in the grid
-    const int64_t cid = cluster_id_x();
-    const int nvec = static_cast<int>(p.nvec);
-    const int v0 = min(nvec, static_cast<int>(q) * slice);
-    const int nv = min(nvec, v0 + slice) - v0;         // vectors of this block's slice (may be 0)
-    const uint32_t my_bytes = static_cast<uint32_t>(nv) * 16u;
-    const float ident = ref_identity<NEG>();
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + size_t(nstage) * stage_bytes);
-    const char* xb = static_cast<const char*>(p.x);
-    uint4* __restrict__ yv = static_cast<uint4*>(p.y);
-    auto valid = [&](int k) { return tid + k * T < nv; };
-    auto vec = [&](int k) { return v0 + tid + k * T; };
-
-    const int64_t n_my = cid < p.rows ? (p.rows - cid + ncl - 1) / ncl : 0;   // same for the whole cluster
-    const int64_t row_bytes = p.nvec * 16;
-    if (tid == 0) {
-        for (int s = 0; s < nstage; ++s) mbar_init(smem_u32(&bars[s]), 1);
-        mbar_init(smem_u32(&xbar[0]), 1);
-        mbar_init(smem_u32(&xbar[1]), 1);
-        mbar_fence_init();
-        fence_proxy_async_smem();
-        pdl_wait();
-        if (nv > 0)
-            for (int s = 0; s < nstage && s < n_my; ++s)
-                bulk_load_row(smem_u32(smem + size_t(s) * stage_bytes),
-                              xb + (cid + int64_t(s) * ncl) * row_bytes + int64_t(v0) * 16, my_bytes, smem_u32(&bars[s]));
-    }
-    __syncthreads();
-    // every block of the cluster is resident, with its mbarriers initialised, before anyone writes
-    // into a peer's shared memory
-    cluster_arrive_relaxed();
-    cluster_wait_acquire();
-    pdl_wait();
-
-    int stage = 0;
-    uint32_t phase = 0;
-    bool alive = true;      // false once a bounded wait has expired: later waits are skipped
-    for (int64_t i = 0; i < n_my; ++i) {
-        const int64_t row = cid + i * ncl;
-        const int par = static_cast<int>(i & 1);
-        const uint32_t xphase = static_cast<uint32_t>(i >> 1) & 1u;
-        // arm this row's exchange barrier: cs deposits of 8 bytes (a deposit may arrive first; the
-        // transaction count is signed)
-        if (tid == 0) mbar_expect_tx(smem_u32(&xbar[par]), cs * 8u);
-        uint4 raw[VPT];
-#pragma unroll
-        for (int k = 0; k < VPT; ++k) raw[k] = make_uint4(0u, 0u, 0u, 0u);
-        if (nv > 0) {
-            if (alive) alive = mbar_wait_warp(smem_u32(&bars[stage]), phase, p.status);
-            const uint4* srow = reinterpret_cast<const uint4*>(smem + size_t(stage) * stage_bytes);
-#pragma unroll
-            for (int k = 0; k < VPT; ++k)
-                if (valid(k)) raw[k] = srow[tid + k * T];
-        }
-        float e[VPT][VE], r_t, s;
-        thread_partial<DT, NEG, VPT>(raw, e, r_t, s, p.c, valid);
-        float R = r_t;
-        block_merge_pairs<NEG>(R, s, wp[par], p.c);
-        if (tid == 0 && nv > 0 && i + nstage < n_my) {
-            fence_proxy_async_smem();
-            bulk_load_row(smem_u32(smem + size_t(stage) * stage_bytes),
-                          xb + (row + int64_t(nstage) * ncl) * row_bytes + int64_t(v0) * 16, my_bytes, smem_u32(&bars[stage]));
-        }
-        // deposit this block's pair in slot q of every block of the cluster (this one included);
-        // rows alternate between two slots/barriers, so a fast peer's next deposit cannot be
-        // counted against this row
-        if (tid < cs)
-            st_async_v2(map_to_rank(smem_u32(&xchg[par][q]), tid), R, s, map_to_rank(smem_u32(&xbar[par]), tid));
-        if (alive) alive = mbar_wait_warp(smem_u32(&xbar[par]), xphase, p.status);
-        R = ident; s = 0.0f;
-        if (lane < static_cast<int>(cs)) ld_shared_v2(smem_u32(&xchg[par][lane]), R, s);
-        warp_merge_pairs<NEG>(R, s, p.c);
         scale_and_store<DT, NEG, VPT>(e, r_t, R, s, p.c, yv + row * p.nvec, valid, vec);
         if (++stage == nstage) { stage = 0; phase ^= 1u; }
     }

@@ -13,6 +13,8 @@ enum : int { DT_F32 = 0, DT_BF16 = 1, DT_F16 = 2 };
 
 // Status bits a kernel may OR into the per-device status word.
 enum : int { DEV_TIMEOUT = 1 };
+// Poll cap of the bounded waits: about two seconds.
+constexpr int kDefaultWaitPolls = 1 << 23;
 
 struct Params {
     const void* x;
@@ -27,6 +29,9 @@ struct Params {
     int64_t pf_rows;   // split-row kernel: the cluster of row i asks L2 for row i + pf_rows (0: off)
     float lag_ns;      // one-shot grids: cluster i < lag_rows starts its loads i * lag_ns late (see first_wave_lag)
     int lag_rows;
+    uint32_t dbg_extra_tx;   // 0 in every product call. The wait-expiry self-test arms each chunk barrier of the
+                             // split-row kernel for this many bytes more than it copies, so that the waits run out.
+    int wait_polls;          // poll cap of the split-row kernel's bounded waits (kDefaultWaitPolls unless that self-test lowered it)
 };
 
 template <int DT> struct Traits;
@@ -436,9 +441,9 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 }
 
 // Arms `bar` for `bytes` and issues the copy in pieces of at most 32 KiB. The expected byte count
-// and the copied byte count come from the same loop.
-__device__ __forceinline__ void bulk_load_row(uint32_t dst, const char* src, uint32_t bytes, uint32_t bar) {
-    mbar_expect_tx(bar, bytes);
+// and the copied byte count come from the same loop (`extra` is zero except in the wait-expiry self-test).
+__device__ __forceinline__ void bulk_load_row(uint32_t dst, const char* src, uint32_t bytes, uint32_t bar, uint32_t extra = 0u) {
+    mbar_expect_tx(bar, bytes + extra);
     for (uint32_t off = 0; off < bytes; off += 32768u) {
         const uint32_t n = min(32768u, bytes - off);
         bulk_load(dst + off, src + off, n, bar);
@@ -467,9 +472,14 @@ __device__ __forceinline__ void first_wave_lag(int64_t cluster, float lag_ns, in
 // time whatever hint it is given, and a lane that polls back to back burns issue slots the other
 // blocks on the SM need (measured: hundreds of instructions per wait). So the first polls are
 // immediate (later chunks of a row have usually landed) and the following ones are spaced by
-// nanosleep, doubling up to 256 ns. At most 2^23 polls, about two seconds. Returns false (and
-// records DEV_TIMEOUT) if the phase did not complete; the caller carries on, skipping further
-// waits, so that every block-wide and cluster-wide barrier is still reached and the kernel ends.
+// nanosleep, doubling up to 256 ns. At most `cap` polls (2^23, about two seconds, unless a self-test
+// passes less). Measured on 256 rows of 512 KiB bf16 (47.1 us): spacings from none at all to
+// 32..128 ns change the time by less than 1%, 128..512 ns costs 4% and 256..1024 ns 9% (every row
+// has three waits on its critical path). The cap is an argument, never a memory word: a version of this loop that looked at a
+// cap in global memory, even only on every 64th poll, made the split-row kernel 7% slower (256 rows
+// of 512 KiB: 50.4 us against 47.1). Returns false (and records DEV_TIMEOUT) if the phase did not
+// complete; the caller carries on, skipping further waits, so that every block-wide and
+// cluster-wide barrier is still reached and the kernel ends.
 __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
     uint32_t done;
     asm volatile("{\n\t.reg .pred p;\n\t"
@@ -479,10 +489,10 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
     return done != 0;
 }
 
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status, int cap = kDefaultWaitPolls) {
     if (mbar_try(bar, parity)) return true;
     unsigned ns = 32;
-    for (int it = 0; it < (1 << 23); ++it) {
+    for (int it = 0; it < cap; ++it) {
         __nanosleep(ns);
         if (mbar_try(bar, parity)) return true;
         if (ns < 256) ns <<= 1;
@@ -493,9 +503,9 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* st
 
 // One lane per warp polls (spinning threads cost issue slots that other blocks' warps need); the
 // result is broadcast so that the whole warp agrees on whether the wait expired.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, int* status) {
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, int* status, int cap = kDefaultWaitPolls) {
     int ok = 1;
-    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, status) ? 1 : 0;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, status, cap) ? 1 : 0;
     return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 

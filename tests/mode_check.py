@@ -31,7 +31,7 @@ def main() -> int:
                     assert status == fs.FS_OK, (rows, cols, dtype, kernel, fs.fs_strerror(status), fs.fs_last_cuda_error())
                     check(xs, dtype, scale, y)
                     ran += 1
-    # many rows per resident block: the resident-grid forms loop and refill their rings
+    # many rows per launch: several generations of resident blocks
     for dtype, rows, cols in ((W.BF16, 40000, 512), (W.FP32, 6000, 8192), (W.BF16, 3000, 32768)):
         x = W.random_case(rows, cols, dtype, seed=5, sigma=2.0, neg_inf_frac=0.01)
         for kernel in (fs.FS_KERNEL_WARP, fs.FS_KERNEL_BLOCK, fs.FS_KERNEL_BLOCK_TMA, fs.FS_KERNEL_CLUSTER):
@@ -45,7 +45,7 @@ def main() -> int:
             ran += 1
     assert fs.fs_device_status() == fs.FS_OK
     print(f"mode_check ok: {ran} cases, env " +
-          " ".join(f"{k}={os.environ[k]}" for k in ("FS_PERSISTENT", "FS_CLUSTER_REGS", "FS_PDL", "FS_PREFETCH_PCT") if k in os.environ))
+          " ".join(f"{k}={v}" for k, v in sorted(os.environ.items()) if k.startswith("FS_")))
     return 0
 
 

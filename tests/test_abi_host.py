@@ -48,7 +48,7 @@ def test_binding_mirrors_the_header():
 
 
 def test_enums_match_header():
-    text = open(HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", open(HEADER).read(), flags=re.S)
     for name, value in re.findall(r"(FS_[A-Z0-9_]+)\s*=\s*(\d+)", text):
         assert getattr(fs, name) == int(value), name
 
@@ -57,6 +57,10 @@ def test_constants_match_header():
     text = open(HEADER).read()
     m = re.search(r"#define FS_STATIC_MAX_ROW_BYTES \((\d+) \* (\d+) \* (\d+)\)", text)
     assert m and int(m.group(1)) * int(m.group(2)) * int(m.group(3)) == fs.FS_STATIC_MAX_ROW_BYTES
+    m = re.search(r"#define FS_STATIC_SCRATCH_BYTES (\d+)", text)
+    assert m and int(m.group(1)) == fs.FS_STATIC_SCRATCH_BYTES
+    assert "#define FS_STATIC_MAX_PAIRS ((FS_STATIC_SCRATCH_BYTES - 256) / 8)" in text
+    assert fs.FS_STATIC_MAX_PAIRS == (fs.FS_STATIC_SCRATCH_BYTES - 256) // 8
 
 
 def test_strings(lib):
