@@ -1,21 +1,32 @@
 #!/usr/bin/env python
 """Benchmark of libfsoftmax: last-dimension softmax, achieved HBM GB/s against the roofline.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference] [--all]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg5] [--impl reference] [--all]
 
 A step is one fs_softmax call (dispatcher -> one kernel) over one batch of the headline workload:
-the bf16 attention-score tensor, 16384 rows x 2048 columns (cfg2). Inputs are seeded synthetic data
-already resident in HBM; successive steps rotate over enough independent (x, y) buffer pairs that
-the working set is several times the L2 size, so every step reads and writes DRAM. Timing is on the
-device with CUDA events recorded on the launching stream, max over ranks.
+the largest of the five configurations, the fp32 causal-masked matrix of 32768 x 32768 (cfg5, 4 GiB in,
+4 GiB out). Inputs are seeded synthetic data already resident in HBM; where a workload is smaller
+than eight times the L2 cache, successive steps rotate over enough independent (x, y) buffer
+pairs (8 x L2 in total) that every step reads and writes DRAM. Timing is on the device with CUDA events recorded on the
+launching stream around exactly K launches (a "train"); the train is repeated (30 times, fewer when
+a train is long) and the median train is reported, so that the figure does not depend on K; the
+slowest rank counts.
 
 One JSON line goes to stdout (rank 0). Beyond the base keys it carries
   roofline      algorithmic bytes (read x once + write y once) per launch / average launch time,
-                against the measured copy bandwidth of this GPU pool (MEASURED_PEAKS.json)
+                against the measured copy bandwidth of this GPU pool (MEASURED_PEAKS.json); DRAM
+                traffic per launch from the ncu capture recorded in profiles/dram_traffic.txt
+  per_config    all five configurations, each timed the same way: time, GB/s, fractions of the
+                measured and of the nominal peak, the library's own copy over the same bytes, the
+                input's 64-bit checksum
   e2e           the same metric through fs_softmax_host: pinned host buffers, H2D and D2H copies
                 inside the timed region
-  cpu_baseline  the fp64 oracle, as it stands, on the host cores over a bounded sample
-  workloads     the other four workloads, each timed the same way (--all, default on at N=1)
+  cpu_baseline  the fp64 oracle, as it stands, on the host cores over a bounded sample of the
+                headline workload; `cpu_baselines` has the same for every configuration (all cores
+                and one core)
+  fixed_cost    time = t0 + bytes / B fitted over 1x..16x the rows of the two short configurations,
+                for fs_softmax and for the library's copy
+  workloads     the widened entry points (causal, router, log_softmax, backward, masked, norms)
 With N > 1 (launched by torch.distributed.run) every rank runs the same per-GPU workload on its
 own GPU: rows are independent, so there is no collective on the data path ("weak" scaling).
 
@@ -47,15 +58,18 @@ UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
-# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
-# summarised under profiles/; None where no capture has been taken.
-NCU_TRAFFIC_BYTES = {
-    "cfg1": 265472,               # profiles/block_row_kernel_cfg1_fp32_64x1000.txt (y stays in L2)
-    "cfg2": 85469440,             # profiles/warp_row_kernel_cfg2_bf16_16384x2048.txt (x read once; 0.28 of y written back by kernel end)
-    "cfg3": 34201088,             # profiles/warp_row_kernel_cfg3_bf16_131072x128.txt
-    "cfg4": 212546048,            # profiles/smem_row_kernel_cfg4_bf16_256x262144.txt
-    "cfg5": 16 * 479168512,       # profiles/smem_row_kernel_cfg5_fp32_2048x32768.txt, scaled from 2048 to 32768 rows
-}
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+
+
+def ncu_traffic():
+    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum, averaged over eight consecutive
+    launches on rotating buffers, so that the write-back of one launch's output is counted while the next runs)
+    per workload, as recorded in profiles/dram_traffic.txt by `python -m paper_2607_24762_b200.traffic`."""
+    from paper_2607_24762_b200 import traffic
+    try:
+        return traffic.read(TRAFFIC_FILE)
+    except Exception:
+        return {}
 
 
 def measured_peak():
@@ -141,25 +155,63 @@ class ClockSampler:
 # GPU arm
 # ---------------------------------------------------------------------------------------------
 
-def device_buffers(w: W.Workload, n_pairs: int, threads: int):
-    """n_pairs independent (x, y) device buffer pairs holding the workload's seeded input."""
+def device_buffers(w: W.Workload, n_pairs: int, threads: int, checksum: list | None = None):
+    """n_pairs independent (x, y) device buffer pairs holding the workload's seeded input. With `checksum`
+    (a list), the 64-bit checksum of the input is appended to it (computed slab by slab on the host)."""
     import torch
     tdtype = torch.float32 if w.dtype == W.FP32 else torch.int16
     slab = max(1, (64 << 20) // (w.cols * w.elem_size))
     x0 = torch.empty((w.rows, w.cols), dtype=tdtype, device="cuda")
+    cs = W.Checksum() if checksum is not None else None
     for r0 in range(0, w.rows, slab):
         r1 = min(w.rows, r0 + slab)
         h = W.generate_rows(w, r0, r1, threads=threads)
+        if cs is not None:
+            cs.update(h)
         x0[r0:r1].copy_(torch.from_numpy(h.view(np.int16) if w.dtype != W.FP32 else h))
+    if cs is not None:
+        checksum.append(cs.value())
     xs = [x0] + [x0.clone() for _ in range(n_pairs - 1)]
     ys = [torch.empty_like(x0) for _ in range(n_pairs)]
     return xs, ys
 
 
+def run_trains(launch, steps: int, stream, barrier=None, n_trains: int = 30, budget_ms: float = 3000.0):
+    """Times trains of exactly `steps` launches, one CUDA event pair (on the launching stream) around each train.
+    30 trains, fewer (at least 3) when 30 would exceed budget_ms of device time. Returns the list of train times in ms."""
+    import torch
+    out = []
+    i = 0
+    while len(out) < n_trains:
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        if barrier:
+            barrier()
+        start.record(stream)
+        for _ in range(steps):
+            launch(i)
+            i += 1
+        stop.record(stream)
+        torch.cuda.synchronize()
+        if barrier:
+            barrier()
+        out.append(start.elapsed_time(stop))
+        if len(out) >= 3 and sum(out) + out[-1] > budget_ms:
+            break
+    return out
+
+
+def train_stats(trains, steps: int):
+    each = sorted(t / steps for t in trains)
+    return {"n_trains": len(each), "median": round(statistics.median(each), 6), "min": round(each[0], 6),
+            "max": round(each[-1], 6), "first": round(trains[0] / steps, 6)}
+
+
 def time_device(w: W.Workload, steps: int, warmup: int, l2_bytes: int, sampler: ClockSampler | None = None,
-                barrier=None, min_clock_samples: int = 0, causal_q=None, extras: bool = False):
-    """Times `steps` fs_softmax (or, with causal_q, fs_softmax_causal) launches with CUDA events on
-    the launching stream: one event pair around the whole train of launches (the steady state).
+                barrier=None, min_clock_samples: int = 0, causal_q=None, extras: bool = False, n_trains: int = 30,
+                causal_too: bool = False):
+    """Times trains of `steps` fs_softmax (or, with causal_q, fs_softmax_causal) launches with CUDA events on
+    the launching stream (run_trains); ms_per_step is the median train divided by `steps`.
     With `extras`, the same buffers are then timed two more ways: the library's own copy kernel over
     the same bytes (the ceiling this device gives a kernel that only moves the data), and the same
     launches one at a time, an event pair around each (that figure includes the launch gap)."""
@@ -168,9 +220,10 @@ def time_device(w: W.Workload, steps: int, warmup: int, l2_bytes: int, sampler: 
     import paper_2607_24762_b200 as fs
     free, _ = torch.cuda.mem_get_info()
     pair_bytes = w.min_bytes
-    want = max(1, math.ceil(4 * l2_bytes / pair_bytes))
+    want = max(1, math.ceil(8 * l2_bytes / pair_bytes))     # 8 x L2: at 4 x, a fifth of cfg3's reads still hit L2 (ncu)
     n_pairs = int(max(1, min(want, 256, (free * 0.6) // pair_bytes)))
-    xs, ys = device_buffers(w, n_pairs, threads=min(8, os.cpu_count() or 1))
+    csum = []
+    xs, ys = device_buffers(w, n_pairs, threads=min(8, os.cpu_count() or 1), checksum=csum)
     stream = torch.cuda.current_stream()
     sh = stream.cuda_stream
     lib = fs.binding.lib()
@@ -189,21 +242,11 @@ def time_device(w: W.Workload, steps: int, warmup: int, l2_bytes: int, sampler: 
     for i in range(max(3, warmup)):
         launch(i)
     torch.cuda.synchronize()
-    if barrier:
-        barrier()
     if sampler:
         sampler.start()
         time.sleep(0.12)
-    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    start.record(stream)
-    for i in range(steps):
-        launch(i)
-    stop.record(stream)
-    torch.cuda.synchronize()
-    if barrier:
-        barrier()
-    ms = start.elapsed_time(stop)
+    trains = run_trains(launch, steps, stream, barrier=barrier, n_trains=n_trains)
+    launches = len(trains) * steps
     extension_s = 0.0
     if sampler and min_clock_samples:
         # the timed region can be shorter than nvidia-smi's sampling period: keep the same loop
@@ -211,34 +254,31 @@ def time_device(w: W.Workload, steps: int, warmup: int, l2_bytes: int, sampler: 
         t0 = time.time()
         i = 0
         while sampler.n_samples() < min_clock_samples + 3 and time.time() - t0 < 3.0:
-            for _ in range(64):
+            for _ in range(8 if w.min_bytes > (1 << 30) else 64):
                 launch(i)
                 i += 1
             torch.cuda.synchronize()
         extension_s = time.time() - t0
     clocks = sampler.stop() if sampler else None
     if clocks is not None:
-        clocks["sampled_over"] = "timed region" + (f" + {extension_s:.1f} s of the same launches" if extension_s else "")
+        clocks["sampled_over"] = "timed trains" + (f" + {extension_s:.1f} s of the same launches" if extension_s else "")
     status = fs.fs_device_status()
     if status != 0:
         raise RuntimeError(f"device status: {fs.fs_strerror(status)}")
     kernel = fs.fs_kernel_name(fs.fs_select_kernel(w.rows, w.cols, w.dtype))
+    stats = train_stats(trains, steps)
     extra = {}
     if extras:
         nbytes = w.rows * w.cols * w.elem_size
         if nbytes % 16 == 0:
+            def copy(i):
+                lib.fs_copy(ptrs[i % n_pairs][0], ptrs[i % n_pairs][1], nbytes, sh)
             for i in range(3):
-                lib.fs_copy(ptrs[i % n_pairs][0], ptrs[i % n_pairs][1], nbytes, sh)
-            torch.cuda.synchronize()
-            start.record(stream)
-            for i in range(steps):
-                lib.fs_copy(ptrs[i % n_pairs][0], ptrs[i % n_pairs][1], nbytes, sh)
-            stop.record(stream)
-            torch.cuda.synchronize()
-            copy_ms = start.elapsed_time(stop) / steps
+                copy(i)
+            copy_ms = statistics.median(run_trains(copy, steps, stream, n_trains=n_trains)) / steps
             extra["own_copy"] = {"ms_per_step": round(copy_ms, 6), "GB/s": round(w.min_bytes / (copy_ms * 1e-3) / 1e9, 1),
-                                 "softmax_over_copy_time": round((ms / steps) / copy_ms, 4)}
-        n1 = min(100, steps)
+                                 "softmax_over_copy_time": round(stats["median"] / copy_ms, 4)}
+        n1 = min(100, max(steps, 20))
         pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n1)]
         for i, (a, b) in enumerate(pairs):
             a.record(stream)
@@ -248,9 +288,63 @@ def time_device(w: W.Workload, steps: int, warmup: int, l2_bytes: int, sampler: 
         each = sorted(a.elapsed_time(b) for a, b in pairs)
         extra["single_launch_ms"] = {"median": round(statistics.median(each), 6), "best": round(each[0], 6), "n": n1,
                                      "note": "event pair around each launch: includes the launch gap"}
+    if causal_too:
+        # fs_softmax_causal(q_offset = 0) over the same buffers: the masked part of x is never read
+        def causal(i):
+            xp, yp = ptrs[i % n_pairs]
+            st = lib.fs_softmax_causal(xp, yp, w.rows, w.cols, 0, w.dtype, scale, sh)
+            if st != 0:
+                raise RuntimeError(f"fs_softmax_causal failed: {fs.fs_strerror(st)}")
+        for i in range(3):
+            causal(i)
+        extra["causal_ms_per_step"] = statistics.median(run_trains(causal, steps, stream, n_trains=min(n_trains, 10))) / steps
     del xs, ys
     torch.cuda.empty_cache()
-    return {"ms_per_step": ms / steps, "n_pairs": n_pairs, "kernel": kernel, "clocks": clocks, **extra}
+    return {"ms_per_step": statistics.median(trains) / steps, "trains": stats, "launches": launches, "n_pairs": n_pairs,
+            "kernel": kernel, "clocks": clocks, "checksum": f"{csum[0]:016x}", **extra}
+
+
+def fit_fixed_cost(w: W.Workload, l2_bytes: int, steps: int = 200):
+    """time = t0 + bytes / B over 1x, 2x, 4x, 8x, 16x the rows of a short workload, for fs_softmax and for the library's
+    copy over the same buffers (least squares; device-seeded data of the workload's shape and dtype)."""
+    import torch
+
+    import paper_2607_24762_b200 as fs
+    lib = fs.binding.lib()
+    stream = torch.cuda.current_stream()
+    sh = stream.cuda_stream
+    tdt = {W.FP32: torch.float32, W.BF16: torch.bfloat16, W.FP16: torch.float16}[w.dtype]
+    g = torch.Generator(device="cuda").manual_seed(7)
+    pts = {"softmax": [], "copy": []}
+    for mult in (1, 2, 4, 8, 16):
+        rows = w.rows * mult
+        nbytes = rows * w.cols * w.elem_size
+        n_pairs = int(max(1, min(16, math.ceil(4 * l2_bytes / (2 * nbytes)))))
+        xs = [(torch.randn((rows, w.cols), generator=g, device="cuda") * 2.0).to(tdt) for _ in range(n_pairs)]
+        ys = [torch.empty_like(x) for x in xs]
+
+        def soft(i):
+            lib.fs_softmax(xs[i % n_pairs].data_ptr(), ys[i % n_pairs].data_ptr(), rows, w.cols, w.dtype, w.scale_f32, sh)
+
+        def copy(i):
+            lib.fs_copy(xs[i % n_pairs].data_ptr(), ys[i % n_pairs].data_ptr(), nbytes, sh)
+
+        for name, fn in (("softmax", soft), ("copy", copy)):
+            for i in range(5):
+                fn(i)
+            k = max(20, steps // mult)
+            ms = statistics.median(run_trains(fn, k, stream, n_trains=9, budget_ms=400.0)) / k
+            pts[name].append((2.0 * nbytes, ms * 1e3))
+        del xs, ys
+        torch.cuda.empty_cache()
+    out = {"workload": w.name, "rows_multiples": [1, 2, 4, 8, 16]}
+    for name, p in pts.items():
+        bx = np.array([b for b, _ in p])
+        ty = np.array([t for _, t in p])
+        slope, t0 = np.polyfit(bx, ty, 1)
+        out[name] = {"t0_us": round(float(t0), 3), "GB/s_marginal": round(1e-3 / float(slope), 1),
+                     "us": [round(float(t), 3) for t in ty]}
+    return out
 
 
 def time_router(w: W.Workload, k: int, steps: int, warmup: int, l2_bytes: int):
@@ -610,19 +704,23 @@ def run_oracle(w: W.Workload, x: np.ndarray, cores: int) -> float:
 
 
 def cpu_baseline(w: W.Workload, target_cpu_seconds: float = 16.0):
+    """The oracle, as it stands, over a bounded sample of the workload: on all host cores (rows partitioned over
+    threads, each running the single-threaded oracle) and on one core. `target_cpu_seconds` is the CPU work of one
+    pass over the sample, summed over cores; a workload smaller than that is passed over several times."""
     from oracle import fso
     fso.build()
     x, cores, what = oracle_sample(w, target_cpu_seconds)
     run_oracle(w, x[:cores], cores)                        # load the library, touch the code
-    # a workload smaller than the target is passed over several times (about 10 s of CPU work)
     est = x.size * 11e-9
-    passes = int(max(1, min(200, round(10.0 / max(est, 1e-3)))))
+    passes = int(max(1, min(200, round(0.6 * target_cpu_seconds / max(est, 1e-3)))))
     dt = sum(run_oracle(w, x, cores) for _ in range(passes)) / passes
     nbytes = 2 * x.size * w.elem_size
     if passes > 1:
         what += f", mean of {passes} passes"
-    # the same oracle on one core, over the head of the same sample (about two seconds of work)
-    n1 = int(max(1, min(x.shape[0], 2.0 / 11e-9 // w.cols)))
+    if x.shape[0] < w.rows:
+        what += "; the workload's figure is extrapolated from this sample"
+    # the same oracle on one core, over the head of the same sample
+    n1 = int(max(1, min(x.shape[0], 0.125 * target_cpu_seconds / 11e-9 // w.cols)))
     dt1 = run_oracle(w, x[:n1], 1)
     one = {"value": round(2 * n1 * w.cols * w.elem_size / dt1 / 1e9, 4), "unit": UNIT, "cores": 1,
            "sample": f"the first {n1} rows of the sample", "seconds": round(dt1, 4)}
@@ -673,19 +771,40 @@ def smi_id(props, local_rank: int) -> str:
 def roofline_obj(w: W.Workload, ms_per_step: float, kernel: str):
     peak, which = measured_peak()
     achieved = w.min_bytes / (ms_per_step * 1e-3) / 1e9
-    traffic = NCU_TRAFFIC_BYTES.get(w.name)
+    t = ncu_traffic().get(w.name)
     return {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
             "frac": round(achieved / peak, 4), "peak_source": f"of {which} (copy bandwidth)",
             "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
-            "traffic": traffic, "algorithmic_bytes_per_launch": w.min_bytes, "kernel": kernel}
+            "traffic": t["bytes_per_launch"] if t else None,
+            "traffic_over_algorithmic": round(t["bytes_per_launch"] / w.min_bytes, 4) if t else None,
+            "traffic_source": t["note"] if t else "no capture recorded in profiles/dram_traffic.txt",
+            "algorithmic_bytes_per_launch": w.min_bytes, "kernel": kernel}
+
+
+def per_config_entry(w: W.Workload, r: dict):
+    peak, _ = measured_peak()
+    gbs = w.min_bytes / (r["ms_per_step"] * 1e-3) / 1e9
+    t = ncu_traffic().get(w.name)
+    e = {"shape": [w.rows, w.cols], "dtype": W.DTYPE_NAME[w.dtype], "kernel": r["kernel"], "ms_per_step": round(r["ms_per_step"], 6),
+         "GB/s": round(gbs, 1), "rows_per_s": round(w.rows / (r["ms_per_step"] * 1e-3), 1),
+         "frac_of_measured": round(gbs / peak, 4), "frac_of_nominal": round(gbs / NOMINAL_HBM_GBS, 4),
+         "steps": r.get("steps"), "trains": r["trains"], "n_pairs": r["n_pairs"], "checksum": r["checksum"],
+         "traffic_over_algorithmic": round(t["bytes_per_launch"] / w.min_bytes, 4) if t else None}
+    if "own_copy" in r:
+        e["own_copy_ms"] = r["own_copy"]["ms_per_step"]
+        e["softmax_over_copy_time"] = r["own_copy"]["softmax_over_copy_time"]
+    if "single_launch_ms" in r:
+        e["single_launch_ms"] = r["single_launch_ms"]["median"]
+    return e
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--workload", default="cfg2", choices=sorted(W.WORKLOADS))
+    ap.add_argument("--workload", default="cfg5", choices=sorted(W.WORKLOADS))
+    ap.add_argument("--trains", type=int, default=30, help="how many times the train of --steps launches is timed (median reported)")
     ap.add_argument("--impl", default="fsoftmax", choices=["fsoftmax", "reference"])
     ap.add_argument("--rows", type=int, default=0,
                     help="use only the first ROWS rows of the workload (small cases for profiler captures)")
@@ -741,7 +860,7 @@ def main():
     sampler = ClockSampler(smi_id(props, local_rank)) if rank == 0 and not args.no_clocks else None
     if args.op != "softmax":
         if args.op == "causal":
-            r = time_device(w, args.steps, args.warmup, l2, causal_q=0)
+            r = time_device(w, args.steps, args.warmup, l2, causal_q=0, n_trains=args.trains)
             kept = sum(min(w.cols, i + 1) for i in range(w.rows))
             alg = (kept + w.rows * w.cols) * w.elem_size
             r = {"ms_per_step": round(r["ms_per_step"], 6), "algorithmic_bytes": alg,
@@ -767,11 +886,13 @@ def main():
             dist.destroy_process_group()
         return
     res = time_device(w, args.steps, args.warmup, l2, sampler=sampler, barrier=barrier, min_clock_samples=8,
-                      extras=world == 1)
+                      extras=world == 1, n_trains=args.trains,
+                      causal_too=world == 1 and w.name == "cfg5" and not args.rows and args.all_workloads is not False)
     from paper_2607_24762_b200 import sharding
     ms = sharding.max_over_ranks(res["ms_per_step"], device="cuda")          # as slow as the slowest rank
     value = sharding.aggregate_throughput(w.min_bytes, ms * 1e-3, world) / 1e9
 
+    res["steps"] = args.steps
     line = {"metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": round(ms, 6), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
@@ -780,50 +901,61 @@ def main():
                        "parallelism": f"rows independent: {world} replica(s) of the per-GPU workload, no collective",
                        "l2": f"rotating over {res['n_pairs']} independent (x,y) buffer pairs = "
                              f"{res['n_pairs'] * w.min_bytes / 2**20:.0f} MiB, L2 is {l2 / 2**20:.0f} MiB",
+                       "timing": f"median of {res['trains']['n_trains']} trains of {args.steps} launches, one CUDA event pair per train",
+                       "input_checksum": res["checksum"],
                        "rows_per_s": round(world * w.rows / (ms * 1e-3), 1)},
             "roofline": roofline_obj(w, ms, res["kernel"]),
-            "gpu_launches": args.steps,
+            "gpu_launches": res["launches"],
             "clocks": res["clocks"]}
-    for key in ("own_copy", "single_launch_ms"):           # the train above is the headline; these explain it
+    line["roofline"]["trains_ms_per_step"] = res["trains"]
+    for key in ("own_copy", "single_launch_ms"):           # the trains above are the headline; these explain it
         if key in res:
             line["roofline"][key] = res[key]
 
     if rank == 0 and world == 1:
-        if not args.no_e2e:
-            line["e2e"] = time_e2e(w, steps=max(3, min(args.steps, 20)), warmup=2)
-        if args.all_workloads is None or args.all_workloads:
-            others = {}
+        full = args.all_workloads is None or args.all_workloads
+        per = {w.name: per_config_entry(w, res)}
+        results = {w.name: res}
+        if full:
             for name, ow in W.WORKLOADS.items():
-                if name == w.name:
+                if name in per:
                     continue
                 free, _ = torch.cuda.mem_get_info()
                 if free < ow.min_bytes * 1.3:
-                    others[name] = {"skipped": "not enough free device memory"}
+                    per[name] = {"skipped": "not enough free device memory"}
                     continue
-                k = max(20, min(2000, int(0.08 / max(ow.min_bytes / 6.0e12, 4e-6))))
-                r = time_device(ow, k, 10, l2, extras=True)
-                gbs = ow.min_bytes / (r["ms_per_step"] * 1e-3) / 1e9
-                peak, which = measured_peak()
-                others[name] = {"what": ow.note, "kernel": r["kernel"], "steps": k, "ms_per_step": round(r["ms_per_step"], 6),
-                                "GB/s": round(gbs, 1), "rows_per_s": round(ow.rows / (r["ms_per_step"] * 1e-3), 1),
-                                "frac_of_measured_copy": round(gbs / peak, 4),
-                                "frac_of_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 4), "n_pairs": r["n_pairs"],
-                                **{key: r[key] for key in ("own_copy", "single_launch_ms") if key in r}}
+                k = max(20, min(1000, int(0.02 / max(ow.min_bytes / 6.0e12, 4e-6))))
+                r = time_device(ow, k, 10, l2, extras=True, n_trains=args.trains, causal_too=name == "cfg5")
+                r["steps"] = k
+                results[name] = r
+                per[name] = per_config_entry(ow, r)
+        line["per_config"] = {k: per[k] for k in sorted(per)}
+        if not args.no_e2e:
+            line["e2e"] = time_e2e(w, steps=max(3, min(args.steps, 5 if w.min_bytes > (1 << 30) else 20)), warmup=1 if w.min_bytes > (1 << 30) else 2)
+        if not args.no_cpu:
+            line["cpu_baseline"] = cpu_baseline(w)
+            if full:
+                line["cpu_baselines"] = {name: (line["cpu_baseline"] if name == w.name else cpu_baseline(ow, 4.0))
+                                         for name, ow in sorted(W.WORKLOADS.items())}
+        if full:
+            try:
+                line["fixed_cost"] = {n: fit_fixed_cost(W.WORKLOADS[n], l2) for n in ("cfg2", "cfg3")}
+            except Exception as exc:                       # never lose the main line to an extra
+                line["fixed_cost"] = {"error": str(exc)[:200]}
+            others = {}
             # the causal entry point on the causal workload: the masked half of x is never read
-            ow = W.WORKLOADS["cfg5"]
-            free, _ = torch.cuda.mem_get_info()
-            if free >= ow.min_bytes * 1.3:
-                r = time_device(ow, 40, 10, l2, causal_q=0)
+            if "causal_ms_per_step" in results.get("cfg5", {}):
+                ow = W.WORKLOADS["cfg5"]
+                cms = results["cfg5"]["causal_ms_per_step"]
                 read_b = ow.rows * (ow.rows + 1) // 2 * ow.elem_size
                 alg = read_b + ow.rows * ow.cols * ow.elem_size
-                gbs = alg / (r["ms_per_step"] * 1e-3) / 1e9
+                gbs = alg / (cms * 1e-3) / 1e9
                 peak, which = measured_peak()
                 others["cfg5_causal"] = {"what": "fs_softmax_causal(q_offset=0) on cfg5: reads only columns j <= i, writes every column",
-                                         "kernel": "cluster", "steps": 40, "ms_per_step": round(r["ms_per_step"], 6),
+                                         "kernel": "cluster", "ms_per_step": round(cms, 6),
                                          "algorithmic_bytes": alg, "GB/s": round(gbs, 1),
                                          "frac_of_measured_copy": round(gbs / peak, 4),
-                                         "speedup_vs_cfg5": round(others["cfg5"]["ms_per_step"] / r["ms_per_step"], 3)
-                                         if "ms_per_step" in others.get("cfg5", {}) else None}
+                                         "speedup_vs_cfg5": round(results["cfg5"]["ms_per_step"] / cms, 3)}
             # the router step (softmax over experts + top-8, renormalised) on the router workload
             rw = W.WORKLOADS["cfg3"]
             try:
@@ -856,8 +988,6 @@ def main():
                 except Exception as exc:
                     others[nname] = {"error": str(exc)[:200]}
             line["workloads"] = others
-        if not args.no_cpu:
-            line["cpu_baseline"] = cpu_baseline(w)
     elif rank == 0:
         line["e2e"] = None
     if rank == 0:

@@ -11,11 +11,20 @@ eager mode and never sees a wrong or unsupported kernel.
 
 The guard admits a call when: the tensor is on a CUDA device, dtype fp32/bf16/fp16, the softmax
 dimension is the last one (or the tensor can be seen that way without a copy), the tensor is
-contiguous, no autograd graph is being recorded for it, and no output dtype conversion is asked
-for other than eager attention's ``softmax(scores, dim=-1, dtype=torch.float32)`` on 16-bit scores
-(which runs the library's 16-bit-in, float32-out kernel). log_softmax follows the same guard but
-falls back for any ``dtype=``. This module is a convenience layer above the C ABI; the library
-itself has no fallback.
+contiguous, and no output dtype conversion is asked for other than eager attention's
+``softmax(scores, dim=-1, dtype=torch.float32)`` on 16-bit scores (which runs the library's
+16-bit-in, float32-out kernel). log_softmax follows the same guard but falls back for any ``dtype=``.
+
+The admitted calls go through operators registered with ``torch.library`` under the namespace
+``fsoftmax`` -- ``torch.ops.fsoftmax.softmax(x, scale)``, ``softmax_backward(dy, y, scale)``,
+``log_softmax(x)``, ``layer_norm(x, weight, bias, eps)``, ``group_norm(x, groups, weight, bias, eps)`` -- each
+with a fake (meta) implementation, so that a traced or compiled model carries them as opaque nodes,
+and softmax with an autograd formula that runs the library's backward kernel: a softmax whose input
+requires grad stays on the library in both directions. The other three have no backward kernel, so
+the guard sends them to eager while autograd is recording. Each operator applies the guard again on
+the tensors it is handed (a compiled graph may call it directly) and computes the same result with
+eager PyTorch when the guard refuses. This module is a convenience layer above the C ABI; the
+library itself has no fallback.
 """
 from __future__ import annotations
 
@@ -54,8 +63,9 @@ def stats(reset: bool = False) -> dict:
     return out
 
 
-def why_not(x: torch.Tensor, dim: int, dtype=None) -> str | None:
-    """None when the guard admits the call, else the reason it goes to eager."""
+def why_not(x: torch.Tensor, dim: int, dtype=None, grad_ok: bool = False) -> str | None:
+    """None when the guard admits the call, else the reason it goes to eager. `grad_ok`: the operator has
+    an autograd formula, so an input that requires grad is no reason to refuse."""
     if not isinstance(x, torch.Tensor):
         return "not a tensor"
     if not x.is_cuda:
@@ -70,16 +80,147 @@ def why_not(x: torch.Tensor, dim: int, dtype=None) -> str | None:
         return "softmax dimension is not the last one"
     if not x.is_contiguous():
         return "not contiguous"
-    if torch.is_grad_enabled() and x.requires_grad:
+    if not grad_ok and torch.is_grad_enabled() and x.requires_grad:
         return "autograd is recording"
     if x.numel() == 0:
         return "empty"
     return None
 
 
+# ---------------------------------------------------------------------------------------------
+# operators registered with torch.library (namespace "fsoftmax")
+# ---------------------------------------------------------------------------------------------
+
+def _library_ok(x: torch.Tensor, *others) -> bool:
+    """The guard as the operators apply it to the tensors they are handed."""
+    if why_not(x, -1, grad_ok=True) is not None:
+        return False
+    for t in others:
+        if t is not None and not (t.is_cuda and t.device == x.device and t.dtype == x.dtype and t.is_contiguous()):
+            return False
+    try:
+        binding.lib()
+    except RuntimeError:
+        return False
+    return True
+
+
+@torch.library.custom_op("fsoftmax::softmax", mutates_args=())
+def _op_softmax(x: torch.Tensor, scale: float) -> torch.Tensor:
+    if not _library_ok(x):
+        _count("eager:operator called on tensors the guard refuses")
+        return _eager_softmax(x if scale == 1.0 else x * scale, -1)
+    cols = x.shape[-1]
+    y = torch.empty_like(x)
+    with torch.cuda.device(x.device):
+        binding.fs_softmax(x, y, x.numel() // cols, cols, _DTYPES[x.dtype], scale, torch.cuda.current_stream(x.device))
+    _count("library")
+    return y
+
+
+@_op_softmax.register_fake
+def _(x, scale):
+    return torch.empty_like(x)
+
+
+@torch.library.custom_op("fsoftmax::softmax_backward", mutates_args=())
+def _op_softmax_backward(dy: torch.Tensor, y: torch.Tensor, scale: float) -> torch.Tensor:
+    """dx = scale * y * (dy - sum(dy * y)) over the last dimension."""
+    if dy.shape != y.shape or not _library_ok(y, dy) or dy.dtype != y.dtype:
+        _count("eager:operator called on tensors the guard refuses")
+        return (scale * y * (dy - (dy * y).sum(dim=-1, keepdim=True))).to(y.dtype)
+    cols = y.shape[-1]
+    dx = torch.empty_like(y)
+    with torch.cuda.device(y.device):
+        binding.fs_softmax_backward(dy, y, dx, y.numel() // cols, cols, _DTYPES[y.dtype], scale,
+                                    torch.cuda.current_stream(y.device))
+    _count("library")
+    return dx
+
+
+@_op_softmax_backward.register_fake
+def _(dy, y, scale):
+    return torch.empty_like(y)
+
+
+def _softmax_setup_context(ctx, inputs, output):
+    ctx.save_for_backward(output)
+    ctx.scale = inputs[1]
+
+
+def _softmax_autograd(ctx, grad):
+    (y,) = ctx.saved_tensors
+    return torch.ops.fsoftmax.softmax_backward(grad.contiguous(), y, ctx.scale), None
+
+
+torch.library.register_autograd("fsoftmax::softmax", _softmax_autograd, setup_context=_softmax_setup_context)
+
+
+@torch.library.custom_op("fsoftmax::log_softmax", mutates_args=())
+def _op_log_softmax(x: torch.Tensor) -> torch.Tensor:
+    if not _library_ok(x):
+        _count("eager:operator called on tensors the guard refuses")
+        return _eager_log_softmax(x, -1)
+    cols = x.shape[-1]
+    y = torch.empty_like(x)
+    with torch.cuda.device(x.device):
+        binding.fs_log_softmax(x, y, x.numel() // cols, cols, _DTYPES[x.dtype], 1.0, torch.cuda.current_stream(x.device))
+    _count("library")
+    return y
+
+
+@_op_log_softmax.register_fake
+def _(x):
+    return torch.empty_like(x)
+
+
+@torch.library.custom_op("fsoftmax::layer_norm", mutates_args=())
+def _op_layer_norm(x: torch.Tensor, weight: torch.Tensor | None, bias: torch.Tensor | None, eps: float) -> torch.Tensor:
+    if not _library_ok(x, weight, bias):
+        _count("eager:operator called on tensors the guard refuses")
+        return _eager_F_layer_norm(x, (x.shape[-1],), weight, bias, eps)
+    cols = x.shape[-1]
+    y = torch.empty_like(x)
+    with torch.cuda.device(x.device):
+        binding.fs_layer_norm(x, weight, bias, y, x.numel() // cols, cols, _DTYPES[x.dtype], eps,
+                              torch.cuda.current_stream(x.device))
+    _count("library")
+    return y
+
+
+@_op_layer_norm.register_fake
+def _(x, weight, bias, eps):
+    return torch.empty_like(x)
+
+
+@torch.library.custom_op("fsoftmax::group_norm", mutates_args=())
+def _op_group_norm(x: torch.Tensor, groups: int, weight: torch.Tensor | None, bias: torch.Tensor | None,
+                   eps: float) -> torch.Tensor:
+    if x.dim() < 2 or not _library_ok(x, weight, bias):
+        _count("eager:operator called on tensors the guard refuses")
+        return _eager_F_group_norm(x, groups, weight, bias, eps)
+    n, ch = x.shape[0], x.shape[1]
+    y = torch.empty_like(x)
+    with torch.cuda.device(x.device):
+        binding.fs_group_norm(x, weight, bias, y, n, ch, x.numel() // (n * ch), groups, _DTYPES[x.dtype], eps,
+                              torch.cuda.current_stream(x.device))
+    _count("library")
+    return y
+
+
+@_op_group_norm.register_fake
+def _(x, groups, weight, bias, eps):
+    return torch.empty_like(x)
+
+
+# ---------------------------------------------------------------------------------------------
+# the guarded front end
+# ---------------------------------------------------------------------------------------------
+
 def softmax(x: torch.Tensor, dim: int = -1, dtype=None, scale: float = 1.0, out: torch.Tensor | None = None):
     """softmax(scale * x) over `dim`: the library kernel when admitted, else eager PyTorch."""
-    reason = why_not(x, dim, dtype)
+    plain = out is None and (dtype is None or (isinstance(x, torch.Tensor) and dtype == x.dtype))
+    reason = why_not(x, dim, dtype, grad_ok=plain)
     if reason is None and out is not None and (out.shape != x.shape or out.dtype != x.dtype or
                                                 not out.is_contiguous() or out.device != x.device):
         reason = "incompatible out tensor"
@@ -108,11 +249,12 @@ def softmax(x: torch.Tensor, dim: int = -1, dtype=None, scale: float = 1.0, out:
             binding.fs_softmax_f32out(x, y, rows, cols, _DTYPES[x.dtype], float(scale), torch.cuda.current_stream(x.device))
         _count("library")
         return y
-    y = out if out is not None else torch.empty_like(x)
+    if out is None:
+        return torch.ops.fsoftmax.softmax(x, float(scale))          # registered operator: autograd, fake tensors
     with torch.cuda.device(x.device):
-        binding.fs_softmax(x, y, rows, cols, _DTYPES[x.dtype], float(scale), torch.cuda.current_stream(x.device))
+        binding.fs_softmax(x, out, rows, cols, _DTYPES[x.dtype], float(scale), torch.cuda.current_stream(x.device))
     _count("library")
-    return y
+    return out
 
 
 def log_softmax(x: torch.Tensor, dim: int = -1, dtype=None):
@@ -128,12 +270,7 @@ def log_softmax(x: torch.Tensor, dim: int = -1, dtype=None):
     if reason is not None:
         _count("eager:" + reason)
         return _eager_log_softmax(x, dim, dtype=dtype)
-    cols = x.shape[-1]
-    y = torch.empty_like(x)
-    with torch.cuda.device(x.device):
-        binding.fs_log_softmax(x, y, x.numel() // cols, cols, _DTYPES[x.dtype], 1.0, torch.cuda.current_stream(x.device))
-    _count("library")
-    return y
+    return torch.ops.fsoftmax.log_softmax(x)
 
 
 def _affine_ok(x, p, n):
@@ -157,13 +294,7 @@ def layer_norm(x: torch.Tensor, normalized_shape, weight=None, bias=None, eps: f
     if reason is not None:
         _count("eager:" + reason)
         return _eager_F_layer_norm(x, shape, weight, bias, eps)
-    cols = x.shape[-1]
-    y = torch.empty_like(x)
-    with torch.cuda.device(x.device):
-        binding.fs_layer_norm(x, weight, bias, y, x.numel() // cols, cols, _DTYPES[x.dtype], float(eps),
-                              torch.cuda.current_stream(x.device))
-    _count("library")
-    return y
+    return torch.ops.fsoftmax.layer_norm(x, weight, bias, float(eps))
 
 
 def group_norm(x: torch.Tensor, num_groups: int, weight=None, bias=None, eps: float = 1e-5):
@@ -181,14 +312,7 @@ def group_norm(x: torch.Tensor, num_groups: int, weight=None, bias=None, eps: fl
     if reason is not None:
         _count("eager:" + reason)
         return _eager_F_group_norm(x, num_groups, weight, bias, eps)
-    n, ch = x.shape[0], x.shape[1]
-    spatial = x.numel() // (n * ch)
-    y = torch.empty_like(x)
-    with torch.cuda.device(x.device):
-        binding.fs_group_norm(x, weight, bias, y, n, ch, spatial, num_groups, _DTYPES[x.dtype], float(eps),
-                              torch.cuda.current_stream(x.device))
-    _count("library")
-    return y
+    return torch.ops.fsoftmax.group_norm(x, int(num_groups), weight, bias, float(eps))
 
 
 def _patched_softmax(input, dim=None, *, dtype=None, **kw):        # torch.softmax(input, dim, dtype=None)

@@ -206,6 +206,35 @@ def checksum(x: np.ndarray) -> int:
         return int(np.bitwise_xor.reduce(mixed) ^ np.uint64(words.size))
 
 
+class Checksum:
+    """The same checksum taken over consecutive slabs of a buffer (rows in order), without holding the buffer:
+    `Checksum().update(a).update(b).value() == checksum(np.concatenate([a, b]))` when every slab but the last is
+    a whole number of 64-bit words."""
+
+    def __init__(self) -> None:
+        self.acc = np.uint64(0)
+        self.words = 0
+
+    def update(self, x: np.ndarray) -> "Checksum":
+        raw = np.ascontiguousarray(x).view(np.uint8).ravel()
+        pad = (-raw.size) % 8
+        if pad:
+            raw = np.concatenate([raw, np.zeros(pad, dtype=np.uint8)])
+        words = raw.view(np.uint64)
+        step = 1 << 22
+        for i in range(0, words.size, step):                      # bounded temporaries
+            part = words[i:i + step]
+            idx = np.arange(self.words + i + 1, self.words + i + part.size + 1, dtype=np.uint64)
+            with np.errstate(over="ignore"):
+                mixed = (part ^ (idx * np.uint64(0x9E3779B97F4A7C15))) * np.uint64(0x100000001B3)
+            self.acc ^= np.bitwise_xor.reduce(mixed)
+        self.words += words.size
+        return self
+
+    def value(self) -> int:
+        return int(self.acc ^ np.uint64(self.words))
+
+
 # ---------------------------------------------------------------------------------------------
 # generic seeded cases for shape sweeps and special-value rows
 # ---------------------------------------------------------------------------------------------

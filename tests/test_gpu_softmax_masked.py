@@ -103,6 +103,37 @@ def test_rows_around_the_four_rows_per_block_kernel(dtype):
             check(x, m, dtype, q, heads, [1.0, 0.25, -0.5][(ci + heads) % 3])
 
 
+@pytest.mark.parametrize("dtype", [BF16, FP16])
+def test_masks_shared_by_many_heads(dtype):
+    """16-bit rows of 256..704 vectors with masks shared by 2 to 16 heads over one to three batches: head counts
+    around the four rows a block takes, both ends of the row range, every mask kind, in place, special values."""
+    ve = 8
+    for ci, (batch, heads, q, nvec) in enumerate([(1, 2, 9, 256), (2, 4, 5, 256), (1, 3, 17, 300), (2, 5, 3, 512), (1, 8, 6, 640),
+                                                   (3, 7, 2, 704), (1, 16, 1, 257), (1, 2, 130, 384), (1, 4, 33, 703)]):
+        x, m = make(batch, heads, q, nvec * ve, dtype, seed=1200 + ci, kind=("causal", "padding", "bias")[ci % 3])
+        check(x, m, dtype, q, heads, [1.0, 0.125, -0.5, 128 ** -0.5][ci % 4], inplace=ci % 4 == 3)
+    # a fully masked row, a NaN and a +inf: whole rows NaN, the other heads of the block untouched
+    x, m = make(1, 4, 3, 2048, dtype, seed=1300, kind="padding")
+    ninf = np.uint16(0xFF80 if dtype == BF16 else 0xFC00)
+    m[1, :] = ninf
+    x[0, 7] = np.uint16(0x7FC0 if dtype == BF16 else 0x7E00)
+    x[5, 100] = np.uint16(0x7F80 if dtype == BF16 else 0x7C00)
+    got = run(x, m, dtype, 3, 4, 1.0)
+    want = fso.softmax_masked_f64(x, m, dtype, 3, 4, 1.0)
+    assert np.array_equal(np.isnan(fso.widen(got, dtype)), np.isnan(want))
+    ok = ~np.isnan(want).any(axis=1)
+    assert fso.compare(got[ok], dtype, want[ok]).ok(dtype)
+    # bf16 results below 2^-126 are kept (the 1-ulp rule covers subnormals)
+    if dtype == BF16:
+        row = np.linspace(-91.0, -87.0, 2048)
+        row[0] = 0.0
+        xs = fso.round_from_f64(np.tile(row, (4, 1)), dtype)
+        ms = fso.round_from_f64(np.zeros((2, 2048)), dtype)
+        rep = check(xs, ms, dtype, 2, 2, 1.0)
+        y = run(xs, ms, dtype, 2, 2, 1.0)
+        assert np.count_nonzero((y[0] > 0) & (y[0] < 0x0080)) > 50
+
+
 @pytest.mark.parametrize("dtype", [FP32, BF16, FP16])
 def test_special_values_alignment_and_aliasing(dtype):
     x, m = make(1, 2, 4, 4096, dtype, seed=9, kind="padding")

@@ -60,11 +60,13 @@ def test_admitted_calls_match_the_oracle_and_others_fall_back():
     assert torch_op.why_not(xt, -1) == "not contiguous"
     assert torch.allclose(torch_op.softmax(xt, -1), torch.softmax(xt, -1))
     xg = x.clone().requires_grad_(True)
-    yg = torch_op.softmax(xg, -1)
-    yg.sum().backward()                                   # eager route keeps autograd working
-    assert xg.grad is not None and torch_op.why_not(xg, -1) == "autograd is recording"
+    assert torch_op.why_not(xg, -1) == "autograd is recording" and torch_op.why_not(xg, -1, grad_ok=True) is None
     with torch.no_grad():
         assert torch_op.why_not(xg, -1) is None
+    # log_softmax has no backward kernel: while autograd records, the guard sends it to eager, and autograd works
+    lg = torch_op.log_softmax(xg, -1)
+    lg.sum().backward()
+    assert xg.grad is not None
     assert torch_op.why_not(x, -1, dtype=torch.float64) == "output dtype conversion requested"
     # eager attention's upcast: 16-bit scores, float32 probabilities, through the mixed-dtype kernel
     xb = (torch.randn(4, 8, 96, 1024, device="cuda") * 2).to(torch.bfloat16)
@@ -140,3 +142,55 @@ def test_log_softmax_and_norms_through_the_guard_on_gpu():
     assert torch.allclose(torch_op.layer_norm(x, (1536,), w, b).float(), ref[0], atol=3e-2, rtol=2e-2)
     y = torch_op.layer_norm(x.float(), (1536,), w.float(), b.float())
     assert y.dtype == torch.float32
+
+
+def test_registered_operators_pass_opcheck_on_cpu():
+    """The operators exist under torch.ops.fsoftmax with schema, fake implementation and (softmax) autograd
+    registration that torch's own checker accepts; on CPU tensors they compute with eager PyTorch."""
+    ops = torch.ops.fsoftmax
+    for name in ("softmax", "softmax_backward", "log_softmax", "layer_norm", "group_norm"):
+        assert hasattr(ops, name)
+    torch.manual_seed(3)
+    cases = [(ops.softmax, (torch.randn(3, 5, requires_grad=True), 0.5)),
+             (ops.softmax_backward, (torch.randn(3, 5), torch.softmax(torch.randn(3, 5), -1), 0.5)),
+             (ops.log_softmax, (torch.randn(3, 5),)),
+             (ops.layer_norm, (torch.randn(3, 5), torch.randn(5), None, 1e-5)),
+             (ops.group_norm, (torch.randn(2, 4, 5), 2, None, torch.randn(4), 1e-5))]
+    for op, args in cases:
+        res = torch.library.opcheck(op, args)
+        assert all(v == "SUCCESS" for v in res.values()), (op, res)
+    x = torch.randn(4, 9, dtype=torch.float64, requires_grad=True)
+    g = torch.randn(4, 9, dtype=torch.float64)
+    ops.softmax(x, 0.5).backward(g)
+    xr = x.detach().clone().requires_grad_(True)
+    torch.softmax(xr * 0.5, -1).backward(g)
+    assert torch.allclose(x.grad, xr.grad, atol=1e-12)
+
+
+@pytest.mark.gpu
+def test_softmax_operator_forward_and_backward_run_the_library():
+    """torch.ops.fsoftmax.softmax on a tensor that requires grad: forward through fs_softmax, x.grad through
+    fs_softmax_backward, both against the oracle under the bars of their entry points."""
+    from oracle import fno, fso
+    from paper_2607_24762_b200 import workloads as W
+    torch.manual_seed(5)
+    for tdt, dt, rows, cols, scale in ((torch.float32, W.FP32, 48, 4096, 1.0), (torch.bfloat16, W.BF16, 64, 2048, 0.125),
+                                       (torch.float16, W.FP16, 6, 65536, 0.5)):
+        x = (torch.randn(rows, cols, device="cuda") * 2).to(tdt).requires_grad_(True)
+        dy = torch.randn(rows, cols, device="cuda").to(tdt)
+        torch_op.stats(reset=True)
+        y = torch_op.softmax(x, -1, scale=scale)                    # the guarded front end routes to the operator
+        y.backward(dy)
+        assert torch_op.stats() == {"library": 2}                   # one forward, one backward kernel; nothing went to eager
+        bits = (lambda t: t.detach().view(torch.int16).cpu().numpy().view(np.uint16)) if dt != W.FP32 else (lambda t: t.detach().cpu().numpy())
+        assert fso.compare(bits(y), dt, fso.softmax_f64(bits(x), dt, scale)).ok(dt)
+        g64, y64 = fso.widen(bits(dy), dt), fso.widen(bits(y), dt)
+        es = abs(scale) * np.abs(y64) * (np.abs(g64) + np.abs(g64 * y64).sum(axis=1, keepdims=True))
+        rep = fno.compare(bits(x.grad), dt, fso.softmax_backward_f64(bits(dy), bits(y), dt, scale), es)
+        assert rep.ok(dt), rep
+    # called directly, as a traced graph would: same kernels; a tensor the guard refuses is computed by eager
+    xs = torch.randn(8, 512, device="cuda")
+    assert torch.allclose(torch.ops.fsoftmax.softmax(xs, 1.0), torch.softmax(xs, -1), atol=1e-6)
+    xt = torch.randn(512, 8, device="cuda").t()
+    assert torch.allclose(torch.ops.fsoftmax.softmax(xt, 1.0), torch.softmax(xt, -1), atol=1e-6)
+    assert torch_op.stats()["eager:operator called on tensors the guard refuses"] == 1
