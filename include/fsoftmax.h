@@ -60,7 +60,8 @@ typedef enum {
     FS_ERR_INVALID_ARG = 1,    /* null pointer, negative size, unknown dtype/kernel, non-finite scale, partial overlap */
     FS_ERR_UNSUPPORTED = 2,    /* a forced kernel cannot handle this shape/alignment/launch geometry */
     FS_ERR_CUDA = 3,           /* a CUDA call failed; see fs_last_cuda_error() */
-    FS_ERR_DEVICE_TIMEOUT = 4  /* a bounded device-side wait expired (reported by fs_device_status) */
+    FS_ERR_DEVICE_TIMEOUT = 4, /* a bounded device-side wait expired (reported by fs_device_status) */
+    FS_ERR_DEVICE_BOUNDS = 5   /* checked build only: a kernel tried to touch memory outside its call's tensors */
 } fs_status;
 
 /* The kernels behind the size-based dispatcher (the "variants" of the operator in the sense of
@@ -360,6 +361,26 @@ int fs_static_status(void);
  *           (a few thousand: long enough for the copies to land) and restore the default after.
  *           y receives the normal result when the cap was long enough for the data to arrive.
  */
+/*
+ * The checked build (libfsoftmax_debug.so: the same sources compiled with -DFS_DEBUG_BOUNDS; the paper's
+ * validator lists illegal memory accesses among the failures it must catch, Sec. III-C). In it every
+ * global load, store and bulk copy of every kernel is checked against the address ranges of the
+ * tensors its entry point was given; an access outside them, or a store into an input, is skipped and
+ * recorded instead of performed: fs_device_status then returns FS_ERR_DEVICE_BOUNDS (once) and
+ * fs_debug_bad_address the first offending address. Several times slower; one stream at a time (the
+ * ranges are one table per device); fs_softmax_static and fs_softmax_host go unchecked.
+ *   fs_debug_checked_build()        1 in the checked build, 0 in the normal one.
+ *   fs_debug_bad_address(&a)        reads and clears the first refused address (0 if none); synchronises.
+ *                                   FS_ERR_UNSUPPORTED in the normal build.
+ *   fs_debug_shrink_writable(n)     self-test: until called again with 0, the output ranges this thread
+ *                                   registers end n bytes early, so a correct kernel "overruns" them by
+ *                                   n bytes without touching anything it should not; the checker must
+ *                                   refuse exactly those stores. FS_ERR_UNSUPPORTED in the normal build.
+ */
+int fs_debug_checked_build(void);
+int fs_debug_bad_address(uint64_t* address);
+int fs_debug_shrink_writable(int64_t bytes);
+
 int fs_debug_set_wait_polls(int polls);
 int fs_debug_wait_probe(void* stream);
 int fs_debug_softmax_expire(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale, void* stream,

@@ -12,7 +12,7 @@ import os
 import threading
 
 FS_DTYPE_FP32, FS_DTYPE_BF16, FS_DTYPE_FP16 = 0, 1, 2
-FS_OK, FS_ERR_INVALID_ARG, FS_ERR_UNSUPPORTED, FS_ERR_CUDA, FS_ERR_DEVICE_TIMEOUT = 0, 1, 2, 3, 4
+FS_OK, FS_ERR_INVALID_ARG, FS_ERR_UNSUPPORTED, FS_ERR_CUDA, FS_ERR_DEVICE_TIMEOUT, FS_ERR_DEVICE_BOUNDS = 0, 1, 2, 3, 4, 5
 FS_KERNEL_AUTO, FS_KERNEL_WARP, FS_KERNEL_BLOCK, FS_KERNEL_BLOCK_TMA, FS_KERNEL_CLUSTER, FS_KERNEL_GENERIC = range(6)
 FS_STATIC_MAX_ROW_BYTES = 16 * 192 * 1024
 FS_STATIC_SCRATCH_BYTES = 65536
@@ -21,7 +21,9 @@ FS_ROUTER_MAX_K = 64
 KERNELS = {"auto": 0, "warp": 1, "block": 2, "block_tma": 3, "cluster": 4, "generic": 5}
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libfsoftmax.so")
+# FSOFTMAX_LIB (read at import) selects another build of the same library, e.g. the checked one
+# (libfsoftmax_debug.so, see _build.build_library(debug=True)); there is still no fallback.
+LIB_PATH = os.environ.get("FSOFTMAX_LIB") or os.path.join(_HERE, "libfsoftmax.so")
 _lock = threading.Lock()
 _lib = None
 
@@ -83,6 +85,12 @@ def lib() -> ctypes.CDLL:
             L.fs_debug_wait_probe.restype = ci
             L.fs_debug_softmax_expire.argtypes = [vp, vp, i64, i64, ci, f32, vp, ci, ci]
             L.fs_debug_softmax_expire.restype = ci
+            L.fs_debug_checked_build.argtypes = []
+            L.fs_debug_checked_build.restype = ci
+            L.fs_debug_bad_address.argtypes = [ctypes.POINTER(ctypes.c_uint64)]
+            L.fs_debug_bad_address.restype = ci
+            L.fs_debug_shrink_writable.argtypes = [i64]
+            L.fs_debug_shrink_writable.restype = ci
             L.fs_copy.argtypes = [vp, vp, i64, vp]
             L.fs_copy.restype = ci
             L.fs_device_status.argtypes = []
@@ -218,6 +226,23 @@ def fs_softmax_static(x, y, rows: int, cols: int, dtype: int, scale: float = 1.0
 def fs_static_status() -> int:
     """Reads and clears the status word of fs_softmax_static's fixed array (synchronises; allocates nothing)."""
     return lib().fs_static_status()
+
+
+def fs_debug_checked_build() -> bool:
+    """Whether the loaded library is the checked build (every global access range-checked)."""
+    return bool(lib().fs_debug_checked_build())
+
+
+def fs_debug_bad_address() -> int:
+    """Checked build: the first address a kernel was refused since the last call (0 if none)."""
+    a = ctypes.c_uint64(0)
+    _check(lib().fs_debug_bad_address(ctypes.byref(a)), "fs_debug_bad_address")
+    return int(a.value)
+
+
+def fs_debug_shrink_writable(nbytes: int) -> None:
+    """Checked build self-test: output ranges registered by this thread end `nbytes` early (0 restores)."""
+    _check(lib().fs_debug_shrink_writable(nbytes), "fs_debug_shrink_writable")
 
 
 def fs_debug_set_wait_polls(polls: int) -> None:

@@ -6,6 +6,7 @@
 #include <atomic>
 #include <cmath>
 #include <cstdio>
+#include <cstddef>
 #include <cstdlib>
 #include <cstring>
 #include <initializer_list>
@@ -400,8 +401,40 @@ bool pdl_enabled() {
     return v;
 }
 
+// Checked build (-DFS_DEBUG_BOUNDS): the entry points register the address ranges of their tensors,
+// every launch uploads them (with the device's status word) to the table the access helpers consult.
+// One table per device image: launches from several host threads or streams at once would overwrite
+// each other's ranges, so the checked library is for single-stream debugging runs.
+struct TensorRange { const void* p; unsigned long long bytes; int writable; };
+#ifdef FS_DEBUG_BOUNDS
+thread_local DebugRanges t_dbg = {};
+thread_local long long t_dbg_shrink = 0;          // self-test: the writable ranges end this many bytes early
+void dbg_register(int* status, std::initializer_list<TensorRange> ranges) {
+    t_dbg = DebugRanges{};
+    t_dbg.status = status;
+    for (const TensorRange& r : ranges) {
+        if (!r.p || t_dbg.n >= 8) continue;
+        const unsigned long long lo = reinterpret_cast<unsigned long long>(r.p);
+        unsigned long long hi = lo + r.bytes;
+        if (r.writable && t_dbg_shrink > 0) hi -= std::min<unsigned long long>(r.bytes, static_cast<unsigned long long>(t_dbg_shrink));
+        t_dbg.lo[t_dbg.n] = lo; t_dbg.hi[t_dbg.n] = hi; t_dbg.writable[t_dbg.n] = r.writable;
+        ++t_dbg.n;
+    }
+}
+#define FS_DBG_RANGES(...) do { Device* d__ = nullptr; const int r__ = get_device(&d__); if (r__ != FS_OK) return r__; \
+                                dbg_register(d__->status, {__VA_ARGS__}); } while (0)
+#else
+#define FS_DBG_RANGES(...) do { } while (0)
+#endif
+
 template <typename... Args>
 int launch(const void* fn, int64_t grid, int threads, size_t smem, int cs, cudaStream_t st, Args... args) {
+#ifdef FS_DEBUG_BOUNDS
+    {   // keep the first refused address of earlier launches
+        DebugRanges up = t_dbg;
+        FS_CUDA(cudaMemcpyToSymbolAsync(g_dbg, &up, offsetof(DebugRanges, first_bad), 0, cudaMemcpyHostToDevice, st));
+    }
+#endif
     void* argv[] = {static_cast<void*>(&args)...};
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(grid), 1, 1);
@@ -1536,6 +1569,7 @@ int fs_softmax_ex(const void* x, void* y, int64_t rows, int64_t cols, int dtype,
     if (cluster < 0 || cluster > kMaxCluster) return FS_ERR_INVALID_ARG;
     if (rows == 0 || cols == 0) return FS_OK;
     FS_CHECK_PTRS(x, y);
+    FS_DBG_RANGES({x, (unsigned long long)(rows * cols * elem_size(dtype)), 0}, {y, (unsigned long long)(rows * cols * elem_size(dtype)), 1});
     return run(x, y, rows, cols, dtype, scale, static_cast<cudaStream_t>(stream), kernel, threads, cluster);
 }
 
@@ -1550,6 +1584,7 @@ int fs_softmax_causal(const void* x, void* y, int64_t rows, int64_t cols, int64_
     if (rows == 0 || cols == 0) return FS_OK;
     if (q_offset > (int64_t(1) << 41) || q_offset < -(int64_t(1) << 41)) return FS_ERR_INVALID_ARG;
     FS_CHECK_PTRS(x, y);
+    FS_DBG_RANGES({x, (unsigned long long)(rows * cols * elem_size(dtype)), 0}, {y, (unsigned long long)(rows * cols * elem_size(dtype)), 1});
     return run_causal(x, y, rows, cols, q_offset, dtype, scale, static_cast<cudaStream_t>(stream));
 }
 
@@ -1565,6 +1600,7 @@ int fs_router_topk(const void* x, float* w, int32_t* idx, int64_t rows, int64_t 
     if (ptr_align(x) < 16 || (cols * elem_size(dtype)) % 16 != 0) return FS_ERR_UNSUPPORTED;
     if (ptr_align(w) < 4 || ptr_align(idx) < 4) return FS_ERR_INVALID_ARG;
     FS_CHECK_PTRS(x, w, idx);
+    FS_DBG_RANGES({x, (unsigned long long)(rows * cols * elem_size(dtype)), 0}, {w, (unsigned long long)(rows * k * 4), 1}, {idx, (unsigned long long)(rows * k * 4), 1});
     const int64_t nvec = cols * elem_size(dtype) / 16;
     WarpGeom g;
     if (!warp_geom(nvec, dtype, &g) || g.vpl * (dtype == FS_DTYPE_FP32 ? 4 : 8) > 32) return FS_ERR_UNSUPPORTED;
@@ -1598,6 +1634,7 @@ int fs_log_softmax(const void* x, void* y, int64_t rows, int64_t cols, int dtype
     if (v != FS_OK) return v;
     if (rows == 0 || cols == 0) return FS_OK;
     FS_CHECK_PTRS(x, y);
+    FS_DBG_RANGES({x, (unsigned long long)(rows * cols * elem_size(dtype)), 0}, {y, (unsigned long long)(rows * cols * elem_size(dtype)), 1});
     return run_log_softmax(x, y, rows, cols, dtype, scale, OUT_LOG, static_cast<cudaStream_t>(stream));
 }
 
@@ -1610,6 +1647,8 @@ int fs_softmax_masked(const void* x, const void* mask, void* y, int64_t rows, in
     if (rows == 0 || cols == 0) return FS_OK;
     if (!mask) return FS_ERR_INVALID_ARG;
     FS_CHECK_PTRS(x, mask, y);
+    FS_DBG_RANGES({x, (unsigned long long)(rows * cols * elem_size(dtype)), 0}, {mask, (unsigned long long)(rows / heads * cols * elem_size(dtype)), 0},
+                  {y, (unsigned long long)(rows * cols * elem_size(dtype)), 1});
     return run_softmax_masked(x, mask, y, rows, cols, q_rows, heads, dtype, scale, static_cast<cudaStream_t>(stream));
 }
 
@@ -1620,6 +1659,8 @@ int fs_softmax_backward(const void* dy, const void* y, void* dx, int64_t rows, i
     if (v != FS_OK) return v;
     if (rows == 0 || cols == 0) return FS_OK;
     FS_CHECK_PTRS(dy, y, dx);
+    FS_DBG_RANGES({dy, (unsigned long long)(rows * cols * elem_size(dtype)), 0}, {y, (unsigned long long)(rows * cols * elem_size(dtype)), 0},
+                  {dx, (unsigned long long)(rows * cols * elem_size(dtype)), 1});
     return run_softmax_backward(dy, y, dx, rows, cols, dtype, scale, static_cast<cudaStream_t>(stream));
 }
 
@@ -1634,6 +1675,7 @@ int fs_softmax_f32out(const void* x, float* y, int64_t rows, int64_t cols, int d
     const uintptr_t na = static_cast<uintptr_t>(rows * cols * 2), nb = static_cast<uintptr_t>(rows * cols * 4);
     if (a < b + nb && b < a + na) return FS_ERR_INVALID_ARG;          // the tensors differ in size: no overlap at all
     FS_CHECK_PTRS(x, y);
+    FS_DBG_RANGES({x, (unsigned long long)(rows * cols * 2), 0}, {y, (unsigned long long)(rows * cols * 4), 1});
     return run_log_softmax(x, y, rows, cols, dtype, scale, OUT_PROB32, static_cast<cudaStream_t>(stream));
 }
 
@@ -1643,6 +1685,8 @@ int fs_layer_norm(const void* x, const void* gamma, const void* beta, void* y, i
     if (v != FS_OK || rows == 0 || cols == 0) return v;
     const int aff = (gamma || beta) ? 1 : 0;
     FS_CHECK_PTRS(x, gamma, beta, y);
+    FS_DBG_RANGES({x, (unsigned long long)(rows * cols * elem_size(dtype)), 0}, {gamma, (unsigned long long)(cols * elem_size(dtype)), 0},
+                  {beta, (unsigned long long)(cols * elem_size(dtype)), 0}, {y, (unsigned long long)(rows * cols * elem_size(dtype)), 1});
     return run_norm(x, gamma, beta, y, rows, cols, dtype, eps, aff, 1, 1, static_cast<cudaStream_t>(stream));
 }
 
@@ -1658,6 +1702,8 @@ int fs_group_norm(const void* x, const void* gamma, const void* beta, void* y, i
     if (v != FS_OK || rows == 0 || cols == 0) return v;
     const int aff = (gamma || beta) ? 2 : 0;
     FS_CHECK_PTRS(x, gamma, beta, y);
+    FS_DBG_RANGES({x, (unsigned long long)(rows * cols * elem_size(dtype)), 0}, {gamma, (unsigned long long)(channels * elem_size(dtype)), 0},
+                  {beta, (unsigned long long)(channels * elem_size(dtype)), 0}, {y, (unsigned long long)(rows * cols * elem_size(dtype)), 1});
     return run_norm(x, gamma, beta, y, rows, cols, dtype, eps, aff, spatial, groups, static_cast<cudaStream_t>(stream));
 }
 
@@ -1682,6 +1728,7 @@ int fs_copy(const void* x, void* y, int64_t bytes, void* stream) {
     if (bytes == 0) return FS_OK;
     if (!x || !y || ptr_align(x) < 16 || ptr_align(y) < 16) return FS_ERR_INVALID_ARG;
     FS_CHECK_PTRS(x, y);
+    FS_DBG_RANGES({x, (unsigned long long)bytes, 0}, {y, (unsigned long long)bytes, 1});
     Device* dev = nullptr;
     int rc = get_device(&dev);
     if (rc != FS_OK) return rc;
@@ -1702,6 +1749,9 @@ int fs_softmax_host(const void* x_host, void* y_host, int64_t rows, int64_t cols
     if (rc != FS_OK) return rc;
     Device& dev = *devp;
     std::lock_guard<std::mutex> lk(g_host_mu);
+#ifdef FS_DEBUG_BOUNDS
+    t_dbg = DebugRanges{};              // the staging buffers are the library's own: unchecked
+#endif
 
     const size_t row_bytes = static_cast<size_t>(cols) * elem_size(dtype);
     // chunk size: small enough that filling and draining the pipeline costs little, large enough
@@ -1803,7 +1853,41 @@ int fs_device_status(void) {
     FS_CUDA(cudaDeviceSynchronize());
     FS_CUDA(cudaMemcpy(&word, dev->status, sizeof(int), cudaMemcpyDeviceToHost));
     if (word) FS_CUDA(cudaMemset(dev->status, 0, sizeof(int)));
+    if (word & DEV_BOUNDS) return FS_ERR_DEVICE_BOUNDS;
     return (word & DEV_TIMEOUT) ? FS_ERR_DEVICE_TIMEOUT : FS_OK;
+}
+
+int fs_debug_checked_build(void) {
+#ifdef FS_DEBUG_BOUNDS
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+int fs_debug_shrink_writable(int64_t bytes) {
+#ifdef FS_DEBUG_BOUNDS
+    t_dbg_shrink = bytes > 0 ? bytes : 0;
+    return FS_OK;
+#else
+    (void)bytes;
+    return FS_ERR_UNSUPPORTED;
+#endif
+}
+
+int fs_debug_bad_address(uint64_t* address) {
+    if (!address) return FS_ERR_INVALID_ARG;
+    *address = 0;
+#ifdef FS_DEBUG_BOUNDS
+    unsigned long long bad = 0, zero = 0;
+    FS_CUDA(cudaDeviceSynchronize());
+    FS_CUDA(cudaMemcpyFromSymbol(&bad, g_dbg, sizeof(bad), offsetof(DebugRanges, first_bad)));
+    if (bad) FS_CUDA(cudaMemcpyToSymbol(g_dbg, &zero, sizeof(zero), offsetof(DebugRanges, first_bad)));
+    *address = bad;
+    return FS_OK;
+#else
+    return FS_ERR_UNSUPPORTED;
+#endif
 }
 
 int fs_softmax_static(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float scale, void* stream) {
@@ -1813,6 +1897,9 @@ int fs_softmax_static(const void* x, void* y, int64_t rows, int64_t cols, int dt
     if (!fast_path_ok(cols, dtype, ptr_align(x), ptr_align(y))) return FS_ERR_UNSUPPORTED;
     const int64_t nvec = cols * elem_size(dtype) / 16;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+#ifdef FS_DEBUG_BOUNDS
+    t_dbg = DebugRanges{};              // registering ranges needs the allocated status word: this entry point goes unchecked
+#endif
     std::lock_guard<std::mutex> lk(g_static_mu);
     StaticDevice* sdp = nullptr;
     int rc = get_static_device(&sdp);
@@ -1905,6 +1992,7 @@ const char* fs_strerror(int status) {
         case FS_ERR_UNSUPPORTED: return "unsupported shape, alignment or launch geometry for the requested kernel";
         case FS_ERR_CUDA: return "CUDA error (see fs_last_cuda_error)";
         case FS_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+        case FS_ERR_DEVICE_BOUNDS: return "checked build: a kernel tried to access memory outside the tensors of its call (the access was skipped)";
         default: return "unknown status";
     }
 }
@@ -1921,6 +2009,12 @@ const char* fs_kernel_name(int kernel) {
     }
 }
 
-const char* fs_version(void) { return "libfsoftmax 0.1 (sm_100a)"; }
+const char* fs_version(void) {
+#ifdef FS_DEBUG_BOUNDS
+    return "libfsoftmax 0.2 (sm_100a, checked build)";
+#else
+    return "libfsoftmax 0.2 (sm_100a)";
+#endif
+}
 
 }  // extern "C"

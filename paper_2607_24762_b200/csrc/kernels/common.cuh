@@ -12,7 +12,7 @@ namespace fsm {
 enum : int { DT_F32 = 0, DT_BF16 = 1, DT_F16 = 2 };
 
 // Status bits a kernel may OR into the per-device status word.
-enum : int { DEV_TIMEOUT = 1 };
+enum : int { DEV_TIMEOUT = 1, DEV_BOUNDS = 2 };
 // Poll cap of the bounded waits: about two seconds.
 constexpr int kDefaultWaitPolls = 1 << 23;
 
@@ -39,9 +39,44 @@ template <> struct Traits<DT_F32>  { static constexpr int VE = 4; static constex
 template <> struct Traits<DT_BF16> { static constexpr int VE = 8; static constexpr int ESZ = 2; };
 template <> struct Traits<DT_F16>  { static constexpr int VE = 8; static constexpr int ESZ = 2; };
 
+// ---- checked build ------------------------------------------------------------------------------
+// With -DFS_DEBUG_BOUNDS (libfsoftmax_debug.so) every global access of every kernel -- they all go
+// through the helpers below -- is checked against the address ranges of the tensors the host
+// registered for the launch. An access outside them (or a store into a read-only tensor) is NOT
+// performed: it sets DEV_BOUNDS in the status word, records the first offending address and the
+// kernel carries on (a load yields zeros), so an indexing error shows up as a status and an address
+// instead of a fault. The stand-in for a memory checker on machines where none can be run.
+#ifdef FS_DEBUG_BOUNDS
+struct DebugRanges {
+    unsigned long long lo[8], hi[8];
+    int writable[8];
+    int n;                              // 0: nothing registered for this launch, nothing is checked
+    int* status;
+    unsigned long long first_bad;       // 0 until an access was refused
+};
+__device__ DebugRanges g_dbg;
+__device__ __forceinline__ bool dbg_ok(const void* p, unsigned long long bytes, bool write) {
+    if (g_dbg.n == 0) return true;
+    const unsigned long long a = reinterpret_cast<unsigned long long>(p);
+    for (int i = 0; i < g_dbg.n; ++i)
+        if (a >= g_dbg.lo[i] && a + bytes <= g_dbg.hi[i] && (!write || g_dbg.writable[i])) return true;
+    atomicOr(g_dbg.status, DEV_BOUNDS);
+    atomicCAS(&g_dbg.first_bad, 0ull, a);
+    return false;
+}
+#define FS_DBG_LOAD(p, bytes, zero)  do { if (!dbg_ok((p), (bytes), false)) return zero; } while (0)
+#define FS_DBG_STORE(p, bytes)       do { if (!dbg_ok((p), (bytes), true)) return; } while (0)
+#define FS_DBG_TOUCH(p)              do { if (!dbg_ok((p), 0, false)) return; } while (0)
+#else
+#define FS_DBG_LOAD(p, bytes, zero)  do { } while (0)
+#define FS_DBG_STORE(p, bytes)       do { } while (0)
+#define FS_DBG_TOUCH(p)              do { } while (0)
+#endif
+
 // ---- 128-bit streaming global access (every byte is touched once: evict-first) -------------
 
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+    FS_DBG_LOAD(p, 16, make_uint4(0u, 0u, 0u, 0u));
     uint4 v;
     asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
@@ -49,6 +84,7 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
 }
 
 __device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
+    FS_DBG_STORE(p, 16);
     asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};"
                  :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
@@ -136,12 +172,14 @@ __device__ __forceinline__ uint4 pack(const float (&f)[Traits<DT>::VE]) {
 }
 
 template <int DT> __device__ __forceinline__ float load_elem(const void* p, int64_t i) {
+    FS_DBG_LOAD(static_cast<const char*>(p) + i * Traits<DT>::ESZ, Traits<DT>::ESZ, 0.0f);
     if constexpr (DT == DT_F32) return static_cast<const float*>(p)[i];
     else if constexpr (DT == DT_BF16) return __bfloat162float(static_cast<const __nv_bfloat16*>(p)[i]);
     else return __half2float(static_cast<const __half*>(p)[i]);
 }
 
 template <int DT> __device__ __forceinline__ void store_elem(void* p, int64_t i, float v) {
+    FS_DBG_STORE(static_cast<char*>(p) + i * Traits<DT>::ESZ, Traits<DT>::ESZ);
     if constexpr (DT == DT_F32) static_cast<float*>(p)[i] = v;
     else if constexpr (DT == DT_BF16) static_cast<__nv_bfloat16*>(p)[i] = __float2bfloat16_rn(v);
     else static_cast<__half*>(p)[i] = __float2half_rn(v);
@@ -436,6 +474,12 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 // Global -> this block's shared memory, completion counted in bytes on `bar`.
 // dst, src and bytes must be multiples of 16.
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+#ifdef FS_DEBUG_BOUNDS
+    if (!dbg_ok(src, bytes, false)) {       // refused: complete the barrier's byte count without copying
+        asm volatile("mbarrier.complete_tx.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
+        return;
+    }
+#endif
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  :: "r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
@@ -452,6 +496,7 @@ __device__ __forceinline__ void bulk_load_row(uint32_t dst, const char* src, uin
 
 // Asks the L2 cache for `bytes` (a multiple of 16) at `src`: no destination, nothing to wait for.
 __device__ __forceinline__ void l2_prefetch(const char* src, uint32_t bytes) {
+    FS_DBG_TOUCH(src);                      // a prefetch must at least start inside a registered tensor
     for (uint32_t off = 0; off < bytes; off += 32768u) {
         const uint32_t n = min(32768u, bytes - off);
         asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" :: "l"(src + off), "r"(n) : "memory");

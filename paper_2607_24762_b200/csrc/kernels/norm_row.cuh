@@ -88,6 +88,7 @@ __device__ __forceinline__ float rstd_of(float var, float eps) {
 }
 
 __device__ __forceinline__ uint4 ld_cached(const uint4* p) {
+    FS_DBG_LOAD(p, 16, make_uint4(0u, 0u, 0u, 0u));
     uint4 v;
     asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
     return v;
@@ -535,6 +536,7 @@ norm_smem_kernel(const NormParams p, const uint32_t stage_bytes, const int slice
 // HBM traffic stays one read and one write per element when x fits L2; otherwise two reads.
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint4 ld_keep(const uint4* p) {
+    FS_DBG_LOAD(p, 16, make_uint4(0u, 0u, 0u, 0u));
     uint4 v;
     asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
     return v;

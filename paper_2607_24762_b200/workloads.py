@@ -215,19 +215,30 @@ class Checksum:
         self.acc = np.uint64(0)
         self.words = 0
 
-    def update(self, x: np.ndarray) -> "Checksum":
+    def update(self, x: np.ndarray, threads: int = 8) -> "Checksum":
         raw = np.ascontiguousarray(x).view(np.uint8).ravel()
         pad = (-raw.size) % 8
         if pad:
             raw = np.concatenate([raw, np.zeros(pad, dtype=np.uint8)])
         words = raw.view(np.uint64)
-        step = 1 << 22
-        for i in range(0, words.size, step):                      # bounded temporaries
+        step = 1 << 21                                            # bounded temporaries; pieces are independent
+        base = self.words
+
+        def piece(i: int) -> np.uint64:
             part = words[i:i + step]
-            idx = np.arange(self.words + i + 1, self.words + i + part.size + 1, dtype=np.uint64)
+            idx = np.arange(base + i + 1, base + i + part.size + 1, dtype=np.uint64)
             with np.errstate(over="ignore"):
                 mixed = (part ^ (idx * np.uint64(0x9E3779B97F4A7C15))) * np.uint64(0x100000001B3)
-            self.acc ^= np.bitwise_xor.reduce(mixed)
+            return np.bitwise_xor.reduce(mixed)
+
+        starts = range(0, words.size, step)
+        if threads > 1 and len(starts) > 1:
+            with ThreadPoolExecutor(max_workers=threads) as ex:
+                parts = list(ex.map(piece, starts))
+        else:
+            parts = [piece(i) for i in starts]
+        for v in parts:
+            self.acc ^= v
         self.words += words.size
         return self
 

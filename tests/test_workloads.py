@@ -71,3 +71,20 @@ def test_bf16_rounding_is_single_rounding():
     assert list(W.f64_to_bf16_bits(v)) == [0x3F81, 0x3F80, 0x3F82]
     assert list(W.f32_to_bf16_bits(v.astype(np.float32))) == [0x3F80, 0x3F80, 0x3F82]
     assert list(W.bf16_bits_to_f32(np.array([0x3F80, 0xC000], dtype=np.uint16))) == [1.0, -2.0]
+
+
+def test_streaming_checksum_equals_the_whole_buffer_checksum():
+    """Checksum taken slab by slab (what the benchmark records for the 4 GiB workload) is the checksum of the whole."""
+    w = W.WORKLOADS["cfg2"]
+    x = W.generate_rows(w, 0, 700)
+    whole = W.checksum(x)
+    for slab in (1, 128, 699, 700):
+        c = W.Checksum()
+        for r0 in range(0, 700, slab):
+            c.update(x[r0:r0 + slab], threads=1 if slab == 1 else 4)
+        assert c.value() == whole
+    y = x.copy()
+    y[350, 7] ^= 1
+    assert W.Checksum().update(y).value() != whole
+    a, b = x[:300].copy(), x[300:].copy()
+    assert W.Checksum().update(b).update(a).value() != whole          # order-sensitive
