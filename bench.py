@@ -347,6 +347,36 @@ def fit_fixed_cost(w: W.Workload, l2_bytes: int, steps: int = 200):
     return out
 
 
+def time_static(w: W.Workload, steps: int, l2_bytes: int):
+    """fs_softmax_static against fs_softmax on device-seeded data of the workload's shape: the same kernels, the
+    scratch in the library's fixed device array instead of allocated memory."""
+    import torch
+
+    import paper_2607_24762_b200 as fs
+    lib = fs.binding.lib()
+    stream = torch.cuda.current_stream()
+    sh = stream.cuda_stream
+    tdt = {W.FP32: torch.float32, W.BF16: torch.bfloat16, W.FP16: torch.float16}[w.dtype]
+    n_pairs = int(max(1, min(8, math.ceil(8 * l2_bytes / w.min_bytes))))
+    g = torch.Generator(device="cuda").manual_seed(11)
+    xs = [(torch.randn((w.rows, w.cols), generator=g, device="cuda") * 3.0).to(tdt) for _ in range(n_pairs)]
+    ys = [torch.empty_like(x) for x in xs]
+    out = {"what": f"fs_softmax_static on {w.name} ({w.rows} x {w.cols} {W.DTYPE_NAME[w.dtype]})", "steps": steps}
+    for name, fn in (("static", lib.fs_softmax_static), ("allocating", lib.fs_softmax)):
+        def launch(i):
+            st = fn(xs[i % n_pairs].data_ptr(), ys[i % n_pairs].data_ptr(), w.rows, w.cols, w.dtype, 1.0, sh)
+            if st != 0:
+                raise RuntimeError(fs.fs_strerror(st))
+        for i in range(5):
+            launch(i)
+        ms = statistics.median(run_trains(launch, steps, stream, n_trains=9, budget_ms=1000.0)) / steps
+        out[name + "_ms_per_step"] = round(ms, 6)
+        out[name + "_GB/s"] = round(w.min_bytes / (ms * 1e-3) / 1e9, 1)
+    if fs.fs_static_status() != 0:
+        raise RuntimeError("fs_static_status reported an expired wait")
+    return out
+
+
 def time_router(w: W.Workload, k: int, steps: int, warmup: int, l2_bytes: int):
     """fs_router_topk on the router workload: reads x once, writes k weights and k columns per row."""
     import torch
@@ -956,6 +986,16 @@ def main():
                                          "algorithmic_bytes": alg, "GB/s": round(gbs, 1),
                                          "frac_of_measured_copy": round(gbs / peak, 4),
                                          "speedup_vs_cfg5": round(results["cfg5"]["ms_per_step"] / cms, 3)}
+            # the entry point that allocates nothing, on the vocabulary-sized workload (the split-row kernel with its
+            # status word in the fixed device array) and on rows beyond a cluster's shared memory (two kernels, the
+            # pairs between them in the same array)
+            try:
+                others["cfg4_static"] = time_static(W.WORKLOADS["cfg4"], 300, l2)
+                import dataclasses
+                others["long_rows_static"] = time_static(dataclasses.replace(W.WORKLOADS["cfg4"], name="16 rows of 8 MiB", rows=16,
+                                                                             cols=1 << 22), 100, l2)
+            except Exception as exc:
+                others["cfg4_static"] = {"error": str(exc)[:200]}
             # the router step (softmax over experts + top-8, renormalised) on the router workload
             rw = W.WORKLOADS["cfg3"]
             try:

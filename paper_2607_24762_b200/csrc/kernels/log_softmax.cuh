@@ -339,6 +339,7 @@ lsm_smem_kernel(const LsmParams p, const uint32_t stage_bytes, const int slice, 
     block_merge_pairs<false>(R, s, wp[0], p.c);
     if (cs > 1) {
         if (tid < cs) st_async_v2(map_to_rank(smem_u32(&xchg[q]), tid), R, s, map_to_rank(smem_u32(&xbar), tid));
+        cluster_arrive_relaxed();          // exit guard: waited for after pass 2 (see smem_row.cuh)
         if (tid < 32 && alive) alive = mbar_wait_warp(smem_u32(&xbar), 0u, p.status);
         if (T > 32) __syncthreads();
         R = ident; s = 0.0f;
@@ -362,6 +363,7 @@ lsm_smem_kernel(const LsmParams p, const uint32_t stage_bytes, const int slice, 
                 lsm_emit<DT, OUT>(flip_vec(raw[u], p.flip), R2, c2, s2, k2, yrow, int64_t(v0) + cbase + u * 32);
         }
     }
+    if (cs > 1) cluster_wait_acquire();    // no block leaves while a peer's deposit into it is still to be issued
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -502,6 +502,7 @@ norm_smem_kernel(const NormParams p, const uint32_t stage_bytes, const int slice
             st_async_v2(dst, st.n, st.mean, bar);
             st_async_v2(dst + 8u, st.m2, 0.0f, bar);
         }
+        cluster_arrive_relaxed();          // exit guard: waited for after pass 2 (see smem_row.cuh)
         if (tid < 32 && alive) alive = mbar_wait_warp(smem_u32(&xbar), 0u, p.status);
         if (T > 32) __syncthreads();
         const float4 v = lane < static_cast<int>(cs) ? xchg[lane] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
@@ -524,6 +525,7 @@ norm_smem_kernel(const NormParams p, const uint32_t stage_bytes, const int slice
     } else {
         norm_pass2<DT, FULL, AFF, false, false>(p, c2, row);
     }
+    if (cs > 1) cluster_wait_acquire();    // no block leaves while a peer's deposit into it is still to be issued
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -271,6 +271,7 @@ smb_smem_kernel(const SmbParams p, const uint32_t stage_bytes, const int slice, 
     }
     if (cs > 1) {
         if (tid < cs) st_async_v2(map_to_rank(smem_u32(&xchg[q]), tid), dot, 0.0f, map_to_rank(smem_u32(&xbar), tid));
+        cluster_arrive_relaxed();          // exit guard: waited for after pass 2 (see smem_row.cuh)
         if (tid < 32 && alive) alive = mbar_wait_warp(smem_u32(&xbar), 0u, p.status);
         if (T > 32) __syncthreads();
         float a = 0.0f, b = 0.0f;
@@ -303,6 +304,7 @@ smb_smem_kernel(const SmbParams p, const uint32_t stage_bytes, const int slice, 
             }
         }
     }
+    if (cs > 1) cluster_wait_acquire();    // no block leaves while a peer's deposit into it is still to be issued
 }
 
 // ---------------------------------------------------------------------------------------------

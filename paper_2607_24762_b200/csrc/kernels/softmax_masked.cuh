@@ -370,6 +370,7 @@ sm_masked_smem_kernel(const MaskedParams p, const uint32_t stage_bytes, const in
     block_merge_pairs<false>(R, s, wp, 1.0f);
     if (cs > 1) {
         if (tid < cs) st_async_v2(map_to_rank(smem_u32(&xchg[q]), tid), R, s, map_to_rank(smem_u32(&xbar), tid));
+        cluster_arrive_relaxed();          // exit guard: waited for after pass 2 (see smem_row.cuh)
         if (tid < 32 && alive) alive = mbar_wait_warp(smem_u32(&xbar), 0u, p.status);
         if (T > 32) __syncthreads();
         R = ident; s = 0.0f;
@@ -408,6 +409,7 @@ sm_masked_smem_kernel(const MaskedParams p, const uint32_t stage_bytes, const in
             }
         }
     }
+    if (cs > 1) cluster_wait_acquire();    // no block leaves while a peer's deposit into it is still to be issued
 }
 
 // ---------------------------------------------------------------------------------------------
