@@ -972,6 +972,9 @@ struct StaticDevice {
     int cluster_ok = 0;
     int* scratch = nullptr;              // device address of fs_static_scratch on this device
     bool configured[3][2][2] = {};       // split-row kernel variants whose attributes are set
+    // resident clusters per launch geometry (an occupancy query, no allocation), for the prefetch distance and the lag
+    struct Geo { const void* fn; int threads, cs; size_t smem; int ncl; } geo[16] = {};
+    int ngeo = 0;
 };
 StaticDevice g_static[kMaxDevices];
 std::mutex g_static_mu;
@@ -1939,6 +1942,24 @@ int fs_softmax_static(const void* x, void* y, int64_t rows, int64_t cols, int dt
         FS_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
         sd.configured[dtype][p.neg][full_variant] = true;
     }
+    int ncl = 0;
+    for (int i = 0; i < sd.ngeo && !ncl; ++i)
+        if (sd.geo[i].fn == fn && sd.geo[i].threads == sg.threads && sd.geo[i].cs == sg.cs && sd.geo[i].smem == smem) ncl = sd.geo[i].ncl;
+    if (!ncl) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(sg.cs * sd.sm_count, 1, 1);
+        cfg.blockDim = dim3(sg.threads, 1, 1);
+        cfg.dynamicSmemBytes = smem;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = sg.cs; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        FS_CUDA(cudaOccupancyMaxActiveClusters(&ncl, fn, &cfg));
+        if (ncl < 1) return FS_ERR_UNSUPPORTED;
+        if (sd.ngeo < 16) sd.geo[sd.ngeo++] = StaticDevice::Geo{fn, sg.threads, sg.cs, smem, ncl};
+    }
+    p.pf_rows = prefetch_rows(ncl);
+    set_first_wave_lag(p, ncl, nvec * 16);
     return launch(fn, rows * sg.cs, sg.threads, smem, sg.cs, st, p,
                   static_cast<uint32_t>(stage_bytes), sg.slice, smem_row_nchunk(sg, dtype));
 }
