@@ -18,7 +18,9 @@ import this module. It never touches CUDA and shares nothing with the CUDA libra
 Pins (tests/test_oracle_norm_pins.py): 50-digit mpmath values stored under tests/golden/, PyTorch's
 float64 CPU operators as an independent library, closed forms (constant rows, two-element rows),
 invariants (zero mean, sum of squares, shift and scale invariance), and a pure-Python loop over a
-tiny group_norm tensor for the channel indexing. Nothing here is "parity unpinned".
+tiny group_norm tensor for the channel indexing; the two error scales that set binary32 tolerances
+(error_scale, backward_error_scale) by hand-computed rows and by bracketing a binary32 evaluation
+against 60-digit arithmetic. Nothing here is "parity unpinned".
 """
 from __future__ import annotations
 
@@ -101,6 +103,18 @@ def error_scale(x: np.ndarray, dtype: int, rows_shape, gamma_full=None, beta_ful
         if beta_full is not None:
             s = s + np.abs(beta_full)
     return s
+
+
+def backward_error_scale(dy: np.ndarray, y: np.ndarray, dtype: int, scale: float) -> np.ndarray:
+    """Per-element magnitude that the rounding error of a binary32 evaluation of the softmax gradient
+    dx = scale * y * (dy - sum_k dy_k y_k) is proportional to: |scale| |y| (|dy| + sum_k |dy_k y_k|). dy and the dot
+    product can cancel, so the error is not proportional to |dx|; the second term carries the rounding of the
+    binary32 products and of their sum. dy, y: [rows, cols] stored elements."""
+    g = fso.widen(np.ascontiguousarray(dy), dtype)
+    p = fso.widen(np.ascontiguousarray(y), dtype)
+    sc = abs(float(np.float32(scale)))
+    with np.errstate(all="ignore"):
+        return sc * np.abs(p) * (np.abs(g) + np.abs(g * p).sum(axis=1, keepdims=True))
 
 
 @dataclass

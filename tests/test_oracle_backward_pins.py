@@ -73,3 +73,54 @@ def test_closed_forms_and_invariants():
     assert np.all(np.isnan(dx[1])) and not np.any(np.isnan(dx[0])) and not np.any(np.isnan(dx[2]))
     y0 = np.array([[1.0, 0.0]], dtype=np.float32)
     assert np.array_equal(fso.softmax_backward_f64(np.array([[2.0, 5.0]], np.float32), y0, FP32, 1.0), [[0.0, 0.0]])
+
+
+# ---------------------------------------------------------------------------------------------
+# backward_error_scale: the magnitude the binary32 tolerance of the backward's parity tests multiplies
+# ---------------------------------------------------------------------------------------------
+
+def test_backward_error_scale_hand_computed():
+    """|scale| |y| (|dy| + sum |dy y|) worked out by hand: y = [1/4, 3/4], dy = [2, -4]: sum |dy y| = 1/2 + 3 = 7/2."""
+    from oracle import fno
+    y = np.array([[0.25, 0.75]], dtype=np.float32)
+    dy = np.array([[2.0, -4.0]], dtype=np.float32)
+    assert np.array_equal(fno.backward_error_scale(dy, y, FP32, 1.0), [[0.25 * 5.5, 0.75 * 7.5]])
+    assert np.array_equal(fno.backward_error_scale(dy, y, FP32, -0.5), [[0.125 * 5.5, 0.375 * 7.5]])
+    # rows are independent, and a one-hot y silences every other column
+    y2 = np.array([[0.25, 0.75], [1.0, 0.0]], dtype=np.float32)
+    dy2 = np.array([[2.0, -4.0], [3.0, 100.0]], dtype=np.float32)
+    assert np.array_equal(fno.backward_error_scale(dy2, y2, FP32, 1.0), [[0.25 * 5.5, 0.75 * 7.5], [6.0, 0.0]])
+
+
+def test_backward_error_scale_brackets_a_binary32_evaluation():
+    """A binary32 evaluation of the gradient, one rounding per operation and three summation orders, against
+    60-digit arithmetic: its worst error is between 3e-8 and 1e-6 of the scale on every family of rows (the parity
+    tests allow 2e-6), also where dy and the dot product cancel. A scale ten times too large or too small, or one
+    without its dot-product term, leaves that band."""
+    import mpmath as mp
+    from oracle import fno
+    rng = np.random.default_rng(11)
+    with mp.workdps(60):
+        for rows, cols, sigma, shift, scale in ((4, 257, 1.0, 0.0, 1.0), (3, 64, 3.0, 0.0, 0.125), (3, 1000, 1.0, 0.0, -0.5),
+                                                (3, 96, 0.05, 7.0, 1.0), (3, 96, 0.01, -50.0, 2.0)):
+            y = fso.softmax_f64(rng.standard_normal((rows, cols)).astype(np.float32) * 2, FP32, 1.0).astype(np.float32)
+            dy = (rng.standard_normal((rows, cols)) * sigma + shift).astype(np.float32)      # shift: dy - dot nearly cancels
+            want = np.empty((rows, cols))
+            for i in range(rows):
+                g = [mp.mpf(float(v)) for v in dy[i]]
+                p = [mp.mpf(float(v)) for v in y[i]]
+                dot = mp.fsum([a * b for a, b in zip(g, p)])
+                want[i] = [float(mp.mpf(float(np.float32(scale))) * b * (a - dot)) for a, b in zip(g, p)]
+            es = fno.backward_error_scale(dy, y, FP32, scale)
+            worst = 0.0
+            for order in (range(cols), range(cols - 1, -1, -1), np.random.default_rng(cols).permutation(cols)):
+                got = np.empty_like(dy)
+                for i in range(rows):
+                    dot = np.float32(0)
+                    for j in order:
+                        dot = np.float32(dot + np.float32(dy[i, j] * y[i, j]))
+                    got[i] = ((dy[i] - dot).astype(np.float32) * y[i]).astype(np.float32) * np.float32(scale)
+                with np.errstate(invalid="ignore", divide="ignore"):
+                    ratio = np.where(es > 0, np.abs(got - want) / es, 0.0)
+                worst = max(worst, float(ratio.max()))
+            assert 3e-8 <= worst <= 1e-6, (rows, cols, sigma, shift, scale, worst)
