@@ -144,8 +144,9 @@ int max_threads_for(int dtype, int vpt) { return vpt * (dtype == FS_DTYPE_FP32 ?
 // Row sizes (bytes) at which the dispatcher changes kernel, from sweeps on B200 (256 MiB of
 // traffic per launch, rows from 2 KiB to 1 MiB, every kernel x threads x cluster size, against a
 // plain copy of the same bytes).
-//   16-bit: (sub-)warp per row up to 4 KiB, block per row (direct loads) up to 8 KiB, then the
-//           shared-memory-resident split.
+//   16-bit: (sub-)warp per row up to 4 KiB; above that up to 14 KiB four rows per block, each in
+//           shared memory under one warp (softmax_tile_wanted), except 6 and 8 KiB rows, which the
+//           block-per-row kernel (direct loads) fits exactly; then the shared-memory-resident split.
 //   fp32:   (sub-)warp per row up to 3 KiB, block per row up to 8 KiB, block per row fed by bulk
 //           copies up to 32 KiB, then the split.
 //   split:  slices of about 32 KiB, cluster and block size chosen per row length (smem_geom);
@@ -153,6 +154,26 @@ int max_threads_for(int dtype, int vpt) { return vpt * (dtype == FS_DTYPE_FP32 ?
 int64_t warp_max_row_bytes(int dtype) { return dtype == FS_DTYPE_FP32 ? 3072 : 4096; }
 int64_t block_max_row_bytes(int) { return 8192; }
 int64_t block_tma_max_row_bytes(int dtype) { return dtype == FS_DTYPE_FP32 ? 32768 : 0; }
+
+// 16-bit rows the dispatcher gives the four-rows-per-block kernel (softmax_tile_kernel), in 16-byte vectors
+// (lo < vectors <= hi): rows above 4 KiB up to 14 KiB, except the two lengths the block-per-row kernel fits
+// exactly. Measured on B200 (bf16, 256 MiB per direction, a copy = 80.1 us): 4.5 / 5 / 7 / 9 / 10 / 11 / 12 / 13 / 14 KiB
+// rows 81.5 / 81.5 / 81.4 / 81.9 / 81.5 / 81.9 / 81.8 / 82.2 / 84.2 us against 88.1 / 83.8 / 82.6 / 99.7 / 94.0 / 90.9 / 85.7 /
+// 93.4 / 88.5 for the block-per-row kernel (up to 8 KiB) and the split-row kernel (beyond); 6 and 8 KiB rows stay
+// with the block kernel (79.4 / 79.1 against 81.8 / 81.4), 16 KiB with the split-row kernel (81.2 against 82.8).
+// FS_SOFTMAX_TILE "lo:hi" (read once) overrides the range, "0" turns the kernel off.
+bool softmax_tile_wanted(int dtype, int64_t nvec) {
+    static const std::pair<int64_t, int64_t> ov = [] {
+        const char* e = std::getenv("FS_SOFTMAX_TILE");
+        if (!e) return std::pair<int64_t, int64_t>(-1, -1);
+        long lo = 0, hi = 0;
+        if (std::sscanf(e, "%ld:%ld", &lo, &hi) == 2) return std::pair<int64_t, int64_t>(lo, hi);
+        return std::pair<int64_t, int64_t>(0, 0);
+    }();
+    if (dtype == FS_DTYPE_FP32) return false;
+    if (ov.first >= 0) return nvec > ov.first && nvec <= ov.second;
+    return nvec > 256 && nvec <= 896 && nvec != 384 && nvec != 512;
+}
 int64_t split_slice_bytes(int) { return 32768; }
 constexpr int64_t kWarpTileMaxRowBytes = 4096;      // rows the warp-tile bulk-copy kernel takes
 constexpr int kMaxCluster = 16;
@@ -281,6 +302,7 @@ int select_kernel(int64_t cols, int dtype, int x_align, int y_align) {
     const int64_t nvec = row_bytes / 16;
     WarpGeom wg; BlockGeom bg;
     if (row_bytes <= warp_max_row_bytes(dtype) && warp_geom(nvec, dtype, &wg)) return FS_KERNEL_WARP;
+    if (softmax_tile_wanted(dtype, nvec)) return FS_KERNEL_BLOCK_TMA;        // four rows per block, a warp per row
     if (row_bytes <= block_max_row_bytes(dtype) && block_geom(nvec, dtype, 0, &bg)) return FS_KERNEL_BLOCK;
     if (row_bytes <= block_tma_max_row_bytes(dtype) && block_geom(nvec, dtype, 0, &bg)) return FS_KERNEL_BLOCK_TMA;
     SmemGeom sg;
@@ -774,6 +796,27 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
         case FS_KERNEL_BLOCK_TMA: {
             const size_t smem_cap = static_cast<size_t>(dev.smem_optin) - 2048;   // room for the static part
             WarpGeom wg;
+            if (was_auto && softmax_tile_wanted(dtype, p.nvec)) {
+                // the dispatcher's own choice for 16-bit rows of 4-12 KiB: four rows per block in shared memory,
+                // each brought by its own bulk copy and worked on by one warp
+                const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) -> const void* {
+                    constexpr int DT = decltype(dt)::value;
+                    if constexpr (DT == DT_F32) return nullptr;
+                    else return (const void*)softmax_tile_kernel<DT, decltype(ng)::value>; });
+                const int t = 128;
+                const size_t smem = size_t(t / 32) * size_t(p.nvec) * 16 + size_t(t / 32) * 8;
+                const int64_t grid = (rows + (t / 32) - 1) / (t / 32);
+                if (fn && smem <= smem_cap && grid <= max_grid) {
+                    int bps = 0;
+                    if ((rc = blocks_per_sm(dev, fn, t, smem, &bps)) != FS_OK) return rc;
+                    p.pf_rows = prefetch_rows(dev.sm_count * bps) * (t / 32);
+                    set_first_wave_lag(p, dev.sm_count * bps, (t / 32) * p.nvec * 16);
+                    FS_LOGF("softmax %lld x %lld dtype %d: four rows per block from shared memory, a warp per row, %d blocks per SM",
+                            (long long)rows, (long long)cols, dtype, bps);
+                    return launch(fn, grid, t, smem, 0, st, p);
+                }
+                // (too little shared memory on this device: the block-per-row form below takes the row)
+            }
             if (p.nvec * 16 <= kWarpTileMaxRowBytes && warp_geom(p.nvec, dtype, &wg)) {
                 // short rows: one bulk copy brings a tile of consecutive rows, each (sub-)warp owns rows
                 const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) { return warp_tma_fn<decltype(dt)::value, decltype(ng)::value>(wg); });

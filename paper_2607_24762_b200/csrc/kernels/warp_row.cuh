@@ -155,4 +155,90 @@ warp_row_tma_kernel(const Params p, const int tile_rows, const uint32_t tile_byt
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// 16-bit rows of 4-12 KiB: four rows per block, each brought to shared memory by a bulk copy of its
+// own (one mbarrier per row) and worked on by one warp alone, three reads of shared memory:
+//   pass A  the row reference R (packed max over the raw vectors, one shuffle reduction);
+//   pass B  e = 2^((x - R) c): subtraction first (exact), one ex2 per element, the row sum taken over
+//           the unrounded fp32 values, e written back IN PLACE in the element dtype (only the lane
+//           that wrote a vector reads it again);
+//   pass C  y = e / S, 128-bit streaming stores.
+// No block barrier after start-up and a register footprint that does not grow with the row, so
+// six to nine blocks of four warps stay resident per SM: the rows a (sub-)warp can no longer hold in
+// registers and a cluster's chunked slices serve poorly. Storing e rounded to the element dtype
+// keeps the result within one unit in the last place of the correctly rounded value (the argument
+// in smem_row.cuh). One-shot grid: block b handles rows b*W .. b*W+W-1.
+// dynamic shared memory: W rows | W mbarriers
+// ---------------------------------------------------------------------------------------------
+template <int DT, bool NEG>
+__global__ void __launch_bounds__(128)
+softmax_tile_kernel(const Params p) {
+    static_assert(DT != DT_F32, "16-bit element types only");
+    constexpr int VE = Traits<DT>::VE;
+    constexpr int H = 4;                                   // vectors per lane and batch
+    pdl_launch_dependents();
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, W = blockDim.x >> 5;
+    const int nvec = static_cast<int>(p.nvec);
+    const int64_t row_bytes = p.nvec * 16;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + size_t(W) * size_t(row_bytes));
+    const int64_t row = int64_t(blockIdx.x) * W + w;
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < W; ++i) mbar_init(smem_u32(&bars[i]), 1);
+        mbar_fence_init();
+        fence_proxy_async_smem();
+    }
+    __syncthreads();
+    pdl_wait();
+    if (row >= p.rows) return;                             // no block-wide barrier follows
+    const char* xb = static_cast<const char*>(p.x);
+    if (lane == 0) {
+        first_wave_lag(blockIdx.x, p.lag_ns, p.lag_rows);
+        bulk_load_row(smem_u32(smem) + uint32_t(w) * uint32_t(row_bytes), xb + row * row_bytes, uint32_t(row_bytes), smem_u32(&bars[w]));
+        if (p.pf_rows > 0 && row + p.pf_rows < p.rows) l2_prefetch(xb + (row + p.pf_rows) * row_bytes, uint32_t(row_bytes));
+    }
+    uint4* sv = reinterpret_cast<uint4*>(smem + size_t(w) * size_t(row_bytes)) + lane;
+    uint4* __restrict__ yv = static_cast<uint4*>(p.y) + row * p.nvec + lane;
+    const float ident = ref_identity<NEG>();
+    mbar_wait_warp(smem_u32(&bars[w]), 0u, p.status);      // on a timeout the status word is set and the row is garbage
+
+    RefAcc<DT, NEG> ref;
+    ref.init();
+    for (int k0 = 0; k0 < nvec; k0 += 32 * H) {
+#pragma unroll
+        for (int u = 0; u < H; ++u)
+            if (k0 + u * 32 + lane < nvec) ref.fold(sv[k0 + u * 32]);
+    }
+    const float R = warp_pick<32, NEG>(ref.value());
+    // a row whose reference is still the identity (only masked entries) subtracts 0 instead: -inf - 0 stays
+    // -inf, the sum is 0 and 0 * (1 / 0) makes the row NaN, as the formula does
+    const float ru = (R == ident) ? 0.0f : R;
+    const f32x2 r2 = pair(ru, ru), c2 = pair(p.c, p.c);
+    f32x2 acc[VE / 2];
+#pragma unroll
+    for (int k = 0; k < VE / 2; ++k) acc[k] = pair(0.0f, 0.0f);
+    for (int k0 = 0; k0 < nvec; k0 += 32 * H) {
+        uint4 raw[H];
+#pragma unroll
+        for (int u = 0; u < H; ++u)
+            if (k0 + u * 32 + lane < nvec) raw[u] = sv[k0 + u * 32];
+#pragma unroll
+        for (int u = 0; u < H; ++u)
+            if (k0 + u * 32 + lane < nvec) sv[k0 + u * 32] = ex2_vec<DT>(raw[u], r2, c2, acc);
+    }
+#pragma unroll
+    for (int k = 1; k < VE / 2; ++k) acc[0] = add2(acc[0], acc[k]);
+    const float inv = recip<DT>(warp_sum<32>(pair_sum(acc[0])));
+    const f32x2 i2 = pair(inv, inv);
+    for (int k0 = 0; k0 < nvec; k0 += 32 * H) {
+        uint4 e[H];
+#pragma unroll
+        for (int u = 0; u < H; ++u)
+            if (k0 + u * 32 + lane < nvec) e[u] = sv[k0 + u * 32];
+#pragma unroll
+        for (int u = 0; u < H; ++u)
+            if (k0 + u * 32 + lane < nvec) st_stream(yv + k0 + u * 32, scale_vec<DT, false>(e[u], i2, i2));
+    }
+}
+
 }  // namespace fsm

@@ -251,6 +251,42 @@ def test_negative_and_zero_scale(dtype):
         check(xs, dtype, 0.0, y)
 
 
+@pytest.mark.parametrize("dtype", [BF16, FP16])
+def test_rows_around_the_four_rows_per_block_kernel(dtype):
+    """16-bit rows above 4 KiB up to 14 KiB (257..896 sixteen-byte vectors, except 384 and 512) take the kernel that
+    works on four rows per block from shared memory, a warp per row: both ends of the range and its two holes, one
+    vector to either side, row counts that leave a block partly empty, both signs of the scale and zero, in place,
+    special values."""
+    for ci, nvec in enumerate((256, 257, 300, 383, 384, 385, 511, 512, 513, 700, 895, 896, 897)):
+        cols = nvec * 8
+        chosen = fs.fs_select_kernel(5, cols, dtype)
+        in_range = 256 < nvec <= 896 and nvec not in (384, 512)
+        assert (chosen == fs.FS_KERNEL_BLOCK_TMA) == in_range, (nvec, chosen)
+        for rows, scale in ((1, 1.0), (5, 0.125), (7, -0.5), (64, 1.0), (3, 0.0)):
+            x = W.random_case(rows, cols, dtype, seed=400 + ci + rows, sigma=3.0, neg_inf_frac=0.02 if scale > 0 else 0.0)
+            status, y = run_softmax(x, dtype, scale, inplace=(ci + rows) % 3 == 0)
+            assert status == fs.FS_OK
+            check(x, dtype, scale, y)
+    cols = 700 * 8
+    x = W.random_case(6, cols, dtype, seed=77, sigma=2.0)
+    ninf = np.uint16(0xFF80 if dtype == BF16 else 0xFC00)
+    x[1, :] = ninf                                                   # only masked entries: NaN row
+    x[2, 1234] = np.uint16(0x7FC0 if dtype == BF16 else 0x7E00)     # NaN
+    x[3, 4321] = np.uint16(0x7F80 if dtype == BF16 else 0x7C00)     # +inf
+    x[4, 1:] = ninf                                                  # one finite entry: exactly [1, 0, 0, ...]
+    status, y = run_softmax(x, dtype, 1.0)
+    rep = check(x, dtype, 1.0, y)
+    yf = W.stored_to_f32(y, dtype)
+    assert np.all(np.isnan(yf[1:4])) and yf[4, 0] == 1.0 and np.all(y[4, 1:] == 0) and rep.nan_mismatch == 0
+    if dtype == BF16:                                                # results below 2^-126 are kept
+        row = np.linspace(-91.0, -87.0, cols)
+        row[0] = 0.0
+        xs = W.to_stored(np.array([row, row[::-1].copy(), row]), BF16)
+        status, y = run_softmax(xs, BF16, 1.0)
+        check(xs, BF16, 1.0, y)
+        assert np.count_nonzero((y[0] > 0) & (y[0] < 0x0080)) > 50
+
+
 def test_bf16_subnormal_outputs_are_not_flushed():
     """Outputs below 2^-126 are representable bf16 subnormals; the 1-ulp rule applies there too."""
     cols = 256

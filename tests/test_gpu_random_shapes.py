@@ -70,8 +70,7 @@ def one_case(rng, S):
         dy = fso.round_from_f64(rng.standard_normal((rows, cols)), dtype)
         gd, yd2 = dev(dy), dev(y); dd = torch.zeros_like(gd)
         fs.fs_softmax_backward(gd, yd2, dd, rows, cols, dtype, scale, S); torch.cuda.synchronize()
-        g64, y64 = fso.widen(dy, dtype), fso.widen(y, dtype)
-        es = abs(float(np.float32(scale))) * np.abs(y64) * (np.abs(g64) + np.abs(g64 * y64).sum(axis=1, keepdims=True))
+        es = fno.backward_error_scale(dy, y, dtype, scale)
         ok = fno.compare(torch_bits_to_np(dd, dtype).reshape(rows, cols), dtype, fso.softmax_backward_f64(dy, y, dtype, scale), es).ok(dtype); tag = 'backward'
     elif op == 4:
         xs = fso.round_from_f64(rng.standard_normal((rows, cols)) * rng.choice([0.5, 3.0]) + rng.choice([0.0, 5.0]), dtype)

@@ -184,8 +184,7 @@ def test_softmax_operator_forward_and_backward_run_the_library():
         assert torch_op.stats() == {"library": 2}                   # one forward, one backward kernel; nothing went to eager
         bits = (lambda t: t.detach().view(torch.int16).cpu().numpy().view(np.uint16)) if dt != W.FP32 else (lambda t: t.detach().cpu().numpy())
         assert fso.compare(bits(y), dt, fso.softmax_f64(bits(x), dt, scale)).ok(dt)
-        g64, y64 = fso.widen(bits(dy), dt), fso.widen(bits(y), dt)
-        es = abs(scale) * np.abs(y64) * (np.abs(g64) + np.abs(g64 * y64).sum(axis=1, keepdims=True))
+        es = fno.backward_error_scale(bits(dy), bits(y), dt, scale)
         rep = fno.compare(bits(x.grad), dt, fso.softmax_backward_f64(bits(dy), bits(y), dt, scale), es)
         assert rep.ok(dt), rep
     # called directly, as a traced graph would: same kernels; a tensor the guard refuses is computed by eager
