@@ -838,6 +838,9 @@ def main():
     ap.add_argument("--impl", default="fsoftmax", choices=["fsoftmax", "reference"])
     ap.add_argument("--rows", type=int, default=0,
                     help="use only the first ROWS rows of the workload (small cases for profiler captures)")
+    ap.add_argument("--cols", type=int, default=0,
+                    help="give the workload's rows this many columns instead (same value distribution; profiler captures of "
+                         "the kernels the five workloads do not reach)")
     ap.add_argument("--all", dest="all_workloads", action="store_true", default=None,
                     help="also time the other workloads (default: on at --gpus 1)")
     ap.add_argument("--no-all", dest="all_workloads", action="store_false")
@@ -853,6 +856,9 @@ def main():
     if args.rows:
         import dataclasses
         w = dataclasses.replace(w, rows=min(w.rows, args.rows), note=w.note + f" (first {args.rows} rows)")
+    if args.cols:
+        import dataclasses
+        w = dataclasses.replace(w, cols=args.cols, name=f"{w.name}_cols{args.cols}", note=w.note + f" (rows of {args.cols} columns instead)")
 
     if args.impl == "reference":
         reference_arm(args, w)
@@ -917,7 +923,7 @@ def main():
         return
     res = time_device(w, args.steps, args.warmup, l2, sampler=sampler, barrier=barrier, min_clock_samples=8,
                       extras=world == 1, n_trains=args.trains,
-                      causal_too=world == 1 and w.name == "cfg5" and not args.rows and args.all_workloads is not False)
+                      causal_too=world == 1 and w.name == "cfg5" and not args.rows and not args.cols and args.all_workloads is not False)
     from paper_2607_24762_b200 import sharding
     ms = sharding.max_over_ranks(res["ms_per_step"], device="cuda")          # as slow as the slowest rank
     value = sharding.aggregate_throughput(w.min_bytes, ms * 1e-3, world) / 1e9
