@@ -70,7 +70,8 @@ typedef enum {
     FS_KERNEL_AUTO = 0,
     FS_KERNEL_WARP = 1,       /* (sub-)warp per row, row held in registers */
     FS_KERNEL_BLOCK = 2,      /* block per row, 128-bit global loads, row held in registers */
-    FS_KERNEL_BLOCK_TMA = 3,  /* block per row (or a tile of short rows per block) staged in shared memory by bulk async copies */
+    FS_KERNEL_BLOCK_TMA = 3,  /* rows staged in shared memory by bulk async copies: a block per row; the dispatcher's own choice for
+                                 16-bit rows of 4.5-14 KiB is four rows per block, a warp per row */
     FS_KERNEL_CLUSTER = 4,    /* row split over a thread-block cluster of 1..16 blocks, slices resident in shared memory,
                                  (max,sum) pairs exchanged through distributed shared memory */
     FS_KERNEL_GENERIC = 5     /* any cols, any alignment; reads the row twice */

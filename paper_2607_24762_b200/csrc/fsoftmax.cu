@@ -175,10 +175,8 @@ bool softmax_tile_wanted(int dtype, int64_t nvec) {
     return nvec > 256 && nvec <= 896 && nvec != 384 && nvec != 512;
 }
 int64_t split_slice_bytes(int) { return 32768; }
-constexpr int64_t kWarpTileMaxRowBytes = 4096;      // rows the warp-tile bulk-copy kernel takes
 constexpr int kMaxCluster = 16;
 constexpr int kSplitThreads = 256;                   // block size of the two-kernel (segment) path
-constexpr int64_t kTileBytes = 16384;               // rows per bulk copy of the warp-tile kernel
 
 int64_t warp_capacity_vecs(int dtype) { return 32 * int64_t(max_vpt(dtype)); }
 
@@ -539,26 +537,6 @@ template <int DT, bool NEG> const void* warp_fn(const WarpGeom& g) {
     return nullptr;
 }
 
-template <int DT, bool NEG> const void* warp_tma_fn(const WarpGeom& g) {
-    if (g.vpl == 1) return (const void*)warp_row_tma_kernel<DT, NEG, 1, 1>;
-    if (g.vpl == 2) return (const void*)warp_row_tma_kernel<DT, NEG, 1, 2>;
-    if (g.vpl == 4) {
-        switch (g.lanes) {
-            case 1:  return (const void*)warp_row_tma_kernel<DT, NEG, 1, 4>;
-            case 2:  return (const void*)warp_row_tma_kernel<DT, NEG, 2, 4>;
-            case 4:  return (const void*)warp_row_tma_kernel<DT, NEG, 4, 4>;
-            case 8:  return (const void*)warp_row_tma_kernel<DT, NEG, 8, 4>;
-            case 16: return (const void*)warp_row_tma_kernel<DT, NEG, 16, 4>;
-            default: return (const void*)warp_row_tma_kernel<DT, NEG, 32, 4>;
-        }
-    }
-    if (g.vpl == 8) return (const void*)warp_row_tma_kernel<DT, NEG, 32, 8>;
-    if constexpr (DT == DT_F32) {
-        if (g.vpl == 16) return (const void*)warp_row_tma_kernel<DT, NEG, 32, 16>;
-    }
-    return nullptr;
-}
-
 #define FS_VPT_TABLE(NAME, KERNEL)                                                          \
     template <int DT, bool NEG> const void* NAME(int vpt) {                                 \
         switch (vpt) {                                                                      \
@@ -795,7 +773,6 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
         }
         case FS_KERNEL_BLOCK_TMA: {
             const size_t smem_cap = static_cast<size_t>(dev.smem_optin) - 2048;   // room for the static part
-            WarpGeom wg;
             if (was_auto && softmax_tile_wanted(dtype, p.nvec)) {
                 // the dispatcher's own choice for 16-bit rows of 4-12 KiB: four rows per block in shared memory,
                 // each brought by its own bulk copy and worked on by one warp
@@ -816,28 +793,6 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
                     return launch(fn, grid, t, smem, 0, st, p);
                 }
                 // (too little shared memory on this device: the block-per-row form below takes the row)
-            }
-            if (p.nvec * 16 <= kWarpTileMaxRowBytes && warp_geom(p.nvec, dtype, &wg)) {
-                // short rows: one bulk copy brings a tile of consecutive rows, each (sub-)warp owns rows
-                const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) { return warp_tma_fn<decltype(dt)::value, decltype(ng)::value>(wg); });
-                if (!fn) return FS_ERR_UNSUPPORTED;
-                const int t = threads ? threads : 128;
-                if (t > 256) return FS_ERR_UNSUPPORTED;
-                const int64_t row_bytes = p.nvec * 16;
-                const int rows_per_pass = (t / 32) * (32 / wg.lanes);
-                int64_t tile_rows = std::max<int64_t>(1, kTileBytes / row_bytes);
-                tile_rows = std::max<int64_t>(rows_per_pass, tile_rows / rows_per_pass * rows_per_pass);
-                tile_rows = std::min<int64_t>(tile_rows, (rows + rows_per_pass - 1) / rows_per_pass * rows_per_pass);
-                const size_t tile_bytes = static_cast<size_t>(tile_rows * row_bytes);
-                if (tile_bytes + 8 > smem_cap || tile_bytes > (size_t(1) << 20) - 16) return FS_ERR_UNSUPPORTED;
-                const size_t smem = tile_bytes + 8;
-                int bps = 0;
-                if ((rc = blocks_per_sm(dev, fn, t, smem, &bps)) != FS_OK) return rc;
-                const int64_t tiles = (rows + tile_rows - 1) / tile_rows;
-                const int64_t grid = std::min<int64_t>(tiles, max_grid);
-                FS_LOGF("softmax %lld x %lld dtype %d: warp kernel fed by bulk copies, tiles of %lld rows", (long long)rows,
-                        (long long)cols, dtype, (long long)tile_rows);
-                return launch(fn, grid, t, smem, 0, st, p, static_cast<int>(tile_rows), static_cast<uint32_t>(tile_bytes));
             }
             BlockGeom g;
             if (!block_geom(p.nvec, dtype, threads, &g)) return FS_ERR_UNSUPPORTED;

@@ -6,11 +6,10 @@
 // store covers whole 32-byte sectors of G adjacent rows. The row maximum and sum are warp-shuffle
 // reductions over the group; one ex2 per element.
 //
-// Two front ends:
-//   warp_row_kernel      128-bit global loads straight into registers
-//   warp_row_tma_kernel  the block's tile of consecutive rows (one contiguous byte range) is
-//                        brought into shared memory by one bulk async copy (no multicast) and the
-//                        warps read their rows from there
+// warp_row_kernel takes its rows by 128-bit global loads straight into registers. (A variant that
+// brought a block's tile of consecutive rows into shared memory with one bulk copy was measured
+// slower on every short-row shape and is gone.) softmax_tile_kernel, at the end of this file,
+// serves the 16-bit rows a warp can no longer hold in registers: one warp per row from shared memory.
 #pragma once
 #include "common.cuh"
 
@@ -97,60 +96,6 @@ warp_row_kernel(const Params p) {
         for (int r = 0; r < R; ++r) {
             const bool row_ok = row0 + int64_t(r) * G < p.rows;
             warp_row_math<DT, NEG, LANES, VPL>(raw[r], p.c, yv + off0 + int64_t(r) * G * p.nvec, row_ok, live);
-        }
-    }
-}
-
-// Dynamic shared memory: the tile (tile_rows * row bytes) followed by one mbarrier.
-// The block's warps split the tile's rows G at a time; a block handles tiles
-// blockIdx.x, blockIdx.x + gridDim.x, ... (normally exactly one).
-template <int DT, bool NEG, int LANES, int VPL>
-__global__ void __launch_bounds__(256)
-warp_row_tma_kernel(const Params p, const int tile_rows, const uint32_t tile_bytes_max) {
-    constexpr int G = 32 / LANES;
-    pdl_launch_dependents();
-    extern __shared__ __align__(128) unsigned char smem[];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int sub = lane / LANES, sl = lane % LANES;
-    const int warps = blockDim.x >> 5;
-    const int nvec = static_cast<int>(p.nvec);
-    const int64_t row_bytes = p.nvec * 16;
-    const int64_t ntiles = (p.rows + tile_rows - 1) / tile_rows;
-    uint64_t* bar = reinterpret_cast<uint64_t*>(smem + tile_bytes_max);
-    const char* xb = static_cast<const char*>(p.x);
-    uint4* __restrict__ yv = static_cast<uint4*>(p.y);
-    auto live = [&](int k) { return sl + k * LANES < nvec; };
-
-    if (threadIdx.x == 0) {
-        mbar_init(smem_u32(bar), 1);
-        mbar_fence_init();
-        fence_proxy_async_smem();
-    }
-    __syncthreads();
-    pdl_wait();
-    uint32_t phase = 0;
-    bool alive = true;
-    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-        const int64_t row_first = tile * tile_rows;
-        const int nrows = static_cast<int>(min(int64_t(tile_rows), p.rows - row_first));
-        if (threadIdx.x == 0)
-            bulk_load_row(smem_u32(smem), xb + row_first * row_bytes, static_cast<uint32_t>(nrows * row_bytes), smem_u32(bar));
-        if (alive) alive = mbar_wait_warp(smem_u32(bar), phase, p.status);
-        phase ^= 1u;
-        const uint4* tile_v = reinterpret_cast<const uint4*>(smem);
-        for (int lr = warp * G + sub; lr - sub < nrows; lr += warps * G) {
-            const bool row_ok = lr < nrows;
-            uint4 raw[VPL];
-#pragma unroll
-            for (int k = 0; k < VPL; ++k) {
-                raw[k] = make_uint4(0u, 0u, 0u, 0u);
-                if (row_ok && live(k)) raw[k] = tile_v[int64_t(lr) * nvec + sl + k * LANES];
-            }
-            warp_row_math<DT, NEG, LANES, VPL>(raw, p.c, yv + (row_first + lr) * p.nvec + sl, row_ok, live);
-        }
-        if (tile + gridDim.x < ntiles) {   // another tile follows: everyone is done reading this one
-            __syncthreads();
-            if (threadIdx.x == 0) fence_proxy_async_smem();
         }
     }
 }
