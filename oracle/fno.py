@@ -117,6 +117,33 @@ def backward_error_scale(dy: np.ndarray, y: np.ndarray, dtype: int, scale: float
         return sc * np.abs(p) * (np.abs(g) + np.abs(g * p).sum(axis=1, keepdims=True))
 
 
+def log_softmax_bound(want: np.ndarray) -> np.ndarray:
+    """Absolute fp32 bound of a log_softmax output: 1e-6 * max(1, |y|) -- three binary32 roundings of
+    (x - R) * scale - ln S plus 2^-22 absolute on log2 S; relative above 1 because outputs reach -50 and beyond.
+    Non-finite oracle values (a -inf output, a NaN row) get 1e-6: they are compared exactly elsewhere."""
+    w = np.asarray(want, dtype=np.float64)
+    with np.errstate(invalid="ignore"):
+        return 1e-6 * np.maximum(1.0, np.where(np.isfinite(w), np.abs(w), 1.0))
+
+
+def masked_softmax_bound(x: np.ndarray, mask: np.ndarray, dtype: int, q_rows: int, heads: int, scale: float,
+                         want: np.ndarray) -> np.ndarray:
+    """Absolute fp32 bound of softmax(scale * x + mask): 1e-6 + 2.5e-7 * Z * y, Z the largest finite |scale * x + mask|
+    of the row. The exponent scale * x + mask is formed in binary32 before the row maximum is taken off, so it
+    carries a rounding of relative size 2^-24 of a number as large as Z: 2^-24 * Z * ln 2 on the exponent of the element
+    and as much again through the row sum. x: [rows, cols] ordered (batch, head, query), mask: [rows / heads, cols]."""
+    X = fso.widen(np.ascontiguousarray(x), dtype)
+    M = fso.widen(np.ascontiguousarray(mask), dtype)
+    rows = X.shape[0]
+    mrow = (np.arange(rows) // (heads * q_rows)) * q_rows + np.arange(rows) % q_rows
+    sc = float(np.float32(scale))
+    w = np.asarray(want, dtype=np.float64)
+    with np.errstate(invalid="ignore", over="ignore"):
+        z = sc * X + M[mrow]
+        zmax = np.max(np.where(np.isfinite(z), np.abs(z), 0.0), axis=1, keepdims=True)
+        return 1e-6 + 2.5e-7 * zmax * np.where(np.isfinite(w), w, 1.0)
+
+
 @dataclass
 class NormReport:
     max_rel_err: float      # max over elements of |got - want| / error_scale
