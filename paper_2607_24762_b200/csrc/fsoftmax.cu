@@ -429,9 +429,8 @@ struct TensorRange { const void* p; unsigned long long bytes; int writable; };
 #ifdef FS_DEBUG_BOUNDS
 thread_local DebugRanges t_dbg = {};
 thread_local long long t_dbg_shrink = 0;          // self-test: the writable ranges end this many bytes early
-void dbg_register(int* status, std::initializer_list<TensorRange> ranges) {
+void dbg_register(std::initializer_list<TensorRange> ranges) {
     t_dbg = DebugRanges{};
-    t_dbg.status = status;
     for (const TensorRange& r : ranges) {
         if (!r.p || t_dbg.n >= 8) continue;
         const unsigned long long lo = reinterpret_cast<unsigned long long>(r.p);
@@ -441,8 +440,7 @@ void dbg_register(int* status, std::initializer_list<TensorRange> ranges) {
         ++t_dbg.n;
     }
 }
-#define FS_DBG_RANGES(...) do { Device* d__ = nullptr; const int r__ = get_device(&d__); if (r__ != FS_OK) return r__; \
-                                dbg_register(d__->status, {__VA_ARGS__}); } while (0)
+#define FS_DBG_RANGES(...) dbg_register({__VA_ARGS__})
 #else
 #define FS_DBG_RANGES(...) do { } while (0)
 #endif
@@ -450,9 +448,13 @@ void dbg_register(int* status, std::initializer_list<TensorRange> ranges) {
 template <typename... Args>
 int launch(const void* fn, int64_t grid, int threads, size_t smem, int cs, cudaStream_t st, Args... args) {
 #ifdef FS_DEBUG_BOUNDS
-    {   // keep the first refused address of earlier launches
-        DebugRanges up = t_dbg;
-        FS_CUDA(cudaMemcpyToSymbolAsync(g_dbg, &up, offsetof(DebugRanges, first_bad), 0, cudaMemcpyHostToDevice, st));
+    {   // the ranges only: the flag word and the first refused address stay as the device has them
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        FS_CUDA(cudaStreamIsCapturing(st, &cap));
+        // inside a stream capture the copy becomes a graph node that reads its source at every replay: the source
+        // must outlive the graph, so it is a small heap block that is never freed (checked build only)
+        const DebugRanges* src = cap == cudaStreamCaptureStatusNone ? &t_dbg : new DebugRanges(t_dbg);
+        FS_CUDA(cudaMemcpyToSymbolAsync(g_dbg, src, offsetof(DebugRanges, flags), 0, cudaMemcpyHostToDevice, st));
     }
 #endif
     void* argv[] = {static_cast<void*>(&args)...};
@@ -1854,6 +1856,14 @@ int fs_device_status(void) {
     FS_CUDA(cudaDeviceSynchronize());
     FS_CUDA(cudaMemcpy(&word, dev->status, sizeof(int), cudaMemcpyDeviceToHost));
     if (word) FS_CUDA(cudaMemset(dev->status, 0, sizeof(int)));
+#ifdef FS_DEBUG_BOUNDS
+    {
+        int flags = 0, zero = 0;
+        FS_CUDA(cudaMemcpyFromSymbol(&flags, g_dbg, sizeof(int), offsetof(DebugRanges, flags)));
+        if (flags) FS_CUDA(cudaMemcpyToSymbol(g_dbg, &zero, sizeof(int), offsetof(DebugRanges, flags)));
+        word |= flags;
+    }
+#endif
     if (word & DEV_BOUNDS) return FS_ERR_DEVICE_BOUNDS;
     return (word & DEV_TIMEOUT) ? FS_ERR_DEVICE_TIMEOUT : FS_OK;
 }
@@ -1899,7 +1909,7 @@ int fs_softmax_static(const void* x, void* y, int64_t rows, int64_t cols, int dt
     const int64_t nvec = cols * elem_size(dtype) / 16;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 #ifdef FS_DEBUG_BOUNDS
-    t_dbg = DebugRanges{};              // registering ranges needs the allocated status word: this entry point goes unchecked
+    t_dbg = DebugRanges{};              // fs_static_status does not read the checker's flag word: this entry point goes unchecked
 #endif
     std::lock_guard<std::mutex> lk(g_static_mu);
     StaticDevice* sdp = nullptr;

@@ -43,24 +43,27 @@ template <> struct Traits<DT_F16>  { static constexpr int VE = 8; static constex
 // With -DFS_DEBUG_BOUNDS (libfsoftmax_debug.so) every global access of every kernel -- they all go
 // through the helpers below -- is checked against the address ranges of the tensors the host
 // registered for the launch. An access outside them (or a store into a read-only tensor) is NOT
-// performed: it sets DEV_BOUNDS in the status word, records the first offending address and the
-// kernel carries on (a load yields zeros), so an indexing error shows up as a status and an address
-// instead of a fault. The stand-in for a memory checker on machines where none can be run.
+// performed: it sets DEV_BOUNDS in the table's own flag word, records the first offending address
+// and the kernel carries on (a load yields zeros), so an indexing error shows up as a status and an
+// address instead of a fault. The stand-in for a memory checker on machines where none can be run.
+// The table holds no pointer that device code dereferences: whatever the host uploads (even a stale
+// or torn copy, as when two streams launch at once), the worst outcome is a false report.
 #ifdef FS_DEBUG_BOUNDS
 struct DebugRanges {
     unsigned long long lo[8], hi[8];
     int writable[8];
     int n;                              // 0: nothing registered for this launch, nothing is checked
-    int* status;
-    unsigned long long first_bad;       // 0 until an access was refused
+    int flags;                          // DEV_BOUNDS once an access was refused   } never uploaded: the host
+    unsigned long long first_bad;       // 0 until an access was refused           } reads and clears them
 };
 __device__ DebugRanges g_dbg;
 __device__ __forceinline__ bool dbg_ok(const void* p, unsigned long long bytes, bool write) {
     if (g_dbg.n == 0) return true;
     const unsigned long long a = reinterpret_cast<unsigned long long>(p);
-    for (int i = 0; i < g_dbg.n; ++i)
+    const int n = min(g_dbg.n, 8);
+    for (int i = 0; i < n; ++i)
         if (a >= g_dbg.lo[i] && a + bytes <= g_dbg.hi[i] && (!write || g_dbg.writable[i])) return true;
-    atomicOr(g_dbg.status, DEV_BOUNDS);
+    atomicOr(&g_dbg.flags, DEV_BOUNDS);
     atomicCAS(&g_dbg.first_bad, 0ull, a);
     return false;
 }

@@ -36,10 +36,8 @@ def run(x, dtype, scale, misalign=0, inplace=False):
 def check(x, dtype, scale, **kw):
     y = run(x, dtype, scale, **kw)
     want = fso.log_softmax_f64(x, dtype, scale)
-    with np.errstate(invalid="ignore"):
-        scale_arr = np.maximum(1.0, np.where(np.isfinite(want), np.abs(want), 1.0))
-    rep = fno.compare(y, dtype, want, scale_arr, rel_tol=1e-6)
-    assert rep.ok(dtype, rel_tol=1e-6), (x.shape, dtype, scale, rep)
+    rep = fno.compare(y, dtype, want, fno.log_softmax_bound(want), rel_tol=1.0)      # the bound is pinned in tests/test_oracle_log_softmax_pins.py
+    assert rep.ok(dtype, rel_tol=1.0), (x.shape, dtype, scale, rep)
     # -inf exactly where the oracle has it
     g64 = fso.widen(y, dtype)
     assert np.array_equal(np.isneginf(g64), np.isneginf(want))

@@ -24,7 +24,7 @@ SCALES = [1.0, 0.5, 128 ** -0.5, -1.0, 0.0]
 def built_library():
     from paper_2607_24762_b200 import _build
     _build.build_library()
-    assert "libfsoftmax.so" in fs.binding.LIB_PATH
+    assert "libfsoftmax" in fs.binding.LIB_PATH      # the normal build, or the checked one (FSOFTMAX_LIB)
     yield
     assert fs.fs_device_status() == fs.FS_OK       # no bounded wait expired in any test
 

@@ -57,9 +57,7 @@ def one_case(rng, S):
         xd = dev(x); yd = torch.zeros_like(xd)
         fs.fs_log_softmax(xd, yd, rows, cols, dtype, scale, S); torch.cuda.synchronize()
         want = fso.log_softmax_f64(x, dtype, scale)
-        with np.errstate(invalid='ignore'):
-            sc = np.maximum(1.0, np.where(np.isfinite(want), np.abs(want), 1.0))
-        ok = fno.compare(torch_bits_to_np(yd, dtype).reshape(rows, cols), dtype, want, sc, rel_tol=1e-6).ok(dtype, rel_tol=1e-6); tag = 'log_softmax'
+        ok = fno.compare(torch_bits_to_np(yd, dtype).reshape(rows, cols), dtype, want, fno.log_softmax_bound(want), rel_tol=1.0).ok(dtype, rel_tol=1.0); tag = 'log_softmax'
     elif op == 2:
         q = int(rng.integers(0, cols + 3)) - 2
         xd = dev(x); yd = torch.zeros_like(xd)
@@ -97,11 +95,7 @@ def one_case(rng, S):
         xd, md = dev(x2), dev(m); yd = torch.zeros_like(xd)
         fs.fs_softmax_masked(xd, md, yd, rows2, cols, q, heads, dtype, scale, S); torch.cuda.synchronize()
         want = fso.softmax_masked_f64(x2, m, dtype, q, heads, scale)
-        mrow = (np.arange(rows2) // (heads * q)) * q + np.arange(rows2) % q
-        with np.errstate(invalid='ignore', over='ignore'):
-            z = float(np.float32(scale)) * fso.widen(x2, dtype) + fso.widen(m, dtype)[mrow]
-            zmax = np.max(np.where(np.isfinite(z), np.abs(z), 0.0), axis=1, keepdims=True)
-            bound = 1e-6 + 2.5e-7 * zmax * np.where(np.isfinite(want), want, 1.0)
+        bound = fno.masked_softmax_bound(x2, m, dtype, q, heads, scale, want)
         ok = fno.compare(torch_bits_to_np(yd, dtype).reshape(rows2, cols), dtype, want, bound, rel_tol=1.0).ok(dtype, rel_tol=1.0); tag = f'masked h={heads}'
     return ok, f"{tag} dtype={dtype} rows={rows} cols={cols} scale={scale}"
 

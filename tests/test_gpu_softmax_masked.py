@@ -56,13 +56,7 @@ def run(x, mask, dtype, q, heads, scale, inplace=False, misalign=0):
 def check(x, mask, dtype, q, heads, scale, **kw):
     got = run(x, mask, dtype, q, heads, scale, **kw)
     want = fso.softmax_masked_f64(x, mask, dtype, q, heads, scale)
-    rows, cols = x.shape
-    sc = float(np.float32(scale))
-    mrow = (np.arange(rows) // (heads * q)) * q + np.arange(rows) % q
-    with np.errstate(invalid="ignore", over="ignore"):
-        z = sc * fso.widen(x, dtype) + fso.widen(mask, dtype)[mrow]
-        zmax = np.max(np.where(np.isfinite(z), np.abs(z), 0.0), axis=1, keepdims=True)
-        bound = 1e-6 + 2.5e-7 * zmax * np.where(np.isfinite(want), want, 1.0)
+    bound = fno.masked_softmax_bound(x, mask, dtype, q, heads, scale, want)      # pinned in tests/test_oracle_masked_pins.py
     rep = fno.compare(got, dtype, want, bound, rel_tol=1.0)
     assert rep.ok(dtype, rel_tol=1.0), (x.shape, dtype, scale, rep)
     g64 = fso.widen(got, dtype)
