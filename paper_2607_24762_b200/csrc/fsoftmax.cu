@@ -95,6 +95,7 @@ int env_int(const char* name, int dflt) {
     const char* e = std::getenv(name);
     return e && e[0] ? std::atoi(e) : dflt;
 }
+bool early_prefetch_enabled() { static const bool v = env_int("FS_EARLY_PF", 1) != 0; return v; }
 bool log_enabled() { static const bool v = env_int("FS_LOG", 0) != 0; return v; }
 bool check_enabled() { static const bool v = env_int("FS_CHECK", 0) != 0; return v; }
 #define FS_LOGF(...) do { if (log_enabled()) { std::fprintf(stderr, "[fsoftmax] " __VA_ARGS__); std::fputc('\n', stderr); } } while (0)
@@ -412,6 +413,7 @@ void set_first_wave_lag(P& p, int resident_clusters, int64_t bytes_per_cluster) 
     static const int bw = [] { const char* e = std::getenv("FS_LAG_BW"); return e ? std::max(0, std::atoi(e)) : 6500; }();
     p.lag_rows = resident_clusters;
     p.lag_ns = bw > 0 ? static_cast<float>(double(bytes_per_cluster) / double(bw)) : 0.0f;
+    p.early_pf = early_prefetch_enabled();
 }
 
 // Programmatic dependent launch (on unless FS_PDL=0): the kernel may be scheduled while the
@@ -729,6 +731,7 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
     p.q_offset = 0;
     p.pf_rows = 0;
     p.dbg_extra_tx = dbg_extra_tx;
+    p.early_pf = early_prefetch_enabled();
     p.wait_polls = dev.wait_polls.load(std::memory_order_relaxed);
     const int64_t max_grid = 0x7fffffff;
 
@@ -890,6 +893,7 @@ int run_causal(const void* x, void* y, int64_t rows, int64_t cols, int64_t q_off
     p.q_offset = q_offset;
     p.pf_rows = 0;
     p.wait_polls = kDefaultWaitPolls;
+    p.early_pf = early_prefetch_enabled();
     SmemGeom sg;
     // (a zero scale goes to the generic kernel: the split kernel masks with -inf, and 0 * -inf is NaN)
     if (fast && p.c != 0.0f && dev.cluster_ok && smem_geom(p.nvec, dtype, 0, 0, &sg) && rows <= 0x7fffffff / sg.cs) {
@@ -1740,7 +1744,7 @@ int fs_copy(const void* x, void* y, int64_t bytes, void* stream) {
     const int64_t grid = std::min<int64_t>((nvec + 1023) / 1024, 0x7fffffff);
     const uint4* xv = static_cast<const uint4*>(x);
     uint4* yv = static_cast<uint4*>(y);
-    return launch(fn, grid, 256, 0, 0, static_cast<cudaStream_t>(stream), xv, yv, nvec);
+    return launch(fn, grid, 256, 0, 0, static_cast<cudaStream_t>(stream), xv, yv, nvec, int(early_prefetch_enabled()));
 }
 
 int fs_softmax_host(const void* x_host, void* y_host, int64_t rows, int64_t cols, int dtype, float scale) {
@@ -1936,6 +1940,7 @@ int fs_softmax_static(const void* x, void* y, int64_t rows, int64_t cols, int dt
     p.q_offset = 0;
     p.pf_rows = 0;
     p.wait_polls = kDefaultWaitPolls;
+    p.early_pf = early_prefetch_enabled();
     const void* fn = smem_row_fn(dtype, p.neg, sg, nvec);
     const size_t stage_bytes = smem_row_stage_bytes(sg, dtype);
     const size_t smem = smem_row_bytes(sg, dtype);

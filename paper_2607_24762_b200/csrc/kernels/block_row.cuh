@@ -156,8 +156,7 @@ block_row_tma_kernel(const Params p, const int nstage, const uint32_t stage_byte
         for (int s = 0; s < nstage; ++s) mbar_init(smem_u32(&bars[s]), 1);
         mbar_fence_init();
         fence_proxy_async_smem();
-        pdl_wait();
-        first_wave_lag(first, p.lag_ns, p.lag_rows);
+        pdl_wait_first_wave<false>(first, p.lag_ns, p.lag_rows, p.early_pf, [&] { if (n_my > 0) pdl_early_prefetch(xb + first * row_bytes, row_bytes); });
         for (int s = 0; s < nstage && s < n_my; ++s)
             bulk_load_row(smem_u32(smem + size_t(s) * stage_bytes),
                           xb + (first + int64_t(s) * gridDim.x) * row_bytes, row_bytes, smem_u32(&bars[s]));
@@ -238,8 +237,10 @@ generic_row_kernel(const Params p) {
 // (four independent loads in flight per thread), blocks handed out by the hardware scheduler
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
-copy_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, const int64_t nvec) {
+copy_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, const int64_t nvec, const int early_pf) {
     pdl_launch_dependents();
+    if (early_pf && threadIdx.x == 0 && int64_t(blockIdx.x) * 1024 < nvec)
+        pdl_early_prefetch(reinterpret_cast<const char*>(x + int64_t(blockIdx.x) * 1024), min(int64_t(1024), nvec - int64_t(blockIdx.x) * 1024) * 16);
     pdl_wait();
     for (int64_t base = int64_t(blockIdx.x) * 1024; base < nvec; base += int64_t(gridDim.x) * 1024) {
         uint4 v[4];

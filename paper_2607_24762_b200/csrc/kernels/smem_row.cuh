@@ -134,8 +134,8 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
         mbar_init(smem_u32(&xbar[1]), 1);
         mbar_fence_init();
         fence_proxy_async_smem();
-        pdl_wait();
-        first_wave_lag(cid, p.lag_ns, p.lag_rows);
+        pdl_wait_first_wave<true>(cid, p.lag_ns, p.lag_rows, p.early_pf, [&] {
+            if (cid < p.rows && nv > 0) pdl_early_prefetch(xb + int64_t(cid) * row_bytes, int64_t(nv) * 16); });
         if (cid < p.rows) issue_row(cid);
         // the row that starts a fraction of a generation of resident clusters later: its slice is on
         // its way to L2 while this one is worked on

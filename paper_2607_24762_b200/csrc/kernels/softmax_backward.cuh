@@ -27,6 +27,7 @@ struct SmbParams {
     int64_t pf_rows;
     float lag_ns;          // first wave of a one-shot grid: cluster i < lag_rows starts i * lag_ns late
     int lag_rows;
+    int early_pf;          // first wave: ask L2 for the block's own input before griddepcontrol.wait (pdl_early_prefetch)
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -111,10 +112,10 @@ smb_tile_kernel(const SmbParams p) {
         fence_proxy_async_smem();
     }
     __syncthreads();
-    pdl_wait();
-    if (row >= p.rows) return;                             // no block-wide barrier follows
     const char* gb = static_cast<const char*>(p.dy) + row * int64_t(row_bytes);
     const char* yb = static_cast<const char*>(p.y) + row * int64_t(row_bytes);
+    pdl_wait();
+    if (row >= p.rows) return;                             // no block-wide barrier follows
     if (lane == 0) {
         first_wave_lag(blockIdx.x, p.lag_ns, p.lag_rows);
         const uint32_t bar = smem_u32(&bars[w]);
@@ -212,8 +213,7 @@ smb_smem_kernel(const SmbParams p, const uint32_t stage_bytes, const int slice, 
         mbar_init(smem_u32(&xbar), 1);
         mbar_fence_init();
         fence_proxy_async_smem();
-        pdl_wait();
-        first_wave_lag(row, p.lag_ns, p.lag_rows);
+        pdl_wait_first_wave<true>(row, p.lag_ns, p.lag_rows, p.early_pf, [&] { if (nv > 0) { pdl_early_prefetch(gb + row * row_bytes, int64_t(nv) * 16); pdl_early_prefetch(yb + row * row_bytes, int64_t(nv) * 16); } });
         for (int ch = 0; ch < nchunk; ++ch) {
             const uint32_t cv = uint32_t(FULL ? chunk_vecs : min(chunk_vecs, nv - ch * chunk_vecs)) * 16u;
             const uint32_t off = uint32_t(ch) * uint32_t(chunk_vecs) * 16u;

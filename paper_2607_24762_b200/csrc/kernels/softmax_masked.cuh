@@ -35,6 +35,7 @@ struct MaskedParams {
     int64_t pf_rows;
     float lag_ns;          // first wave of a one-shot grid: cluster i < lag_rows starts i * lag_ns late
     int lag_rows;
+    int early_pf;          // first wave: ask L2 for the block's own input before griddepcontrol.wait (pdl_early_prefetch)
 };
 
 __device__ __forceinline__ int64_t mask_row_of(const MaskedParams& p, int64_t row) {
@@ -170,9 +171,9 @@ sm_masked_tile_kernel(const MaskedParams p) {
         fence_proxy_async_smem();
     }
     __syncthreads();
+    const char* xb = static_cast<const char*>(p.x);
     pdl_wait();
     if (row >= p.rows) return;                             // no block-wide barrier follows
-    const char* xb = static_cast<const char*>(p.x);
     if (lane == 0) {
         first_wave_lag(blockIdx.x, p.lag_ns, p.lag_rows);
         bulk_load_row(smem_u32(smem) + uint32_t(w) * uint32_t(row_bytes), xb + row * row_bytes, uint32_t(row_bytes), smem_u32(&bars[w]));
@@ -285,8 +286,7 @@ sm_masked_smem_kernel(const MaskedParams p, const uint32_t stage_bytes, const in
         mbar_init(smem_u32(&xbar), 1);
         mbar_fence_init();
         fence_proxy_async_smem();
-        pdl_wait();
-        first_wave_lag(row, p.lag_ns, p.lag_rows);
+        pdl_wait_first_wave<true>(row, p.lag_ns, p.lag_rows, p.early_pf, [&] { if (nv > 0) { pdl_early_prefetch(xb + row * row_bytes, int64_t(nv) * 16); } });
         for (int ch = 0; ch < nchunk; ++ch) {
             const int cv = FULL ? chunk_vecs : min(chunk_vecs, nv - ch * chunk_vecs);
             bulk_load_row(smem_u32(smem) + uint32_t(ch) * uint32_t(chunk_vecs) * 16u,

@@ -134,9 +134,9 @@ softmax_tile_kernel(const Params p) {
         fence_proxy_async_smem();
     }
     __syncthreads();
+    const char* xb = static_cast<const char*>(p.x);
     pdl_wait();
     if (row >= p.rows) return;                             // no block-wide barrier follows
-    const char* xb = static_cast<const char*>(p.x);
     if (lane == 0) {
         first_wave_lag(blockIdx.x, p.lag_ns, p.lag_rows);
         bulk_load_row(smem_u32(smem) + uint32_t(w) * uint32_t(row_bytes), xb + row * row_bytes, uint32_t(row_bytes), smem_u32(&bars[w]));
