@@ -35,6 +35,11 @@
  *     cudaPointerGetAttributes (memory the current device cannot address is FS_ERR_INVALID_ARG);
  *     FS_SIM_NO_CLUSTER=1 and FS_SIM_SMEM_OPTIN=<bytes> make the library behave as on a device
  *     without cluster launch / with less shared memory, so that its downgrade paths can be tested.
+ *   - Stream order is all a caller has to respect. Kernels are launched with programmatic dependent
+ *     launch: they may become resident while the previous kernel of the stream drains, and read their
+ *     inputs only after it has completed. Before that point the first wave of the long-row kernels
+ *     asks the L2 cache for its own input (a prefetch, never a read: whatever the previous kernel
+ *     still writes there is what the later read returns). FS_PDL=0 / FS_EARLY_PF=0 turn the two off.
  */
 #ifndef FSOFTMAX_H_
 #define FSOFTMAX_H_

@@ -75,6 +75,16 @@ warp_row_kernel(const Params p) {
     uint4* __restrict__ yv = static_cast<uint4*>(p.y);
     const int nvec = static_cast<int>(p.nvec);
     auto live = [&](int k) { return sl + k * LANES < nvec; };
+    if (LANES * VPL >= 128 && p.early_pf && lane == 0) {
+        // rows of 2 KiB and more: this warp's first tile (contiguous rows) is asked of L2 ahead of the
+        // dependency wait (pdl_early_prefetch); measured 21.77 -> 21.57 us on 16384 rows of 4 KiB bf16,
+        // while 256-byte rows lose (12.02 -> 12.09 us on 131072 of them) and go without
+        const int64_t tile0 = int64_t(blockIdx.x) * warps + (threadIdx.x >> 5);
+        if (tile0 < ntiles) {
+            const int64_t r0 = tile0 * rows_per_tile;
+            pdl_early_prefetch(reinterpret_cast<const char*>(xv + r0 * p.nvec), min(rows_per_tile, p.rows - r0) * p.nvec * 16);
+        }
+    }
     pdl_wait();
 
     for (int64_t tile = int64_t(blockIdx.x) * warps + (threadIdx.x >> 5); tile < ntiles;
