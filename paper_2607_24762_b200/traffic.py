@@ -4,7 +4,7 @@ The record lives in ``profiles/dram_traffic.txt`` (text, one line per workload);
 for ``roofline.traffic``. It is written by this module from the CSV logs of
 
     ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum --print-units base --clock-control none \
-        -k regex:<kernel> -s <warm-up launches> -c 8 --csv --log-file <log>.csv \
+        --cache-control none -k regex:<kernel> -s <warm-up launches> -c 8 --csv --log-file <log>.csv \
         python bench.py --workload cfgN [--rows R] --steps 8 --trains 1 --warmup 3 --no-all --no-e2e --no-cpu --no-clocks
 
 (one capture per workload, after the same command has exited 0 without ncu): eight CONSECUTIVE launches
