@@ -1499,6 +1499,27 @@ template <int DT> const void* masked_warp_fn(const WarpGeom& g) {
     }
 }
 
+// the four-rows-per-block kernel of fs_softmax_masked by number of batches (of 128 vectors) and whether the row fills them
+template <int DT> const void* masked_tile_fn(int nb, bool full) {
+    if constexpr (DT == DT_F32) {
+        return nullptr;
+    } else {
+        switch (nb * 2 + (full ? 1 : 0)) {
+            case 4:  return (const void*)sm_masked_tile_kernel<DT, 2, false>;
+            case 5:  return (const void*)sm_masked_tile_kernel<DT, 2, true>;
+            case 6:  return (const void*)sm_masked_tile_kernel<DT, 3, false>;
+            case 7:  return (const void*)sm_masked_tile_kernel<DT, 3, true>;
+            case 8:  return (const void*)sm_masked_tile_kernel<DT, 4, false>;
+            case 9:  return (const void*)sm_masked_tile_kernel<DT, 4, true>;
+            case 10: return (const void*)sm_masked_tile_kernel<DT, 5, false>;
+            case 11: return (const void*)sm_masked_tile_kernel<DT, 5, true>;
+            case 12: return (const void*)sm_masked_tile_kernel<DT, 6, false>;
+            case 13: return (const void*)sm_masked_tile_kernel<DT, 6, true>;
+            default: return nullptr;
+        }
+    }
+}
+
 int run_softmax_masked(const void* x, const void* mask, void* y, int64_t rows, int64_t cols, int64_t q_rows, int64_t heads,
                        int dtype, float scale, cudaStream_t st) {
     Device* devp = nullptr;
@@ -1514,13 +1535,15 @@ int run_softmax_masked(const void* x, const void* mask, void* y, int64_t rows, i
     p.c = static_cast<float>(static_cast<double>(scale) * kLog2e);
     p.status = dev.status; p.pf_rows = 0;
     if (fast && masked_tile_wanted(dtype, p.nvec)) {        // rows of 4-11 KiB: a warp per row from shared memory
-        const void* fn = by_dtype(dtype, [&](auto dt) -> const void* { return (const void*)sm_masked_tile_kernel<decltype(dt)::value>; });
+        const int nb = static_cast<int>((p.nvec + 127) / 128);          // batches of 4 vectors per lane
+        const bool full = p.nvec % 128 == 0;
+        const void* fn = by_dtype(dtype, [&](auto dt) -> const void* { return masked_tile_fn<decltype(dt)::value>(nb, full); });
         const int t = 128;
         const size_t smem = size_t(t / 32) * size_t(p.nvec) * 16 + size_t(t / 32) * 8;
-        int bps = 0;
-        if ((rc = blocks_per_sm(dev, fn, t, smem, &bps)) != FS_OK) return rc;
         const int64_t grid = (rows + (t / 32) - 1) / (t / 32);
-        if (grid <= 0x7fffffff) {
+        if (fn && grid <= 0x7fffffff) {                     // (a forced range beyond six batches goes to the kernels below)
+            int bps = 0;
+            if ((rc = blocks_per_sm(dev, fn, t, smem, &bps)) != FS_OK) return rc;
             p.pf_rows = prefetch_rows(dev.sm_count * bps) * (t / 32);
             set_first_wave_lag(p, dev.sm_count * bps, (t / 32) * p.nvec * 16);
             return launch(fn, grid, t, smem, 0, st, p);

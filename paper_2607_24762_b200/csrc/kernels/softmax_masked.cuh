@@ -145,17 +145,27 @@ sm_masked_warp_long_kernel(const MaskedParams p) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// Rows of 4-11 KiB: four rows per block, each brought to shared memory by a bulk copy of its own
-// (one mbarrier per row) and worked on by one warp alone, with the arithmetic of the warp kernel
-// above: pass A takes the maximum exponent, pass B puts e = 2^(t - R) back in place of x in shared
-// memory in the element dtype, pass C scales and stores. The mask vectors come through the
-// read-only path in passes A and B. No block barrier after start-up; the register footprint does
-// not grow with the row. One-shot grid: block b handles rows b*W .. b*W+W-1.
-// dynamic shared memory: W rows | W mbarriers
+// 16-bit rows of 4-10 KiB: four rows per block, each brought to shared memory by a bulk copy of its
+// own (one mbarrier per row) and worked on by one warp alone, in NB batches of 4 vectors per lane.
+// The exponents t = x c + m log2(e) are formed ONCE (the mask vectors are read once, through the
+// read-only path): a lane takes the largest t of its 32 elements of the batch as that batch's
+// reference r_b, puts e = 2^(t - r_b) back in place of x in shared memory in the element dtype and
+// folds the batch's sum into its running (r, s) pair with the online-softmax merge
+// (Milakov-Gimelshein); the lanes' pairs are merged by shuffles, and the last sweep stores
+// y = e * 2^(r_b - R) / S, the per-batch factor being one ex2 per lane and batch. This is the
+// split-row kernel's arithmetic (smem_row.cuh: chunk references, in-place e, the bf16 bias of 2^64
+// and the separate small factor) with a lane's batch in the role of a thread's chunk; the bias is
+// folded into the reference (r_b - 64 is what is subtracted and what is merged), which saves the
+// addition per element. A first version took the row maximum in a sweep of its own and formed t
+// twice: 21.5 thread instructions per element and 27.9 us on 8 x 2048 rows of 4 KiB bf16 with a
+// shared mask, issue-bound; this one takes 23.4 us (rows of 5 / 8 / 10 KiB: 35.5 -> 31.8, 33.7 -> 26.7, 41.8 -> 32.9 us).
+// FULL: the row is exactly NB batches (no bounds checks). No block barrier after start-up.
+// One-shot grid: block b handles rows b*W .. b*W+W-1. dynamic shared memory: W rows | W mbarriers
 // ---------------------------------------------------------------------------------------------
-template <int DT>
+template <int DT, int NB, bool FULL>
 __global__ void __launch_bounds__(128)
 sm_masked_tile_kernel(const MaskedParams p) {
+    static_assert(DT != DT_F32, "16-bit element types only");
     constexpr int NP = Traits<DT>::VE / 2;
     constexpr int H = 4;                                   // vectors per lane and batch
     pdl_launch_dependents();
@@ -183,63 +193,77 @@ sm_masked_tile_kernel(const MaskedParams p) {
     const uint4* __restrict__ mr = static_cast<const uint4*>(p.mask) + mask_row_of(p, row) * p.nvec + lane;
     uint4* __restrict__ yv = static_cast<uint4*>(p.y) + row * p.nvec + lane;
     const f32x2 c2 = pair(p.c, p.c);
+    const float ident = __int_as_float(0xff800000);
+    const uint32_t ninf = DT == DT_BF16 ? 0xff80ff80u : 0xfc00fc00u;     // a vector past the row's end: x = 0, mask = -inf
     mbar_wait_warp(smem_u32(&bars[w]), 0u, p.status);      // on a timeout the status word is set and the row is garbage
 
-    float r = __int_as_float(0xff800000);
-    for (int k0 = 0; k0 < nvec; k0 += 32 * H) {
+    float rb[NB];                                          // what batch b's e are relative to (ident: nothing but -inf or NaN)
+    float r = ident, s = 0.0f;
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+        const int k0 = b * 32 * H;
         uint4 xr[H], mk[H];
 #pragma unroll
         for (int u = 0; u < H; ++u) {
-            xr[u] = make_uint4(0u, 0u, 0u, 0u); mk[u] = xr[u];
-            if (k0 + u * 32 + lane < nvec) { xr[u] = sv[k0 + u * 32]; mk[u] = ld_cached(mr + k0 + u * 32); }
+            xr[u] = make_uint4(0u, 0u, 0u, 0u); mk[u] = make_uint4(ninf, ninf, ninf, ninf);
+            if (FULL || k0 + u * 32 + lane < nvec) { xr[u] = sv[k0 + u * 32]; mk[u] = ld_cached(mr + k0 + u * 32); }
         }
+        f32x2 t[H][NP];
+        float m = ident;
+#pragma unroll
+        for (int u = 0; u < H; ++u) m = fmaxf(m, masked_exponents<DT>(xr[u], mk[u], c2, t[u]));
+        // all of these elements masked (or none finite): subtract 0 instead of the identity. bf16: e carries
+        // 2^64 so that outputs below 2^-126 survive in e (see ex2_elem); the bias sits in the reference.
+        const float sub = ((m == ident) ? 0.0f : m) - (DT == DT_BF16 ? 64.0f : 0.0f);
+        rb[b] = (m == ident) ? ident : sub;
+        const f32x2 s2 = pair(sub, sub);
+        f32x2 acc[2] = {pair(0.0f, 0.0f), pair(0.0f, 0.0f)};
 #pragma unroll
         for (int u = 0; u < H; ++u) {
-            if (k0 + u * 32 + lane < nvec) {
-                f32x2 t[NP];
-                r = fmaxf(r, masked_exponents<DT>(xr[u], mk[u], c2, t));
+#pragma unroll
+            for (int j = 0; j < NP; ++j) {
+                float lo, hi;
+                unpair(sub2(t[u][j], s2), lo, hi);
+                t[u][j] = pair(ex2_ftz(lo), ex2_ftz(hi));
+                acc[j & 1] = add2(acc[j & 1], t[u][j]);
             }
+            if (FULL || k0 + u * 32 + lane < nvec) sv[k0 + u * 32] = narrow_pairs<DT>(t[u]);     // this lane alone reads it back
         }
+        const float part = pair_sum(add2(acc[0], acc[1]));
+        // online merge of (rb[b], part) into (r, s): only the sum left behind is rescaled
+        const float rn = fmaxf(r, rb[b]);
+        const bool keep = (rn == r);
+        const float lo = keep ? rb[b] : r;
+        const float f = (lo == ident) ? 1.0f : ex2_ftz(lo - rn);
+        s = keep ? fmaf(part, f, s) : fmaf(s, f, part);
+        r = rn;
     }
-    r = warp_pick<32, false>(r);
-    const f32x2 r2 = pair(r, r);
-    f32x2 acc[2] = {pair(0.0f, 0.0f), pair(0.0f, 0.0f)};
-    for (int k0 = 0; k0 < nvec; k0 += 32 * H) {
-        uint4 xr[H], mk[H];
+    warp_merge_pairs<false>(r, s, 1.0f);
+    const float inv = recip<DT>(s);
 #pragma unroll
-        for (int u = 0; u < H; ++u) {
-            xr[u] = make_uint4(0u, 0u, 0u, 0u); mk[u] = xr[u];
-            if (k0 + u * 32 + lane < nvec) { xr[u] = sv[k0 + u * 32]; mk[u] = ld_cached(mr + k0 + u * 32); }
-        }
-#pragma unroll
-        for (int u = 0; u < H; ++u) {
-            if (k0 + u * 32 + lane < nvec) {
-                f32x2 t[NP];
-                masked_exponents<DT>(xr[u], mk[u], c2, t);
-#pragma unroll
-                for (int j = 0; j < NP; ++j) {
-                    float lo, hi;
-                    unpair(sub2(t[j], r2), lo, hi);
-                    if (DT == DT_BF16) { lo += 64.0f; hi += 64.0f; }        // keeps subnormal bf16 outputs (see ex2_elem)
-                    t[j] = pair(ex2_ftz(lo), ex2_ftz(hi));
-                    acc[j & 1] = add2(acc[j & 1], t[j]);
-                }
-                sv[k0 + u * 32] = narrow_pairs<DT>(t);     // this lane alone reads it back
-            }
-        }
-    }
-    const float inv = recip<DT>(warp_sum<32>(pair_sum(add2(acc[0], acc[1]))));
-    const f32x2 i2 = pair(inv, inv);
-    for (int k0 = 0; k0 < nvec; k0 += 32 * H) {
+    for (int b = 0; b < NB; ++b) {
+        const int k0 = b * 32 * H;
+        const float fac = (rb[b] == ident) ? 1.0f : ex2_noflush(rb[b] - r);
+        // bf16: e carries 2^64 and inv 2^-64; a factor this small is applied separately so that
+        // fac * inv cannot underflow before it meets e
+        const bool one_mul = DT != DT_BF16 || fac >= 0x1p-40f || !(fac == fac);
+        const float f1 = one_mul ? fac * inv : inv;
+        const f32x2 f2 = pair(f1, f1), g2 = pair(fac, fac);
         uint4 e[H];
 #pragma unroll
         for (int u = 0; u < H; ++u) {
             e[u] = make_uint4(0u, 0u, 0u, 0u);
-            if (k0 + u * 32 + lane < nvec) e[u] = sv[k0 + u * 32];
+            if (FULL || k0 + u * 32 + lane < nvec) e[u] = sv[k0 + u * 32];
         }
+        if (one_mul) {
 #pragma unroll
-        for (int u = 0; u < H; ++u)
-            if (k0 + u * 32 + lane < nvec) st_stream(yv + k0 + u * 32, scale_vec<DT, false>(e[u], i2, i2));
+            for (int u = 0; u < H; ++u)
+                if (FULL || k0 + u * 32 + lane < nvec) st_stream(yv + k0 + u * 32, scale_vec<DT, false>(e[u], f2, f2));
+        } else {                                           // rare: both multiplications before the one rounding
+#pragma unroll
+            for (int u = 0; u < H; ++u)
+                if (FULL || k0 + u * 32 + lane < nvec) st_stream(yv + k0 + u * 32, scale_vec<DT, true>(e[u], f2, g2));
+        }
     }
 }
 
