@@ -68,6 +68,10 @@ __device__ __forceinline__ float masked_exponents(const uint4& xraw, const uint4
 // read-only path (they are shared by the heads and hit L1/L2). Pass A takes the maximum exponent,
 // pass B forms e = 2^(t - R), adds it up and puts it back in place of x in the element dtype
 // (the in-place store of the split-row kernel, in registers), pass C scales and stores.
+// The single sweep of sm_masked_tile_kernel below (exponents formed once, per-batch references) was
+// tried here too and is slower: holding a batch's 32 exponents takes 72 registers against 56 and the
+// resident warps are what hides the latency of this kernel (bf16 rows of 1 / 2 / 3 KiB: 10.1 -> 11.2,
+// 16.5 -> 18.4, 23.5 -> 27.5 us; fp32 rows of 4 KiB 23.2 -> 24.2 us).
 template <int DT, int LANES, int VPL>
 __device__ __forceinline__ void sm_masked_warp_body(const MaskedParams& p) {
     constexpr int NP = Traits<DT>::VE / 2;
