@@ -576,24 +576,27 @@ template <int DT> const void* router_fn(const WarpGeom& g) {
     return nullptr;
 }
 
-// k <= 8: the sorting-network kernel, same geometries
-template <int DT> const void* router8_fn(const WarpGeom& g) {
-    if (g.vpl == 1) return (const void*)router_top8_kernel<DT, 1, 1>;
-    if (g.vpl == 2) return (const void*)router_top8_kernel<DT, 1, 2>;
+// k <= 8: the sorting-network kernel, same geometries; FULL when the row fills them exactly
+template <int DT, bool FULL> const void* router8_fn(const WarpGeom& g) {
+    if (g.vpl == 1) return (const void*)router_top8_kernel<DT, 1, 1, FULL>;
+    if (g.vpl == 2) return (const void*)router_top8_kernel<DT, 1, 2, FULL>;
     if (g.vpl == 4) {
         switch (g.lanes) {
-            case 1:  return (const void*)router_top8_kernel<DT, 1, 4>;
-            case 2:  return (const void*)router_top8_kernel<DT, 2, 4>;
-            case 4:  return (const void*)router_top8_kernel<DT, 4, 4>;
-            case 8:  return (const void*)router_top8_kernel<DT, 8, 4>;
-            case 16: return (const void*)router_top8_kernel<DT, 16, 4>;
-            default: return (const void*)router_top8_kernel<DT, 32, 4>;
+            case 1:  return (const void*)router_top8_kernel<DT, 1, 4, FULL>;
+            case 2:  return (const void*)router_top8_kernel<DT, 2, 4, FULL>;
+            case 4:  return (const void*)router_top8_kernel<DT, 4, 4, FULL>;
+            case 8:  return (const void*)router_top8_kernel<DT, 8, 4, FULL>;
+            case 16: return (const void*)router_top8_kernel<DT, 16, 4, FULL>;
+            default: return (const void*)router_top8_kernel<DT, 32, 4, FULL>;
         }
     }
     if constexpr (DT == DT_F32) {
-        if (g.vpl == 8) return (const void*)router_top8_kernel<DT, 32, 8>;
+        if (g.vpl == 8) return (const void*)router_top8_kernel<DT, 32, 8, FULL>;
     }
     return nullptr;
+}
+template <int DT> const void* router8_fn(const WarpGeom& g, bool full) {
+    return full ? router8_fn<DT, true>(g) : router8_fn<DT, false>(g);
 }
 
 // Calls f(std::integral_constant<int, DT>, std::bool_constant<NEG>) for the run-time dtype and sign.
@@ -1641,11 +1644,12 @@ int fs_router_topk(const void* x, float* w, int32_t* idx, int64_t rows, int64_t 
     // kernel that takes one maximum per round, which serves any k)
     static const bool rounds_only = env_int("FS_ROUTER_ROUNDS", 0) != 0;
     const bool net = k <= 8 && !rounds_only;
+    const bool full = nvec == int64_t(g.lanes) * g.vpl;        // no padding vectors in a row's lanes
     const void* fn = nullptr;
     switch (dtype) {
-        case FS_DTYPE_FP32: fn = net ? router8_fn<DT_F32>(g) : router_fn<DT_F32>(g); break;
-        case FS_DTYPE_BF16: fn = net ? router8_fn<DT_BF16>(g) : router_fn<DT_BF16>(g); break;
-        default:            fn = net ? router8_fn<DT_F16>(g) : router_fn<DT_F16>(g); break;
+        case FS_DTYPE_FP32: fn = net ? router8_fn<DT_F32>(g, full) : router_fn<DT_F32>(g); break;
+        case FS_DTYPE_BF16: fn = net ? router8_fn<DT_BF16>(g, full) : router_fn<DT_BF16>(g); break;
+        default:            fn = net ? router8_fn<DT_F16>(g, full) : router_fn<DT_F16>(g); break;
     }
     if (!fn) return FS_ERR_UNSUPPORTED;
     RouterParams p;

@@ -189,18 +189,25 @@ template <class K> __device__ __forceinline__ void merge8_desc(K (&a)[8], const 
     bitonic8_desc(a);
 }
 
+// A key is built in two steps so that its column part costs no arithmetic per element: the column of
+// element i of vector v in lane sl is v * LANES * VE + sl * VE + i, three bit fields that do not overlap
+// (all powers of two), so the complement 0xffff - col is 0xffff ^ (v * LANES * VE + i) ^ (sl * VE): the
+// first part is an immediate folded into the key's last logic operation (local), and the lane's part is
+// put into the eight keys that survive the lane's own sort (with_lane). Among one lane's elements the
+// local part alone orders equal values by column.
 template <int DT> struct RouterKey {                       // 16-bit inputs: value and column in one word
     using type = uint32_t;
-    static __device__ __forceinline__ type make(float z, int col) {
-        if (DT == DT_BF16) {       // z is a bf16 value: the high half of its binary32 key is its 16-bit key
+    static __device__ __forceinline__ type local(float z, int c) {
+        if (DT == DT_BF16) {       // z is a bf16 value (low half of its binary32 image zero): flip the sign bit, or the whole high half
             const uint32_t b = __float_as_uint(z);
-            const uint32_t o = b ^ (static_cast<uint32_t>(static_cast<int32_t>(b) >> 31) | 0x80000000u);
-            return (o & 0xffff0000u) | (0xffffu - static_cast<uint32_t>(col));
+            const uint32_t m = (static_cast<uint32_t>(static_cast<int32_t>(b) >> 31) & 0x7fff0000u) | 0x80000000u;
+            return b ^ m ^ (0xffffu ^ static_cast<uint32_t>(c));
         }
         const uint32_t h = static_cast<uint32_t>(__half_as_ushort(__float2half_rn(z))); // z is an fp16 value: exact
         const uint32_t o = (h & 0x8000u) ? (~h & 0xffffu) : (h | 0x8000u);
-        return (o << 16) | (0xffffu - static_cast<uint32_t>(col));
+        return (o << 16) | (0xffffu ^ static_cast<uint32_t>(c));
     }
+    static __device__ __forceinline__ type with_lane(type k, int lane_cols) { return k ^ static_cast<uint32_t>(lane_cols); }
     static __device__ __forceinline__ int col(type k) { return static_cast<int>(0xffffu - (k & 0xffffu)); }
     static __device__ __forceinline__ float value(type k) {
         const uint32_t o = k >> 16;
@@ -211,14 +218,19 @@ template <int DT> struct RouterKey {                       // 16-bit inputs: val
 };
 template <> struct RouterKey<DT_F32> {
     using type = unsigned long long;
-    static __device__ __forceinline__ type make(float z, int col) {
-        return (static_cast<type>(order_key(z)) << 32) | static_cast<type>(0xffffffffu - static_cast<uint32_t>(col));
+    static __device__ __forceinline__ type local(float z, int c) {
+        return (static_cast<type>(order_key(z)) << 32) | static_cast<type>(0xffffffffu ^ static_cast<uint32_t>(c));
     }
+    static __device__ __forceinline__ type with_lane(type k, int lane_cols) { return k ^ static_cast<type>(static_cast<uint32_t>(lane_cols)); }
     static __device__ __forceinline__ int col(type k) { return static_cast<int>(0xffffffffu - static_cast<uint32_t>(k)); }
     static __device__ __forceinline__ float value(type k) { return order_unkey(static_cast<uint32_t>(k >> 32)); }
 };
 
-template <int DT, int LANES, int VPL>
+// FULL: every row has exactly LANES * VPL vectors (no padding keys, no per-vector predicates); the rows
+// past the end that the last group of a warp may hold read the last row instead and store nothing.
+// The row maximum the softmax needs is not reduced separately: it is the value of the first key once
+// the row's eight best are known, so the sum of exponentials follows the selection.
+template <int DT, int LANES, int VPL, bool FULL>
 __global__ void __launch_bounds__(128)
 router_top8_kernel(const RouterParams p) {
     constexpr int VE = Traits<DT>::VE;
@@ -241,30 +253,18 @@ router_top8_kernel(const RouterParams p) {
     for (int64_t grp = int64_t(blockIdx.x) * warps + (tid >> 5); grp < ngroups; grp += int64_t(gridDim.x) * warps) {
         const int64_t row = grp * G + sub;
         const bool row_ok = row < p.rows;
+        const int64_t row_ld = FULL ? (row_ok ? row : p.rows - 1) : row;
         float z[VPL][VE];
         bool live[VPL];
-        float top = __int_as_float(0xff800000);
 #pragma unroll
         for (int v = 0; v < VPL; ++v) {
-            live[v] = row_ok && sl + v * LANES < nvec;
+            live[v] = FULL || (row_ok && sl + v * LANES < nvec);
             uint4 raw = make_uint4(0u, 0u, 0u, 0u);
-            if (live[v]) raw = ld_stream(xv + row * p.nvec + sl + v * LANES);
+            if (live[v]) raw = ld_stream(xv + row_ld * p.nvec + sl + v * LANES);
             unpack<DT>(raw, z[v]);
 #pragma unroll
-            for (int i = 0; i < VE; ++i) {
-                z[v][i] = fmaf(z[v][i], sg, 0.0f);          // sign of the scale; -0 becomes +0; inf * 0 = NaN
-                if (live[v]) top = fmaxf(top, z[v][i]);     // fmaxf drops NaN
-            }
+            for (int i = 0; i < VE; ++i) z[v][i] = fmaf(z[v][i], sg, 0.0f);   // sign of the scale; -0 becomes +0; inf * 0 = NaN
         }
-        top = warp_pick<LANES, false>(top);
-        float s = 0.0f;
-#pragma unroll
-        for (int v = 0; v < VPL; ++v)
-#pragma unroll
-            for (int i = 0; i < VE; ++i)
-                if (live[v]) s += ex2_ftz_r((z[v][i] - top) * cabs);
-        s = warp_sum<LANES>(s);
-        const float inv_s = 1.0f / s;                      // NaN when the row is NaN
 
         // ---- this lane's eight best
         K best[8];
@@ -278,7 +278,8 @@ router_top8_kernel(const RouterParams p) {
                 if (f < E) {
                     const int v = f / VE, i = f % VE;
                     const float kz = fmaxf(z[v][i], __int_as_float(0xff800000));       // NaN counts as -inf (fmaxf drops it)
-                    if (live[v]) grp8[j] = RK::make(kz, (v * LANES + sl) * VE + i);
+                    const K key = RK::local(kz, v * LANES * VE + i);
+                    grp8[j] = (FULL || live[v]) ? key : K(0);                            // padding is never selected
                 }
             }
             sort8_desc(grp8);
@@ -289,6 +290,8 @@ router_top8_kernel(const RouterParams p) {
                 merge8_desc(best, grp8);
             }
         }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) best[j] = RK::with_lane(best[j], sl * VE);
         // ---- the row's eight best: merge across the lanes of the group
 #pragma unroll
         for (int o = 1; o < LANES; o <<= 1) {
@@ -297,8 +300,17 @@ router_top8_kernel(const RouterParams p) {
             for (int j = 0; j < 8; ++j) other[j] = __shfl_xor_sync(0xffffffffu, best[j], o);
             merge8_desc(best, other);
         }
-        // ---- weights and output: entry r by lane r mod LANES
+        // ---- the softmax sum against the row maximum (the first key; -inf for a row of NaN or -inf only)
         const float key0 = RK::value(best[0]);
+        float s = 0.0f;
+#pragma unroll
+        for (int v = 0; v < VPL; ++v)
+#pragma unroll
+            for (int i = 0; i < VE; ++i)
+                if (FULL || live[v]) s += ex2_ftz_r((z[v][i] - key0) * cabs);
+        s = warp_sum<LANES>(s);
+        const float inv_s = 1.0f / s;                      // NaN when the row is NaN
+        // ---- weights and output: entry r by lane r mod LANES
         float e[8];
         float sel = 0.0f;
 #pragma unroll
