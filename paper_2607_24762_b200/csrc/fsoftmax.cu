@@ -96,6 +96,7 @@ int env_int(const char* name, int dflt) {
     return e && e[0] ? std::atoi(e) : dflt;
 }
 bool early_prefetch_enabled() { static const bool v = env_int("FS_EARLY_PF", 1) != 0; return v; }
+bool wide_store_enabled() { static const bool v = env_int("FS_WIDE_STORE", 1) != 0; return v; }
 bool log_enabled() { static const bool v = env_int("FS_LOG", 0) != 0; return v; }
 bool check_enabled() { static const bool v = env_int("FS_CHECK", 0) != 0; return v; }
 #define FS_LOGF(...) do { if (log_enabled()) { std::fprintf(stderr, "[fsoftmax] " __VA_ARGS__); std::fputc('\n', stderr); } } while (0)
@@ -1310,6 +1311,7 @@ int run_log_softmax(const void* x, void* y, int64_t rows, int64_t cols, int dtyp
     p.c = static_cast<float>(static_cast<double>(p.scale) * kLog2e);
     p.flip = std::signbit(scale) && scale != 0.0f ? (dtype == FS_DTYPE_FP32 ? 0x80000000u : 0x80008000u) : 0u;
     p.status = dev.status; p.pf_rows = 0;
+    p.wide = (out == OUT_PROB32 && reinterpret_cast<uintptr_t>(y) % 32 == 0 && wide_store_enabled()) ? 1 : 0;   // (a row of y is a multiple of 32 bytes)
     if (fast && lsm_tile_wanted(dtype, p.nvec) && (out == OUT_LOG || dtype != FS_DTYPE_FP32)) {   // a warp per row from shared memory
         const void* fn = by_dtype(dtype, [&](auto dt) -> const void* {
             constexpr int DT = decltype(dt)::value;
@@ -1656,6 +1658,7 @@ int fs_router_topk(const void* x, float* w, int32_t* idx, int64_t rows, int64_t 
     p.x = x; p.w = w; p.idx = idx; p.rows = rows; p.nvec = nvec; p.k = k;
     p.c = static_cast<float>(static_cast<double>(scale) * kLog2e);
     p.renorm = renormalize ? 1 : 0;
+    p.wide = (net && k == 8 && reinterpret_cast<uintptr_t>(w) % 32 == 0 && reinterpret_cast<uintptr_t>(idx) % 32 == 0 && wide_store_enabled()) ? 1 : 0;
     const int t = 128;
     const size_t smem = net ? 0 : static_cast<size_t>(g.vpl) * (dtype == FS_DTYPE_FP32 ? 4 : 8) * t * sizeof(uint32_t);   // <= 16 KiB
     const int64_t groups = (rows + (32 / g.lanes) - 1) / (32 / g.lanes);

@@ -93,6 +93,15 @@ __device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
                  :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
+// 32 bytes at a 32-byte-aligned address in one instruction (256-bit global stores: sm_100): a warp
+// whose lanes each own 32 consecutive output bytes writes 1 KiB of whole sectors per instruction,
+// where two 16-byte stores per lane each fill half of every sector they touch.
+__device__ __forceinline__ void st_stream32(uint4* p, const uint4& a, const uint4& b) {
+    FS_DBG_STORE(p, 32);
+    asm volatile("st.global.cs.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 :: "l"(p), "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w) : "memory");
+}
+
 __device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"

@@ -38,6 +38,7 @@ struct LsmParams {
     float lag_ns;          // first wave of a one-shot grid: cluster i < lag_rows starts i * lag_ns late
     int lag_rows;
     int early_pf;          // first wave: ask L2 for the block's own input before griddepcontrol.wait (pdl_early_prefetch)
+    int wide;              // OUT_PROB32: y is 32-byte aligned, a vector's eight floats leave in one 256-bit store
 };
 
 __device__ __forceinline__ float lg2_approx(float v) {
@@ -69,8 +70,9 @@ __device__ __forceinline__ void lsm_accumulate(const uint4& raw, f32x2 r2, f32x2
 
 // One vector of output from one (sign-adjusted) vector of x. `ybase` is the row's first output
 // element; `v` the vector's index in the row. k2 is -ln S (OUT_LOG) or 1/S (OUT_PROB32).
+// wide (OUT_PROB32, y 32-byte aligned): the vector's eight floats leave in one 256-bit store.
 template <int DT, int OUT>
-__device__ __forceinline__ void lsm_emit(const uint4& raw, f32x2 r2, f32x2 c2, f32x2 s2, f32x2 k2, void* ybase, int64_t v) {
+__device__ __forceinline__ void lsm_emit(const uint4& raw, f32x2 r2, f32x2 c2, f32x2 s2, f32x2 k2, void* ybase, int64_t v, bool wide) {
     constexpr int NP = Traits<DT>::VE / 2;
     f32x2 d[NP];
     widen_pairs<DT>(raw, d);
@@ -90,8 +92,12 @@ __device__ __forceinline__ void lsm_emit(const uint4& raw, f32x2 r2, f32x2 c2, f
         uint4 a, b;
         unpair_bits(d[0], a.x, a.y); unpair_bits(d[1], a.z, a.w);
         unpair_bits(d[NP - 2], b.x, b.y); unpair_bits(d[NP - 1], b.z, b.w);
-        st_stream(out, a);
-        st_stream(out + 1, b);
+        if (wide) {
+            st_stream32(out, a, b);
+        } else {
+            st_stream(out, a);
+            st_stream(out + 1, b);
+        }
     }
 }
 
@@ -143,7 +149,7 @@ __device__ __forceinline__ void lsm_warp_body(const LsmParams& p) {
             char* yrow = static_cast<char*>(p.y) + row * ypitch;
 #pragma unroll
             for (int k = 0; k < VPL; ++k)
-                if (sl + k * LANES < nvec) lsm_emit<DT, OUT>(raw[k], r2, c2, s2, k2, yrow, sl + k * LANES);
+                if (sl + k * LANES < nvec) lsm_emit<DT, OUT>(raw[k], r2, c2, s2, k2, yrow, sl + k * LANES, p.wide != 0);
         }
     }
 }
@@ -237,7 +243,7 @@ lsm_tile_kernel(const LsmParams p) {
         }
 #pragma unroll
         for (int u = 0; u < H; ++u)
-            if (k0 + u * 32 + lane < nvec) lsm_emit<DT, OUT>(raw[u], r2, c2, s2, k2, yrow, k0 + u * 32 + lane);
+            if (k0 + u * 32 + lane < nvec) lsm_emit<DT, OUT>(raw[u], r2, c2, s2, k2, yrow, k0 + u * 32 + lane, p.wide != 0);
     }
 }
 
@@ -360,7 +366,7 @@ lsm_smem_kernel(const LsmParams p, const uint32_t stage_bytes, const int slice, 
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             if (FULL || cbase + u * 32 < nv)
-                lsm_emit<DT, OUT>(flip_vec(raw[u], p.flip), R2, c2, s2, k2, yrow, int64_t(v0) + cbase + u * 32);
+                lsm_emit<DT, OUT>(flip_vec(raw[u], p.flip), R2, c2, s2, k2, yrow, int64_t(v0) + cbase + u * 32, p.wide != 0);
         }
     }
     if (cs > 1) cluster_wait_acquire();    // no block leaves while a peer's deposit into it is still to be issued

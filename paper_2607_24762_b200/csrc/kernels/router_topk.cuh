@@ -30,6 +30,7 @@ struct RouterParams {
     int k;
     float c;           // scale * log2(e)
     int renorm;
+    int wide;          // k == 8 and w, idx 32-byte aligned: a row's eight weights (columns) leave in one 256-bit store
 };
 
 __device__ __forceinline__ uint32_t order_key(float v) {        // monotone float -> uint32, all results >= 1
@@ -320,11 +321,24 @@ router_top8_kernel(const RouterParams p) {
         }
         // 0 * inv_s carries a NaN row into the renormalised weights (inv_s is finite otherwise)
         const float f = p.renorm ? 1.0f / sel + 0.0f * inv_s : inv_s;
+        if (p.wide) {
+            // every lane of the group holds the whole list: one lane stores the row's 32 bytes of weights, another
+            // its 32 bytes of columns (whole sectors, two store instructions instead of sixteen partial ones)
+            if (row_ok && sl == 0)
+                st_stream32(reinterpret_cast<uint4*>(p.w + row * 8),
+                            make_uint4(__float_as_uint(e[0] * f), __float_as_uint(e[1] * f), __float_as_uint(e[2] * f), __float_as_uint(e[3] * f)),
+                            make_uint4(__float_as_uint(e[4] * f), __float_as_uint(e[5] * f), __float_as_uint(e[6] * f), __float_as_uint(e[7] * f)));
+            if (row_ok && sl == (LANES > 1 ? 1 : 0))
+                st_stream32(reinterpret_cast<uint4*>(p.idx + row * 8),
+                            make_uint4(uint32_t(RK::col(best[0])), uint32_t(RK::col(best[1])), uint32_t(RK::col(best[2])), uint32_t(RK::col(best[3]))),
+                            make_uint4(uint32_t(RK::col(best[4])), uint32_t(RK::col(best[5])), uint32_t(RK::col(best[6])), uint32_t(RK::col(best[7]))));
+        } else {
 #pragma unroll
-        for (int r = 0; r < 8; ++r) {
-            if (row_ok && r < p.k && (r % LANES) == sl) {
-                p.idx[row * p.k + r] = RK::col(best[r]);
-                p.w[row * p.k + r] = e[r] * f;
+            for (int r = 0; r < 8; ++r) {
+                if (row_ok && r < p.k && (r % LANES) == sl) {
+                    p.idx[row * p.k + r] = RK::col(best[r]);
+                    p.w[row * p.k + r] = e[r] * f;
+                }
             }
         }
     }

@@ -22,14 +22,18 @@ def built_library():
     assert fs.fs_device_status() == fs.FS_OK
 
 
-def check(x, dtype, scale, misalign=0):
+def check(x, dtype, scale, misalign=0, y_offset=0):
+    """y_offset: floats in front of y (0: 32-byte aligned, one 256-bit store per vector; 4: 16-byte aligned, two
+    128-bit stores; 1: element-wise kernel)."""
     rows, cols = x.shape
     xd = np_to_torch_bits(np.concatenate([np.zeros(misalign, x.dtype), x.ravel()])).cuda()
-    yd = torch.full((rows * cols + 8,), 7.0, dtype=torch.float32, device="cuda")           # 8 guard floats behind
-    fs.fs_softmax_f32out(xd.data_ptr() + 2 * misalign, yd, rows, cols, dtype, scale, torch.cuda.current_stream())
+    yd = torch.full((y_offset + rows * cols + 8,), 7.0, dtype=torch.float32, device="cuda")  # guard floats in front and behind
+    fs.binding._check(fs.binding.lib().fs_softmax_f32out(xd.data_ptr() + 2 * misalign, yd.data_ptr() + 4 * y_offset, rows, cols, dtype,
+                                                        scale, torch.cuda.current_stream().cuda_stream), "fs_softmax_f32out")
     torch.cuda.synchronize()
     got = yd.cpu().numpy()
-    assert np.all(got[rows * cols:] == 7.0)
+    assert np.all(got[:y_offset] == 7.0) and np.all(got[y_offset + rows * cols:] == 7.0)
+    got = got[y_offset:]
     rep = fso.compare(got[:rows * cols].reshape(rows, cols), FP32, fso.softmax_f64(x, dtype, scale))
     assert rep.ok(FP32), (x.shape, dtype, scale, rep)
     return rep
@@ -55,6 +59,16 @@ def test_rows_around_the_four_rows_per_block_kernel(dtype):
             scale = [1.0, 0.25, -0.5, 0.0][(ci + rows) % 4]
             x = W.random_case(rows, nvec * 8, dtype, seed=60 * nvec + rows, sigma=2.0, neg_inf_frac=0.03 if scale > 0 else 0.0)
             check(x, dtype, scale)
+
+
+@pytest.mark.parametrize("dtype", [BF16, FP16])
+def test_output_alignments(dtype):
+    """y at a 32-byte boundary leaves in 256-bit stores, at a 16-byte boundary in pairs of 128-bit stores, anywhere
+    else through the element-wise kernel: the warp kernel, the four-rows-per-block kernel and the split-row kernel."""
+    for ci, (rows, cols) in enumerate(((67, 2048), (9, 3072), (5, 65536), (3, 100000))):
+        x = W.random_case(rows, cols, dtype, seed=4100 + ci, sigma=2.0, neg_inf_frac=0.02)
+        for y_offset in (0, 4, 8, 12, 1):
+            check(x, dtype, [1.0, 0.5][ci % 2], y_offset=y_offset)
 
 
 @pytest.mark.parametrize("dtype", [BF16, FP16])
