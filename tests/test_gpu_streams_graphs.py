@@ -129,3 +129,34 @@ def test_two_kernel_paths_on_two_streams_do_not_share_scratch():
         check(xs[i], W.FP32, 1.0, torch_bits_to_np(yd[i], W.FP32))
         rep = fno.compare(torch_bits_to_np(nd[i], W.FP32), W.FP32, fno.layer_norm_f64(xs[i], W.FP32), fno.error_scale(xs[i], W.FP32, xs[i].shape))
         assert rep.ok(W.FP32), rep
+
+
+def test_a_launch_reads_what_the_previous_launch_of_the_stream_wrote():
+    """Kernels start under programmatic dependent launch while the previous kernel of the stream drains, and the
+    long-row kernels ask L2 for their input before they wait for it. The input of each launch here IS the output
+    of the launch before it, written into a buffer that held NaN until then: a chain run back to back must give,
+    bit for bit, what the same launches give with a synchronisation between them."""
+    cases = [(W.BF16, 256, 262144), (W.BF16, 2048, 32768), (W.FP32, 4096, 8192), (W.BF16, 16384, 2048), (W.FP32, 300, 50000),
+             (W.BF16, 16384, 5120)]
+    s = torch.cuda.current_stream()
+    for dtype, rows, cols in cases:
+        x = np_to_torch_bits(W.random_case(rows, cols, dtype, seed=rows + cols, sigma=3.0)).cuda()
+        bufs = [torch.empty_like(x) for _ in range(4)]
+        want = []
+        src = x
+        for b in bufs:                                                       # one at a time
+            fs.fs_softmax(src, b, rows, cols, dtype, 4.0, s)
+            torch.cuda.synchronize()
+            want.append(b.clone())
+            src = b
+        for rep in range(3):
+            for b in bufs:
+                b.view(torch.int16 if dtype != W.FP32 else torch.int32).fill_(-1)      # NaN patterns
+            src = x
+            for b in bufs:                                                   # back to back
+                fs.fs_softmax(src, b, rows, cols, dtype, 4.0, s)
+                src = b
+            torch.cuda.synchronize()
+            for b, w in zip(bufs, want):
+                assert torch.equal(b.view(torch.uint8), w.view(torch.uint8)), (dtype, rows, cols, rep)
+    assert fs.fs_device_status() == fs.FS_OK
