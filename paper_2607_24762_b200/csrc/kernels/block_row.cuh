@@ -132,6 +132,8 @@ block_row_kernel(const Params p) {
 
 // ---------------------------------------------------------------------------------------------
 // block per row, rows staged in a shared-memory ring by bulk async copies
+// Every warp waits for the row's mbarrier by itself: one polling warp and a block barrier, the form
+// that pays in the split-row kernel, is slower here (fp32 rows of 12 / 16 KiB: 31.6 -> 33.1, 41.0 -> 42.9 us).
 // dynamic shared memory: [nstage][stage_bytes] row buffers | nstage mbarriers (8 B each)
 // ---------------------------------------------------------------------------------------------
 template <int DT, bool NEG, int VPT>
