@@ -97,6 +97,7 @@ int env_int(const char* name, int dflt) {
 }
 bool early_prefetch_enabled() { static const bool v = env_int("FS_EARLY_PF", 1) != 0; return v; }
 bool wide_store_enabled() { static const bool v = env_int("FS_WIDE_STORE", 1) != 0; return v; }
+bool shift_enabled() { static const bool v = env_int("FS_SHIFT", 1) != 0; return v; }
 bool log_enabled() { static const bool v = env_int("FS_LOG", 0) != 0; return v; }
 bool check_enabled() { static const bool v = env_int("FS_CHECK", 0) != 0; return v; }
 #define FS_LOGF(...) do { if (log_enabled()) { std::fprintf(stderr, "[fsoftmax] " __VA_ARGS__); std::fputc('\n', stderr); } } while (0)
@@ -155,6 +156,7 @@ int max_threads_for(int dtype, int vpt) { return vpt * (dtype == FS_DTYPE_FP32 ?
 //           rows beyond 16 x 32 KiB grow the slice.
 int64_t warp_max_row_bytes(int dtype) { return dtype == FS_DTYPE_FP32 ? 3072 : 4096; }
 int64_t block_max_row_bytes(int) { return 8192; }
+constexpr int64_t kSpanMaxRowBytes = 512;            // span_rows_kernel: 128 such rows in a block's shared memory
 int64_t block_tma_max_row_bytes(int dtype) { return dtype == FS_DTYPE_FP32 ? 32768 : 0; }
 
 // 16-bit rows the dispatcher gives the four-rows-per-block kernel (softmax_tile_kernel), in 16-byte vectors
@@ -557,6 +559,7 @@ template <int DT, bool NEG> const void* warp_fn(const WarpGeom& g) {
     }
 FS_VPT_TABLE(block_fn, block_row_kernel)
 FS_VPT_TABLE(block_tma_fn, block_row_tma_kernel)
+FS_VPT_TABLE(block_shift_fn, block_row_shift_kernel)
 
 template <int DT> const void* router_fn(const WarpGeom& g) {
     if (g.vpl == 1) return (const void*)router_topk_kernel<DT, 1, 1>;
@@ -743,6 +746,38 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
     // cluster holds (the dispatcher's own choice only) are cut into segments over two kernels instead.
     const auto run_generic = [&](bool allow_split, int t) -> int {
         if (allow_split && fast && cols * esz >= (int64_t(1) << 20)) return run_softmax_split(dev, x, y, rows, cols, dtype, scale, st);
+        // Rows whose byte length is not a multiple of 16, in tensors that are themselves 16-byte aligned: the block
+        // kernel on the aligned vectors that cover each row (block_row_shift_kernel), as long as a block's registers
+        // hold the row. A zero scale, a forced block size and FS_SHIFT=0 keep the element-wise kernel.
+        if (t == 0 && shift_enabled() && (cols * esz) % 16 != 0 && cols * esz <= kSpanMaxRowBytes && ptr_align(x) >= 16 &&
+            ptr_align(y) >= 16) {
+            // short rows: a block takes 128 consecutive rows as one span of the tensor (span_rows_kernel)
+            const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) -> const void* {
+                return (const void*)span_rows_kernel<decltype(dt)::value, decltype(ng)::value>; });
+            const int tb = 128;
+            const size_t smem = (size_t(tb) * size_t(cols * esz) + 15 + 15) / 16 * 16 + 16;
+            const int64_t grid = (rows + tb - 1) / tb;
+            if (grid <= max_grid && smem <= static_cast<size_t>(dev.smem_optin) - 2048) {
+                int bps = 0;
+                if ((rc = blocks_per_sm(dev, fn, tb, smem, &bps)) != FS_OK) return rc;
+                FS_LOGF("softmax %lld x %lld dtype %d: spans of %d short rows (rows not a multiple of 16 bytes), %zu B shared",
+                        (long long)rows, (long long)cols, dtype, tb, smem);
+                return launch(fn, grid, tb, smem, 0, st, p, int64_t(rows * cols * esz / 16));
+            }
+        }
+        if (t == 0 && shift_enabled() && p.c != 0.0f && (cols * esz) % 16 != 0 && ptr_align(x) >= 16 && ptr_align(y) >= 16 &&
+            cols < (int64_t(1) << 24)) {
+            const int ve = 16 / esz;
+            BlockGeom g;
+            if (block_geom((cols + 2 * (ve - 1)) / ve + 1, dtype, 0, &g)) {
+                const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) { return block_shift_fn<decltype(dt)::value, decltype(ng)::value>(g.vpt); });
+                if (fn) {
+                    FS_LOGF("softmax %lld x %lld dtype %d: block kernel on shifted vectors (rows not a multiple of 16 bytes), %d threads x %d vectors",
+                            (long long)rows, (long long)cols, dtype, g.threads, g.vpt);
+                    return launch(fn, std::min<int64_t>(rows, max_grid), g.threads, 0, 0, st, p, int64_t(rows * cols * esz / 16));
+                }
+            }
+        }
         const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) { return (const void*)generic_row_kernel<decltype(dt)::value, decltype(ng)::value, false>; });
         if (t == 0) {
             t = 32;

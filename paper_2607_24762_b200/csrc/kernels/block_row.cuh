@@ -131,6 +131,183 @@ block_row_kernel(const Params p) {
 }
 
 // ---------------------------------------------------------------------------------------------
+// block per row for rows whose byte length is NOT a multiple of 16 (x and y themselves 16-byte
+// aligned): the row is read as the aligned 16-byte vectors that cover it. Row i starts `head`
+// elements into its first vector and may end inside its last one; those two vectors are shared
+// with the neighbouring rows, so their foreign elements are replaced by the reference identity
+// (they drop out of the maximum and add 0 to the sum) and they are the only ones stored element by
+// element -- a full-vector store there would write the neighbours' outputs. Everything between
+// is the block kernel above: 128-bit accesses, one pass, one ex2 per element. The tensor's very
+// last vector, when the tensor ends inside it, is assembled from scalar loads: no byte beyond the
+// tensor is touched. (A zero scale never comes here: the identity times 0 is NaN.)
+// tensor_vecs = whole 16-byte vectors in the tensor.
+// ---------------------------------------------------------------------------------------------
+template <int DT, bool NEG, int VPT>
+__global__ void __launch_bounds__(BlockCfg<DT, VPT>::MAX_THREADS, 1)
+block_row_shift_kernel(const Params p, const int64_t tensor_vecs) {
+    constexpr int VE = Traits<DT>::VE;
+    constexpr int ESZ = Traits<DT>::ESZ;
+    __shared__ float2 wp[2][32];
+    pdl_launch_dependents();
+    const int T = blockDim.x, tid = threadIdx.x;
+    const int cols = static_cast<int>(p.cols);
+    const uint4* __restrict__ xv = static_cast<const uint4*>(p.x);
+    uint4* __restrict__ yv = static_cast<uint4*>(p.y);
+    const int64_t total = p.rows * p.cols;
+    auto vec = [&](int k) { return tid + k * T; };
+    int par = 0;
+    pdl_wait();
+    for (int64_t row = blockIdx.x; row < p.rows; row += gridDim.x, par ^= 1) {
+        const int64_t e0 = row * p.cols;                                  // the row's first element
+        const int64_t gv0 = (e0 * ESZ) >> 4;                              // the vector that holds it
+        const int head = static_cast<int>(e0 - gv0 * VE);                 // elements of that vector before the row
+        const int nvr = (head + cols + VE - 1) / VE;                      // vectors that cover the row
+        const int tail_keep = head + cols - (nvr - 1) * VE;               // elements of the last vector up to the row's end
+        auto valid = [&](int k) { return tid + k * T < nvr; };
+        uint4 raw[VPT];
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            raw[k] = make_uint4(0u, 0u, 0u, 0u);
+            if (valid(k)) {
+                const int64_t gv = gv0 + vec(k);
+                if (gv < tensor_vecs) {
+                    raw[k] = ld_stream(xv + gv);
+                } else {                                                  // the tensor ends inside this vector
+                    float t[VE];
+#pragma unroll
+                    for (int i = 0; i < VE; ++i) t[i] = gv * VE + i < total ? load_elem<DT>(p.x, gv * VE + i) : 0.0f;
+                    raw[k] = pack<DT>(t);
+                }
+                if (vec(k) == 0 && head > 0) mask_head<DT, NEG>(raw[k], head);
+                if (vec(k) == nvr - 1 && tail_keep < VE) mask_tail<DT, NEG>(raw[k], tail_keep);
+            }
+        }
+        float e[VPT][VE], r_t, s;
+        thread_partial<DT, NEG, VPT>(raw, e, r_t, s, p.c, valid);
+        float R = r_t;
+        block_merge_pairs<NEG>(R, s, wp[par], p.c);
+        const float fac = ref_factor(r_t, R, p.c, ref_identity<NEG>());
+        const float inv = recip<DT>(s);
+        // bf16: e carries 2^64 and inv 2^-64; a factor this small is applied separately (see scale_and_store)
+        const bool one_mul = DT != DT_BF16 || fac >= 0x1p-40f || !(fac == fac);
+        const float f1 = one_mul ? fac * inv : inv, f2 = one_mul ? 1.0f : fac;
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            if (valid(k)) {
+#pragma unroll
+                for (int i = 0; i < VE; ++i) e[k][i] = one_mul ? e[k][i] * f1 : (e[k][i] * f1) * f2;
+                const int v = vec(k);
+                const int lo = (v == 0) ? head : 0, hi = (v == nvr - 1) ? tail_keep : VE;
+                if (lo == 0 && hi == VE) {
+                    st_stream(yv + gv0 + v, pack<DT>(e[k]));
+                } else {
+#pragma unroll
+                    for (int i = 0; i < VE; ++i)
+                        if (i >= lo && i < hi) store_elem<DT>(p.y, (gv0 + v) * VE + i, e[k][i]);
+                }
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Short rows whose byte length is not a multiple of 16 (x and y themselves 16-byte aligned): a
+// block takes blockDim.x CONSECUTIVE rows, i.e. one contiguous span of the tensor. The span is read as
+// the aligned 16-byte vectors that cover it (coalesced, whole sectors) into shared memory, every
+// thread works on its own row there -- the element-wise kernel's arithmetic, thread-local: the
+// reference, the sum, then y = 2^((x - R) c) / S written back in place in the element dtype -- and
+// the span leaves as 16-byte vectors again. Only the span's first and last vector can be shared
+// with the neighbouring blocks: those are stored element by element, own elements only. The
+// tensor's very last vector, when the tensor ends inside it, is assembled from scalar loads.
+// dynamic shared memory: the span, rounded out to whole vectors. tensor_vecs = whole vectors in the tensor.
+// ---------------------------------------------------------------------------------------------
+template <int DT> __device__ __forceinline__ float smem_elem(const unsigned char* sm, int i) {
+    if constexpr (DT == DT_F32) return reinterpret_cast<const float*>(sm)[i];
+    else if constexpr (DT == DT_BF16) return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(sm)[i]);
+    else return __half2float(reinterpret_cast<const __half*>(sm)[i]);
+}
+template <int DT> __device__ __forceinline__ void smem_put(unsigned char* sm, int i, float v) {
+    if constexpr (DT == DT_F32) reinterpret_cast<float*>(sm)[i] = v;
+    else if constexpr (DT == DT_BF16) reinterpret_cast<__nv_bfloat16*>(sm)[i] = __float2bfloat16_rn(v);
+    else reinterpret_cast<__half*>(sm)[i] = __float2half_rn(v);
+}
+
+template <int DT, bool NEG>
+__global__ void __launch_bounds__(128)
+span_rows_kernel(const Params p, const int64_t tensor_vecs) {
+    constexpr int VE = Traits<DT>::VE;
+    constexpr int ESZ = Traits<DT>::ESZ;
+    extern __shared__ __align__(128) unsigned char smem[];
+    pdl_launch_dependents();
+    const int T = blockDim.x, tid = threadIdx.x;
+    const int cols = static_cast<int>(p.cols);
+    const int64_t r0 = int64_t(blockIdx.x) * T;
+    const int nr = static_cast<int>(min(int64_t(T), p.rows - r0));          // rows of this block
+    const int64_t e0 = r0 * p.cols, e1 = (r0 + nr) * p.cols;                // its elements: [e0, e1)
+    const int64_t gv0 = (e0 * ESZ) >> 4, gv1 = (e1 * ESZ + 15) >> 4;        // the vectors that cover them
+    const int nv = static_cast<int>(gv1 - gv0);
+    const int head = static_cast<int>(e0 - gv0 * VE);                       // elements of the first vector before the span
+    const int tail_keep = static_cast<int>(e1 - (gv1 - 1) * VE);            // elements of the last vector inside the span
+    const int64_t total = p.rows * p.cols;
+    const uint4* __restrict__ xv = static_cast<const uint4*>(p.x);
+    uint4* __restrict__ yv = static_cast<uint4*>(p.y);
+    uint4* sv = reinterpret_cast<uint4*>(smem);
+    pdl_wait();
+    for (int vb = tid; vb < nv; vb += 8 * T) {                              // eight loads in flight per thread
+        uint4 t8[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int v = vb + u * T;
+            const int64_t gv = gv0 + v;
+            t8[u] = make_uint4(0u, 0u, 0u, 0u);
+            if (v < nv && gv < tensor_vecs) t8[u] = ld_stream(xv + gv);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int v = vb + u * T;
+            const int64_t gv = gv0 + v;
+            if (v < nv) {
+                if (gv >= tensor_vecs) {                                    // the tensor ends inside this vector
+                    float t[VE];
+#pragma unroll
+                    for (int i = 0; i < VE; ++i) t[i] = gv * VE + i < total ? load_elem<DT>(p.x, gv * VE + i) : 0.0f;
+                    t8[u] = pack<DT>(t);
+                }
+                sv[v] = t8[u];
+            }
+        }
+    }
+    __syncthreads();
+    if (tid < nr) {
+        const int sb = head + tid * cols;                                   // this thread's row, in elements of the span buffer
+        const float ident = ref_identity<NEG>();
+        float r = ident;
+        for (int j = 0; j < cols; ++j) r = ref_pick<NEG>(r, smem_elem<DT>(smem, sb + j));
+        const float ru = (r == ident) ? 0.0f : r;
+        float s0 = 0.0f, s1 = 0.0f;                                         // two chains: the additions need not wait for each other
+        int j = 0;
+        for (; j + 1 < cols; j += 2) {
+            s0 += ex2_noflush((smem_elem<DT>(smem, sb + j) - ru) * p.c);
+            s1 += ex2_noflush((smem_elem<DT>(smem, sb + j + 1) - ru) * p.c);
+        }
+        if (j < cols) s0 += ex2_noflush((smem_elem<DT>(smem, sb + j) - ru) * p.c);
+        const float inv = 1.0f / (s0 + s1);
+        for (int j = 0; j < cols; ++j)
+            smem_put<DT>(smem, sb + j, ex2_noflush((smem_elem<DT>(smem, sb + j) - ru) * p.c) * inv);
+    }
+    __syncthreads();
+    for (int v = tid; v < nv; v += T) {
+        const int64_t gv = gv0 + v;
+        const int lo = (v == 0) ? head : 0, hi = (v == nv - 1) ? tail_keep : VE;
+        if (lo == 0 && hi == VE) {
+            st_stream(yv + gv, sv[v]);
+        } else {
+            for (int i = lo; i < hi; ++i) store_elem<DT>(p.y, gv * VE + i, smem_elem<DT>(smem, v * VE + i));
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // block per row, rows staged in a shared-memory ring by bulk async copies
 // Every warp waits for the row's mbarrier by itself: one polling warp and a block barrier, the form
 // that pays in the split-row kernel, is slower here (fp32 rows of 12 / 16 KiB: 31.6 -> 33.1, 41.0 -> 42.9 us).

@@ -136,6 +136,24 @@ __device__ __forceinline__ void mask_tail(uint4& v, int keep) {
     }
 }
 
+// The mirror image: the first `skip` elements (1 .. VE-1) become the reference identity.
+template <int DT, bool NEG>
+__device__ __forceinline__ void mask_head(uint4& v, int skip) {
+    uint32_t* w = reinterpret_cast<uint32_t*>(&v);
+    if constexpr (DT == DT_F32) {
+        const uint32_t id = NEG ? 0x7f800000u : 0xff800000u;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) if (k < skip) w[k] = id;
+    } else {
+        const uint32_t id16 = (DT == DT_BF16) ? (NEG ? 0x7f80u : 0xff80u) : (NEG ? 0x7c00u : 0xfc00u);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            if (2 * k + 1 < skip) w[k] = id16 | (id16 << 16);
+            else if (2 * k < skip) w[k] = (w[k] & 0xffff0000u) | id16;
+        }
+    }
+}
+
 // ---- dtype unpack / pack of one 16-byte vector ------------------------------------------------
 
 template <int DT>

@@ -18,7 +18,7 @@ from gpu_util import check, run_softmax  # noqa: E402
 def main() -> int:
     ran = 0
     shapes = [(1, 8), (300, 128), (2000, 256), (77, 1000), (600, 2048), (513, 4096), (129, 16384), (70, 40000),
-              (37, 65536), (9, 262144), (5, 100000)]
+              (37, 65536), (9, 262144), (5, 100000), (130, 37), (21, 1001), (3, 50257)]
     for dtype in (W.FP32, W.BF16, W.FP16):
         for rows, cols in shapes:
             x = W.random_case(rows, cols, dtype, seed=rows + cols, sigma=2.5, neg_inf_frac=0.03)

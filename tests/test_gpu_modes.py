@@ -1,5 +1,5 @@
 """The library's environment switches select other launch forms of the same kernels: launches without
-programmatic dependent launch (FS_PDL=0), no prefetch ahead of the dependency wait (FS_EARLY_PF=0), the L2 prefetch off or a whole generation ahead (FS_PREFETCH_PCT=0 / 100),
+programmatic dependent launch (FS_PDL=0), no prefetch ahead of the dependency wait (FS_EARLY_PF=0), rows that are not a multiple of 16 bytes on the element-wise kernel only (FS_SHIFT=0), the L2 prefetch off or a whole generation ahead (FS_PREFETCH_PCT=0 / 100),
 the first wave of a one-shot grid started all at once (FS_LAG_BW=0), a device simulated without cluster launch or
 with little shared memory (FS_SIM_NO_CLUSTER=1, FS_SIM_SMEM_OPTIN), pointer validation and logging (FS_CHECK=1,
 FS_LOG=1). Each form gets the same oracle parity sweep, in a child process because the switches are read once per
@@ -21,6 +21,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
     {"FS_CHECK": "1", "FS_LOG": "1"},
     {"FS_PDL": "0"},
     {"FS_EARLY_PF": "0"},
+    {"FS_SHIFT": "0"},
     {"FS_PREFETCH_PCT": "0"},
     {"FS_PREFETCH_PCT": "100"},
     {"FS_LAG_BW": "0"},
