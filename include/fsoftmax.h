@@ -80,7 +80,7 @@ typedef enum {
     FS_KERNEL_CLUSTER = 4,    /* row split over a thread-block cluster of 1..16 blocks, slices resident in shared memory,
                                  (max,sum) pairs exchanged through distributed shared memory */
     FS_KERNEL_GENERIC = 5     /* any cols, any alignment. Element-wise accesses, the row read twice -- except rows whose byte length
-                                 is not a multiple of 16 in 16-byte aligned tensors, which (up to 64 KiB per row, 128 KiB for fp32)
+                                 is not a multiple of 16 in 16-byte aligned tensors, which (up to what a cluster's shared memory holds)
                                  are read and written as the aligned 16-byte vectors that cover them, unless a block size is forced */
 } fs_kernel;
 

@@ -156,7 +156,11 @@ int max_threads_for(int dtype, int vpt) { return vpt * (dtype == FS_DTYPE_FP32 ?
 //           rows beyond 16 x 32 KiB grow the slice.
 int64_t warp_max_row_bytes(int dtype) { return dtype == FS_DTYPE_FP32 ? 3072 : 4096; }
 int64_t block_max_row_bytes(int) { return 8192; }
-constexpr int64_t kSpanMaxRowBytes = 512;            // span_rows_kernel: 128 such rows in a block's shared memory
+constexpr int64_t kSpanMaxRowBytes = 512;
+// rows up to this size that are not a multiple of 16 bytes stay with the shifted block kernel; longer ones go to the
+// shifted split-row kernel where the device has cluster launch (FS_SHIFT_BLOCK_MAX overrides, bytes). Measured on
+// B200, block / split-row: fp32 rows of 4 KB 32.7 / 54.2 us, bf16 rows of 8 KB 75.7 / 76.8, of 24 KB 208 / 70.5, of 60 KB 228 / 97.
+int64_t shift_block_max_row_bytes() { static const int64_t v = env_int("FS_SHIFT_BLOCK_MAX", 8192); return v; }            // span_rows_kernel: 128 such rows in a block's shared memory
 int64_t block_tma_max_row_bytes(int dtype) { return dtype == FS_DTYPE_FP32 ? 32768 : 0; }
 
 // 16-bit rows the dispatcher gives the four-rows-per-block kernel (softmax_tile_kernel), in 16-byte vectors
@@ -765,11 +769,35 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
                 return launch(fn, grid, tb, smem, 0, st, p, int64_t(rows * cols * esz / 16));
             }
         }
-        if (t == 0 && shift_enabled() && p.c != 0.0f && (cols * esz) % 16 != 0 && ptr_align(x) >= 16 && ptr_align(y) >= 16 &&
-            cols < (int64_t(1) << 24)) {
-            const int ve = 16 / esz;
+        const bool shift_ok = t == 0 && shift_enabled() && p.c != 0.0f && (cols * esz) % 16 != 0 && ptr_align(x) >= 16 &&
+                              ptr_align(y) >= 16 && cols < (int64_t(1) << 24);
+        const int64_t nvr_max = (cols + 2 * (16 / esz - 1)) / (16 / esz);      // vectors that cover a row, at most
+        if (shift_ok && dev.cluster_ok && cols * esz > shift_block_max_row_bytes()) {
+            // long rows: the split-row kernel on the aligned vectors that cover each row (one cluster per row)
+            SmemGeom sg;
+            if (smem_geom(nvr_max, dtype, 0, 0, &sg) && rows <= max_grid / sg.cs) {
+                const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) -> const void* {
+                    return (const void*)smem_row_kernel<decltype(dt)::value, decltype(ng)::value, false, false, true>; });
+                const size_t stage_bytes = smem_row_stage_bytes(sg, dtype);
+                const size_t smem = smem_row_bytes(sg, dtype);
+                if (smem <= static_cast<size_t>(dev.smem_optin) - 2048) {
+                    int ncl = 0;
+                    if ((rc = active_clusters(dev, fn, sg.threads, smem, sg.cs, &ncl)) != FS_OK) return rc;
+                    Params ps = p;
+                    ps.nvec = 0;                                   // the kernel takes every row's own vector range
+                    ps.tensor_vecs = rows * cols * esz / 16;
+                    ps.pf_rows = prefetch_rows(ncl);
+                    set_first_wave_lag(ps, ncl, nvr_max * 16);
+                    FS_LOGF("softmax %lld x %lld dtype %d: split-row kernel on shifted vectors (rows not a multiple of 16 bytes), %d blocks per row x %d "
+                            "threads, %zu B shared", (long long)rows, (long long)cols, dtype, sg.cs, sg.threads, smem);
+                    return launch(fn, rows * sg.cs, sg.threads, smem, sg.cs, st, ps, static_cast<uint32_t>(stage_bytes), sg.slice,
+                                  smem_row_nchunk(sg, dtype));
+                }
+            }
+        }
+        if (shift_ok) {
             BlockGeom g;
-            if (block_geom((cols + 2 * (ve - 1)) / ve + 1, dtype, 0, &g)) {
+            if (block_geom(nvr_max + 1, dtype, 0, &g)) {
                 const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) { return block_shift_fn<decltype(dt)::value, decltype(ng)::value>(g.vpt); });
                 if (fn) {
                     FS_LOGF("softmax %lld x %lld dtype %d: block kernel on shifted vectors (rows not a multiple of 16 bytes), %d threads x %d vectors",

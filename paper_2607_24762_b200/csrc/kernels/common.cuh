@@ -31,6 +31,7 @@ struct Params {
     int lag_rows;
     uint32_t dbg_extra_tx;   // 0 in every product call. The wait-expiry self-test arms each chunk barrier of the
                              // split-row kernel for this many bytes more than it copies, so that the waits run out.
+    int64_t tensor_vecs;     // kernels on shifted vectors: whole 16-byte vectors in the tensor (the last one may be partial)
     int early_pf;            // first wave: ask L2 for the block's own input before griddepcontrol.wait (see pdl_early_prefetch)
     int wait_polls;          // poll cap of the split-row kernel's bounded waits (kDefaultWaitPolls unless that self-test lowered it)
 };

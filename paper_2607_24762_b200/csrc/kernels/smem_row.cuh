@@ -70,10 +70,20 @@ __host__ __device__ constexpr uint32_t smem_row_tail_bytes(int threads, int nchu
 // (arrive right after the deposits, wait before the row ends; in a normal run every peer has
 // arrived long before) keeps a block that gave up from exiting while a peer's deposit into its
 // shared memory is still to be issued.
-template <int DT, bool NEG, bool FULL, bool CAUSAL>
+//
+// SHIFT (one cluster per row, not FULL, not CAUSAL): rows whose byte length is not a multiple of 16,
+// in 16-byte aligned tensors. Row i is then covered by the aligned vectors gv0 .. gv0 + nvr - 1 of the
+// tensor, starts `head` elements into the first of them and may end inside the last; these two
+// vectors are shared with the neighbouring rows. Their foreign elements are replaced by the
+// reference identity as they are read (they drop out of the maximum and add 0 to the sum), and
+// they are the only vectors stored element by element, own elements only. A bulk copy never
+// touches the vector in which the tensor ends: that one is assembled from scalar loads.
+template <int DT, bool NEG, bool FULL, bool CAUSAL, bool SHIFT = false>
 __global__ void __launch_bounds__(256, 3)
 smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, const int nchunk_alloc) {
+    static_assert(!SHIFT || (!FULL && !CAUSAL), "shifted rows: the general, unmasked variant only");
     constexpr int VE = Traits<DT>::VE;
+    constexpr int ESZ = Traits<DT>::ESZ;
     constexpr int U = smem_row_u(DT);
     pdl_launch_dependents();
     extern __shared__ __align__(128) unsigned char smem[];
@@ -93,10 +103,21 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
     int nfill = 0;           // causal: masked vectors of this block's slice, to be filled
     int tail_at = -1;        // causal: local index of the vector that straddles the boundary
     int tail_keep = 0;       //         and how many of its elements are kept
+    int64_t gv0 = 0;         // SHIFT: the tensor's vector that holds the row's first element,
+    int head = 0;            //        the elements of that vector before the row,
+    int nvr = 0;             //        the vectors that cover the row,
+    int last_keep = VE;      //        and the elements of the last one up to the row's end
+    if (SHIFT) {
+        const int64_t e0 = int64_t(cid) * p.cols;
+        gv0 = (e0 * ESZ) >> 4;
+        head = static_cast<int>(e0 - gv0 * VE);
+        nvr = static_cast<int>((head + p.cols + VE - 1) / VE);
+        last_keep = static_cast<int>(head + p.cols - int64_t(nvr - 1) * VE);
+    }
     if (FULL) {
         v0 = static_cast<int>(q) * slice; nv = slice; nchunk = nchunk_alloc;
     } else {
-        const int nvec = static_cast<int>(p.nvec);
+        const int nvec = SHIFT ? nvr : static_cast<int>(p.nvec);
         v0 = min(nvec, static_cast<int>(q) * slice);
         nv = min(nvec, v0 + slice) - v0;                  // vectors of this block's slice (may be 0)
         if (CAUSAL) {
@@ -115,13 +136,23 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + stage_bytes);
     float* rcs = reinterpret_cast<float*>(smem + stage_bytes + kSmemRowBarBytes) + tid;   // [chunk][thread]
     uint4* sv = reinterpret_cast<uint4*>(smem) + tpos;
-    const char* xb = static_cast<const char*>(p.x) + int64_t(v0) * 16;
-    uint4* __restrict__ yv = static_cast<uint4*>(p.y) + v0 + tpos;
-    const int64_t row_bytes = p.nvec * 16;
+    // SHIFT: the row's offset is in gv0 already (one row per cluster) and row_bytes is 0
+    const char* xb = static_cast<const char*>(p.x) + (gv0 + v0) * 16;
+    uint4* __restrict__ yv = static_cast<uint4*>(p.y) + gv0 + v0 + tpos;
+    const int64_t row_bytes = SHIFT ? 0 : p.nvec * 16;
 
     auto issue_row = [&](int64_t row) {                    // thread 0: one bulk copy per chunk
         for (int ch = 0; ch < nchunk; ++ch) {
-            const int cv = FULL ? chunk_vecs : min(chunk_vecs, nv - ch * chunk_vecs);
+            int cv = FULL ? chunk_vecs : min(chunk_vecs, nv - ch * chunk_vecs);
+            if (SHIFT && gv0 + v0 + ch * chunk_vecs + cv > p.tensor_vecs) {
+                // the tensor ends inside this chunk's last vector: scalar loads for that one, into shared memory
+                --cv;
+                const int64_t gv = gv0 + v0 + ch * chunk_vecs + cv;
+                float t[VE];
+#pragma unroll
+                for (int i = 0; i < VE; ++i) t[i] = gv * VE + i < p.rows * p.cols ? load_elem<DT>(p.x, gv * VE + i) : 0.0f;
+                reinterpret_cast<uint4*>(smem)[ch * chunk_vecs + cv] = pack<DT>(t);
+            }
             bulk_load_row(smem_u32(smem) + uint32_t(ch) * uint32_t(chunk_vecs) * 16u,
                           xb + row * row_bytes + int64_t(ch) * chunk_vecs * 16,
                           uint32_t(cv) * 16u, smem_u32(&bars[ch]), p.dbg_extra_tx);
@@ -134,13 +165,18 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
         mbar_init(smem_u32(&xbar[1]), 1);
         mbar_fence_init();
         fence_proxy_async_smem();
+        // (SHIFT: the span may include the vector in which the tensor ends; a prefetch reads nothing)
         pdl_wait_first_wave<true>(cid, p.lag_ns, p.lag_rows, p.early_pf, [&] {
-            if (cid < p.rows && nv > 0) pdl_early_prefetch(xb + int64_t(cid) * row_bytes, int64_t(nv) * 16); });
+            if (cid < p.rows && nv > 0) pdl_early_prefetch(xb + int64_t(cid) * row_bytes, int64_t(SHIFT ? max(nv - 1, 1) : nv) * 16); });
         if (cid < p.rows) issue_row(cid);
         // the row that starts a fraction of a generation of resident clusters later: its slice is on
         // its way to L2 while this one is worked on
         const int64_t pr = int64_t(cid) + p.pf_rows;
-        if (p.pf_rows > 0 && pr < p.rows) {
+        if (SHIFT) {
+            // the later row's own covering vectors, this block's share of them (the last vector left out: see above)
+            if (p.pf_rows > 0 && pr < p.rows && nv > 1)
+                l2_prefetch(static_cast<const char*>(p.x) + (((pr * p.cols * ESZ) >> 4) + v0) * 16, uint32_t(nv - 1) * 16u);
+        } else if (p.pf_rows > 0 && pr < p.rows) {
             int pnv = nv;
             if (CAUSAL) {
                 const int64_t pkeep = max(int64_t(0), min(p.cols, pr + p.q_offset + 1));
@@ -177,6 +213,7 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
             // warp 0 polls, the other warps wait at the hardware barrier (no issue slots spent)
             if (tid < 32 && alive) alive = mbar_wait_warp(smem_u32(&bars[ch]), phase, p.status, p.wait_polls);
             if (T > 32) __syncthreads();
+            else if (SHIFT) __syncwarp();      // (lane 0 may have written the tensor's last vector itself)
             uint4* sc = sv + ch * chunk_vecs;
             const int cbase = ch * chunk_vecs + tpos;
             if (!FULL) {
@@ -195,6 +232,14 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
 #pragma unroll
                 for (int u = 0; u < U; ++u)
                     if (cbase + u * US == tail_at) mask_tail<DT, NEG>(raw[u], tail_keep);
+            }
+            if (SHIFT) {   // the row's first and last vector: the neighbours' elements drop out
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int vr = v0 + cbase + u * US;
+                    if (vr == 0 && head > 0) mask_head<DT, NEG>(raw[u], head);
+                    if (vr == nvr - 1 && last_keep < VE) mask_tail<DT, NEG>(raw[u], last_keep);
+                }
             }
             RefAcc<DT, NEG> ref;
             ref.init();
@@ -236,7 +281,7 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
 
         // ---- pass 2: scale the stored e, chunk by chunk with the chunk's own reference
         const float inv = recip<DT>(s);
-        uint4* yrow = yv + row * p.nvec;
+        uint4* yrow = yv + (SHIFT ? int64_t(0) : row * p.nvec);
         for (int ch = 0; ch < nchunk; ++ch) {
             const uint4* sc = sv + ch * chunk_vecs;
             const float rc = rcs[ch * T];
@@ -251,16 +296,32 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
 #pragma unroll
             for (int u = 0; u < U; ++u) raw[u] = sc[u * US];
             const f32x2 f2 = pair(f1, f1);
+            // SHIFT: the row's first and last vector hold the neighbours' elements too: own elements only, one by one
+            auto put = [&](int u, const uint4& out) {
+                if (SHIFT) {
+                    const int vr = v0 + cbase + u * US;
+                    const int lo = (vr == 0) ? head : 0, hi = (vr == nvr - 1) ? last_keep : VE;
+                    if (lo != 0 || hi != VE) {
+                        float f[VE];
+                        unpack<DT>(out, f);
+#pragma unroll
+                        for (int i = 0; i < VE; ++i)
+                            if (i >= lo && i < hi) store_elem<DT>(p.y, (gv0 + vr) * VE + i, f[i]);
+                        return;
+                    }
+                }
+                st_stream(yc + u * US, out);
+            };
             if (DT == DT_BF16 && !one_mul) {
                 // rare: both multiplications before the one rounding
                 const f32x2 g2 = pair(fac, fac);
 #pragma unroll
                 for (int u = 0; u < U; ++u)
-                    if (FULL || cbase + u * US < nv) st_stream(yc + u * US, scale_vec<DT, true>(raw[u], f2, g2));
+                    if (FULL || cbase + u * US < nv) put(u, scale_vec<DT, true>(raw[u], f2, g2));
             } else {
 #pragma unroll
                 for (int u = 0; u < U; ++u)
-                    if (FULL || cbase + u * US < nv) st_stream(yc + u * US, scale_vec<DT, false>(raw[u], f2, f2));
+                    if (FULL || cbase + u * US < nv) put(u, scale_vec<DT, false>(raw[u], f2, f2));
             }
         }
 

@@ -1,7 +1,7 @@
 """Rows whose byte length is not a multiple of 16, in tensors that are themselves 16-byte aligned: rows up to 512
 bytes are taken 128 at a time as one contiguous span of the tensor (the span's first and last vector are shared with
-the neighbouring blocks), longer ones by the block kernel on the aligned vectors that cover each row (the first and
-last vector of a row are shared with its neighbours). Element-wise parity against the oracle with guard bands around the buffers: every head offset a row
+the neighbouring blocks), longer ones by the block kernel, and beyond 16 KiB by the split-row kernel, on the aligned
+vectors that cover each row (the first and last vector of a row are shared with its neighbours). Element-wise parity against the oracle with guard bands around the buffers: every head offset a row
 can have, rows shorter than a vector, rows that end at the tensor's last partial vector, every dtype, negative
 scales, in place, special values, and the row lengths on both sides of what a block's registers hold."""
 import numpy as np
@@ -71,11 +71,27 @@ def test_in_place_special_values_and_the_element_wise_fallbacks(dtype):
         st, y = run_softmax(xs, dtype, scale, inplace=inplace)
         assert st == fs.FS_OK
         check(xs, dtype, scale, y)
+    xl = W.random_case(9, 30011, dtype, seed=79, sigma=2.0)            # long rows: a cluster per row on shifted vectors
+    xl[1, 0] = bits[0]; xl[2, 30010] = bits[1]; xl[3, :] = bits[2]; xl[4, 1:30000] = bits[2]; xl[5, 0] = bits[2]; xl[5, 30010] = bits[2]
+    for scale, inplace in ((1.0, False), (-1.0, False), (0.0, False), (0.5, True)):
+        st, y = run_softmax(xl, dtype, scale, inplace=inplace)
+        assert st == fs.FS_OK
+        check(xl, dtype, scale, y)
     for kw in (dict(scale=0.0), dict(scale=1.0, offset=1), dict(scale=1.0, threads=64, kernel=fs.FS_KERNEL_GENERIC)):
         scale = kw.pop("scale")                                       # zero scale, unaligned tensors, forced block size
         st, y = run_softmax(x, dtype, scale, **kw)
         assert st == fs.FS_OK
         check(x, dtype, scale, y)
+
+
+@pytest.mark.parametrize("dtype", [FP32, BF16])
+def test_many_long_rows(dtype):
+    """More rows than resident clusters, every head offset a row can have (the row length is odd)."""
+    for rows, cols in ((301, 20001), (130, 50257), (40, 262145)):
+        x = W.random_case(rows, cols, dtype, seed=rows + cols, sigma=2.5, neg_inf_frac=0.01)
+        st, y = run_softmax(x, dtype, 1.0)
+        assert st == fs.FS_OK
+        check(x, dtype, 1.0, y)
 
 
 def test_subnormal_bf16_outputs_survive():
@@ -87,3 +103,10 @@ def test_subnormal_bf16_outputs_survive():
     assert st == fs.FS_OK
     check(x, BF16, 1.0, y)
     assert np.count_nonzero((y[0] > 0) & (y[0] < 0x0080)) > 20
+    row = np.linspace(-91.0, -87.0, 30011)                             # the same on the split-row kernel
+    row[0] = 0.0
+    x = fso.round_from_f64(np.tile(row, (3, 1)), BF16)
+    st, y = run_softmax(x, BF16, 1.0)
+    assert st == fs.FS_OK
+    check(x, BF16, 1.0, y)
+    assert np.count_nonzero((y[0] > 0) & (y[0] < 0x0080)) > 500
