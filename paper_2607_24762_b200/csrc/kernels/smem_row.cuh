@@ -233,7 +233,11 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
                 for (int u = 0; u < U; ++u)
                     if (cbase + u * US == tail_at) mask_tail<DT, NEG>(raw[u], tail_keep);
             }
-            if (SHIFT) {   // the row's first and last vector: the neighbours' elements drop out
+            // SHIFT: does this chunk hold the row's first or last vector (and is that one shared with a neighbour)?
+            // A block-uniform question, so that every other chunk runs the plain code.
+            const int vch = v0 + ch * chunk_vecs;
+            const bool edge = SHIFT && ((vch == 0 && head > 0) || (last_keep < VE && nvr - 1 >= vch && nvr - 1 < vch + chunk_vecs));
+            if (edge) {    // the neighbours' elements drop out
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
                     const int vr = v0 + cbase + u * US;
@@ -297,8 +301,11 @@ smem_row_kernel(const Params p, const uint32_t stage_bytes, const int slice, con
             for (int u = 0; u < U; ++u) raw[u] = sc[u * US];
             const f32x2 f2 = pair(f1, f1);
             // SHIFT: the row's first and last vector hold the neighbours' elements too: own elements only, one by one
+            // (only in a chunk that holds such a vector: block-uniform)
+            const int vch = v0 + ch * chunk_vecs;
+            const bool edge = SHIFT && ((vch == 0 && head > 0) || (last_keep < VE && nvr - 1 >= vch && nvr - 1 < vch + chunk_vecs));
             auto put = [&](int u, const uint4& out) {
-                if (SHIFT) {
+                if (edge) {
                     const int vr = v0 + cbase + u * US;
                     const int lo = (vr == 0) ? head : 0, hi = (vr == nvr - 1) ? last_keep : VE;
                     if (lo != 0 || hi != VE) {
