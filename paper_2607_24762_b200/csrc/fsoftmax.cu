@@ -758,7 +758,7 @@ int run(const void* x, void* y, int64_t rows, int64_t cols, int dtype, float sca
             // short rows: a block takes 128 consecutive rows as one span of the tensor (span_rows_kernel)
             const void* fn = by_variant(dtype, p.neg, [&](auto dt, auto ng) -> const void* {
                 return (const void*)span_rows_kernel<decltype(dt)::value, decltype(ng)::value>; });
-            const int tb = 128;
+            const int tb = 128;        // (32 or 64 rows per block change nothing: the per-thread loops are what takes the time)
             const size_t smem = (size_t(tb) * size_t(cols * esz) + 15 + 15) / 16 * 16 + 16;
             const int64_t grid = (rows + tb - 1) / tb;
             if (grid <= max_grid && smem <= static_cast<size_t>(dev.smem_optin) - 2048) {

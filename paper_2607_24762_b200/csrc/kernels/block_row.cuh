@@ -282,18 +282,25 @@ span_rows_kernel(const Params p, const int64_t tensor_vecs) {
         const int sb = head + tid * cols;                                   // this thread's row, in elements of the span buffer
         const float ident = ref_identity<NEG>();
         float r = ident;
+#pragma unroll 4
         for (int j = 0; j < cols; ++j) r = ref_pick<NEG>(r, smem_elem<DT>(smem, sb + j));
         const float ru = (r == ident) ? 0.0f : r;
+        // The sum may flush terms below 2^-126 (the largest term is 1); the outputs may too, except bf16's, whose
+        // subnormals are still representable values of the output format.
         float s0 = 0.0f, s1 = 0.0f;                                         // two chains: the additions need not wait for each other
         int j = 0;
+#pragma unroll 2
         for (; j + 1 < cols; j += 2) {
-            s0 += ex2_noflush((smem_elem<DT>(smem, sb + j) - ru) * p.c);
-            s1 += ex2_noflush((smem_elem<DT>(smem, sb + j + 1) - ru) * p.c);
+            s0 += ex2_ftz((smem_elem<DT>(smem, sb + j) - ru) * p.c);
+            s1 += ex2_ftz((smem_elem<DT>(smem, sb + j + 1) - ru) * p.c);
         }
-        if (j < cols) s0 += ex2_noflush((smem_elem<DT>(smem, sb + j) - ru) * p.c);
+        if (j < cols) s0 += ex2_ftz((smem_elem<DT>(smem, sb + j) - ru) * p.c);
         const float inv = 1.0f / (s0 + s1);
-        for (int j = 0; j < cols; ++j)
-            smem_put<DT>(smem, sb + j, ex2_noflush((smem_elem<DT>(smem, sb + j) - ru) * p.c) * inv);
+#pragma unroll 4
+        for (int j = 0; j < cols; ++j) {
+            const float t = (smem_elem<DT>(smem, sb + j) - ru) * p.c;
+            smem_put<DT>(smem, sb + j, (DT == DT_BF16 ? ex2_noflush(t) : ex2_ftz(t)) * inv);
+        }
     }
     __syncthreads();
     for (int v = tid; v < nv; v += T) {
